@@ -1,0 +1,231 @@
+/*
+ * ooco.h -- C ABI of the B200 (sm_100a) paged decode-attention library.
+ *
+ * The library implements the one operator that dominates a decode step in an
+ * online/offline co-located LLM serving instance: grouped-query attention of
+ * one new query token per sequence over that sequence's paged KV cache, plus
+ * the append of the new token's K/V into the cache, plus the Roofline byte /
+ * FLOP count a bottleneck-aware scheduler feeds its latency predictor with.
+ *
+ * Conventions that hold for every entry point
+ *   - "device" pointers are CUDA global-memory addresses valid on the current
+ *     device; "host" pointers are ordinary CPU addresses.  The caller owns
+ *     every buffer.  Entry points in this header never allocate device memory.
+ *   - bf16 tensors are passed as `const void*` / `void*` to 16-bit words.
+ *   - `cuda_stream` is a `cudaStream_t` cast to `void*` (NULL = legacy default
+ *     stream).  All device work is enqueued on it; no entry point synchronises
+ *     with the host unless its comment says so.
+ *   - Return value: OOCO_OK (0) or a negative OOCO_E_* code.  Argument
+ *     validation happens on the host before anything is launched; a call that
+ *     returns an error has enqueued nothing.
+ */
+#ifndef OOCO_H_
+#define OOCO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OOCO_VERSION 1
+
+enum {
+  OOCO_OK = 0,
+  OOCO_E_NULLPTR = -1,     /* a required pointer is NULL                          */
+  OOCO_E_SHAPE = -2,       /* an extent is <= 0, Hq % Hkv != 0, bad stride, ...   */
+  OOCO_E_UNSUPPORTED = -3, /* legal shape outside what the kernels are built for  */
+  OOCO_E_WORKSPACE = -4,   /* workspace / staging buffer too small or misaligned  */
+  OOCO_E_CUDA = -5,        /* a CUDA runtime / driver call or a launch failed     */
+  OOCO_E_DEVICE = -6       /* the device-side status word reports a problem       */
+};
+
+/*
+ * Shape of one attention operator invocation (one transformer layer).
+ * Symbols follow the paper's symbol table (Table "Symbol definitions"):
+ * Hq = num_q_heads, Hkv = num_kv_heads; the table's D_h ("hidden dim for
+ * attention") equals Hq * head_dim.  All extents count elements, not bytes.
+ *
+ * The KV pool is the non-contiguous KV-cache memory pool of section 2.1
+ * (continuous batching): `num_blocks` physical blocks of `block_size` token
+ * slots each.  Element (block n, kv head h, slot s, dim i) of k_cache and of
+ * v_cache lives at
+ *     n * kv_block_stride + h * kv_head_stride + s * kv_token_stride + i.
+ * The tuned layout is head-major [num_blocks, Hkv, block_size, head_dim]
+ * (kv_token_stride = head_dim, kv_head_stride = block_size * head_dim); a
+ * token-major pool [num_blocks, block_size, Hkv, head_dim] is accepted too.
+ *
+ * Supported by the kernels: head_dim in {64, 128}; block_size in
+ * {16, 32, 64, 128, 256}; 1 <= Hq / Hkv <= 16; every stride a multiple of 8
+ * elements (16 bytes) and the cache base addresses 16-byte aligned.
+ */
+typedef struct {
+  int32_t batch;              /* B: sequences in the decode batch                  */
+  int32_t num_q_heads;        /* Hq                                                */
+  int32_t num_kv_heads;       /* Hkv; query head hq reads kv head hq / (Hq / Hkv)  */
+  int32_t head_dim;           /* per-head dimension                                */
+  int32_t block_size;         /* token slots per physical block                    */
+  int32_t num_blocks;         /* physical blocks in the pool                       */
+  int32_t max_blocks_per_seq; /* row width of block_table                          */
+  int32_t reserved;           /* must be 0                                         */
+  int64_t kv_block_stride;
+  int64_t kv_head_stride;
+  int64_t kv_token_stride;
+} ooco_shape_t;
+
+/*
+ * Roofline cost of one decode-attention invocation (Table "Operator
+ * Modeling", attention row, with S_q = 1 and S_kv = context length, summed
+ * over the batch).  bytes_paper = bytes_q + bytes_out + bytes_kv is the
+ * table's memory entry; bytes_index (block table and length reads) is not in
+ * the paper's model and is reported beside it.
+ */
+typedef struct {
+  int64_t flops;        /* sum_b 4 * Hq * head_dim * T_b                            */
+  int64_t bytes_q;      /* d * B * Hq * head_dim                                    */
+  int64_t bytes_out;    /* d * B * Hq * head_dim                                    */
+  int64_t bytes_kv;     /* sum_b 2 * d * Hkv * head_dim * T_b                       */
+  int64_t bytes_index;  /* 4 * (B + sum_b ceil(T_b / block_size))                   */
+  int64_t bytes_paper;  /* bytes_q + bytes_out + bytes_kv                           */
+  int64_t total_tokens; /* sum_b T_b                                                */
+} ooco_cost_t;
+
+/*
+ * KV-cache append (section 2.1: a decode execution "reuses and expands" the
+ * KV cache).  For every sequence b and kv head h the head_dim 16-bit words of
+ * k_new[b, h, :] are copied verbatim to slot positions[b] % block_size of
+ * physical block block_table[b, positions[b] / block_size] of k_cache, and
+ * likewise for V.  No other word of either cache is written.
+ *
+ *   k_new, v_new   device, bf16 [B, Hkv, head_dim], contiguous, read-only
+ *   k_cache,v_cache device, bf16 pool (layout: see ooco_shape_t), written
+ *   block_table    device, int32 [B, max_blocks_per_seq], read-only
+ *   positions      device, int32 [B], read-only; a sequence with a negative
+ *                  position or one at or beyond max_blocks_per_seq * block_size
+ *                  is skipped, as is one whose table entry is outside
+ *                  [0, num_blocks)
+ * No two sequences may target the same (block, slot).
+ */
+int ooco_kv_append(const ooco_shape_t* shape, const void* k_new, const void* v_new,
+                   void* k_cache, void* v_cache, const int32_t* block_table,
+                   const int32_t* positions, void* cuda_stream);
+
+/*
+ * Upper bound, in bytes, of the workspace ooco_decode_attention needs for
+ * `shape` whatever the context lengths are.  Host arithmetic only.  Returns 0
+ * for an invalid or unsupported shape.
+ */
+size_t ooco_decode_workspace_bytes(const ooco_shape_t* shape);
+
+/*
+ * Paged decode attention (sections 2.1 and 2.3: one query token per sequence,
+ * the whole cached context of every sequence is read, GQA; section 3.3.1: the
+ * operator is one fused kernel whose score matrix stays on chip).
+ * For every sequence b, query head hq, with kv head h = hq / (Hq / Hkv):
+ *     s_t   = scale * <q[b, hq, :], K_b,t,h>          t in [0, T_b)
+ *     w     = softmax_t(s)
+ *     out[b, hq, :] = sum_t w_t * V_b,t,h
+ * where token t of sequence b lives in slot t % block_size of physical block
+ * block_table[b, t / block_size] and T_b = context_lens[b].  Inputs are bf16,
+ * products and sums are accumulated in fp32, the result is rounded to bf16
+ * (round to nearest even).  T_b = 0 gives out[b] = 0.
+ *
+ *   q              device, bf16 [B, Hq, head_dim], contiguous
+ *   k_cache,v_cache device, bf16 pool, read-only (blocks may be shared
+ *                  between sequences)
+ *   block_table    device, int32 [B, max_blocks_per_seq]; only the first
+ *                  ceil(T_b / block_size) entries of row b are read
+ *   context_lens   device, int32 [B]; values are clamped to
+ *                  [0, max_blocks_per_seq * block_size]
+ *   out            device, bf16 [B, Hq, head_dim], written
+ *   workspace      device, >= ooco_decode_workspace_bytes(shape) bytes,
+ *                  256-byte aligned; scratch, contents undefined afterwards
+ *                  except for the status word ooco_workspace_status reads.
+ *                  Calls that may overlap on the GPU need separate workspaces.
+ * Pool slots at or beyond T_b and table entries beyond the last used block
+ * are never interpreted (they may hold NaN / garbage).  A table entry outside
+ * [0, num_blocks) that IS needed reads as zeros and never faults.
+ * Three launches are enqueued (plan, split-KV partial attention, LSE merge);
+ * the call is asynchronous.
+ */
+int ooco_decode_attention(const ooco_shape_t* shape, const void* q, const void* k_cache,
+                          const void* v_cache, const int32_t* block_table,
+                          const int32_t* context_lens, float scale, void* out,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Reads back the device-side status word an earlier ooco_decode_attention /
+ * ooco_decode_step_host call left in `workspace`.  SYNCHRONISES `cuda_stream`.
+ * *status_host is 0 when every kernel ran to completion, otherwise a bit mask
+ * (1: plan overflowed the work list, 2: a bounded wait inside the attention
+ * kernel gave up).  Returns OOCO_E_DEVICE when *status_host != 0.
+ */
+int ooco_workspace_status(const void* workspace, void* cuda_stream, int32_t* status_host);
+
+/*
+ * Attention row of the paper's operator model (Table "Operator Modeling"),
+ * summed over the batch with S_q = 1, S_kv = context_lens_host[b]; this is the
+ * attention term of the latency predictor L(.) of Algorithms "Offline Request
+ * Migration Decision" and "Mix Decoding Selection".  Pure host arithmetic on
+ * 64-bit integers; touches no device.
+ *
+ *   context_lens_host  HOST, int32 [B]; negative lengths count as 0
+ *   bytes_per_value    the table's d (2 for bf16)
+ *   cost_out           HOST, written
+ * The printed table multiplies the K/V term by Hq / Hkv; with D_h = Hq *
+ * head_dim that cannot be right (GQA would increase traffic), so the K/V term
+ * here is 2 * d * S_kv * D_h * Hkv / Hq, which equals the bytes of the cache
+ * slots the operator addresses and coincides with the printed formula when
+ * Hq = Hkv.
+ */
+int ooco_decode_bytes_model(const ooco_shape_t* shape, const int32_t* context_lens_host,
+                            int32_t bytes_per_value, ooco_cost_t* cost_out);
+
+/*
+ * Bytes of device staging memory ooco_decode_step_host needs for `shape`
+ * (0 for an invalid shape).  Host arithmetic only.
+ */
+size_t ooco_step_staging_bytes(const ooco_shape_t* shape);
+
+/*
+ * One whole decode step of this operator driven from HOST buffers: copies the
+ * step's inputs to the device, appends the new token's K/V at positions[b]
+ * (ooco_kv_append), attends over context_lens[b] tokens
+ * (ooco_decode_attention; a serving step passes context_lens = positions + 1,
+ * section 2.1), and copies `out` back.  Everything is enqueued on
+ * `cuda_stream` in that order and the call returns after the stream has been
+ * SYNCHRONISED, so out_host is valid on return.
+ *
+ *   q_host, k_new_host, v_new_host   HOST (pinned for full copy speed), bf16
+ *                                    [B,Hq,D], [B,Hkv,D], [B,Hkv,D]
+ *   block_table_host                 HOST int32 [B, max_blocks_per_seq]
+ *   positions_host, context_lens_host HOST int32 [B]
+ *   k_cache, v_cache                 DEVICE pool (the persistent serving state)
+ *   out_host                         HOST bf16 [B,Hq,D], written
+ *   staging                          DEVICE scratch, >= ooco_step_staging_bytes
+ *   workspace                        DEVICE, as for ooco_decode_attention
+ */
+int ooco_decode_step_host(const ooco_shape_t* shape, const void* q_host,
+                          const void* k_new_host, const void* v_new_host,
+                          const int32_t* block_table_host, const int32_t* positions_host,
+                          const int32_t* context_lens_host, void* k_cache, void* v_cache,
+                          float scale, void* out_host, void* staging, size_t staging_bytes,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Number of kernels the last successful ooco_decode_attention call on this
+ * thread enqueued (for launch accounting in benchmarks); 0 before any call.
+ */
+int ooco_last_launch_count(void);
+
+/* Static, human-readable name of a status code.  Never NULL. */
+const char* ooco_status_string(int status);
+
+/* OOCO_VERSION the library was built from. */
+int ooco_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OOCO_H_ */

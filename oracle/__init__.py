@@ -1,0 +1,139 @@
+"""fp64 CPU oracle of the paged decode path (TEST INFRASTRUCTURE ONLY).
+
+Thin ctypes/numpy access to ``ooco_oracle.c``.  Only the tests, the smoke check
+and the benchmark's CPU-baseline / reference legs may import this package; the
+product package never does, and nothing here imports the product package.
+bf16 tensors are exchanged as ``numpy.uint16`` arrays of the raw bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ooco_oracle.c")
+_LIB_PATH = os.path.join(_HERE, "libooco_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ooco_oracle.c with gcc (OpenMP, no fast-math) next to its source."""
+    stale = (not os.path.exists(_LIB_PATH)) or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC)
+    if force or stale:
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fno-fast-math", "-shared", "-fPIC",
+               "-o", _LIB_PATH, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i32, i64, f64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
+        lib.oracle_decode_attention.restype = ctypes.c_int
+        lib.oracle_decode_attention.argtypes = [i32] * 7 + [i64] * 3 + [vp] * 5 + [f64, vp, i64, vp, vp, vp]
+        lib.oracle_kv_append.restype = i64
+        lib.oracle_kv_append.argtypes = [i32] * 6 + [i64] * 3 + [vp] * 6
+        lib.oracle_bytes_model.restype = ctypes.c_int
+        lib.oracle_bytes_model.argtypes = [i32] * 5 + [vp, i32, vp]
+        lib.oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    """Threads the attention oracle uses (OpenMP's maximum)."""
+    return int(_load().oracle_num_threads())
+
+
+def _ptr(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def _u16(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, a.dtype
+    return a
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+@dataclass
+class AttentionResult:
+    out: np.ndarray   # float64 [B, Hq, D]
+    lse: np.ndarray   # float64 [B, Hq], natural-log-sum-exp of the scaled scores
+    wsum: np.ndarray  # float64 [B, Hq], sum of the softmax weights
+
+
+def decode_attention(q, k_cache, v_cache, block_table, context_lens, scale, *, num_kv_heads,
+                     block_size, strides, pairs=None) -> AttentionResult:
+    """Softmax attention of one query token per sequence over its paged KV cache.
+
+    q: uint16 [B, Hq, D]; k_cache / v_cache: flat or shaped uint16 pools addressed through
+    ``strides`` = (block, head, token) element strides; block_table: int32 [B, MB];
+    context_lens: int32 [B]; pairs: optional int32 [n, 2] list of (b, hq) rows to compute
+    (all other rows of the result are NaN).
+    """
+    lib = _load()
+    q = _u16(q)
+    B, Hq, D = q.shape
+    k_cache, v_cache = _u16(k_cache), _u16(v_cache)
+    block_table, context_lens = _i32(block_table), _i32(context_lens)
+    assert block_table.ndim == 2 and block_table.shape[0] == B and context_lens.shape == (B,)
+    MB = block_table.shape[1]
+    bstr, hstr, tstr = (int(s) for s in strides)
+    num_blocks = k_cache.size // bstr
+    assert k_cache.size == v_cache.size
+    out = np.full((B, Hq, D), np.nan, dtype=np.float64)
+    lse = np.full((B, Hq), np.nan, dtype=np.float64)
+    wsum = np.full((B, Hq), np.nan, dtype=np.float64)
+    if pairs is not None:
+        pairs = _i32(pairs).reshape(-1, 2)
+        pp, npairs = _ptr(pairs), pairs.shape[0]
+    else:
+        pp, npairs = None, 0
+    rc = lib.oracle_decode_attention(B, Hq, num_kv_heads, D, block_size, num_blocks, MB, bstr, hstr,
+                                     tstr, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+                                     _ptr(context_lens), float(scale), pp, npairs, _ptr(out),
+                                     _ptr(lse), _ptr(wsum))
+    if rc != 0:
+        raise ValueError(f"oracle_decode_attention failed with {rc}")
+    return AttentionResult(out, lse, wsum)
+
+
+def kv_append(k_new, v_new, k_cache, v_cache, block_table, positions, *, block_size, strides) -> int:
+    """In-place append of k_new / v_new uint16 [B, Hkv, D] into the uint16 pools. Returns rows written."""
+    lib = _load()
+    k_new, v_new = _u16(k_new), _u16(v_new)
+    B, Hkv, D = k_new.shape
+    assert k_cache.dtype == np.uint16 and v_cache.dtype == np.uint16
+    assert k_cache.flags.c_contiguous and v_cache.flags.c_contiguous and k_cache.flags.writeable
+    block_table, positions = _i32(block_table), _i32(positions)
+    MB = block_table.shape[1]
+    bstr, hstr, tstr = (int(s) for s in strides)
+    num_blocks = k_cache.size // bstr
+    return int(lib.oracle_kv_append(B, Hkv, D, block_size, num_blocks, MB, bstr, hstr, tstr,
+                                    _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
+                                    _ptr(block_table), _ptr(positions)))
+
+
+COST_FIELDS = ("flops", "bytes_q", "bytes_out", "bytes_kv", "bytes_index", "bytes_paper", "total_tokens")
+
+
+def bytes_model(context_lens, *, num_q_heads, num_kv_heads, head_dim, block_size, bytes_per_value=2) -> dict:
+    """Attention row of the paper's operator table summed over the batch, as a dict of ints."""
+    lib = _load()
+    context_lens = _i32(context_lens)
+    cost = np.zeros(7, dtype=np.int64)
+    rc = lib.oracle_bytes_model(context_lens.shape[0], num_q_heads, num_kv_heads, head_dim, block_size,
+                                _ptr(context_lens), bytes_per_value, _ptr(cost))
+    if rc != 0:
+        raise ValueError(f"oracle_bytes_model failed with {rc}")
+    return {k: int(v) for k, v in zip(COST_FIELDS, cost)}
