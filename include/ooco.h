@@ -219,6 +219,16 @@ int ooco_decode_step_host(const ooco_shape_t* shape, const void* q_host,
  */
 int ooco_last_launch_count(void);
 
+/*
+ * Launch-shape override for benchmark sweeps (process-wide; the defaults are the tuned
+ * values).  knob: 0 consumer warps per CTA {2,4,8}; 1 pipeline stages (0 = as many as
+ * fit); 2 CTAs per SM {1..4}; 3 / 4 minimum / maximum split-KV chunk in tokens (multiples
+ * of 128); 5 target work items per CTA; 6 non-zero = one TMA copy per 64-dim half.
+ * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
+ * unknown knob or a value outside its range.
+ */
+int ooco_set_tuning(int knob, int value);
+
 /* Static, human-readable name of a status code.  Never NULL. */
 const char* ooco_status_string(int status);
 

@@ -1,0 +1,203 @@
+"""ctypes binding of the `ooco_*` C ABI: argument marshalling only.
+
+Every function takes torch tensors (device memory owned by the caller), passes their raw
+pointers through the C boundary and raises `OocoError` on a non-zero status.  There is no
+fallback: without the built CUDA library the import of the library fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libooco.so")
+
+EXPORTS = (
+    "ooco_kv_append", "ooco_decode_workspace_bytes", "ooco_decode_attention", "ooco_workspace_status",
+    "ooco_decode_bytes_model", "ooco_step_staging_bytes", "ooco_decode_step_host",
+    "ooco_last_launch_count", "ooco_set_tuning", "ooco_status_string", "ooco_version",
+)
+
+
+class OocoError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class ooco_shape_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "batch", "num_q_heads", "num_kv_heads", "head_dim", "block_size", "num_blocks",
+        "max_blocks_per_seq", "reserved")] + [(n, ctypes.c_int64) for n in (
+            "kv_block_stride", "kv_head_stride", "kv_token_stride")]
+
+
+class ooco_cost_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in (
+        "flops", "bytes_q", "bytes_out", "bytes_kv", "bytes_index", "bytes_paper", "total_tokens")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library (built by `paper_2511_21862_b200.build`); no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2511_21862_b200.build` "
+                              "(there is no non-CUDA fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32p = ctypes.c_void_p, ctypes.c_void_p
+        sp = ctypes.POINTER(ooco_shape_t)
+        L.ooco_kv_append.restype = ctypes.c_int
+        L.ooco_kv_append.argtypes = [sp, vp, vp, vp, vp, i32p, i32p, vp]
+        L.ooco_decode_workspace_bytes.restype = ctypes.c_size_t
+        L.ooco_decode_workspace_bytes.argtypes = [sp]
+        L.ooco_decode_attention.restype = ctypes.c_int
+        L.ooco_decode_attention.argtypes = [sp, vp, vp, vp, i32p, i32p, ctypes.c_float, vp, vp,
+                                            ctypes.c_size_t, vp]
+        L.ooco_workspace_status.restype = ctypes.c_int
+        L.ooco_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+        L.ooco_decode_bytes_model.restype = ctypes.c_int
+        L.ooco_decode_bytes_model.argtypes = [sp, i32p, ctypes.c_int32, ctypes.POINTER(ooco_cost_t)]
+        L.ooco_step_staging_bytes.restype = ctypes.c_size_t
+        L.ooco_step_staging_bytes.argtypes = [sp]
+        L.ooco_decode_step_host.restype = ctypes.c_int
+        L.ooco_decode_step_host.argtypes = [sp, vp, vp, vp, i32p, i32p, i32p, vp, vp, ctypes.c_float, vp,
+                                            vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
+        L.ooco_last_launch_count.restype = ctypes.c_int
+        L.ooco_set_tuning.restype = ctypes.c_int
+        L.ooco_set_tuning.argtypes = [ctypes.c_int, ctypes.c_int]
+        L.ooco_status_string.restype = ctypes.c_char_p
+        L.ooco_status_string.argtypes = [ctypes.c_int]
+        L.ooco_version.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().ooco_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise OocoError(status, where)
+
+
+@dataclass(frozen=True)
+class Shape:
+    batch: int
+    num_q_heads: int
+    num_kv_heads: int
+    head_dim: int
+    block_size: int
+    num_blocks: int
+    max_blocks_per_seq: int
+    kv_block_stride: int
+    kv_head_stride: int
+    kv_token_stride: int
+
+    def c(self) -> ooco_shape_t:
+        return ooco_shape_t(self.batch, self.num_q_heads, self.num_kv_heads, self.head_dim, self.block_size,
+                            self.num_blocks, self.max_blocks_per_seq, 0, self.kv_block_stride,
+                            self.kv_head_stride, self.kv_token_stride)
+
+
+KNOBS = {"warps": 0, "stages": 1, "ctas_per_sm": 2, "chunk_min": 3, "chunk_max": 4, "items_per_cta": 5,
+         "split_halves": 6}
+
+
+def set_tuning(**kw):
+    for k, v in kw.items():
+        _check(lib().ooco_set_tuning(KNOBS[k], int(v)), f"ooco_set_tuning({k}={v})")
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype=None) -> int:
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, (t.dtype, dtype)
+    return t.data_ptr()
+
+
+def workspace_bytes(shape: Shape) -> int:
+    n = lib().ooco_decode_workspace_bytes(ctypes.byref(shape.c()))
+    if n == 0:
+        raise OocoError(-3, "ooco_decode_workspace_bytes")
+    return int(n)
+
+
+def step_staging_bytes(shape: Shape) -> int:
+    n = lib().ooco_step_staging_bytes(ctypes.byref(shape.c()))
+    if n == 0:
+        raise OocoError(-3, "ooco_step_staging_bytes")
+    return int(n)
+
+
+def kv_append(shape: Shape, k_new, v_new, k_cache, v_cache, block_table, positions, stream=None):
+    _check(lib().ooco_kv_append(
+        ctypes.byref(shape.c()), _dev(k_new, torch.bfloat16), _dev(v_new, torch.bfloat16),
+        _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32),
+        _dev(positions, torch.int32), _stream_ptr(stream)), "ooco_kv_append")
+
+
+def decode_attention(shape: Shape, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace,
+                     stream=None):
+    _check(lib().ooco_decode_attention(
+        ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_cache, torch.bfloat16),
+        _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
+        float(scale), _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        _stream_ptr(stream)), "ooco_decode_attention")
+
+
+def workspace_status(workspace, stream=None) -> int:
+    """Synchronises the stream and returns the device status word (0 = clean)."""
+    v = ctypes.c_int32(0)
+    rc = lib().ooco_workspace_status(_dev(workspace), _stream_ptr(stream), ctypes.byref(v))
+    if rc not in (0, -6):
+        raise OocoError(rc, "ooco_workspace_status")
+    return int(v.value)
+
+
+def decode_bytes_model(shape: Shape, context_lens_host, bytes_per_value: int = 2) -> dict:
+    """Host-only: `context_lens_host` is a CPU int32 tensor."""
+    t = context_lens_host
+    assert not t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()
+    c = ooco_cost_t()
+    _check(lib().ooco_decode_bytes_model(ctypes.byref(shape.c()), t.data_ptr(), bytes_per_value,
+                                         ctypes.byref(c)), "ooco_decode_bytes_model")
+    return {n: int(getattr(c, n)) for n, _ in ooco_cost_t._fields_}
+
+
+def decode_step_host(shape: Shape, q_host, k_new_host, v_new_host, block_table_host, positions_host,
+                     context_lens_host, k_cache, v_cache, scale, out_host, staging, workspace, stream=None):
+    """One append + attention step from host (ideally pinned) buffers; returns with out_host filled."""
+    for t in (q_host, k_new_host, v_new_host, block_table_host, positions_host, context_lens_host, out_host):
+        assert not t.is_cuda and t.is_contiguous()
+    _check(lib().ooco_decode_step_host(
+        ctypes.byref(shape.c()), q_host.data_ptr(), k_new_host.data_ptr(), v_new_host.data_ptr(),
+        block_table_host.data_ptr(), positions_host.data_ptr(), context_lens_host.data_ptr(),
+        _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), float(scale), out_host.data_ptr(),
+        _dev(staging), staging.numel() * staging.element_size(), _dev(workspace),
+        workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step_host")
+
+
+def last_launch_count() -> int:
+    return int(lib().ooco_last_launch_count())
+
+
+def shape_of(batch) -> Shape:
+    """Shape struct of a `paper_2511_21862_b200.inputs.DecodeBatch`."""
+    cfg = batch.cfg
+    bstr, hstr, tstr = batch.strides
+    return Shape(batch.context_lens.numel(), cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.block_size,
+                 batch.num_blocks, batch.max_blocks_per_seq, bstr, hstr, tstr)

@@ -1,0 +1,568 @@
+// Paged decode attention for sm_100a: plan -> split-KV partial attention -> LSE merge.
+//
+// Work item = (sequence b, kv head h, token chunk [t0, t1)).  One CTA processes an item with
+// one producer warp that streams K / V tiles global -> shared through TMA (128-byte swizzle)
+// into a ring of stages, and NCW consumer warps that each own 16 tokens of every stage:
+//   S[16 tok x 8 heads]  = K_tile (A, ldmatrix) x Q^T (B, registers)          mma.sync bf16
+//   online softmax over tokens (warp shuffles), P packed to bf16, transposed by movmatrix
+//   O^T[D x 8 heads]    += V_tile^T (A, ldmatrix.trans) x P (B)               mma.sync bf16
+// so every K / V byte is read from HBM once, by one CTA, for the whole GQA group.
+// CTAs are persistent and pull items from a device-side list through an atomic counter.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ptx.cuh"
+
+namespace ooco {
+
+constexpr int kStatusPlanOverflow = 1;
+constexpr int kStatusWaitTimeout = 2;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every in-kernel wait gives up after 2 s
+
+struct WsHeader {  // first 256 bytes of the workspace
+  int32_t status;
+  int32_t n_items;
+  int32_t next_item;
+  int32_t chunk_tokens;
+  int32_t n_split_seqs;
+  int32_t pad[59];
+};
+static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
+
+struct DecodeParams {
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  const int32_t* block_table;
+  const int32_t* context_lens;
+  WsHeader* hdr;
+  int4* items;            // [max_items] {b, h, t0, t1}
+  int32_t* seq_first;     // [B + 1] first chunk index of each sequence (exclusive scan)
+  float* part_o;          // [max_items, G, D] normalised partial outputs
+  float* part_lse;        // [max_items, G] log2-domain log-sum-exp of each partial
+  int32_t B, Hq, Hkv, G, D, bs, MB;
+  int32_t max_items;
+  int32_t tile_rows;      // token rows per TMA box = min(bs, stage tokens)
+  int32_t split_halves;   // 1: one 4-d TMA per 64-dim half; 0: one 5-d TMA per box
+  int32_t nstages;
+  int32_t grid_main;      // CTAs of the attention kernel (first items are assigned statically)
+  int32_t chunk_min, chunk_max, items_per_cta;
+  float scale_log2e;
+};
+
+// ------------------------------------------------------------------------------------ plan
+// One CTA.  Chooses the chunk length from the total work, splits every sequence into
+// near-equal chunks that are multiples of `stage_tok`, and writes the item list.
+template <int kThreads>
+__global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stage_tok) {
+  __shared__ long long s_red[kThreads / 32];
+  __shared__ int s_scan[kThreads / 32];
+  __shared__ long long s_total;
+  __shared__ int s_run;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const long long cap = (long long)p.MB * p.bs;
+
+  long long acc = 0;
+  for (int b = tid; b < p.B; b += kThreads) {
+    long long t = p.context_lens[b];
+    acc += t < 0 ? 0 : (t > cap ? cap : t);
+  }
+  for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) s_red[wid] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    long long t = 0;
+    for (int i = 0; i < kThreads / 32; ++i) t += s_red[i];
+    s_total = t;
+    s_run = 0;
+  }
+  __syncthreads();
+  // chunk length: about items_per_cta items per CTA, within [chunk_min, chunk_max]
+  long long want = (s_total * p.Hkv) / ((long long)p.grid_main * p.items_per_cta) + 1;
+  want = ((want + stage_tok - 1) / stage_tok) * stage_tok;
+  if (want < p.chunk_min) want = p.chunk_min;
+  if (want > p.chunk_max) want = p.chunk_max;
+  const int chunk = (int)want;
+
+  // exclusive scan of chunks per sequence, kThreads sequences at a time
+  for (int base = 0; base < p.B; base += kThreads) {
+    const int b = base + tid;
+    int n = 0;
+    if (b < p.B) {
+      long long t = p.context_lens[b];
+      t = t < 0 ? 0 : (t > cap ? cap : t);
+      n = (int)((t + chunk - 1) / chunk);
+    }
+    int inc = n;
+    for (int o = 1; o < 32; o <<= 1) {
+      int v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    if (lane == 31) s_scan[wid] = inc;
+    __syncthreads();
+    if (wid == 0) {
+      int v = lane < kThreads / 32 ? s_scan[lane] : 0;
+      int w = v;
+      for (int o = 1; o < 32; o <<= 1) {
+        int u = __shfl_up_sync(0xffffffffu, w, o);
+        if (lane >= o) w += u;
+      }
+      if (lane < kThreads / 32) s_scan[lane] = w - v;  // exclusive warp offsets
+    }
+    __syncthreads();
+    const int run = s_run;
+    if (b < p.B) p.seq_first[b] = run + s_scan[wid] + inc - n;
+    __syncthreads();
+    if (tid == kThreads - 1) s_run = run + s_scan[wid] + inc;
+    __syncthreads();
+  }
+  const int n_chunks = s_run;
+  if (tid == 0) p.seq_first[p.B] = n_chunks;
+  __syncthreads();
+  long long n_items = (long long)n_chunks * p.Hkv;
+  const bool overflow = n_items > p.max_items;
+  if (overflow) n_items = 0;
+  if (tid == 0) {
+    p.hdr->status = overflow ? kStatusPlanOverflow : 0;
+    p.hdr->n_items = (int)n_items;
+    p.hdr->next_item = p.grid_main;
+    p.hdr->chunk_tokens = chunk;
+  }
+  // items, ordered (sequence, chunk, kv head); the sequence of a chunk is found by bisection
+  for (long long i = tid; i < n_items; i += kThreads) {
+    const int ci = (int)(i / p.Hkv), h = (int)(i % p.Hkv);
+    int lo = 0, hi = p.B;  // largest b with seq_first[b] <= ci
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (p.seq_first[mid] <= ci) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    long long t = p.context_lens[b];
+    t = t > cap ? cap : t;
+    const int T = (int)t;
+    const int n = p.seq_first[b + 1] - p.seq_first[b];
+    const int c = ci - p.seq_first[b];
+    int len = (T + n - 1) / n;                              // near-equal chunks ...
+    len = ((len + stage_tok - 1) / stage_tok) * stage_tok;  // ... in whole stages
+    int t0 = c * len, t1 = t0 + len;
+    if (t0 > T) t0 = T;
+    if (t1 > T) t1 = T;
+    p.items[i] = make_int4(b, h, t0, t1);
+  }
+  // sequences without context produce zeros
+  const int row = p.Hq * p.D;
+  for (int b = wid; b < p.B; b += kThreads / 32) {
+    if (p.context_lens[b] > 0) continue;
+    for (int i = lane; i < row; i += 32) p.out[(size_t)b * row + i] = __float2bfloat16(0.f);
+  }
+}
+
+// Bounded mbarrier wait whose verdict is the same in every lane of the (converged) warp.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity, abort_flag, kWaitLimitNs));
+}
+
+// ------------------------------------------------------------------------------------ main
+// Shared-memory carve-up, shared by host (sizing) and device.
+template <int D, int NCW, int NT>
+struct SmemLayout {
+  static constexpr int kStageTok = 16 * NCW;
+  static constexpr int kTileBytes = kStageTok * D * 2;      // K (or V) bytes of one stage
+  static constexpr int kStageBytes = 2 * kTileBytes;
+  static constexpr int kHeads = NT * 8;
+  static constexpr int kOStride = D + 4;                     // floats; keeps the merge stores conflict-free
+  static constexpr int kMergeBytes = NCW * kHeads * (kOStride + 2) * 4;
+  __host__ __device__ static int q_slot_bytes(int G) { return ((G * D * 2 + 127) / 128) * 128; }
+  __host__ __device__ static size_t total(int nstages, int G) {
+    return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16) + kMergeBytes + 64;
+  }
+};
+
+template <int D, int NCW, int NT>
+__global__ void __launch_bounds__((NCW + 1) * 32, 1)
+decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                   const DecodeParams p) {
+  using L = SmemLayout<D, NCW, NT>;
+  constexpr int kStageTok = L::kStageTok;
+  constexpr int KS = D / 16;  // k-steps of the score MMA = m-tiles of the value MMA
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int s_abort;
+
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const int nst = p.nstages;
+  const int qslot = L::q_slot_bytes(p.G);
+  const uint32_t s_stage = base;
+  const uint32_t s_q = s_stage + (uint32_t)nst * L::kStageBytes;
+  const uint32_t s_merge = s_q + (uint32_t)nst * qslot;
+  const uint32_t s_meta = s_merge + L::kMergeBytes;
+  const uint32_t s_full = s_meta + (uint32_t)nst * 16;
+  const uint32_t s_empty = s_full + (uint32_t)nst * 8;
+  const uint32_t s_mbar = s_empty + (uint32_t)nst * 8;
+  float* g_merge = reinterpret_cast<float*>(gen + (s_merge - base));
+  int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
+  uint8_t* g_q = gen + (s_q - base);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int i = 0; i < nst; ++i) {
+      mbar_init(s_full + 8 * i, 1);
+      mbar_init(s_empty + 8 * i, NCW);
+    }
+    mbar_init(s_mbar, NCW * 32);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const int n_items = p.hdr->n_items;
+
+  if (warp == NCW) {
+    // ================================================================= producer warp
+    if (lane == 0) {
+      prefetch_tmap(&tm_k);
+      prefetch_tmap(&tm_v);
+    }
+    const int boxes_per_stage = kStageTok / p.tile_rows;
+    const uint32_t box_bytes = (uint32_t)p.tile_rows * D * 2;
+    int it = 0;
+    int item = blockIdx.x;
+    int4 d = make_int4(0, 0, 0, 0);
+    int blk_cur = 0;
+    if (item < n_items) {
+      d = p.items[item];
+      const int tb = d.z + lane * p.tile_rows;
+      if (lane < boxes_per_stage && tb < d.w) blk_cur = p.block_table[(size_t)d.x * p.MB + tb / p.bs];
+    }
+    bool ok = true;
+    while (item < n_items && ok) {
+      int nxt = 0;
+      if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
+      int4 nd = make_int4(0, 0, 0, 0);
+      int blk_nxt_item = 0;
+      const int b = d.x, h = d.y, t0 = d.z, t1 = d.w;
+      const int nstage_item = (t1 - t0 + kStageTok - 1) / kStageTok;
+      const int32_t* row = p.block_table + (size_t)b * p.MB;
+      for (int s = 0; s < nstage_item; ++s, ++it) {
+        const int tok0 = t0 + s * kStageTok;
+        const int ntok = min(kStageTok, t1 - tok0);
+        const int nbox = (ntok + p.tile_rows - 1) / p.tile_rows;
+        // table entries of the following stage, one stage ahead of their use
+        int blk_n = 0;
+        {
+          const int tb = tok0 + kStageTok + lane * p.tile_rows;
+          if (s + 1 < nstage_item && lane < boxes_per_stage && tb < t1) blk_n = row[tb / p.bs];
+        }
+        const int slot = it % nst;
+        const uint32_t ph = (uint32_t)(it / nst) & 1u;
+        if (!warp_wait(s_empty + 8 * slot, ph ^ 1u, &s_abort)) {
+          ok = false;
+          break;
+        }
+        const uint32_t full = s_full + 8 * slot;
+        if (lane == 0) {
+          const int flags = (s == 0 ? 1 : 0) | (s == nstage_item - 1 ? 2 : 0);
+          g_meta[slot] = make_int4(item, b, h, ntok | (flags << 16));
+          uint32_t bytes = 2u * nbox * box_bytes;
+          if (s == 0) bytes += (uint32_t)p.G * D * 2;
+          mbar_arrive_expect_tx(full, bytes);
+        }
+        __syncwarp();
+        if (lane < nbox) {
+          const int tb = tok0 + lane * p.tile_rows;
+          const int c_tok = tb % p.bs;
+          const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + lane * box_bytes;
+          const uint32_t dv = dk + L::kTileBytes;
+          if (D == 128 && !p.split_halves) {
+            tma_load_5d(dk, &tm_k, full, 0, c_tok, 0, h, blk_cur);
+            tma_load_5d(dv, &tm_v, full, 0, c_tok, 0, h, blk_cur);
+          } else {
+#pragma unroll
+            for (int j = 0; j < D / 64; ++j) {
+              tma_load_4d(dk + j * (box_bytes / (D / 64)), &tm_k, full, 64 * j, c_tok, h, blk_cur);
+              tma_load_4d(dv + j * (box_bytes / (D / 64)), &tm_v, full, 64 * j, c_tok, h, blk_cur);
+            }
+          }
+        }
+        if (s == 0 && lane == 0)
+          bulk_g2s(s_q + (uint32_t)slot * qslot, p.q + ((size_t)b * p.Hq + (size_t)h * p.G) * D,
+                   (uint32_t)p.G * D * 2, full);
+        // look ahead to the next item: its descriptor, then its first table entries
+        if (s == 0) {
+          nxt = __shfl_sync(0xffffffffu, nxt, 0);
+          if (nxt < n_items) nd = p.items[nxt];
+        }
+        if (s == (nstage_item > 1 ? 1 : 0) && nxt < n_items) {
+          const int tb = nd.z + lane * p.tile_rows;
+          if (lane < boxes_per_stage && tb < nd.w) blk_nxt_item = p.block_table[(size_t)nd.x * p.MB + tb / p.bs];
+        }
+        blk_cur = blk_n;
+      }
+      if (nstage_item <= 0) nxt = __shfl_sync(0xffffffffu, nxt, 0);  // (items are never empty)
+      item = nxt;
+      d = nd;
+      blk_cur = blk_nxt_item;
+    }
+    // end marker (one stage, seen by every consumer warp)
+    if (ok) {
+      const int slot = it % nst;
+      const uint32_t ph = (uint32_t)(it / nst) & 1u;
+      if (warp_wait(s_empty + 8 * slot, ph ^ 1u, &s_abort)) {
+        if (lane == 0) {
+          g_meta[slot] = make_int4(-1, 0, 0, 0);
+          mbar_arrive(s_full + 8 * slot);
+        }
+        ++it;
+      } else {
+        ok = false;
+      }
+    }
+    if (!ok) {
+      // stop path: record it, then wait (bounded) until every copy already issued has landed
+      if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+      int dummy_abort = 0;
+      const int pending = it < nst ? it : nst;
+      for (int k = 0; k < pending; ++k) {
+        const int j = it - 1 - k;
+        mbar_wait_bounded(s_full + 8 * (j % nst), (uint32_t)(j / nst) & 1u, &dummy_abort, kWaitLimitNs / 8);
+      }
+    }
+    return;
+  }
+
+  // =================================================================== consumer warps
+  const int g = lane >> 2, t = lane & 3;
+  float m_run[NT][2], l_run[NT][2];
+  float o_acc[NT][KS][4];
+  uint32_t qf[NT][KS][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    m_run[nt][0] = m_run[nt][1] = -INFINITY;
+    l_run[nt][0] = l_run[nt][1] = 0.f;
+#pragma unroll
+    for (int k = 0; k < KS; ++k) {
+      o_acc[nt][k][0] = o_acc[nt][k][1] = o_acc[nt][k][2] = o_acc[nt][k][3] = 0.f;
+      qf[nt][k][0] = qf[nt][k][1] = 0u;
+    }
+  }
+  // per-lane row / chunk selectors of the two ldmatrix patterns
+  const int r0 = 16 * warp;                        // first token row of this warp inside a stage
+  const int box = r0 / p.tile_rows;
+  const int rb = r0 % p.tile_rows;
+  const uint32_t box_bytes = (uint32_t)p.tile_rows * D * 2;
+  const uint32_t half_bytes = (uint32_t)p.tile_rows * 128;   // one 64-dim half of a box
+  const int lr_k = (lane & 7) + ((lane >> 3) & 1) * 8, cs_k = lane >> 4;
+  const int lr_v = (lane & 7) + (lane >> 4) * 8, cs_v = (lane >> 3) & 1;
+  const uint32_t off_k = box * box_bytes + (uint32_t)(rb + lr_k) * 128;
+  const uint32_t off_v = box * box_bytes + (uint32_t)(rb + lr_v) * 128;
+  uint32_t mphase = 0;  // parity of the next merge-barrier phase to wait for
+  bool merge_pending_read = false;
+
+  for (int it = 0;; ++it) {
+    const int slot = it % nst;
+    if (!warp_wait(s_full + 8 * slot, (uint32_t)(it / nst) & 1u, &s_abort)) {
+      if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+      return;
+    }
+    const int4 meta = g_meta[slot];
+    if (meta.x < 0) break;
+    const int ntok = meta.w & 0xffff;
+    const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+    if (first) {
+      const uint8_t* qs = g_q + (size_t)slot * qslot;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const int head = 8 * nt + g;
+        m_run[nt][0] = m_run[nt][1] = -INFINITY;
+        l_run[nt][0] = l_run[nt][1] = 0.f;
+#pragma unroll
+        for (int k = 0; k < KS; ++k) {
+          o_acc[nt][k][0] = o_acc[nt][k][1] = o_acc[nt][k][2] = o_acc[nt][k][3] = 0.f;
+          uint32_t v0 = 0u, v1 = 0u;
+          if (head < p.G) {
+            const uint8_t* src = qs + ((size_t)head * D + 16 * k + 2 * t) * 2;
+            v0 = *reinterpret_cast<const uint32_t*>(src);
+            v1 = *reinterpret_cast<const uint32_t*>(src + 16);
+          }
+          qf[nt][k][0] = v0;
+          qf[nt][k][1] = v1;
+        }
+      }
+    }
+    const int valid = min(16, ntok - r0);
+    if (valid > 0) {
+      const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;
+      const uint32_t vst = kst + L::kTileBytes;
+      // ---- scores: S = K_tile x Q^T
+      float sc[NT][2][4];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sc[nt][0][e] = sc[nt][1][e] = 0.f;
+#pragma unroll
+      for (int k = 0; k < KS; ++k) {
+        const int c = 2 * k + cs_k;
+        const uint32_t addr = kst + off_k + (uint32_t)(c >> 3) * half_bytes + (uint32_t)(((c & 7) ^ (lr_k & 7)) << 4);
+        uint32_t a0, a1, a2, a3;
+        ldmatrix_x4(addr, a0, a1, a2, a3);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(sc[nt][k & 1], a0, a1, a2, a3, qf[nt][k][0], qf[nt][k][1]);
+      }
+      uint32_t pb[NT][2];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        float s0 = (sc[nt][0][0] + sc[nt][1][0]) * p.scale_log2e;  // token g,   head 2t
+        float s1 = (sc[nt][0][1] + sc[nt][1][1]) * p.scale_log2e;  // token g,   head 2t+1
+        float s2 = (sc[nt][0][2] + sc[nt][1][2]) * p.scale_log2e;  // token g+8, head 2t
+        float s3 = (sc[nt][0][3] + sc[nt][1][3]) * p.scale_log2e;  // token g+8, head 2t+1
+        if (g >= valid) s0 = s1 = -INFINITY;
+        if (g + 8 >= valid) s2 = s3 = -INFINITY;
+        float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+        }
+        const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
+        const float al0 = ex2(m_run[nt][0] - mn0), al1 = ex2(m_run[nt][1] - mn1);
+        m_run[nt][0] = mn0;
+        m_run[nt][1] = mn1;
+        const uint32_t p01 = pack_bf16x2(ex2(s0 - mn0), ex2(s1 - mn1));  // token g
+        const uint32_t p23 = pack_bf16x2(ex2(s2 - mn0), ex2(s3 - mn1));  // token g+8
+        // sums use the rounded weights, so numerator and denominator agree exactly
+        l_run[nt][0] = l_run[nt][0] * al0 + __uint_as_float(p01 << 16) + __uint_as_float(p23 << 16);
+        l_run[nt][1] = l_run[nt][1] * al1 + __uint_as_float(p01 & 0xffff0000u) + __uint_as_float(p23 & 0xffff0000u);
+        if (__any_sync(0xffffffffu, (al0 != 1.f) | (al1 != 1.f))) {
+#pragma unroll
+          for (int k = 0; k < KS; ++k) {
+            o_acc[nt][k][0] *= al0;
+            o_acc[nt][k][1] *= al1;
+            o_acc[nt][k][2] *= al0;
+            o_acc[nt][k][3] *= al1;
+          }
+        }
+        pb[nt][0] = movmatrix_trans(p01);  // tokens 2t,2t+1   of head g
+        pb[nt][1] = movmatrix_trans(p23);  // tokens 2t+8,+9   of head g
+      }
+      // ---- values: O^T += V_tile^T x P ; rows past the context are cleared in registers
+      uint32_t mk01 = 0xffffffffu, mk23 = 0xffffffffu;
+      if (valid < 16) {
+        mk01 = (2 * t < valid ? 0x0000ffffu : 0u) | (2 * t + 1 < valid ? 0xffff0000u : 0u);
+        mk23 = (2 * t + 8 < valid ? 0x0000ffffu : 0u) | (2 * t + 9 < valid ? 0xffff0000u : 0u);
+      }
+#pragma unroll
+      for (int k = 0; k < KS; ++k) {
+        const int c = 2 * k + cs_v;
+        const uint32_t addr = vst + off_v + (uint32_t)(c >> 3) * half_bytes + (uint32_t)(((c & 7) ^ (lr_v & 7)) << 4);
+        uint32_t a0, a1, a2, a3;
+        ldmatrix_x4_trans(addr, a0, a1, a2, a3);
+        a0 &= mk01;
+        a1 &= mk01;
+        a2 &= mk23;
+        a3 &= mk23;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(o_acc[nt][k], a0, a1, a2, a3, pb[nt][0], pb[nt][1]);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(s_empty + 8 * slot);
+
+    if (last) {
+      // ---- combine the NCW warps' running states, then write the item's result
+      if (merge_pending_read) {  // previous item's readers must be done with the buffer
+        if (!warp_wait(s_mbar, mphase, &s_abort)) {
+          if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+          return;
+        }
+        mphase ^= 1u;
+      }
+      float* mo = g_merge + (size_t)warp * L::kHeads * L::kOStride;
+      float* mm = g_merge + (size_t)NCW * L::kHeads * L::kOStride + (size_t)warp * L::kHeads * 2;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        float l0 = l_run[nt][0], l1 = l_run[nt][1];
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          l0 += __shfl_xor_sync(0xffffffffu, l0, o);
+          l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+        }
+        const int h0 = 8 * nt + 2 * t;
+        if (g == 0) {
+          mm[2 * h0] = m_run[nt][0];
+          mm[2 * h0 + 1] = l0;
+          mm[2 * h0 + 2] = m_run[nt][1];
+          mm[2 * h0 + 3] = l1;
+        }
+#pragma unroll
+        for (int k = 0; k < KS; ++k) {
+          mo[(size_t)h0 * L::kOStride + 16 * k + g] = o_acc[nt][k][0];
+          mo[(size_t)(h0 + 1) * L::kOStride + 16 * k + g] = o_acc[nt][k][1];
+          mo[(size_t)h0 * L::kOStride + 16 * k + g + 8] = o_acc[nt][k][2];
+          mo[(size_t)(h0 + 1) * L::kOStride + 16 * k + g + 8] = o_acc[nt][k][3];
+        }
+      }
+      mbar_arrive(s_mbar);
+      if (!warp_wait(s_mbar, mphase, &s_abort)) {
+        if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+        return;
+      }
+      mphase ^= 1u;
+      const int item = meta.x, b = meta.y, h = meta.z;
+      const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
+      const float* all_m = g_merge + (size_t)NCW * L::kHeads * L::kOStride;
+      for (int idx = threadIdx.x; idx < p.G * D; idx += NCW * 32) {
+        const int head = idx / D, dim = idx % D;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NCW; ++w) M = fmaxf(M, all_m[(w * L::kHeads + head) * 2]);
+        float den = 0.f, num = 0.f;
+#pragma unroll
+        for (int w = 0; w < NCW; ++w) {
+          const float sw = ex2(all_m[(w * L::kHeads + head) * 2] - M);
+          den += sw * all_m[(w * L::kHeads + head) * 2 + 1];
+          num += sw * g_merge[((size_t)w * L::kHeads + head) * L::kOStride + dim];
+        }
+        const float o = num / den;
+        if (n_chunks == 1) {
+          p.out[((size_t)b * p.Hq + (size_t)h * p.G + head) * D + dim] = __float2bfloat16_rn(o);
+        } else {
+          p.part_o[((size_t)item * p.G + head) * D + dim] = o;
+          if (dim == 0) p.part_lse[(size_t)item * p.G + head] = M + lg2(den);
+        }
+      }
+      mbar_arrive(s_mbar);
+      merge_pending_read = true;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ merge
+// One CTA per (sequence, kv head); sequences that were not split are skipped.
+//   out = sum_c 2^(lse_c - M) o_c / sum_c 2^(lse_c - M),  M = max_c lse_c
+__global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
+  const int b = blockIdx.x / p.Hkv, h = blockIdx.x % p.Hkv;
+  const int first = p.seq_first[b];
+  const int n = p.seq_first[b + 1] - first;
+  if (n <= 1 || p.hdr->n_items == 0) return;
+  for (int idx = threadIdx.x; idx < p.G * p.D; idx += blockDim.x) {
+    const int head = idx / p.D, dim = idx % p.D;
+    float M = -INFINITY;
+    for (int c = 0; c < n; ++c) {
+      const size_t item = (size_t)(first + c) * p.Hkv + h;
+      M = fmaxf(M, p.part_lse[item * p.G + head]);
+    }
+    float den = 0.f, num = 0.f;
+    for (int c = 0; c < n; ++c) {
+      const size_t item = (size_t)(first + c) * p.Hkv + h;
+      const float w = exp2f(p.part_lse[item * p.G + head] - M);
+      den += w;
+      num += w * p.part_o[(item * p.G + head) * p.D + dim];
+    }
+    p.out[((size_t)b * p.Hq + (size_t)h * p.G + head) * p.D + dim] = __float2bfloat16_rn(num / den);
+  }
+}
+
+}  // namespace ooco

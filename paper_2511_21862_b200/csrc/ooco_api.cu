@@ -1,0 +1,411 @@
+// Host side of the ooco_* C ABI: argument validation, tensor-map encoding, launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstring>
+
+#include "../../include/ooco.h"
+#include "decode_kernels.cuh"
+
+namespace ooco {
+
+// ------------------------------------------------------------------------------------ tuning
+// Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
+enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
+            kKnobSplitHalves, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {1}, {256}, {8192}, {6}, {0}};
+constexpr int kGridCap = 1024;  // upper bound on CTAs assumed by the host-only workspace bound
+
+static thread_local int tl_last_launches = 0;
+
+struct DeviceInfo {
+  int sm_count = 0;
+  int smem_optin = 0;
+};
+static DeviceInfo device_info(int dev) {
+  static DeviceInfo cache[64];
+  static std::atomic<int> ready[64];
+  if (dev >= 0 && dev < 64 && ready[dev].load(std::memory_order_acquire)) return cache[dev];
+  DeviceInfo d;
+  cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev);
+  cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (dev >= 0 && dev < 64) {
+    cache[dev] = d;
+    ready[dev].store(1, std::memory_order_release);
+  }
+  return d;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_fn() {
+  static std::atomic<EncodeTiledFn> fn{nullptr};
+  EncodeTiledFn f = fn.load(std::memory_order_acquire);
+  if (f) return f;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !ptr)
+    return nullptr;
+  f = reinterpret_cast<EncodeTiledFn>(ptr);
+  fn.store(f, std::memory_order_release);
+  return f;
+}
+
+static bool supported_block(int bs) { return bs == 16 || bs == 32 || bs == 64 || bs == 128 || bs == 256; }
+
+static int validate_shape(const ooco_shape_t* s) {
+  if (!s) return OOCO_E_NULLPTR;
+  if (s->batch <= 0 || s->num_q_heads <= 0 || s->num_kv_heads <= 0 || s->head_dim <= 0 ||
+      s->block_size <= 0 || s->num_blocks <= 0 || s->max_blocks_per_seq <= 0 || s->reserved != 0)
+    return OOCO_E_SHAPE;
+  if (s->num_q_heads % s->num_kv_heads) return OOCO_E_SHAPE;
+  if (s->kv_block_stride <= 0 || s->kv_head_stride <= 0 || s->kv_token_stride < s->head_dim)
+    return OOCO_E_SHAPE;
+  if (s->head_dim != 64 && s->head_dim != 128) return OOCO_E_UNSUPPORTED;
+  if (!supported_block(s->block_size)) return OOCO_E_UNSUPPORTED;
+  if (s->num_q_heads / s->num_kv_heads > 16) return OOCO_E_UNSUPPORTED;
+  if ((s->kv_block_stride | s->kv_head_stride | s->kv_token_stride) & 7) return OOCO_E_UNSUPPORTED;
+  if ((int64_t)s->max_blocks_per_seq * s->block_size > (int64_t)1 << 30) return OOCO_E_UNSUPPORTED;
+  return OOCO_OK;
+}
+
+// Workspace carve-up (all offsets multiples of 256 bytes).
+struct WsLayout {
+  size_t off_first, off_items, off_lse, off_o, total;
+  int max_items;
+};
+static WsLayout ws_layout(const ooco_shape_t* s) {
+  const int G = s->num_q_heads / s->num_kv_heads;
+  const int64_t cmax = g_knobs[kKnobChunkMax].load();
+  const int64_t ipc = g_knobs[kKnobItemsPerCta].load();
+  const int64_t per_seq = ((int64_t)s->max_blocks_per_seq * s->block_size + cmax - 1) / cmax;
+  int64_t extra = (int64_t)s->num_kv_heads * s->batch * per_seq;
+  if (extra < kGridCap * ipc) extra = kGridCap * ipc;
+  const int64_t max_items = (int64_t)s->num_kv_heads * s->batch + extra + 64;
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  WsLayout w;
+  w.max_items = (int)(max_items > INT32_MAX ? INT32_MAX : max_items);
+  w.off_first = 256;
+  w.off_items = w.off_first + up(((size_t)s->batch + 1) * 4);
+  w.off_lse = w.off_items + up((size_t)w.max_items * 16);
+  w.off_o = w.off_lse + up((size_t)w.max_items * G * 4);
+  w.total = w.off_o + up((size_t)w.max_items * G * s->head_dim * 4);
+  return w;
+}
+
+static int encode_kv_map(CUtensorMap* tm, const ooco_shape_t* s, const void* base, int tile_rows,
+                         bool five_d) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return OOCO_E_CUDA;
+  const cuuint64_t es = 2;
+  CUresult r;
+  if (five_d) {  // (64 dims, token, half, head, block): one box = [2][tile_rows][64]
+    cuuint64_t dims[5] = {64, (cuuint64_t)s->block_size, (cuuint64_t)s->head_dim / 64,
+                          (cuuint64_t)s->num_kv_heads, (cuuint64_t)s->num_blocks};
+    cuuint64_t strides[4] = {(cuuint64_t)s->kv_token_stride * es, 64 * es, (cuuint64_t)s->kv_head_stride * es,
+                             (cuuint64_t)s->kv_block_stride * es};
+    cuuint32_t box[5] = {64, (cuuint32_t)tile_rows, (cuuint32_t)s->head_dim / 64, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {  // (dims, token, head, block): one box = [tile_rows][64]
+    cuuint64_t dims[4] = {(cuuint64_t)s->head_dim, (cuuint64_t)s->block_size, (cuuint64_t)s->num_kv_heads,
+                          (cuuint64_t)s->num_blocks};
+    cuuint64_t strides[3] = {(cuuint64_t)s->kv_token_stride * es, (cuuint64_t)s->kv_head_stride * es,
+                             (cuuint64_t)s->kv_block_stride * es};
+    cuuint32_t box[4] = {64, (cuuint32_t)tile_rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
+  return r == CUDA_SUCCESS ? OOCO_OK : OOCO_E_CUDA;
+}
+
+template <int D, int NCW, int NT>
+static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
+                       int ctas_per_sm, int want_stages, cudaStream_t st, int dev) {
+  using L = SmemLayout<D, NCW, NT>;
+  const size_t budget = (size_t)di.smem_optin / ctas_per_sm - (ctas_per_sm > 1 ? 1024 : 0);
+  int nst = want_stages > 0 ? want_stages : 32;
+  while (nst > 2 && L::total(nst, p.G) > budget) --nst;
+  if (L::total(nst, p.G) > (size_t)di.smem_optin) return OOCO_E_UNSUPPORTED;
+  p.nstages = nst;
+  const size_t smem = L::total(nst, p.G);
+  auto kern = decode_main_kernel<D, NCW, NT>;
+  static std::atomic<size_t> configured[64];
+  if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
+      return OOCO_E_CUDA;
+    if (dev >= 0 && dev < 64) configured[dev].store((size_t)di.smem_optin);
+  }
+  kern<<<p.grid_main, (NCW + 1) * 32, smem, st>>>(tk, tv, p);
+  return cudaGetLastError() == cudaSuccess ? OOCO_OK : OOCO_E_CUDA;
+}
+
+template <int D, int NCW>
+static int launch_main_nt(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
+                          int cps, int stages, cudaStream_t st, int dev) {
+  if (p.G <= 8) return launch_main<D, NCW, 1>(tk, tv, p, di, cps, stages, st, dev);
+  return launch_main<D, NCW, 2>(tk, tv, p, di, cps, stages, st, dev);
+}
+
+template <int D>
+static int launch_main_ncw(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
+                           const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev) {
+  switch (ncw) {
+    case 2: return launch_main_nt<D, 2>(tk, tv, p, di, cps, stages, st, dev);
+    case 8: return launch_main_nt<D, 8>(tk, tv, p, di, cps, stages, st, dev);
+    default: return launch_main_nt<D, 4>(tk, tv, p, di, cps, stages, st, dev);
+  }
+}
+
+// ------------------------------------------------------------------------------------ append
+// One thread per 16-byte vector of the new K and of the new V rows.
+__global__ void __launch_bounds__(256)
+kv_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint16_t* k_cache,
+                 uint16_t* v_cache, const int32_t* __restrict__ block_table,
+                 const int32_t* __restrict__ positions, int B, int Hkv, int D, int bs, int NB, int MB,
+                 int64_t bstr, int64_t hstr, int64_t tstr) {
+  const int vec_per_row = D / 8;
+  const long long n = (long long)B * Hkv * vec_per_row;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int v = (int)(i % vec_per_row);
+    const int h = (int)((i / vec_per_row) % Hkv);
+    const int b = (int)(i / ((long long)vec_per_row * Hkv));
+    const int pos = positions[b];
+    if (pos < 0 || (long long)pos >= (long long)MB * bs) continue;
+    const int blk = block_table[(size_t)b * MB + pos / bs];
+    if (blk < 0 || blk >= NB) continue;
+    const int64_t dst = (int64_t)blk * bstr + (int64_t)h * hstr + (int64_t)(pos % bs) * tstr + 8 * v;
+    *reinterpret_cast<uint4*>(k_cache + dst) = k_new[i];
+    *reinterpret_cast<uint4*>(v_cache + dst) = v_new[i];
+  }
+}
+
+static int current_device(int* dev) { return cudaGetDevice(dev) == cudaSuccess ? OOCO_OK : OOCO_E_CUDA; }
+
+}  // namespace ooco
+
+using namespace ooco;
+
+extern "C" {
+
+int ooco_version(void) { return OOCO_VERSION; }
+
+const char* ooco_status_string(int status) {
+  switch (status) {
+    case OOCO_OK: return "ok";
+    case OOCO_E_NULLPTR: return "null pointer argument";
+    case OOCO_E_SHAPE: return "invalid shape";
+    case OOCO_E_UNSUPPORTED: return "shape not supported by the kernels";
+    case OOCO_E_WORKSPACE: return "workspace or staging buffer too small or misaligned";
+    case OOCO_E_CUDA: return "CUDA call or launch failed";
+    case OOCO_E_DEVICE: return "device-side status word reports a problem";
+    default: return "unknown status";
+  }
+}
+
+int ooco_last_launch_count(void) { return tl_last_launches; }
+
+int ooco_set_tuning(int knob, int value) {
+  if (knob < 0 || knob >= kKnobCount) return OOCO_E_SHAPE;
+  if (knob == kKnobWarps && value != 2 && value != 4 && value != 8) return OOCO_E_SHAPE;
+  if (knob == kKnobStages && (value < 0 || value > 64)) return OOCO_E_SHAPE;
+  if (knob == kKnobCtasPerSm && (value < 1 || value > 4)) return OOCO_E_SHAPE;
+  if ((knob == kKnobChunkMin || knob == kKnobChunkMax) && (value < 128 || value > (1 << 20) || value % 128))
+    return OOCO_E_SHAPE;
+  if (knob == kKnobItemsPerCta && (value < 1 || value > 64)) return OOCO_E_SHAPE;
+  g_knobs[knob].store(value);
+  return OOCO_OK;
+}
+
+int ooco_kv_append(const ooco_shape_t* s, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                   const int32_t* block_table, const int32_t* positions, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
+    return OOCO_E_UNSUPPORTED;
+  const long long n = (long long)s->batch * s->num_kv_heads * (s->head_dim / 8);
+  long long blocks = (n + 255) / 256;
+  if (blocks > 4096) blocks = 4096;
+  kv_append_kernel<<<(int)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(
+      (const uint4*)k_new, (const uint4*)v_new, (uint16_t*)k_cache, (uint16_t*)v_cache, block_table, positions,
+      s->batch, s->num_kv_heads, s->head_dim, s->block_size, s->num_blocks, s->max_blocks_per_seq,
+      s->kv_block_stride, s->kv_head_stride, s->kv_token_stride);
+  return cudaGetLastError() == cudaSuccess ? OOCO_OK : OOCO_E_CUDA;
+}
+
+size_t ooco_decode_workspace_bytes(const ooco_shape_t* s) {
+  if (validate_shape(s)) return 0;
+  return ws_layout(s).total;
+}
+
+int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
+                          const int32_t* block_table, const int32_t* context_lens, float scale, void* out,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q) & 15) return OOCO_E_UNSUPPORTED;
+  const WsLayout w = ws_layout(s);
+  if (workspace_bytes < w.total || ((uintptr_t)workspace & 255)) return OOCO_E_WORKSPACE;
+  int dev = 0;
+  if ((rc = current_device(&dev))) return rc;
+  const DeviceInfo di = device_info(dev);
+  if (di.sm_count <= 0) return OOCO_E_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+
+  const int ncw = g_knobs[kKnobWarps].load();
+  const int cps = g_knobs[kKnobCtasPerSm].load();
+  const int stage_tok = 16 * ncw;
+  DecodeParams p;
+  memset(&p, 0, sizeof p);
+  uint8_t* ws = (uint8_t*)workspace;
+  p.q = (const __nv_bfloat16*)q;
+  p.out = (__nv_bfloat16*)out;
+  p.block_table = block_table;
+  p.context_lens = context_lens;
+  p.hdr = (WsHeader*)ws;
+  p.seq_first = (int32_t*)(ws + w.off_first);
+  p.items = (int4*)(ws + w.off_items);
+  p.part_lse = (float*)(ws + w.off_lse);
+  p.part_o = (float*)(ws + w.off_o);
+  p.B = s->batch;
+  p.Hq = s->num_q_heads;
+  p.Hkv = s->num_kv_heads;
+  p.G = p.Hq / p.Hkv;
+  p.D = s->head_dim;
+  p.bs = s->block_size;
+  p.MB = s->max_blocks_per_seq;
+  p.max_items = w.max_items;
+  p.tile_rows = s->block_size < stage_tok ? s->block_size : stage_tok;
+  p.grid_main = di.sm_count * cps;
+  if (p.grid_main > kGridCap) p.grid_main = kGridCap;
+  p.chunk_min = g_knobs[kKnobChunkMin].load();
+  p.chunk_max = g_knobs[kKnobChunkMax].load();
+  if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
+  p.items_per_cta = g_knobs[kKnobItemsPerCta].load();
+  p.scale_log2e = scale * 1.4426950408889634f;
+
+  CUtensorMap tk, tv;
+  bool five_d = s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
+  if (five_d && encode_kv_map(&tk, s, k_cache, p.tile_rows, true) != OOCO_OK) five_d = false;
+  if (five_d) {
+    if ((rc = encode_kv_map(&tv, s, v_cache, p.tile_rows, true))) return rc;
+  } else {
+    if ((rc = encode_kv_map(&tk, s, k_cache, p.tile_rows, false))) return rc;
+    if ((rc = encode_kv_map(&tv, s, v_cache, p.tile_rows, false))) return rc;
+  }
+  p.split_halves = five_d ? 0 : 1;
+
+  plan_kernel<1024><<<1, 1024, 0, st>>>(p, stage_tok);
+  if (cudaGetLastError() != cudaSuccess) return OOCO_E_CUDA;
+  const int stages = g_knobs[kKnobStages].load();
+  if (s->head_dim == 128)
+    rc = launch_main_ncw<128>(ncw, tk, tv, p, di, cps, stages, st, dev);
+  else
+    rc = launch_main_ncw<64>(ncw, tk, tv, p, di, cps, stages, st, dev);
+  if (rc) return rc;
+  lse_merge_kernel<<<p.B * p.Hkv, 256, 0, st>>>(p);
+  if (cudaGetLastError() != cudaSuccess) return OOCO_E_CUDA;
+  tl_last_launches = 3;
+  return OOCO_OK;
+}
+
+int ooco_workspace_status(const void* workspace, void* cuda_stream, int32_t* status_host) {
+  if (!workspace || !status_host) return OOCO_E_NULLPTR;
+  int32_t v = 0;
+  if (cudaMemcpyAsync(&v, workspace, sizeof v, cudaMemcpyDeviceToHost, (cudaStream_t)cuda_stream) != cudaSuccess)
+    return OOCO_E_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return OOCO_E_CUDA;
+  *status_host = v;
+  return v == 0 ? OOCO_OK : OOCO_E_DEVICE;
+}
+
+int ooco_decode_bytes_model(const ooco_shape_t* s, const int32_t* context_lens_host, int32_t bytes_per_value,
+                            ooco_cost_t* c) {
+  if (!s || !context_lens_host || !c) return OOCO_E_NULLPTR;
+  if (s->batch <= 0 || s->num_q_heads <= 0 || s->num_kv_heads <= 0 || s->head_dim <= 0 || s->block_size <= 0 ||
+      bytes_per_value <= 0 || s->num_q_heads % s->num_kv_heads)
+    return OOCO_E_SHAPE;
+  const int64_t d = bytes_per_value;
+  const int64_t q_row = (int64_t)s->num_q_heads * s->head_dim;     // D_h of the operator table
+  const int64_t kv_row = (int64_t)s->num_kv_heads * s->head_dim;   // D_h * Hkv / Hq
+  int64_t tokens = 0, blocks = 0;
+  for (int32_t b = 0; b < s->batch; ++b) {
+    const int64_t t = context_lens_host[b] > 0 ? context_lens_host[b] : 0;
+    tokens += t;
+    blocks += (t + s->block_size - 1) / s->block_size;
+  }
+  c->total_tokens = tokens;
+  c->flops = 4 * q_row * tokens;
+  c->bytes_q = d * s->batch * q_row;
+  c->bytes_out = c->bytes_q;
+  c->bytes_kv = 2 * d * kv_row * tokens;
+  c->bytes_index = 4 * ((int64_t)s->batch + blocks);
+  c->bytes_paper = c->bytes_q + c->bytes_out + c->bytes_kv;
+  return OOCO_OK;
+}
+
+size_t ooco_step_staging_bytes(const ooco_shape_t* s) {
+  if (validate_shape(s)) return 0;
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  const size_t qb = (size_t)s->batch * s->num_q_heads * s->head_dim * 2;
+  const size_t kb = (size_t)s->batch * s->num_kv_heads * s->head_dim * 2;
+  return up(qb) * 2 + up(kb) * 2 + up((size_t)s->batch * s->max_blocks_per_seq * 4) + 2 * up((size_t)s->batch * 4);
+}
+
+int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void* k_new_host,
+                          const void* v_new_host, const int32_t* block_table_host,
+                          const int32_t* positions_host, const int32_t* context_lens_host, void* k_cache,
+                          void* v_cache, float scale, void* out_host, void* staging, size_t staging_bytes,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  if (!q_host || !k_new_host || !v_new_host || !block_table_host || !positions_host || !context_lens_host ||
+      !k_cache || !v_cache || !out_host || !staging || !workspace)
+    return OOCO_E_NULLPTR;
+  if (staging_bytes < ooco_step_staging_bytes(s) || ((uintptr_t)staging & 255)) return OOCO_E_WORKSPACE;
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t qb = (size_t)s->batch * s->num_q_heads * s->head_dim * 2;
+  const size_t kb = (size_t)s->batch * s->num_kv_heads * s->head_dim * 2;
+  const size_t tb = (size_t)s->batch * s->max_blocks_per_seq * 4;
+  const size_t lb = (size_t)s->batch * 4;
+  uint8_t* base = (uint8_t*)staging;
+  uint8_t* d_q = base;
+  uint8_t* d_out = d_q + up(qb);
+  uint8_t* d_kn = d_out + up(qb);
+  uint8_t* d_vn = d_kn + up(kb);
+  uint8_t* d_tab = d_vn + up(kb);
+  uint8_t* d_pos = d_tab + up(tb);
+  uint8_t* d_len = d_pos + up(lb);
+  bool ok = true;
+  ok &= cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_kn, k_new_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_vn, v_new_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_tab, block_table_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_pos, positions_host, lb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_len, context_lens_host, lb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) return OOCO_E_CUDA;
+  if ((rc = ooco_kv_append(s, d_kn, d_vn, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_pos, st)))
+    return rc;
+  if ((rc = ooco_decode_attention(s, d_q, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_len, scale,
+                                  d_out, workspace, workspace_bytes, st)))
+    return rc;
+  if (cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return OOCO_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return OOCO_E_CUDA;
+  tl_last_launches = 4;
+  return OOCO_OK;
+}
+
+}  // extern "C"

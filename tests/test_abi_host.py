@@ -1,0 +1,122 @@
+"""Host-only checks of the C ABI: exported symbols, the byte/FLOP model, argument validation."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_21862_b200 import binding, build, inputs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "ooco.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ooco_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = declared_functions()
+    assert len(names) >= 10
+    L = binding.lib()
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(names) == set(binding.EXPORTS)
+    assert L.ooco_version() == 1
+    assert binding.status_string(0) == "ok" and "unknown" in binding.status_string(-99)
+
+
+def read_golden():
+    rows = []
+    for line in open(os.path.join(ROOT, "tests", "golden", "bytes_model.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        a, b, c = (p.split() for p in line.split("|"))
+        rows.append(([int(x) for x in a], [int(x) for x in b], [int(x) for x in c]))
+    return rows
+
+
+@pytest.mark.parametrize("row", read_golden(), ids=lambda r: "-".join(map(str, r[0])))
+def test_bytes_model_golden(row):
+    (Hq, Hkv, D, bs, d), lens, want = row
+    keys = oracle.COST_FIELDS
+    got_o = oracle.bytes_model(lens, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, block_size=bs, bytes_per_value=d)
+    assert [got_o[k] for k in keys] == want
+    sh = binding.Shape(len(lens), Hq, Hkv, D, bs, 1, 1, Hkv * bs * D, bs * D, D)
+    got_l = binding.decode_bytes_model(sh, torch.tensor(lens, dtype=torch.int32), d)
+    assert [got_l[k] for k in keys] == want
+
+
+def test_bytes_model_equals_enumeration_of_addressed_slots():
+    """bytes_kv = bytes of the distinct cache words a batch addresses; index = table + length words."""
+    cfg = inputs.DecodeConfig("enum", 12, 3, 64, 16, (inputs.LengthGroup(5, 1, 90),), seed=21, pool_fill=0.6)
+    batch = inputs.make_batch(cfg)
+    lens = batch.context_lens
+    touched = set()
+    table_words = 0
+    for b in range(5):
+        T = int(lens[b])
+        table_words += -(-T // 16)
+        for t in range(T):
+            blk = int(batch.block_table[b, t // 16])
+            for h in range(3):
+                touched.add((blk, h, t % 16))
+    kv_bytes = 2 * len(touched) * 64 * 2                      # K and V, D elements of 2 bytes
+    o = oracle.bytes_model(lens.numpy(), num_q_heads=12, num_kv_heads=3, head_dim=64, block_size=16)
+    l = binding.decode_bytes_model(binding.shape_of(batch), lens.contiguous())
+    for got in (o, l):
+        assert got["bytes_kv"] == kv_bytes
+        assert got["bytes_index"] == 4 * (5 + table_words)
+        assert got["bytes_q"] == got["bytes_out"] == batch.q.numel() * 2
+        assert got["flops"] == 2 * 2 * 12 * 64 * int(lens.sum())   # QK^T and PV, 2 flops per MAC
+        assert got["bytes_paper"] == got["bytes_q"] + got["bytes_out"] + got["bytes_kv"]
+
+
+def test_bytes_model_mha_matches_printed_table_entry():
+    """With Hq == Hkv the table's printed ratio is 1: memory = 2d(Sq*Dh + Skv*Dh)."""
+    lens = torch.tensor([7, 300, 4096], dtype=torch.int32)
+    Hq, D, d = 16, 128, 2
+    sh = binding.Shape(3, Hq, Hq, D, 16, 1, 1, Hq * 16 * D, 16 * D, D)
+    got = binding.decode_bytes_model(sh, lens, d)
+    Dh = Hq * D
+    assert got["bytes_paper"] == sum(2 * d * (1 * Dh + int(t) * Dh) for t in lens)
+    assert got["flops"] == sum(4 * Dh * 1 * int(t) for t in lens)
+
+
+def test_argument_validation_without_a_device():
+    L = binding.lib()
+    good = binding.Shape(2, 8, 2, 64, 16, 8, 4, 2 * 16 * 64, 16 * 64, 64)
+    assert binding.workspace_bytes(good) > 256 and binding.step_staging_bytes(good) > 0
+    one = ctypes.c_void_p(256)
+    def attn(shape, ptr=one, ws_bytes=1 << 40):
+        return L.ooco_decode_attention(ctypes.byref(shape.c()), ptr, ptr, ptr, ptr, ptr, 1.0, ptr, ptr, ws_bytes, None)
+    import dataclasses
+    assert attn(good, ptr=None) == -1                                                   # NULLPTR
+    assert attn(dataclasses.replace(good, num_q_heads=7)) == -2                         # Hq % Hkv
+    assert attn(dataclasses.replace(good, batch=0)) == -2
+    assert attn(dataclasses.replace(good, head_dim=96, kv_token_stride=96)) == -3       # UNSUPPORTED
+    assert attn(dataclasses.replace(good, block_size=8)) == -3
+    assert attn(dataclasses.replace(good, num_q_heads=64, num_kv_heads=2)) == -3        # group of 32
+    assert attn(dataclasses.replace(good, kv_token_stride=68)) == -3                    # not 16-byte multiple
+    assert attn(good, ws_bytes=1024) == -4                                              # WORKSPACE
+    assert L.ooco_kv_append(ctypes.byref(good.c()), None, one, one, one, one, one, None) == -1
+    assert L.ooco_decode_bytes_model(ctypes.byref(good.c()), None, 2, None) == -1
+    assert L.ooco_set_tuning(99, 1) == -2 and L.ooco_set_tuning(0, 3) == -2
+    bad = dataclasses.replace(good, head_dim=96, kv_token_stride=96)
+    assert L.ooco_decode_workspace_bytes(ctypes.byref(bad.c())) == 0
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libooco.so")
+    with pytest.raises(ImportError):
+        binding.lib()

@@ -1,0 +1,65 @@
+"""Helpers shared by the parity tests: run the CUDA path, run the oracle, compare."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2511_21862_b200 import binding, inputs
+
+MAX_ABS_TOL = 1e-2    # bf16 in / fp32 accumulate / bf16 out vs the fp64 oracle: max |err|
+MEAN_ABS_TOL = 1e-3   # and mean |err|, over all B * Hq * D outputs
+
+
+def bf16_to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+def gpu_attention(batch, context_lens=None, scale=None, check_status=True):
+    """out (bf16, device) of ooco_decode_attention on a device-resident batch."""
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device=batch.q.device)
+    out = torch.full_like(batch.q, float("nan"))
+    lens = batch.context_lens if context_lens is None else context_lens
+    binding.decode_attention(sh, batch.q, batch.k_cache, batch.v_cache, batch.block_table, lens,
+                             batch.cfg.scale if scale is None else scale, out, ws)
+    if check_status:
+        assert binding.workspace_status(ws) == 0
+    torch.cuda.synchronize()
+    return out
+
+
+def oracle_attention(batch, context_lens=None, scale=None, seqs=None):
+    """fp64 oracle on a host copy; with `seqs`, only those sequences (other rows NaN), using a
+    compacted copy of just their blocks (plain torch indexing) so huge pools need not be copied."""
+    cfg = batch.cfg
+    lens = (batch.context_lens if context_lens is None else context_lens).cpu()
+    table = batch.block_table.cpu()
+    k, v = batch.k_cache, batch.v_cache
+    pairs = None
+    if seqs is not None:
+        seqs = [int(s) for s in seqs]
+        bs = cfg.block_size
+        new_table = table.clone()
+        ids = []
+        for b in seqs:
+            n = (int(lens[b]) + bs - 1) // bs
+            new_table[b, :n] = torch.arange(len(ids), len(ids) + n, dtype=torch.int32)
+            ids.extend(table[b, :n].tolist())
+        idx = torch.tensor(ids if ids else [0], dtype=torch.long, device=k.device)
+        k, v, table = k.index_select(0, idx), v.index_select(0, idx), new_table
+        pairs = np.array([(b, h) for b in seqs for h in range(cfg.num_q_heads)], dtype=np.int32)
+    return oracle.decode_attention(
+        inputs.as_u16(batch.q), inputs.as_u16(k), inputs.as_u16(v), table.numpy(), lens.numpy(),
+        cfg.scale if scale is None else scale, num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size,
+        strides=batch.strides, pairs=pairs)
+
+
+def assert_parity(out_gpu: torch.Tensor, ref: np.ndarray, rows=None, what=""):
+    got = bf16_to_f64(out_gpu)
+    if rows is not None:
+        got, ref = got[rows], ref[rows]
+    assert not np.isnan(ref).any(), "oracle rows missing"
+    assert not np.isnan(got).any(), f"{what}: NaN in the CUDA output"
+    err = np.abs(got - ref)
+    assert err.max() <= MAX_ABS_TOL, f"{what}: max abs err {err.max():.3e}"
+    assert err.mean() <= MEAN_ABS_TOL, f"{what}: mean abs err {err.mean():.3e}"
+    return float(err.max()), float(err.mean())
