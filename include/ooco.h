@@ -229,6 +229,12 @@ int ooco_last_launch_count(void);
  */
 int ooco_set_tuning(int knob, int value);
 
+/*
+ * Text naming the CUDA call that made the last OOCO_E_CUDA on this thread fail, with its
+ * error code ("" if none yet).  The pointer stays valid for the thread's lifetime.
+ */
+const char* ooco_last_error_detail(void);
+
 /* Static, human-readable name of a status code.  Never NULL. */
 const char* ooco_status_string(int status);
 

@@ -18,14 +18,15 @@ LIB_PATH = os.path.join(_HERE, "libooco.so")
 EXPORTS = (
     "ooco_kv_append", "ooco_decode_workspace_bytes", "ooco_decode_attention", "ooco_workspace_status",
     "ooco_decode_bytes_model", "ooco_step_staging_bytes", "ooco_decode_step_host",
-    "ooco_last_launch_count", "ooco_set_tuning", "ooco_status_string", "ooco_version",
+    "ooco_last_launch_count", "ooco_last_error_detail", "ooco_set_tuning", "ooco_status_string", "ooco_version",
 )
 
 
 class OocoError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {status_string(status)} ({status})")
+        detail = lib().ooco_last_error_detail().decode() if status == -5 else ""
+        super().__init__(f"{where}: {status_string(status)} ({status}) {detail}".rstrip())
 
 
 class ooco_shape_t(ctypes.Structure):
@@ -70,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.ooco_decode_step_host.argtypes = [sp, vp, vp, vp, i32p, i32p, i32p, vp, vp, ctypes.c_float, vp,
                                             vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
         L.ooco_last_launch_count.restype = ctypes.c_int
+        L.ooco_last_error_detail.restype = ctypes.c_char_p
         L.ooco_set_tuning.restype = ctypes.c_int
         L.ooco_set_tuning.argtypes = [ctypes.c_int, ctypes.c_int]
         L.ooco_status_string.restype = ctypes.c_char_p

@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <cstdint>
+#include <cstdio>
 #include <cstring>
 
 #include "../../include/ooco.h"
@@ -19,6 +20,13 @@ static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {1}, {256}, {8192}, {6}
 constexpr int kGridCap = 1024;  // upper bound on CTAs assumed by the host-only workspace bound
 
 static thread_local int tl_last_launches = 0;
+static thread_local char tl_detail[160] = "";
+
+// Remembers where a CUDA-side failure happened (read back through ooco_last_error_detail).
+static int fail_cuda(const char* where, long code) {
+  snprintf(tl_detail, sizeof tl_detail, "%s failed with code %ld", where, code);
+  return OOCO_E_CUDA;
+}
 
 struct DeviceInfo {
   int sm_count = 0;
@@ -101,7 +109,7 @@ static WsLayout ws_layout(const ooco_shape_t* s) {
 static int encode_kv_map(CUtensorMap* tm, const ooco_shape_t* s, const void* base, int tile_rows,
                          bool five_d) {
   EncodeTiledFn enc = encode_fn();
-  if (!enc) return OOCO_E_CUDA;
+  if (!enc) return fail_cuda("cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)", -1);
   const cuuint64_t es = 2;
   CUresult r;
   if (five_d) {  // (64 dims, token, half, head, block): one box = [2][tile_rows][64]
@@ -125,28 +133,40 @@ static int encode_kv_map(CUtensorMap* tm, const ooco_shape_t* s, const void* bas
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   }
-  return r == CUDA_SUCCESS ? OOCO_OK : OOCO_E_CUDA;
+  return r == CUDA_SUCCESS ? OOCO_OK : fail_cuda(five_d ? "cuTensorMapEncodeTiled(5d)" : "cuTensorMapEncodeTiled(4d)", (long)r);
 }
 
 template <int D, int NCW, int NT>
 static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                        int ctas_per_sm, int want_stages, cudaStream_t st, int dev) {
   using L = SmemLayout<D, NCW, NT>;
-  const size_t budget = (size_t)di.smem_optin / ctas_per_sm - (ctas_per_sm > 1 ? 1024 : 0);
+  auto kern = decode_main_kernel<D, NCW, NT>;
+  // the opt-in limit covers static + dynamic shared memory of the kernel
+  static std::atomic<int> static_smem{-1};
+  if (static_smem.load() < 0) {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncGetAttributes", (long)e);
+    static_smem.store((int)fa.sharedSizeBytes);
+  }
+  const size_t dyn_max = (size_t)di.smem_optin - (size_t)static_smem.load();
+  // per-CTA share of the SM's shared memory (1 KiB per CTA is reserved by the system)
+  const size_t budget = ctas_per_sm > 1 ? ((size_t)di.smem_optin + 1024) / ctas_per_sm - 1024 - static_smem.load()
+                                        : dyn_max;
   int nst = want_stages > 0 ? want_stages : 32;
   while (nst > 2 && L::total(nst, p.G) > budget) --nst;
-  if (L::total(nst, p.G) > (size_t)di.smem_optin) return OOCO_E_UNSUPPORTED;
+  if (L::total(nst, p.G) > dyn_max) return OOCO_E_UNSUPPORTED;
   p.nstages = nst;
   const size_t smem = L::total(nst, p.G);
-  auto kern = decode_main_kernel<D, NCW, NT>;
   static std::atomic<size_t> configured[64];
   if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
-      return OOCO_E_CUDA;
-    if (dev >= 0 && dev < 64) configured[dev].store((size_t)di.smem_optin);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
+    if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
   kern<<<p.grid_main, (NCW + 1) * 32, smem, st>>>(tk, tv, p);
-  return cudaGetLastError() == cudaSuccess ? OOCO_OK : OOCO_E_CUDA;
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the attention kernel", (long)e);
 }
 
 template <int D, int NCW>
@@ -215,6 +235,8 @@ const char* ooco_status_string(int status) {
 
 int ooco_last_launch_count(void) { return tl_last_launches; }
 
+const char* ooco_last_error_detail(void) { return tl_detail; }
+
 int ooco_set_tuning(int knob, int value) {
   if (knob < 0 || knob >= kKnobCount) return OOCO_E_SHAPE;
   if (knob == kKnobWarps && value != 2 && value != 4 && value != 8) return OOCO_E_SHAPE;
@@ -241,7 +263,8 @@ int ooco_kv_append(const ooco_shape_t* s, const void* k_new, const void* v_new, 
       (const uint4*)k_new, (const uint4*)v_new, (uint16_t*)k_cache, (uint16_t*)v_cache, block_table, positions,
       s->batch, s->num_kv_heads, s->head_dim, s->block_size, s->num_blocks, s->max_blocks_per_seq,
       s->kv_block_stride, s->kv_head_stride, s->kv_token_stride);
-  return cudaGetLastError() == cudaSuccess ? OOCO_OK : OOCO_E_CUDA;
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the append kernel", (long)e);
 }
 
 size_t ooco_decode_workspace_bytes(const ooco_shape_t* s) {
@@ -308,7 +331,8 @@ int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_ca
   p.split_halves = five_d ? 0 : 1;
 
   plan_kernel<1024><<<1, 1024, 0, st>>>(p, stage_tok);
-  if (cudaGetLastError() != cudaSuccess) return OOCO_E_CUDA;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
   if (s->head_dim == 128)
     rc = launch_main_ncw<128>(ncw, tk, tv, p, di, cps, stages, st, dev);
@@ -316,7 +340,8 @@ int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_ca
     rc = launch_main_ncw<64>(ncw, tk, tv, p, di, cps, stages, st, dev);
   if (rc) return rc;
   lse_merge_kernel<<<p.B * p.Hkv, 256, 0, st>>>(p);
-  if (cudaGetLastError() != cudaSuccess) return OOCO_E_CUDA;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda("launch of the merge kernel", (long)e);
   tl_last_launches = 3;
   return OOCO_OK;
 }
