@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the paged decode path (KV append + paged GQA decode attention) on B200.
+
+A "step" is one pass of the whole hot path for one transformer layer over one synthetic decode
+batch: ooco_kv_append of the new token's K/V, then ooco_decode_attention (plan + split-KV
+attention + LSE merge).  Successive steps use different pool replicas (as successive layers of a
+model do), so the KV working set of the timed region is far larger than L2.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1] [--impl ours|reference]
+
+Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs an independent replica of the
+workload (its own seed); there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2511_21862_b200 import inputs
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+METRIC = "paged decode-attn achieved HBM TB/s"
+# DRAM bytes (read + write) of one attention-kernel launch on cfg1 from the ncu capture summarised
+# in profiles/; None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the benchmark runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        super().__init__(daemon=True)
+        self.period, self.index = period_s, index
+        self.samples = []          # (t, sm_mhz, reasons_bitmask, power_w)
+        self._stop_evt = threading.Event()
+        self.max_mhz = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._stop_evt.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    rs = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    rs = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                try:
+                    pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                except Exception:
+                    pw = None
+                self.samples.append((time.perf_counter(), mhz, rs, pw))
+            except Exception:
+                pass
+            self._stop_evt.wait(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+
+    def summary(self, t0, t1):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        win = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
+        mhz = sorted(s[1] for s in win)
+        bits = 0
+        for s in win:
+            bits |= s[2]
+        names = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+                 0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+                 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        reasons = [n for b, n in names.items() if bits & b]
+        pw = [s[3] for s in win if s[3] is not None]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(win), "power_w_max": max(pw) if pw else None}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate(world, step_ms_local, units_local):
+    """(max over ranks of the step time, sum over ranks of the units) -- gloo/nccl all-reduce."""
+    if world == 1:
+        return step_ms_local, units_local
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([step_ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def replica_count(pool_bytes: int, free_bytes: int) -> int:
+    """Pool replicas so that the rotating KV working set is >= 4 GiB (>> the 126 MB L2)."""
+    want = max(2, -(-(4 << 30) // max(1, pool_bytes)))
+    fit = max(1, int(free_bytes * 0.6) // max(1, pool_bytes))
+    return max(1, min(want, fit, 16))
+
+
+def run_reference(args, rank, world):
+    """The oracle as it stands, on the host cores, on a bounded sample of the workload per step."""
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    cfg = inputs.CONFIGS[args.workload]
+    batch = inputs.make_batch(cfg, "cpu", poison=False)
+    lens = batch.context_lens.numpy()
+    # sample: whole sequences, shortest first, up to ~budget tokens * heads per step
+    budget = args.ref_token_heads
+    order = np.argsort(lens, kind="stable")
+    chosen, acc = [], 0
+    for b in order:
+        cost = int(lens[b]) * cfg.num_q_heads
+        if chosen and acc + cost > budget:
+            break
+        chosen.append(int(b)); acc += cost
+    pairs = np.array([(b, h) for b in chosen for h in range(cfg.num_q_heads)], dtype=np.int32)
+    tok = int(sum(int(lens[b]) for b in chosen))
+    sample_bytes = tok * 2 * 2 * cfg.num_kv_heads * cfg.head_dim + 2 * 2 * len(chosen) * cfg.num_q_heads * cfg.head_dim
+    q, k, v = inputs.as_u16(batch.q), inputs.as_u16(batch.k_cache), inputs.as_u16(batch.v_cache)
+    table = batch.block_table.numpy()
+
+    def step():
+        oracle.decode_attention(q, k, v, table, lens, cfg.scale, num_kv_heads=cfg.num_kv_heads,
+                                block_size=cfg.block_size, strides=batch.strides, pairs=pairs)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    ms = dt / args.steps * 1e3
+    val = sample_bytes / (ms * 1e-3) / 1e12
+    sample = f"{len(chosen)} shortest sequences of {cfg.name} ({tok} tokens, all {cfg.num_q_heads} q heads) per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "description": cfg.description, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TB/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": "TB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+        "decode_tokens_per_s": len(chosen) / (ms * 1e-3),
+    }
+    print(json.dumps(line))
+
+
+def cpu_baseline(cfg, batch_host_fn, budget_s=15.0):
+    """Oracle timed on the host cores on a bounded sample of the same workload (rank 0, N = 1)."""
+    import numpy as np
+    import oracle
+    hb = batch_host_fn()
+    lens = hb["lens"]
+    order = np.argsort(lens, kind="stable")
+    per_unit = None
+    # calibrate on the shortest sequence, then take whole sequences up to ~budget_s of CPU work
+    def run(seqs):
+        pairs = np.array([(b, h) for b in seqs for h in range(cfg.num_q_heads)], dtype=np.int32)
+        t0 = time.perf_counter()
+        oracle.decode_attention(hb["q"], hb["k"], hb["v"], hb["table"], lens, cfg.scale,
+                                num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size,
+                                strides=hb["strides"], pairs=pairs)
+        return time.perf_counter() - t0
+    first = [int(order[len(order) // 2])]
+    t_cal = run(first)
+    per_unit = t_cal / max(1, int(lens[first[0]]))
+    chosen, acc = [], 0.0
+    for b in order[::-1]:                                   # longest first: fewest partial sequences
+        est = per_unit * int(lens[b])
+        if chosen and acc + est > budget_s:
+            continue
+        chosen.append(int(b)); acc += est
+        if acc > budget_s:
+            break
+    dt = run(chosen)
+    tok = int(sum(int(lens[b]) for b in chosen))
+    nbytes = tok * 2 * 2 * cfg.num_kv_heads * cfg.head_dim + 2 * 2 * len(chosen) * cfg.num_q_heads * cfg.head_dim
+    return {"value": nbytes / dt / 1e12, "unit": "TB/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{len(chosen)} of {len(lens)} sequences of {cfg.name} ({tok} of {int(lens.sum())} tokens, "
+                      f"all q heads), {dt:.1f} s",
+            "decode_tokens_per_s": len(chosen) / dt}
+
+
+def run_ours(args, rank, local_rank, world):
+    from paper_2511_21862_b200 import binding, build
+    build.build()
+    binding.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = inputs.replace(inputs.CONFIGS[args.workload], seed=inputs.CONFIGS[args.workload].seed + 100 * rank)
+    batch = inputs.make_batch(cfg, dev, poison=False)
+    sh = binding.shape_of(batch)
+    B = sh.batch
+    lens_host = batch.context_lens.cpu().contiguous()
+    cost = binding.decode_bytes_model(sh, lens_host)
+    append_bytes = 2 * 2 * B * cfg.num_kv_heads * cfg.head_dim * 2        # K and V rows, read + written
+    step_bytes = cost["bytes_paper"] + append_bytes
+
+    pool_bytes = 2 * batch.k_cache.numel() * 2
+    free, _ = torch.cuda.mem_get_info(dev)
+    R = replica_count(pool_bytes, free)
+    pools = [(batch.k_cache, batch.v_cache)] + [(batch.k_cache.clone(), batch.v_cache.clone()) for _ in range(R - 1)]
+    ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device=dev)
+    out = torch.empty_like(batch.q)
+    positions = batch.context_lens                                        # append at T_b ...
+    lens1 = (batch.context_lens + 1).contiguous()                         # ... then attend T_b + 1 tokens
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        k, v = pools[i % R]
+        binding.kv_append(sh, batch.k_new, batch.v_new, k, v, batch.block_table, positions, stream)
+        binding.decode_attention(sh, batch.q, k, v, batch.block_table, lens1, cfg.scale, out, ws, stream)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    binding.profile_enable(args.steps)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin = time.perf_counter()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t_end = time.perf_counter()
+    ms_local = e0.elapsed_time(e1) / args.steps
+    recs = binding.profile_read(args.steps)
+    binding.profile_enable(0)
+    assert binding.workspace_status(ws) == 0
+    clocks = sampler.summary(t_begin, t_end)
+
+    # ---- end to end through the host-buffer entry point (pinned inputs in, result out, every step)
+    pin = lambda t: t.cpu().contiguous().pin_memory()
+    hq, hk, hv, ht = pin(batch.q), pin(batch.k_new), pin(batch.v_new), pin(batch.block_table)
+    hp, hl = pin(positions), pin(lens1)
+    hout = torch.empty(batch.q.shape, dtype=torch.bfloat16).pin_memory()
+    stg = torch.empty(binding.step_staging_bytes(sh), dtype=torch.uint8, device=dev)
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, ht, hp, hl))
+    d2h = hout.numel() * hout.element_size()
+    e2e_steps = max(3, min(args.steps, 200))
+
+    def e2e_step(i):
+        k, v = pools[i % R]
+        binding.decode_step_host(sh, hq, hk, hv, ht, hp, hl, k, v, cfg.scale, hout, stg, ws, stream)
+    for i in range(3):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_ms_local = (time.perf_counter() - t0) / e2e_steps * 1e3
+    sampler.stop()
+
+    ms, total_bytes = aggregate(world, ms_local, float(step_bytes))
+    e2e_ms, _ = aggregate(world, e2e_ms_local, 0.0)
+    _, total_seqs = aggregate(world, 0.0, float(B))
+    if rank != 0:
+        return
+    value = total_bytes / (ms * 1e-3) / 1e12
+    peak, peak_kind = measured_peak()
+    attn_ms = sorted(r[1] for r in recs)
+    attn_avg = sum(attn_ms) / len(attn_ms)
+    kernel_bytes = cost["bytes_kv"] + cost["bytes_q"] + cost["bytes_out"]
+    achieved = kernel_bytes / (attn_avg * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "TB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "description": cfg.description, "batch": B,
+                   "total_tokens": cost["total_tokens"], "step": "kv_append + decode_attention, one layer",
+                   "l2": f"inputs larger than L2: steps rotate over {R} pool replicas ({R * pool_bytes / 2**30:.2f} GiB)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "pct_of_nominal_8tbps": 100.0 * value * 1e3 / (NOMINAL_HBM_GBS * world),
+        "pct_of_measured_copy": 100.0 * value * 1e3 / (peak * world),
+        "decode_tokens_per_s": total_seqs / (ms * 1e-3),
+        "step_bytes": step_bytes,
+        "kernel_ms": {"plan": sum(r[0] for r in recs) / len(recs), "attention": attn_avg,
+                      "attention_median": attn_ms[len(attn_ms) // 2], "merge": sum(r[2] for r in recs) / len(recs)},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbps": achieved / NOMINAL_HBM_GBS,
+                     "kernel": "decode_main_kernel", "algorithmic_bytes_per_launch": kernel_bytes,
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
+        "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e12, "unit": "TB/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
+        "gpu_launches": args.steps * 4,
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        def host_batch():
+            return {"q": inputs.as_u16(batch.q), "k": inputs.as_u16(batch.k_cache), "v": inputs.as_u16(batch.v_cache),
+                    "table": batch.block_table.cpu().numpy(), "lens": lens_host.numpy(), "strides": batch.strides}
+        line["cpu_baseline"] = cpu_baseline(cfg, host_batch, args.cpu_seconds)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg1", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--ref-token-heads", type=int, default=400000,
+                    help="reference arm: (tokens x q heads) of oracle work per step")
+    args = ap.parse_args()
+    rank, local_rank, world = dist_env()
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 5
+        args.warmup = args.warmup if args.warmup is not None else 1
+        run_reference(args, rank, world)
+        return
+    args.steps = args.steps if args.steps is not None else (2000 if args.workload in ("cfg0", "cfg1") else 200)
+    args.warmup = max(3, args.warmup if args.warmup is not None else 20)
+    run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

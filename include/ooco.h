@@ -220,10 +220,25 @@ int ooco_decode_step_host(const ooco_shape_t* shape, const void* q_host,
 int ooco_last_launch_count(void);
 
 /*
+ * Per-kernel timing of ooco_decode_attention for benchmarks.  ooco_profile_enable(n > 0)
+ * creates CUDA events for up to n calls (process-wide; host objects only, no device
+ * memory) and makes every later ooco_decode_attention call record four events on its
+ * stream: before the plan kernel, before the attention kernel, after it, after the merge
+ * kernel; n = 0 switches recording off and destroys the events.  ooco_profile_read
+ * SYNCHRONISES on the recorded events, writes for each recorded call, oldest first, the
+ * three durations in milliseconds (plan, attention, merge) to ms_out[3 * i + 0..2] for at
+ * most max_records calls, stores the number written in *n_out and forgets all records.
+ * Do not enable while a stream is being captured into a graph.
+ */
+int ooco_profile_enable(int max_records);
+int ooco_profile_read(float* ms_out, int max_records, int* n_out);
+
+/*
  * Launch-shape override for benchmark sweeps (process-wide; the defaults are the tuned
  * values).  knob: 0 consumer warps per CTA {2,4,8}; 1 pipeline stages (0 = as many as
  * fit); 2 CTAs per SM {1..4}; 3 / 4 minimum / maximum split-KV chunk in tokens (multiples
- * of 128); 5 target work items per CTA; 6 non-zero = one TMA copy per 64-dim half.
+ * of 128); 5 target work items per CTA; 6 non-zero = one TMA copy per 64-dim half;
+ * 7 16-token tiles per consumer warp and stage {1,2}.
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.
  */

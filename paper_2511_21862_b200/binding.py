@@ -19,6 +19,7 @@ EXPORTS = (
     "ooco_kv_append", "ooco_decode_workspace_bytes", "ooco_decode_attention", "ooco_workspace_status",
     "ooco_decode_bytes_model", "ooco_step_staging_bytes", "ooco_decode_step_host",
     "ooco_last_launch_count", "ooco_last_error_detail", "ooco_set_tuning", "ooco_status_string", "ooco_version",
+    "ooco_profile_enable", "ooco_profile_read",
 )
 
 
@@ -77,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.ooco_status_string.restype = ctypes.c_char_p
         L.ooco_status_string.argtypes = [ctypes.c_int]
         L.ooco_version.restype = ctypes.c_int
+        L.ooco_profile_enable.restype = ctypes.c_int
+        L.ooco_profile_enable.argtypes = [ctypes.c_int]
+        L.ooco_profile_read.restype = ctypes.c_int
+        L.ooco_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
         _lib = L
     return _lib
 
@@ -110,7 +115,7 @@ class Shape:
 
 
 KNOBS = {"warps": 0, "stages": 1, "ctas_per_sm": 2, "chunk_min": 3, "chunk_max": 4, "items_per_cta": 5,
-         "split_halves": 6}
+         "split_halves": 6, "tiles_per_warp": 7}
 
 
 def set_tuning(**kw):
@@ -191,6 +196,18 @@ def decode_step_host(shape: Shape, q_host, k_new_host, v_new_host, block_table_h
         _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), float(scale), out_host.data_ptr(),
         _dev(staging), staging.numel() * staging.element_size(), _dev(workspace),
         workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step_host")
+
+
+def profile_enable(max_records: int):
+    _check(lib().ooco_profile_enable(int(max_records)), "ooco_profile_enable")
+
+
+def profile_read(max_records: int):
+    """[(plan_ms, attention_ms, merge_ms), ...] of the calls recorded since the last read."""
+    buf = (ctypes.c_float * (3 * max_records))()
+    n = ctypes.c_int(0)
+    _check(lib().ooco_profile_read(buf, max_records, ctypes.byref(n)), "ooco_profile_read")
+    return [(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(n.value)]
 
 
 def last_launch_count() -> int:

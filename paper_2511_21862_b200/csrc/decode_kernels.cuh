@@ -165,30 +165,143 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 // ------------------------------------------------------------------------------------ main
-// Shared-memory carve-up, shared by host (sizing) and device.
-template <int D, int NCW, int NT>
+// Shared-memory carve-up, shared by host (sizing) and device.  TPW = 16-token tiles each
+// consumer warp owns per stage.
+template <int D, int NCW, int NT, int TPW>
 struct SmemLayout {
-  static constexpr int kStageTok = 16 * NCW;
+  static constexpr int kStageTok = 16 * NCW * TPW;
   static constexpr int kTileBytes = kStageTok * D * 2;      // K (or V) bytes of one stage
   static constexpr int kStageBytes = 2 * kTileBytes;
   static constexpr int kHeads = NT * 8;
-  static constexpr int kOStride = D + 4;                     // floats; keeps the merge stores conflict-free
-  static constexpr int kMergeBytes = NCW * kHeads * (kOStride + 2) * 4;
+  static constexpr int kOStride = 64 + 4;                    // floats per head row of one 64-dim pass
+  static constexpr int kMergeOBytes = NCW * kHeads * kOStride * 4;
+  static constexpr int kMergeBytes = kMergeOBytes + NCW * kHeads * 2 * 4;
   __host__ __device__ static int q_slot_bytes(int G) { return ((G * D * 2 + 127) / 128) * 128; }
   __host__ __device__ static size_t total(int nstages, int G) {
     return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16) + kMergeBytes + 64;
   }
 };
 
-template <int D, int NCW, int NT>
+// One consumer warp's work on its TPW tiles of a stage.  kTail: some of the warp's rows lie
+// beyond the chunk (`valid` < 16 * TPW of them count); masked rows get weight 0 and their V
+// words are cleared in registers, so NaN / stale bytes there never reach an accumulator.
+template <int D, int NT, int TPW, bool kTail>
+__device__ __forceinline__ void consume_tiles(uint32_t kst, uint32_t vst, const uint32_t (&tile_k)[TPW],
+                                              const uint32_t (&tile_v)[TPW], const uint32_t (&kpat)[D / 16],
+                                              const uint32_t (&vpat)[D / 16],
+                                              const uint32_t (&qf)[NT][D / 16][2], float (&m_run)[NT][2],
+                                              float (&l_run)[NT][2], float (&o_acc)[NT][D / 16][4],
+                                              float scale_log2e, int valid, int g, int t) {
+  constexpr int KS = D / 16;
+  constexpr int NACC = TPW == 1 ? 2 : 1;  // a lone tile splits its k-steps over two accumulators
+  // ---- scores: S = K_tile x Q^T
+  float sc[TPW][NT][NACC][4];
+#pragma unroll
+  for (int u = 0; u < TPW; ++u)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int a = 0; a < NACC; ++a)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sc[u][nt][a][e] = 0.f;
+#pragma unroll
+  for (int k = 0; k < KS; ++k) {
+#pragma unroll
+    for (int u = 0; u < TPW; ++u) {
+      if (kTail && valid <= 16 * u) continue;
+      uint32_t a0, a1, a2, a3;
+      ldmatrix_x4(kst + tile_k[u] + kpat[k], a0, a1, a2, a3);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+        mma_bf16(sc[u][nt][k % NACC], a0, a1, a2, a3, qf[nt][k][0], qf[nt][k][1]);
+    }
+  }
+  uint32_t pb[TPW][NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    float s[TPW][4];  // [u]: (token g, head 2t) (token g, head 2t+1) (token g+8, 2t) (token g+8, 2t+1)
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < TPW; ++u) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float v = sc[u][nt][0][e];
+        if (NACC == 2) v += sc[u][nt][NACC - 1][e];
+        s[u][e] = v * scale_log2e;
+      }
+      if (kTail) {
+        if (16 * u + g >= valid) s[u][0] = s[u][1] = -INFINITY;
+        if (16 * u + g + 8 >= valid) s[u][2] = s[u][3] = -INFINITY;
+      }
+      mx0 = fmaxf(mx0, fmaxf(s[u][0], s[u][2]));
+      mx1 = fmaxf(mx1, fmaxf(s[u][1], s[u][3]));
+    }
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+    }
+    const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
+    const float al0 = ex2(m_run[nt][0] - mn0), al1 = ex2(m_run[nt][1] - mn1);
+    m_run[nt][0] = mn0;
+    m_run[nt][1] = mn1;
+    float add0 = 0.f, add1 = 0.f;
+#pragma unroll
+    for (int u = 0; u < TPW; ++u) {
+      const uint32_t p01 = pack_bf16x2(ex2(s[u][0] - mn0), ex2(s[u][1] - mn1));  // token g
+      const uint32_t p23 = pack_bf16x2(ex2(s[u][2] - mn0), ex2(s[u][3] - mn1));  // token g+8
+      // sums use the rounded weights, so numerator and denominator agree exactly
+      add0 += __uint_as_float(p01 << 16) + __uint_as_float(p23 << 16);
+      add1 += __uint_as_float(p01 & 0xffff0000u) + __uint_as_float(p23 & 0xffff0000u);
+      pb[u][nt][0] = movmatrix_trans(p01);  // tokens 2t,2t+1 of head g
+      pb[u][nt][1] = movmatrix_trans(p23);  // tokens 2t+8,2t+9 of head g
+    }
+    l_run[nt][0] = l_run[nt][0] * al0 + add0;
+    l_run[nt][1] = l_run[nt][1] * al1 + add1;
+    if (__any_sync(0xffffffffu, (al0 != 1.f) | (al1 != 1.f))) {
+#pragma unroll
+      for (int k = 0; k < KS; ++k) {
+        o_acc[nt][k][0] *= al0;
+        o_acc[nt][k][1] *= al1;
+        o_acc[nt][k][2] *= al0;
+        o_acc[nt][k][3] *= al1;
+      }
+    }
+  }
+  // ---- values: O^T += V_tile^T x P
+#pragma unroll
+  for (int u = 0; u < TPW; ++u) {
+    if (kTail && valid <= 16 * u) continue;
+    uint32_t mk01 = 0xffffffffu, mk23 = 0xffffffffu;
+    if (kTail) {
+      const int v = valid - 16 * u;
+      mk01 = (2 * t < v ? 0x0000ffffu : 0u) | (2 * t + 1 < v ? 0xffff0000u : 0u);
+      mk23 = (2 * t + 8 < v ? 0x0000ffffu : 0u) | (2 * t + 9 < v ? 0xffff0000u : 0u);
+    }
+#pragma unroll
+    for (int k = 0; k < KS; ++k) {
+      uint32_t a0, a1, a2, a3;
+      ldmatrix_x4_trans(vst + tile_v[u] + vpat[k], a0, a1, a2, a3);
+      if (kTail) {
+        a0 &= mk01;
+        a1 &= mk01;
+        a2 &= mk23;
+        a3 &= mk23;
+      }
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) mma_bf16(o_acc[nt][k], a0, a1, a2, a3, pb[u][nt][0], pb[u][nt][1]);
+    }
+  }
+}
+
+template <int D, int NCW, int NT, int TPW>
 __global__ void __launch_bounds__((NCW + 1) * 32, 1)
 decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const DecodeParams p) {
-  using L = SmemLayout<D, NCW, NT>;
+  using L = SmemLayout<D, NCW, NT, TPW>;
   constexpr int kStageTok = L::kStageTok;
   constexpr int KS = D / 16;  // k-steps of the score MMA = m-tiles of the value MMA
   extern __shared__ uint8_t smem_raw[];
-  __shared__ int s_abort;
 
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -205,11 +318,12 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   float* g_merge = reinterpret_cast<float*>(gen + (s_merge - base));
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
   uint8_t* g_q = gen + (s_q - base);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(gen + (s_mbar + 8 - base));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    s_abort = 0;
+    *s_abort = 0;
     for (int i = 0; i < nst; ++i) {
       mbar_init(s_full + 8 * i, 1);
       mbar_init(s_empty + 8 * i, NCW);
@@ -258,7 +372,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         }
         const int slot = it % nst;
         const uint32_t ph = (uint32_t)(it / nst) & 1u;
-        if (!warp_wait(s_empty + 8 * slot, ph ^ 1u, &s_abort)) {
+        if (!warp_wait(s_empty + 8 * slot, ph ^ 1u, s_abort)) {
           ok = false;
           break;
         }
@@ -310,7 +424,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (ok) {
       const int slot = it % nst;
       const uint32_t ph = (uint32_t)(it / nst) & 1u;
-      if (warp_wait(s_empty + 8 * slot, ph ^ 1u, &s_abort)) {
+      if (warp_wait(s_empty + 8 * slot, ph ^ 1u, s_abort)) {
         if (lane == 0) {
           g_meta[slot] = make_int4(-1, 0, 0, 0);
           mbar_arrive(s_full + 8 * slot);
@@ -348,22 +462,33 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       qf[nt][k][0] = qf[nt][k][1] = 0u;
     }
   }
-  // per-lane row / chunk selectors of the two ldmatrix patterns
-  const int r0 = 16 * warp;                        // first token row of this warp inside a stage
-  const int box = r0 / p.tile_rows;
-  const int rb = r0 % p.tile_rows;
+  // Per-lane byte offsets of the ldmatrix rows inside a stage's K / V tile.  A box holds
+  // [D/64 halves][tile_rows][64 dims] with the 128-byte swizzle (16-byte chunk ^= row & 7).
+  const int r0 = 16 * TPW * warp;  // first token row of this warp inside a stage
   const uint32_t box_bytes = (uint32_t)p.tile_rows * D * 2;
-  const uint32_t half_bytes = (uint32_t)p.tile_rows * 128;   // one 64-dim half of a box
+  const uint32_t half_bytes = (uint32_t)p.tile_rows * 128;
   const int lr_k = (lane & 7) + ((lane >> 3) & 1) * 8, cs_k = lane >> 4;
   const int lr_v = (lane & 7) + (lane >> 4) * 8, cs_v = (lane >> 3) & 1;
-  const uint32_t off_k = box * box_bytes + (uint32_t)(rb + lr_k) * 128;
-  const uint32_t off_v = box * box_bytes + (uint32_t)(rb + lr_v) * 128;
+  uint32_t tile_k[TPW], tile_v[TPW], kpat[KS], vpat[KS];
+#pragma unroll
+  for (int u = 0; u < TPW; ++u) {
+    const int r = r0 + 16 * u;
+    const uint32_t bo = (uint32_t)(r / p.tile_rows) * box_bytes;
+    tile_k[u] = bo + (uint32_t)(r % p.tile_rows + lr_k) * 128;
+    tile_v[u] = bo + (uint32_t)(r % p.tile_rows + lr_v) * 128;
+  }
+#pragma unroll
+  for (int k = 0; k < KS; ++k) {
+    const int ck = 2 * k + cs_k, cv = 2 * k + cs_v;
+    kpat[k] = (uint32_t)(ck >> 3) * half_bytes + (uint32_t)(((ck & 7) ^ (lr_k & 7)) << 4);
+    vpat[k] = (uint32_t)(cv >> 3) * half_bytes + (uint32_t)(((cv & 7) ^ (lr_v & 7)) << 4);
+  }
   uint32_t mphase = 0;  // parity of the next merge-barrier phase to wait for
   bool merge_pending_read = false;
 
   for (int it = 0;; ++it) {
     const int slot = it % nst;
-    if (!warp_wait(s_full + 8 * slot, (uint32_t)(it / nst) & 1u, &s_abort)) {
+    if (!warp_wait(s_full + 8 * slot, (uint32_t)(it / nst) & 1u, s_abort)) {
       if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
       return;
     }
@@ -392,95 +517,27 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         }
       }
     }
-    const int valid = min(16, ntok - r0);
+    const int valid = ntok - r0;  // this warp's rows [0, valid) of 16 * TPW hold tokens of the chunk
     if (valid > 0) {
       const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;
       const uint32_t vst = kst + L::kTileBytes;
-      // ---- scores: S = K_tile x Q^T
-      float sc[NT][2][4];
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) sc[nt][0][e] = sc[nt][1][e] = 0.f;
-#pragma unroll
-      for (int k = 0; k < KS; ++k) {
-        const int c = 2 * k + cs_k;
-        const uint32_t addr = kst + off_k + (uint32_t)(c >> 3) * half_bytes + (uint32_t)(((c & 7) ^ (lr_k & 7)) << 4);
-        uint32_t a0, a1, a2, a3;
-        ldmatrix_x4(addr, a0, a1, a2, a3);
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) mma_bf16(sc[nt][k & 1], a0, a1, a2, a3, qf[nt][k][0], qf[nt][k][1]);
-      }
-      uint32_t pb[NT][2];
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        float s0 = (sc[nt][0][0] + sc[nt][1][0]) * p.scale_log2e;  // token g,   head 2t
-        float s1 = (sc[nt][0][1] + sc[nt][1][1]) * p.scale_log2e;  // token g,   head 2t+1
-        float s2 = (sc[nt][0][2] + sc[nt][1][2]) * p.scale_log2e;  // token g+8, head 2t
-        float s3 = (sc[nt][0][3] + sc[nt][1][3]) * p.scale_log2e;  // token g+8, head 2t+1
-        if (g >= valid) s0 = s1 = -INFINITY;
-        if (g + 8 >= valid) s2 = s3 = -INFINITY;
-        float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
-#pragma unroll
-        for (int o = 4; o < 32; o <<= 1) {
-          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
-          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
-        }
-        const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
-        const float al0 = ex2(m_run[nt][0] - mn0), al1 = ex2(m_run[nt][1] - mn1);
-        m_run[nt][0] = mn0;
-        m_run[nt][1] = mn1;
-        const uint32_t p01 = pack_bf16x2(ex2(s0 - mn0), ex2(s1 - mn1));  // token g
-        const uint32_t p23 = pack_bf16x2(ex2(s2 - mn0), ex2(s3 - mn1));  // token g+8
-        // sums use the rounded weights, so numerator and denominator agree exactly
-        l_run[nt][0] = l_run[nt][0] * al0 + __uint_as_float(p01 << 16) + __uint_as_float(p23 << 16);
-        l_run[nt][1] = l_run[nt][1] * al1 + __uint_as_float(p01 & 0xffff0000u) + __uint_as_float(p23 & 0xffff0000u);
-        if (__any_sync(0xffffffffu, (al0 != 1.f) | (al1 != 1.f))) {
-#pragma unroll
-          for (int k = 0; k < KS; ++k) {
-            o_acc[nt][k][0] *= al0;
-            o_acc[nt][k][1] *= al1;
-            o_acc[nt][k][2] *= al0;
-            o_acc[nt][k][3] *= al1;
-          }
-        }
-        pb[nt][0] = movmatrix_trans(p01);  // tokens 2t,2t+1   of head g
-        pb[nt][1] = movmatrix_trans(p23);  // tokens 2t+8,+9   of head g
-      }
-      // ---- values: O^T += V_tile^T x P ; rows past the context are cleared in registers
-      uint32_t mk01 = 0xffffffffu, mk23 = 0xffffffffu;
-      if (valid < 16) {
-        mk01 = (2 * t < valid ? 0x0000ffffu : 0u) | (2 * t + 1 < valid ? 0xffff0000u : 0u);
-        mk23 = (2 * t + 8 < valid ? 0x0000ffffu : 0u) | (2 * t + 9 < valid ? 0xffff0000u : 0u);
-      }
-#pragma unroll
-      for (int k = 0; k < KS; ++k) {
-        const int c = 2 * k + cs_v;
-        const uint32_t addr = vst + off_v + (uint32_t)(c >> 3) * half_bytes + (uint32_t)(((c & 7) ^ (lr_v & 7)) << 4);
-        uint32_t a0, a1, a2, a3;
-        ldmatrix_x4_trans(addr, a0, a1, a2, a3);
-        a0 &= mk01;
-        a1 &= mk01;
-        a2 &= mk23;
-        a3 &= mk23;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) mma_bf16(o_acc[nt][k], a0, a1, a2, a3, pb[nt][0], pb[nt][1]);
-      }
+      if (valid >= 16 * TPW)
+        consume_tiles<D, NT, TPW, false>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
+                                         p.scale_log2e, valid, g, t);
+      else
+        consume_tiles<D, NT, TPW, true>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
+                                        p.scale_log2e, valid, g, t);
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(s_empty + 8 * slot);
 
     if (last) {
-      // ---- combine the NCW warps' running states, then write the item's result
-      if (merge_pending_read) {  // previous item's readers must be done with the buffer
-        if (!warp_wait(s_mbar, mphase, &s_abort)) {
-          if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
-          return;
-        }
-        mphase ^= 1u;
-      }
+      // ---- combine the NCW warps' running states (64 dims per pass), then write the item's result
+      const int item = meta.x, b = meta.y, h = meta.z;
+      const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
       float* mo = g_merge + (size_t)warp * L::kHeads * L::kOStride;
-      float* mm = g_merge + (size_t)NCW * L::kHeads * L::kOStride + (size_t)warp * L::kHeads * 2;
+      float* all_m = g_merge + L::kMergeOBytes / 4;
+      float lsum[NT][2];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         float l0 = l_run[nt][0], l1 = l_run[nt][1];
@@ -489,52 +546,66 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           l0 += __shfl_xor_sync(0xffffffffu, l0, o);
           l1 += __shfl_xor_sync(0xffffffffu, l1, o);
         }
-        const int h0 = 8 * nt + 2 * t;
-        if (g == 0) {
-          mm[2 * h0] = m_run[nt][0];
-          mm[2 * h0 + 1] = l0;
-          mm[2 * h0 + 2] = m_run[nt][1];
-          mm[2 * h0 + 3] = l1;
+        lsum[nt][0] = l0;
+        lsum[nt][1] = l1;
+      }
+#pragma unroll
+      for (int pass = 0; pass < D / 64; ++pass) {
+        if (merge_pending_read) {  // earlier readers must be done with the buffer
+          if (!warp_wait(s_mbar, mphase, s_abort)) {
+            if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+            return;
+          }
+          mphase ^= 1u;
         }
 #pragma unroll
-        for (int k = 0; k < KS; ++k) {
-          mo[(size_t)h0 * L::kOStride + 16 * k + g] = o_acc[nt][k][0];
-          mo[(size_t)(h0 + 1) * L::kOStride + 16 * k + g] = o_acc[nt][k][1];
-          mo[(size_t)h0 * L::kOStride + 16 * k + g + 8] = o_acc[nt][k][2];
-          mo[(size_t)(h0 + 1) * L::kOStride + 16 * k + g + 8] = o_acc[nt][k][3];
-        }
-      }
-      mbar_arrive(s_mbar);
-      if (!warp_wait(s_mbar, mphase, &s_abort)) {
-        if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
-        return;
-      }
-      mphase ^= 1u;
-      const int item = meta.x, b = meta.y, h = meta.z;
-      const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
-      const float* all_m = g_merge + (size_t)NCW * L::kHeads * L::kOStride;
-      for (int idx = threadIdx.x; idx < p.G * D; idx += NCW * 32) {
-        const int head = idx / D, dim = idx % D;
-        float M = -INFINITY;
+        for (int nt = 0; nt < NT; ++nt) {
+          const int h0 = 8 * nt + 2 * t;
+          if (pass == 0 && g == 0) {
+            float* mm = all_m + ((size_t)warp * L::kHeads + h0) * 2;
+            mm[0] = m_run[nt][0];
+            mm[1] = lsum[nt][0];
+            mm[2] = m_run[nt][1];
+            mm[3] = lsum[nt][1];
+          }
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) M = fmaxf(M, all_m[(w * L::kHeads + head) * 2]);
-        float den = 0.f, num = 0.f;
+          for (int kk = 0; kk < 4; ++kk) {
+            const int k = 4 * pass + kk;
+            mo[(size_t)h0 * L::kOStride + 16 * kk + g] = o_acc[nt][k][0];
+            mo[(size_t)(h0 + 1) * L::kOStride + 16 * kk + g] = o_acc[nt][k][1];
+            mo[(size_t)h0 * L::kOStride + 16 * kk + g + 8] = o_acc[nt][k][2];
+            mo[(size_t)(h0 + 1) * L::kOStride + 16 * kk + g + 8] = o_acc[nt][k][3];
+          }
+        }
+        mbar_arrive(s_mbar);
+        if (!warp_wait(s_mbar, mphase, s_abort)) {
+          if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+          return;
+        }
+        mphase ^= 1u;
+        for (int idx = threadIdx.x; idx < p.G * 64; idx += NCW * 32) {
+          const int head = idx >> 6, dl = idx & 63, dim = 64 * pass + dl;
+          float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) {
-          const float sw = ex2(all_m[(w * L::kHeads + head) * 2] - M);
-          den += sw * all_m[(w * L::kHeads + head) * 2 + 1];
-          num += sw * g_merge[((size_t)w * L::kHeads + head) * L::kOStride + dim];
+          for (int w = 0; w < NCW; ++w) M = fmaxf(M, all_m[(w * L::kHeads + head) * 2]);
+          float den = 0.f, num = 0.f;
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            const float sw = ex2(all_m[(w * L::kHeads + head) * 2] - M);
+            den += sw * all_m[(w * L::kHeads + head) * 2 + 1];
+            num += sw * g_merge[((size_t)w * L::kHeads + head) * L::kOStride + dl];
+          }
+          const float o = num / den;
+          if (n_chunks == 1) {
+            p.out[((size_t)b * p.Hq + (size_t)h * p.G + head) * D + dim] = __float2bfloat16_rn(o);
+          } else {
+            p.part_o[((size_t)item * p.G + head) * D + dim] = o;
+            if (dim == 0) p.part_lse[(size_t)item * p.G + head] = M + lg2(den);
+          }
         }
-        const float o = num / den;
-        if (n_chunks == 1) {
-          p.out[((size_t)b * p.Hq + (size_t)h * p.G + head) * D + dim] = __float2bfloat16_rn(o);
-        } else {
-          p.part_o[((size_t)item * p.G + head) * D + dim] = o;
-          if (dim == 0) p.part_lse[(size_t)item * p.G + head] = M + lg2(den);
-        }
+        mbar_arrive(s_mbar);
+        merge_pending_read = true;
       }
-      mbar_arrive(s_mbar);
-      merge_pending_read = true;
     }
   }
 }

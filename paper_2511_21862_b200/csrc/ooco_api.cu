@@ -6,6 +6,8 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "../../include/ooco.h"
 #include "decode_kernels.cuh"
@@ -15,8 +17,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {1}, {256}, {8192}, {6}, {0}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}};
 constexpr int kGridCap = 1024;  // upper bound on CTAs assumed by the host-only workspace bound
 
 static thread_local int tl_last_launches = 0;
@@ -27,6 +29,15 @@ static int fail_cuda(const char* where, long code) {
   snprintf(tl_detail, sizeof tl_detail, "%s failed with code %ld", where, code);
   return OOCO_E_CUDA;
 }
+
+// Optional per-call kernel timing (benchmarks): 4 events per ooco_decode_attention call.
+struct Profiler {
+  std::mutex mu;
+  std::vector<cudaEvent_t> ev;  // 4 per record: before plan, before attention, after attention, after merge
+  int capacity = 0, used = 0;
+};
+static Profiler g_prof;
+static std::atomic<int> g_prof_on{0};
 
 struct DeviceInfo {
   int sm_count = 0;
@@ -136,11 +147,11 @@ static int encode_kv_map(CUtensorMap* tm, const ooco_shape_t* s, const void* bas
   return r == CUDA_SUCCESS ? OOCO_OK : fail_cuda(five_d ? "cuTensorMapEncodeTiled(5d)" : "cuTensorMapEncodeTiled(4d)", (long)r);
 }
 
-template <int D, int NCW, int NT>
+template <int D, int NCW, int NT, int TPW>
 static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                        int ctas_per_sm, int want_stages, cudaStream_t st, int dev) {
-  using L = SmemLayout<D, NCW, NT>;
-  auto kern = decode_main_kernel<D, NCW, NT>;
+  using L = SmemLayout<D, NCW, NT, TPW>;
+  auto kern = decode_main_kernel<D, NCW, NT, TPW>;
   // the opt-in limit covers static + dynamic shared memory of the kernel
   static std::atomic<int> static_smem{-1};
   if (static_smem.load() < 0) {
@@ -169,20 +180,26 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the attention kernel", (long)e);
 }
 
-template <int D, int NCW>
+template <int D, int NCW, int TPW>
 static int launch_main_nt(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                           int cps, int stages, cudaStream_t st, int dev) {
-  if (p.G <= 8) return launch_main<D, NCW, 1>(tk, tv, p, di, cps, stages, st, dev);
-  return launch_main<D, NCW, 2>(tk, tv, p, di, cps, stages, st, dev);
+  if (p.G <= 8) return launch_main<D, NCW, 1, TPW>(tk, tv, p, di, cps, stages, st, dev);
+  return launch_main<D, NCW, 2, TPW>(tk, tv, p, di, cps, stages, st, dev);
 }
 
 template <int D>
-static int launch_main_ncw(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
+static int launch_main_ncw(int ncw, int tpw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
                            const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev) {
+  if (tpw == 2) {
+    switch (ncw) {
+      case 2: return launch_main_nt<D, 2, 2>(tk, tv, p, di, cps, stages, st, dev);
+      default: return launch_main_nt<D, 4, 2>(tk, tv, p, di, cps, stages, st, dev);
+    }
+  }
   switch (ncw) {
-    case 2: return launch_main_nt<D, 2>(tk, tv, p, di, cps, stages, st, dev);
-    case 8: return launch_main_nt<D, 8>(tk, tv, p, di, cps, stages, st, dev);
-    default: return launch_main_nt<D, 4>(tk, tv, p, di, cps, stages, st, dev);
+    case 2: return launch_main_nt<D, 2, 1>(tk, tv, p, di, cps, stages, st, dev);
+    case 8: return launch_main_nt<D, 8, 1>(tk, tv, p, di, cps, stages, st, dev);
+    default: return launch_main_nt<D, 4, 1>(tk, tv, p, di, cps, stages, st, dev);
   }
 }
 
@@ -237,6 +254,38 @@ int ooco_last_launch_count(void) { return tl_last_launches; }
 
 const char* ooco_last_error_detail(void) { return tl_detail; }
 
+int ooco_profile_enable(int max_records) {
+  if (max_records < 0 || max_records > (1 << 20)) return OOCO_E_SHAPE;
+  std::lock_guard<std::mutex> lk(g_prof.mu);
+  g_prof_on.store(0, std::memory_order_release);
+  for (cudaEvent_t e : g_prof.ev) cudaEventDestroy(e);
+  g_prof.ev.clear();
+  g_prof.capacity = g_prof.used = 0;
+  if (max_records == 0) return OOCO_OK;
+  g_prof.ev.resize(4 * (size_t)max_records);
+  for (auto& e : g_prof.ev)
+    if (cudaEventCreate(&e) != cudaSuccess) return fail_cuda("cudaEventCreate", -1);
+  g_prof.capacity = max_records;
+  g_prof_on.store(1, std::memory_order_release);
+  return OOCO_OK;
+}
+
+int ooco_profile_read(float* ms_out, int max_records, int* n_out) {
+  if (!ms_out || !n_out) return OOCO_E_NULLPTR;
+  std::lock_guard<std::mutex> lk(g_prof.mu);
+  int n = g_prof.used < max_records ? g_prof.used : max_records;
+  for (int i = 0; i < n; ++i) {
+    cudaEvent_t* e = &g_prof.ev[4 * (size_t)i];
+    if (cudaEventSynchronize(e[3]) != cudaSuccess) return fail_cuda("cudaEventSynchronize", -1);
+    for (int k = 0; k < 3; ++k)
+      if (cudaEventElapsedTime(&ms_out[3 * i + k], e[k], e[k + 1]) != cudaSuccess)
+        return fail_cuda("cudaEventElapsedTime", -1);
+  }
+  *n_out = n;
+  g_prof.used = 0;
+  return OOCO_OK;
+}
+
 int ooco_set_tuning(int knob, int value) {
   if (knob < 0 || knob >= kKnobCount) return OOCO_E_SHAPE;
   if (knob == kKnobWarps && value != 2 && value != 4 && value != 8) return OOCO_E_SHAPE;
@@ -245,6 +294,7 @@ int ooco_set_tuning(int knob, int value) {
   if ((knob == kKnobChunkMin || knob == kKnobChunkMax) && (value < 128 || value > (1 << 20) || value % 128))
     return OOCO_E_SHAPE;
   if (knob == kKnobItemsPerCta && (value < 1 || value > 64)) return OOCO_E_SHAPE;
+  if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
   return OOCO_OK;
 }
@@ -289,7 +339,9 @@ int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_ca
 
   const int ncw = g_knobs[kKnobWarps].load();
   const int cps = g_knobs[kKnobCtasPerSm].load();
-  const int stage_tok = 16 * ncw;
+  int tpw = g_knobs[kKnobTilesPerWarp].load();
+  if (ncw == 8) tpw = 1;
+  const int stage_tok = 16 * ncw * tpw;
   DecodeParams p;
   memset(&p, 0, sizeof p);
   uint8_t* ws = (uint8_t*)workspace;
@@ -330,18 +382,27 @@ int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_ca
   }
   p.split_halves = five_d ? 0 : 1;
 
+  cudaEvent_t* pe = nullptr;
+  if (g_prof_on.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lk(g_prof.mu);
+    if (g_prof.used < g_prof.capacity) pe = &g_prof.ev[4 * (size_t)g_prof.used++];
+  }
+  if (pe) cudaEventRecord(pe[0], st);
   plan_kernel<1024><<<1, 1024, 0, st>>>(p, stage_tok);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
+  if (pe) cudaEventRecord(pe[1], st);
   if (s->head_dim == 128)
-    rc = launch_main_ncw<128>(ncw, tk, tv, p, di, cps, stages, st, dev);
+    rc = launch_main_ncw<128>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);
   else
-    rc = launch_main_ncw<64>(ncw, tk, tv, p, di, cps, stages, st, dev);
+    rc = launch_main_ncw<64>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);
   if (rc) return rc;
+  if (pe) cudaEventRecord(pe[2], st);
   lse_merge_kernel<<<p.B * p.Hkv, 256, 0, st>>>(p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the merge kernel", (long)e);
+  if (pe) cudaEventRecord(pe[3], st);
   tl_last_launches = 3;
   return OOCO_OK;
 }

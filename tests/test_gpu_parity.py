@@ -20,6 +20,10 @@ def _built():
     binding.lib()
 
 
+DEFAULT_KNOBS = dict(warps=4, stages=0, ctas_per_sm=2, chunk_min=256, chunk_max=8192, items_per_cta=6, split_halves=0,
+                     tiles_per_warp=1)
+
+
 def fixed(*vals):
     return (G(len(vals), min(vals), max(vals), "fixed", tuple(vals)),)
 
@@ -57,14 +61,16 @@ def test_attention_matches_oracle(cfg):
             assert torch.count_nonzero(out[b].float()) == 0
 
 
-@pytest.mark.parametrize("knobs", [dict(warps=2), dict(warps=8), dict(warps=4, ctas_per_sm=2), dict(warps=2, ctas_per_sm=3),
-                                   dict(split_halves=1), dict(stages=2), dict(chunk_min=128, chunk_max=128)],
+@pytest.mark.parametrize("knobs", [dict(warps=2), dict(warps=8, ctas_per_sm=1), dict(warps=4, ctas_per_sm=1),
+                                   dict(warps=2, ctas_per_sm=3), dict(split_halves=1), dict(stages=2),
+                                   dict(chunk_min=128, chunk_max=128), dict(tiles_per_warp=2),
+                                   dict(tiles_per_warp=2, warps=2, ctas_per_sm=3)],
                          ids=lambda k: "-".join(f"{a}{b}" for a, b in k.items()))
 def test_launch_shapes_agree_with_oracle(knobs):
-    default = dict(warps=4, stages=0, ctas_per_sm=1, chunk_min=256, chunk_max=8192, items_per_cta=6, split_halves=0)
+    default = dict(DEFAULT_KNOBS)
     try:
         binding.set_tuning(**{**default, **knobs})
-        for cfg in (SMALL[3], SMALL[5], SMALL[13], SMALL[2]):
+        for cfg in (SMALL[3], SMALL[5], SMALL[13], SMALL[2], SMALL[7], SMALL[10]):
             batch = inputs.make_batch(cfg, "cuda", poison=True, table_pad=-1)
             assert_parity(gpu_attention(batch), oracle_attention(batch).out, what=f"{cfg.name} {knobs}")
     finally:
