@@ -155,6 +155,19 @@ int ooco_decode_attention(const ooco_shape_t* shape, const void* q, const void* 
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * One decode step of this operator with DEVICE buffers: the KV append of ooco_kv_append
+ * (the new token's K / V written at positions[b]) fused into the first launch of
+ * ooco_decode_attention, which then attends over context_lens[b] tokens; a serving step
+ * passes context_lens = positions + 1 (section 2.1: decode reuses and expands the cache).
+ * Same arguments, layouts, ownership and errors as the two calls it replaces; three
+ * launches instead of four.  The attention sees the appended rows.
+ */
+int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new, const void* v_new,
+                     void* k_cache, void* v_cache, const int32_t* block_table,
+                     const int32_t* positions, const int32_t* context_lens, float scale, void* out,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Reads back the device-side status word an earlier ooco_decode_attention /
  * ooco_decode_step_host call left in `workspace`.  SYNCHRONISES `cuda_stream`.
  * *status_host is 0 when every kernel ran to completion, otherwise a bit mask
@@ -191,9 +204,8 @@ size_t ooco_step_staging_bytes(const ooco_shape_t* shape);
 /*
  * One whole decode step of this operator driven from HOST buffers: copies the
  * step's inputs to the device, appends the new token's K/V at positions[b]
- * (ooco_kv_append), attends over context_lens[b] tokens
- * (ooco_decode_attention; a serving step passes context_lens = positions + 1,
- * section 2.1), and copies `out` back.  Everything is enqueued on
+ * and attends over context_lens[b] tokens (ooco_decode_step; a serving step
+ * passes context_lens = positions + 1, section 2.1), and copies `out` back.  Everything is enqueued on
  * `cuda_stream` in that order and the call returns after the stream has been
  * SYNCHRONISED, so out_host is valid on return.
  *
@@ -238,7 +250,8 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * values).  knob: 0 consumer warps per CTA {2,4,8}; 1 pipeline stages (0 = as many as
  * fit); 2 CTAs per SM {1..4}; 3 / 4 minimum / maximum split-KV chunk in tokens (multiples
  * of 128); 5 target work items per CTA; 6 non-zero = one TMA copy per 64-dim half;
- * 7 16-token tiles per consumer warp and stage {1,2}.
+ * 7 16-token tiles per consumer warp and stage {1,2}; 8 non-zero = launch the attention and
+ * merge kernels with programmatic dependent launch (their prologues overlap the predecessor).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.
  */

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libooco.so")
 
 EXPORTS = (
     "ooco_kv_append", "ooco_decode_workspace_bytes", "ooco_decode_attention", "ooco_workspace_status",
-    "ooco_decode_bytes_model", "ooco_step_staging_bytes", "ooco_decode_step_host",
+    "ooco_decode_bytes_model", "ooco_step_staging_bytes", "ooco_decode_step_host", "ooco_decode_step",
     "ooco_last_launch_count", "ooco_last_error_detail", "ooco_set_tuning", "ooco_status_string", "ooco_version",
     "ooco_profile_enable", "ooco_profile_read",
 )
@@ -62,6 +62,9 @@ def lib() -> ctypes.CDLL:
         L.ooco_decode_attention.restype = ctypes.c_int
         L.ooco_decode_attention.argtypes = [sp, vp, vp, vp, i32p, i32p, ctypes.c_float, vp, vp,
                                             ctypes.c_size_t, vp]
+        L.ooco_decode_step.restype = ctypes.c_int
+        L.ooco_decode_step.argtypes = [sp, vp, vp, vp, vp, vp, i32p, i32p, i32p, ctypes.c_float, vp, vp,
+                                       ctypes.c_size_t, vp]
         L.ooco_workspace_status.restype = ctypes.c_int
         L.ooco_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.ooco_decode_bytes_model.restype = ctypes.c_int
@@ -115,7 +118,7 @@ class Shape:
 
 
 KNOBS = {"warps": 0, "stages": 1, "ctas_per_sm": 2, "chunk_min": 3, "chunk_max": 4, "items_per_cta": 5,
-         "split_halves": 6, "tiles_per_warp": 7}
+         "split_halves": 6, "tiles_per_warp": 7, "pdl": 8}
 
 
 def set_tuning(**kw):
@@ -164,6 +167,16 @@ def decode_attention(shape: Shape, q, k_cache, v_cache, block_table, context_len
         _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
         float(scale), _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_attention")
+
+
+def decode_step(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table, positions, context_lens, scale, out,
+                workspace, stream=None):
+    """Fused append (at `positions`) + attention (over `context_lens`) on device buffers."""
+    _check(lib().ooco_decode_step(
+        ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_new, torch.bfloat16), _dev(v_new, torch.bfloat16),
+        _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32),
+        _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), _dev(out, torch.bfloat16),
+        _dev(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step")
 
 
 def workspace_status(workspace, stream=None) -> int:

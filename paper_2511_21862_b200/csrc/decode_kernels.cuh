@@ -40,6 +40,7 @@ struct DecodeParams {
   WsHeader* hdr;
   int4* items;            // [max_items] {b, h, t0, t1}
   int32_t* seq_first;     // [B + 1] first chunk index of each sequence (exclusive scan)
+  int32_t* split_list;    // [B] sequences that were split into more than one chunk
   float* part_o;          // [max_items, G, D] normalised partial outputs
   float* part_lse;        // [max_items, G] log2-domain log-sum-exp of each partial
   int32_t B, Hq, Hkv, G, D, bs, MB;
@@ -52,12 +53,55 @@ struct DecodeParams {
   float scale_log2e;
 };
 
+// ------------------------------------------------------------------------------------ append
+struct AppendParams {
+  const uint4* k_new;   // NULL: no append in this launch
+  const uint4* v_new;
+  uint16_t* k_cache;
+  uint16_t* v_cache;
+  const int32_t* block_table;
+  const int32_t* positions;
+  int32_t B, Hkv, D, bs, NB, MB;
+  int64_t bstr, hstr, tstr;
+};
+
+// Copies the new K / V rows into their slots, one thread per 16-byte vector; `block` of
+// `nblocks` CTAs cooperate grid-stride.
+__device__ __forceinline__ void kv_append_body(const AppendParams& a, int block, int nblocks) {
+  const int vec_per_row = a.D / 8;
+  const long long n = (long long)a.B * a.Hkv * vec_per_row;
+  for (long long i = block * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)nblocks * blockDim.x) {
+    const int v = (int)(i % vec_per_row);
+    const int h = (int)((i / vec_per_row) % a.Hkv);
+    const int b = (int)(i / ((long long)vec_per_row * a.Hkv));
+    const int pos = a.positions[b];
+    if (pos < 0 || (long long)pos >= (long long)a.MB * a.bs) continue;
+    const int blk = a.block_table[(size_t)b * a.MB + pos / a.bs];
+    if (blk < 0 || blk >= a.NB) continue;
+    const int64_t dst = (int64_t)blk * a.bstr + (int64_t)h * a.hstr + (int64_t)(pos % a.bs) * a.tstr + 8 * v;
+    *reinterpret_cast<uint4*>(a.k_cache + dst) = a.k_new[i];
+    *reinterpret_cast<uint4*>(a.v_cache + dst) = a.v_new[i];
+  }
+}
+
+__global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams a) {
+  kv_append_body(a, blockIdx.x, gridDim.x);
+}
+
 // ------------------------------------------------------------------------------------ plan
-// One CTA.  Chooses the chunk length from the total work, splits every sequence into
+// CTA 0 plans; CTAs 1.. (present only in the fused step) do the KV append.  The plan chooses the chunk length from the total work, splits every sequence into
 // near-equal chunks that are multiples of `stage_tok`, and writes the item list.
 template <int kThreads>
-__global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stage_tok) {
+__global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stage_tok, int first_in_smem,
+                                                        const AppendParams ap) {
+  extern __shared__ int s_first[];  // copy of seq_first when it fits (first_in_smem)
+  grid_dep_launch();
+  if (blockIdx.x > 0) {
+    kv_append_body(ap, blockIdx.x - 1, gridDim.x - 1);
+    return;
+  }
   __shared__ long long s_red[kThreads / 32];
+  __shared__ int s_nsplit;
   __shared__ int s_scan[kThreads / 32];
   __shared__ long long s_total;
   __shared__ int s_run;
@@ -77,6 +121,7 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     for (int i = 0; i < kThreads / 32; ++i) t += s_red[i];
     s_total = t;
     s_run = 0;
+    s_nsplit = 0;
   }
   __syncthreads();
   // chunk length: about items_per_cta items per CTA, within [chunk_min, chunk_max]
@@ -113,14 +158,23 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     }
     __syncthreads();
     const int run = s_run;
-    if (b < p.B) p.seq_first[b] = run + s_scan[wid] + inc - n;
+    if (b < p.B) {
+      const int f = run + s_scan[wid] + inc - n;
+      p.seq_first[b] = f;
+      if (first_in_smem) s_first[b] = f;
+      if (n > 1) p.split_list[atomicAdd(&s_nsplit, 1)] = b;
+    }
     __syncthreads();
     if (tid == kThreads - 1) s_run = run + s_scan[wid] + inc;
     __syncthreads();
   }
   const int n_chunks = s_run;
-  if (tid == 0) p.seq_first[p.B] = n_chunks;
+  if (tid == 0) {
+    p.seq_first[p.B] = n_chunks;
+    if (first_in_smem) s_first[p.B] = n_chunks;
+  }
   __syncthreads();
+  const int* first = first_in_smem ? s_first : p.seq_first;
   long long n_items = (long long)n_chunks * p.Hkv;
   const bool overflow = n_items > p.max_items;
   if (overflow) n_items = 0;
@@ -129,6 +183,7 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     p.hdr->n_items = (int)n_items;
     p.hdr->next_item = p.grid_main;
     p.hdr->chunk_tokens = chunk;
+    p.hdr->n_split_seqs = overflow ? 0 : s_nsplit;
   }
   // items, ordered (sequence, chunk, kv head); the sequence of a chunk is found by bisection
   for (long long i = tid; i < n_items; i += kThreads) {
@@ -136,14 +191,14 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     int lo = 0, hi = p.B;  // largest b with seq_first[b] <= ci
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (p.seq_first[mid] <= ci) lo = mid; else hi = mid;
+      if (first[mid] <= ci) lo = mid; else hi = mid;
     }
     const int b = lo;
     long long t = p.context_lens[b];
     t = t > cap ? cap : t;
     const int T = (int)t;
-    const int n = p.seq_first[b + 1] - p.seq_first[b];
-    const int c = ci - p.seq_first[b];
+    const int n = first[b + 1] - first[b];
+    const int c = ci - first[b];
     int len = (T + n - 1) / n;                              // near-equal chunks ...
     len = ((len + stage_tok - 1) / stage_tok) * stage_tok;  // ... in whole stages
     int t0 = c * len, t1 = t0 + len;
@@ -332,6 +387,8 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     fence_mbar_init();
   }
   __syncthreads();
+  grid_dep_wait();    // the plan (and a fused append) must have completed
+  grid_dep_launch();  // the merge kernel may queue up behind this grid
   const int n_items = p.hdr->n_items;
 
   if (warp == NCW) {
@@ -611,28 +668,60 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------ merge
-// One CTA per (sequence, kv head); sequences that were not split are skipped.
-//   out = sum_c 2^(lse_c - M) o_c / sum_c 2^(lse_c - M),  M = max_c lse_c
+// LSE merge of the partial results of split sequences.  One warp per (split sequence, query
+// head): lanes own D / 32 consecutive dims; chunks are taken 32 at a time (one lse per lane),
+//   out = sum_c 2^(lse_c - M) o_c / sum_c 2^(lse_c - M),  M = max_c lse_c.
+template <int D>
 __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
-  const int b = blockIdx.x / p.Hkv, h = blockIdx.x % p.Hkv;
-  const int first = p.seq_first[b];
-  const int n = p.seq_first[b + 1] - first;
-  if (n <= 1 || p.hdr->n_items == 0) return;
-  for (int idx = threadIdx.x; idx < p.G * p.D; idx += blockDim.x) {
-    const int head = idx / p.D, dim = idx % p.D;
-    float M = -INFINITY;
-    for (int c = 0; c < n; ++c) {
-      const size_t item = (size_t)(first + c) * p.Hkv + h;
-      M = fmaxf(M, p.part_lse[item * p.G + head]);
+  constexpr int V = D / 32;  // dims per lane
+  const int lane = threadIdx.x & 31;
+  grid_dep_wait();
+  const int warps_total = gridDim.x * (blockDim.x >> 5);
+  const int n_units = p.hdr->n_split_seqs * p.Hq;
+  for (int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); u < n_units; u += warps_total) {
+    const int b = p.split_list[u / p.Hq], hq = u % p.Hq;
+    const int h = hq / p.G, head = hq % p.G;
+    const int first = p.seq_first[b];
+    const int n = p.seq_first[b + 1] - first;
+    float M = -INFINITY, den = 0.f, acc[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = 0.f;
+    for (int c0 = 0; c0 < n; c0 += 32) {
+      const int cnt = min(32, n - c0);
+      float lse = -INFINITY;
+      if (lane < cnt) lse = p.part_lse[((size_t)(first + c0 + lane) * p.Hkv + h) * p.G + head];
+      float gm = lse;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
+      const float Mn = fmaxf(M, gm);
+      const float resc = exp2f(M - Mn);
+      M = Mn;
+      const float w_lane = exp2f(lse - M);  // 0 for lanes beyond cnt
+      float ws = w_lane;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
+      den = den * resc + ws;
+#pragma unroll
+      for (int i = 0; i < V; ++i) acc[i] *= resc;
+      const float* src = p.part_o + (((size_t)(first + c0) * p.Hkv + h) * p.G + head) * D + lane * V;
+      const size_t cstride = (size_t)p.Hkv * p.G * D;
+#pragma unroll 8
+      for (int j = 0; j < cnt; ++j) {
+        const float w = __shfl_sync(0xffffffffu, w_lane, j);
+        if (V == 4) {
+          const float4 o = *reinterpret_cast<const float4*>(src + j * cstride);
+          acc[0] += w * o.x; acc[1] += w * o.y; acc[2] += w * o.z; acc[V - 1] += w * o.w;
+        } else {
+          const float2 o = *reinterpret_cast<const float2*>(src + j * cstride);
+          acc[0] += w * o.x; acc[V - 1] += w * o.y;
+        }
+      }
     }
-    float den = 0.f, num = 0.f;
-    for (int c = 0; c < n; ++c) {
-      const size_t item = (size_t)(first + c) * p.Hkv + h;
-      const float w = exp2f(p.part_lse[item * p.G + head] - M);
-      den += w;
-      num += w * p.part_o[(item * p.G + head) * p.D + dim];
-    }
-    p.out[((size_t)b * p.Hq + (size_t)h * p.G + head) * p.D + dim] = __float2bfloat16_rn(num / den);
+    __nv_bfloat16* dst = p.out + ((size_t)b * p.Hq + hq) * D + lane * V;
+    const float inv = 1.f / den;
+#pragma unroll
+    for (int i = 0; i < V; i += 2)
+      *reinterpret_cast<__nv_bfloat162*>(dst + i) = __floats2bfloat162_rn(acc[i] * inv, acc[i + 1] * inv);
   }
 }
 

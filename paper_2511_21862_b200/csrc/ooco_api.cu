@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <utility>
 #include <vector>
 
 #include "../../include/ooco.h"
@@ -17,11 +18,12 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}};
-constexpr int kGridCap = 1024;  // upper bound on CTAs assumed by the host-only workspace bound
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}};
+constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
 static thread_local int tl_last_launches = 0;
+static thread_local bool tl_events_between_kernels = false;  // profiling: no programmatic overlap
 static thread_local char tl_detail[160] = "";
 
 // Remembers where a CUDA-side failure happened (read back through ooco_last_error_detail).
@@ -95,7 +97,7 @@ static int validate_shape(const ooco_shape_t* s) {
 
 // Workspace carve-up (all offsets multiples of 256 bytes).
 struct WsLayout {
-  size_t off_first, off_items, off_lse, off_o, total;
+  size_t off_first, off_split, off_items, off_lse, off_o, total;
   int max_items;
 };
 static WsLayout ws_layout(const ooco_shape_t* s) {
@@ -110,7 +112,8 @@ static WsLayout ws_layout(const ooco_shape_t* s) {
   WsLayout w;
   w.max_items = (int)(max_items > INT32_MAX ? INT32_MAX : max_items);
   w.off_first = 256;
-  w.off_items = w.off_first + up(((size_t)s->batch + 1) * 4);
+  w.off_split = w.off_first + up(((size_t)s->batch + 1) * 4);
+  w.off_items = w.off_split + up((size_t)s->batch * 4);
   w.off_lse = w.off_items + up((size_t)w.max_items * 16);
   w.off_o = w.off_lse + up((size_t)w.max_items * G * 4);
   w.total = w.off_o + up((size_t)w.max_items * G * s->head_dim * 4);
@@ -175,8 +178,9 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
     if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
-  kern<<<p.grid_main, (NCW + 1) * 32, smem, st>>>(tk, tv, p);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_ex(kern, dim3(p.grid_main), dim3((NCW + 1) * 32), smem, st,
+                            g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the attention kernel", (long)e);
 }
 
@@ -203,28 +207,50 @@ static int launch_main_ncw(int ncw, int tpw, const CUtensorMap& tk, const CUtens
   }
 }
 
-// ------------------------------------------------------------------------------------ append
-// One thread per 16-byte vector of the new K and of the new V rows.
-__global__ void __launch_bounds__(256)
-kv_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint16_t* k_cache,
-                 uint16_t* v_cache, const int32_t* __restrict__ block_table,
-                 const int32_t* __restrict__ positions, int B, int Hkv, int D, int bs, int NB, int MB,
-                 int64_t bstr, int64_t hstr, int64_t tstr) {
-  const int vec_per_row = D / 8;
-  const long long n = (long long)B * Hkv * vec_per_row;
-  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
-       i += (long long)gridDim.x * blockDim.x) {
-    const int v = (int)(i % vec_per_row);
-    const int h = (int)((i / vec_per_row) % Hkv);
-    const int b = (int)(i / ((long long)vec_per_row * Hkv));
-    const int pos = positions[b];
-    if (pos < 0 || (long long)pos >= (long long)MB * bs) continue;
-    const int blk = block_table[(size_t)b * MB + pos / bs];
-    if (blk < 0 || blk >= NB) continue;
-    const int64_t dst = (int64_t)blk * bstr + (int64_t)h * hstr + (int64_t)(pos % bs) * tstr + 8 * v;
-    *reinterpret_cast<uint4*>(k_cache + dst) = k_new[i];
-    *reinterpret_cast<uint4*>(v_cache + dst) = v_new[i];
-  }
+// Launch with the programmatic-stream-serialization attribute (the kernel itself waits for its
+// predecessor with griddepcontrol.wait) when `pdl`, else an ordinary launch.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
+static AppendParams make_append_params(const ooco_shape_t* s, const void* k_new, const void* v_new,
+                                       void* k_cache, void* v_cache, const int32_t* block_table,
+                                       const int32_t* positions) {
+  AppendParams a;
+  a.k_new = (const uint4*)k_new;
+  a.v_new = (const uint4*)v_new;
+  a.k_cache = (uint16_t*)k_cache;
+  a.v_cache = (uint16_t*)v_cache;
+  a.block_table = block_table;
+  a.positions = positions;
+  a.B = s->batch;
+  a.Hkv = s->num_kv_heads;
+  a.D = s->head_dim;
+  a.bs = s->block_size;
+  a.NB = s->num_blocks;
+  a.MB = s->max_blocks_per_seq;
+  a.bstr = s->kv_block_stride;
+  a.hstr = s->kv_head_stride;
+  a.tstr = s->kv_token_stride;
+  return a;
+}
+
+static int append_blocks(const ooco_shape_t* s, int threads) {
+  const long long n = (long long)s->batch * s->num_kv_heads * (s->head_dim / 8);
+  long long blocks = (n + threads - 1) / threads;
+  return (int)(blocks > 2048 ? 2048 : blocks);
 }
 
 static int current_device(int* dev) { return cudaGetDevice(dev) == cudaSuccess ? OOCO_OK : OOCO_E_CUDA; }
@@ -306,13 +332,8 @@ int ooco_kv_append(const ooco_shape_t* s, const void* k_new, const void* v_new, 
   if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
   if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
     return OOCO_E_UNSUPPORTED;
-  const long long n = (long long)s->batch * s->num_kv_heads * (s->head_dim / 8);
-  long long blocks = (n + 255) / 256;
-  if (blocks > 4096) blocks = 4096;
-  kv_append_kernel<<<(int)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(
-      (const uint4*)k_new, (const uint4*)v_new, (uint16_t*)k_cache, (uint16_t*)v_cache, block_table, positions,
-      s->batch, s->num_kv_heads, s->head_dim, s->block_size, s->num_blocks, s->max_blocks_per_seq,
-      s->kv_block_stride, s->kv_head_stride, s->kv_token_stride);
+  const AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
+  kv_append_kernel<<<append_blocks(s, 256), 256, 0, (cudaStream_t)cuda_stream>>>(ap);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the append kernel", (long)e);
 }
@@ -322,9 +343,10 @@ size_t ooco_decode_workspace_bytes(const ooco_shape_t* s) {
   return ws_layout(s).total;
 }
 
-int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
-                          const int32_t* block_table, const int32_t* context_lens, float scale, void* out,
-                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+// Plan (+ optional fused append) -> split-KV attention -> LSE merge on `cuda_stream`.
+static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
+                       const int32_t* block_table, const int32_t* context_lens, float scale, void* out,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream, const AppendParams* append) {
   int rc = validate_shape(s);
   if (rc) return rc;
   if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
@@ -351,6 +373,7 @@ int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_ca
   p.context_lens = context_lens;
   p.hdr = (WsHeader*)ws;
   p.seq_first = (int32_t*)(ws + w.off_first);
+  p.split_list = (int32_t*)(ws + w.off_split);
   p.items = (int4*)(ws + w.off_items);
   p.part_lse = (float*)(ws + w.off_lse);
   p.part_o = (float*)(ws + w.off_o);
@@ -387,8 +410,15 @@ int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_ca
     std::lock_guard<std::mutex> lk(g_prof.mu);
     if (g_prof.used < g_prof.capacity) pe = &g_prof.ev[4 * (size_t)g_prof.used++];
   }
+  tl_events_between_kernels = pe != nullptr;
   if (pe) cudaEventRecord(pe[0], st);
-  plan_kernel<1024><<<1, 1024, 0, st>>>(p, stage_tok);
+  const size_t first_bytes = ((size_t)p.B + 1) * 4;
+  const int first_in_smem = first_bytes <= 40 * 1024;
+  AppendParams ap;
+  memset(&ap, 0, sizeof ap);
+  if (append) ap = *append;
+  const int plan_grid = 1 + (append ? append_blocks(s, 1024) : 0);
+  plan_kernel<1024><<<plan_grid, 1024, first_in_smem ? first_bytes : 0, st>>>(p, stage_tok, first_in_smem, ap);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
@@ -399,12 +429,42 @@ int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_ca
     rc = launch_main_ncw<64>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);
   if (rc) return rc;
   if (pe) cudaEventRecord(pe[2], st);
-  lse_merge_kernel<<<p.B * p.Hkv, 256, 0, st>>>(p);
-  e = cudaGetLastError();
+  {
+    long long warps = (long long)p.B * p.Hq;  // upper bound on (split sequence, query head) units
+    int blocks = (int)((warps + 7) / 8);
+    if (blocks > di.sm_count * 8) blocks = di.sm_count * 8;
+    const bool pdl = g_knobs[kKnobPdl].load() != 0 && !pe;
+    if (s->head_dim == 128)
+      e = launch_ex(lse_merge_kernel<128>, dim3(blocks), dim3(256), 0, st, pdl, p);
+    else
+      e = launch_ex(lse_merge_kernel<64>, dim3(blocks), dim3(256), 0, st, pdl, p);
+  }
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the merge kernel", (long)e);
   if (pe) cudaEventRecord(pe[3], st);
   tl_last_launches = 3;
   return OOCO_OK;
+}
+
+int ooco_decode_attention(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
+                          const int32_t* block_table, const int32_t* context_lens, float scale, void* out,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                     cuda_stream, nullptr);
+}
+
+int ooco_decode_step(const ooco_shape_t* s, const void* q, const void* k_new, const void* v_new, void* k_cache,
+                     void* v_cache, const int32_t* block_table, const int32_t* positions,
+                     const int32_t* context_lens, float scale, void* out, void* workspace,
+                     size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
+    return OOCO_E_UNSUPPORTED;
+  const AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
+  return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                     cuda_stream, &ap);
 }
 
 int ooco_workspace_status(const void* workspace, void* cuda_stream, int32_t* status_host) {
@@ -483,14 +543,12 @@ int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void*
   ok &= cudaMemcpyAsync(d_pos, positions_host, lb, cudaMemcpyHostToDevice, st) == cudaSuccess;
   ok &= cudaMemcpyAsync(d_len, context_lens_host, lb, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (!ok) return OOCO_E_CUDA;
-  if ((rc = ooco_kv_append(s, d_kn, d_vn, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_pos, st)))
-    return rc;
-  if ((rc = ooco_decode_attention(s, d_q, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_len, scale,
-                                  d_out, workspace, workspace_bytes, st)))
+  if ((rc = ooco_decode_step(s, d_q, d_kn, d_vn, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_pos,
+                             (const int32_t*)d_len, scale, d_out, workspace, workspace_bytes, st)))
     return rc;
   if (cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return OOCO_E_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return OOCO_E_CUDA;
-  tl_last_launches = 4;
+  tl_last_launches = 3;
   return OOCO_OK;
 }
 

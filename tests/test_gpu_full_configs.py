@@ -46,8 +46,10 @@ def test_large_config_sampled_sequences(name):
     mx, mean = assert_parity(out, ref.out, rows=seqs, what=name)
     print(f"{name} sampled {len(seqs)} sequences: max abs {mx:.3e} mean abs {mean:.3e}")
     # property that holds at any size: every output lies in the convex hull of its V values
-    bound = batch.v_cache[torch.isfinite(batch.v_cache)].abs().max().float()
-    assert out.float().abs().max() <= bound * 1.01
+    step = 1 << 13                                                                      # blocks per chunk
+    bound = max(float(torch.nan_to_num(batch.v_cache[s:s + step].float(), nan=0.0).abs().max())
+                for s in range(0, batch.num_blocks, step))
+    assert float(out.float().abs().max()) <= bound * 1.01
 
     if name == "cfg4":
         # one-token append for every sequence at position T_b: whole pool compared word for word

@@ -21,7 +21,7 @@ def _built():
 
 
 DEFAULT_KNOBS = dict(warps=4, stages=0, ctas_per_sm=2, chunk_min=256, chunk_max=8192, items_per_cta=6, split_halves=0,
-                     tiles_per_warp=1)
+                     tiles_per_warp=1, pdl=1)
 
 
 def fixed(*vals):
@@ -64,7 +64,7 @@ def test_attention_matches_oracle(cfg):
 @pytest.mark.parametrize("knobs", [dict(warps=2), dict(warps=8, ctas_per_sm=1), dict(warps=4, ctas_per_sm=1),
                                    dict(warps=2, ctas_per_sm=3), dict(split_halves=1), dict(stages=2),
                                    dict(chunk_min=128, chunk_max=128), dict(tiles_per_warp=2),
-                                   dict(tiles_per_warp=2, warps=2, ctas_per_sm=3)],
+                                   dict(tiles_per_warp=2, warps=2, ctas_per_sm=3), dict(pdl=0)],
                          ids=lambda k: "-".join(f"{a}{b}" for a, b in k.items()))
 def test_launch_shapes_agree_with_oracle(knobs):
     default = dict(DEFAULT_KNOBS)
@@ -182,7 +182,29 @@ def test_serving_step_from_host_buffers():
     ref = oracle.decode_attention(inputs.as_u16(batch.q), k_ref, v_ref, batch.block_table.cpu().numpy(),
                                   lens1.numpy(), cfg.scale, num_kv_heads=8, block_size=16, strides=batch.strides)
     assert_parity(out_h, ref.out, what="host step")
-    assert binding.last_launch_count() == 4
+    assert binding.last_launch_count() == 3
+
+
+def test_fused_step_on_device_buffers():
+    """ooco_decode_step = append at T (bit-exact over the whole pool) + attention over T + 1 tokens."""
+    cfg = C("fused", 40, 8, 128, 16, (G(21, 1, 3000),), seed=52, pool_fill=0.85)
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(batch.q, float("nan"))
+    lens1 = (batch.context_lens + 1).contiguous()
+    k_ref, v_ref = inputs.as_u16(batch.k_cache).copy(), inputs.as_u16(batch.v_cache).copy()
+    for _ in range(2):                                                         # same slots twice: idempotent
+        binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, batch.k_cache, batch.v_cache, batch.block_table,
+                            batch.context_lens, lens1, cfg.scale, out, ws)
+    assert binding.workspace_status(ws) == 0
+    oracle.kv_append(inputs.as_u16(batch.k_new), inputs.as_u16(batch.v_new), k_ref, v_ref,
+                     batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), block_size=16,
+                     strides=batch.strides)
+    assert np.array_equal(inputs.as_u16(batch.k_cache), k_ref) and np.array_equal(inputs.as_u16(batch.v_cache), v_ref)
+    ref = oracle.decode_attention(inputs.as_u16(batch.q), k_ref, v_ref, batch.block_table.cpu().numpy(),
+                                  lens1.cpu().numpy(), cfg.scale, num_kv_heads=8, block_size=16, strides=batch.strides)
+    assert_parity(out, ref.out, what="fused step")
 
 
 def test_many_sequences_plan_scan():
