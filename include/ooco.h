@@ -168,6 +168,43 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Paged decode attention for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a packaging variant of ooco_decode_attention.)
+ *
+ * Who needs it: an inference engine that hands the whole device to its KV-cache pool at
+ * start-up has nothing left for cudaMalloc to give; a latency-critical decode loop cannot
+ * afford the device-wide synchronisation an allocation or a free implies; and a plug-in
+ * running under a host framework may be forbidden to allocate outside that framework's own
+ * pool.  Such a caller cannot provide the workspace ooco_decode_attention asks for.
+ *
+ * This entry point takes the same inputs and output but no workspace: the scratch is an
+ * array of OOCO_STATIC_SCRATCH_BYTES built into the library's device image (every GPU that
+ * loads the library holds it until the process exits).  The call allocates nothing, neither
+ * through cudaMalloc / cudaFree nor through any allocating library routine, and computes
+ * exactly what ooco_decode_attention computes, with the same launches.
+ *
+ *   - A shape whose ooco_decode_workspace_bytes exceeds OOCO_STATIC_SCRATCH_BYTES is refused
+ *     with OOCO_E_WORKSPACE before anything is launched, and ooco_last_error_detail names
+ *     both sizes.  The exact test is ooco_decode_workspace_bytes(shape) <=
+ *     OOCO_STATIC_SCRATCH_BYTES; with head_dim 128 and block tables of up to 8 K tokens that
+ *     admits about 300 sequences of 32 q / 8 kv heads (64 sequences need 8.2 MiB) and about
+ *     50 sequences of 64 q / 8 kv heads.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current, as for every call); make that first call outside any stream capture.
+ *   - All calls on a device share the one array: two calls that may overlap on the GPU (other
+ *     streams, other host threads) race on it and corrupt each other's results.  Calls on one
+ *     stream are ordered and safe.  The array keeps the previous call's contents; nothing in
+ *     it needs to start at zero, because the first kernel of each call rewrites every field
+ *     that is read later.
+ *   - The device status word of this variant is not exposed.
+ */
+#define OOCO_STATIC_SCRATCH_BYTES (16u << 20)
+int ooco_decode_attention_static(const ooco_shape_t* shape, const void* q, const void* k_cache,
+                                 const void* v_cache, const int32_t* block_table,
+                                 const int32_t* context_lens, float scale, void* out,
+                                 void* cuda_stream);
+
+/*
  * Reads back the device-side status word an earlier ooco_decode_attention /
  * ooco_decode_step_host call left in `workspace`.  SYNCHRONISES `cuda_stream`.
  * *status_host is 0 when every kernel ran to completion, otherwise a bit mask

@@ -19,14 +19,14 @@ EXPORTS = (
     "ooco_kv_append", "ooco_decode_workspace_bytes", "ooco_decode_attention", "ooco_workspace_status",
     "ooco_decode_bytes_model", "ooco_step_staging_bytes", "ooco_decode_step_host", "ooco_decode_step",
     "ooco_last_launch_count", "ooco_last_error_detail", "ooco_set_tuning", "ooco_status_string", "ooco_version",
-    "ooco_profile_enable", "ooco_profile_read",
+    "ooco_profile_enable", "ooco_profile_read", "ooco_decode_attention_static",
 )
 
 
 class OocoError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        detail = lib().ooco_last_error_detail().decode() if status == -5 else ""
+        detail = lib().ooco_last_error_detail().decode() if status in (-4, -5) else ""
         super().__init__(f"{where}: {status_string(status)} ({status}) {detail}".rstrip())
 
 
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.ooco_decode_step.restype = ctypes.c_int
         L.ooco_decode_step.argtypes = [sp, vp, vp, vp, vp, vp, i32p, i32p, i32p, ctypes.c_float, vp, vp,
                                        ctypes.c_size_t, vp]
+        L.ooco_decode_attention_static.restype = ctypes.c_int
+        L.ooco_decode_attention_static.argtypes = [sp, vp, vp, vp, i32p, i32p, ctypes.c_float, vp, vp]
         L.ooco_workspace_status.restype = ctypes.c_int
         L.ooco_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.ooco_decode_bytes_model.restype = ctypes.c_int
@@ -177,6 +179,21 @@ def decode_step(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table, po
         _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32),
         _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), _dev(out, torch.bfloat16),
         _dev(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step")
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def decode_attention_static(shape: Shape, q, k_cache, v_cache, block_table, context_lens, scale, out, stream=None):
+    """ooco_decode_attention without a workspace argument, for callers that cannot allocate device
+    memory (the whole device already belongs to a KV pool, an allocation's implicit synchronisation is
+    not affordable, or the host framework forbids allocations outside its pool).  The scratch is a
+    16 MiB array built into the library; shapes that need more raise OocoError(-4).  Calls that may
+    overlap on the GPU race on that array; the first call on a device should precede stream capture."""
+    _check(lib().ooco_decode_attention_static(
+        ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_cache, torch.bfloat16),
+        _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
+        float(scale), _dev(out, torch.bfloat16), _stream_ptr(stream)), "ooco_decode_attention_static")
 
 
 def workspace_status(workspace, stream=None) -> int:

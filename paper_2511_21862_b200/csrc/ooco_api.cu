@@ -253,6 +253,31 @@ static int append_blocks(const ooco_shape_t* s, int threads) {
   return (int)(blocks > 2048 ? 2048 : blocks);
 }
 
+// Built-in scratch for ooco_decode_attention_static: it lives in the library's device image, so
+// using it needs no allocation call.  In host code the name below is only a stand-in for the
+// symbol; the device address comes from cudaGetSymbolAddress (static_scratch_ptr).
+static __device__ __align__(256) unsigned char g_static_scratch[OOCO_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+static int static_scratch_ptr(void** ptr_out) {
+  static std::mutex mu;
+  static void* cache[64];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail_cuda("cudaGetDevice", (long)e);
+  std::lock_guard<std::mutex> lk(mu);
+  if (dev >= 0 && dev < 64 && cache[dev]) {
+    *ptr_out = cache[dev];
+    return OOCO_OK;
+  }
+  void* ptr = nullptr;
+  e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
+  if (e != cudaSuccess || !ptr) return fail_cuda("cudaGetSymbolAddress(built-in scratch)", (long)e);
+  if (dev >= 0 && dev < 64) cache[dev] = ptr;
+  *ptr_out = ptr;
+  return OOCO_OK;
+}
+
 static int current_device(int* dev) { return cudaGetDevice(dev) == cudaSuccess ? OOCO_OK : OOCO_E_CUDA; }
 
 }  // namespace ooco
@@ -465,6 +490,24 @@ int ooco_decode_step(const ooco_shape_t* s, const void* q, const void* k_new, co
   const AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
   return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
                      cuda_stream, &ap);
+}
+
+int ooco_decode_attention_static(const ooco_shape_t* s, const void* q, const void* k_cache,
+                                 const void* v_cache, const int32_t* block_table,
+                                 const int32_t* context_lens, float scale, void* out, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  const size_t need = ws_layout(s).total;
+  if (need > (size_t)OOCO_STATIC_SCRATCH_BYTES) {
+    snprintf(tl_detail, sizeof tl_detail,
+             "shape needs %zu bytes of scratch, the built-in scratch holds %zu: use ooco_decode_attention",
+             need, (size_t)OOCO_STATIC_SCRATCH_BYTES);
+    return OOCO_E_WORKSPACE;
+  }
+  void* scratch = nullptr;
+  if ((rc = static_scratch_ptr(&scratch))) return rc;
+  return ooco_decode_attention(s, q, k_cache, v_cache, block_table, context_lens, scale, out, scratch,
+                               (size_t)OOCO_STATIC_SCRATCH_BYTES, cuda_stream);
 }
 
 int ooco_workspace_status(const void* workspace, void* cuda_stream, int32_t* status_host) {
