@@ -38,7 +38,7 @@ struct DecodeParams {
   const int32_t* block_table;
   const int32_t* context_lens;
   WsHeader* hdr;
-  int4* items;            // [max_items] {b, h, t0, t1}
+  int4* items;            // [max_items] {b, partial slot = chunk index * Hkv + h, t0, t1}, longest first
   int32_t* seq_first;     // [B + 1] first chunk index of each sequence (exclusive scan)
   int32_t* split_list;    // [B] sequences that were split into more than one chunk
   float* part_o;          // [max_items, G, D] normalised partial outputs
@@ -185,15 +185,21 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     p.hdr->chunk_tokens = chunk;
     p.hdr->n_split_seqs = overflow ? 0 : s_nsplit;
   }
-  // items, ordered (sequence, chunk, kv head); the sequence of a chunk is found by bisection
-  for (long long i = tid; i < n_items; i += kThreads) {
-    const int ci = (int)(i / p.Hkv), h = (int)(i % p.Hkv);
-    int lo = 0, hi = p.B;  // largest b with seq_first[b] <= ci
+  // Items in order of decreasing length (longest first keeps the tail of the dynamic schedule
+  // short): counting sort of the chunks by length in stages.  An item carries its partial-result
+  // slot (chunk index * Hkv + head), which does not depend on the order.
+  __shared__ int s_hist[kThreads];    // bucket r = kThreads - 1 - min(stages, kThreads - 1)
+  __shared__ int s_cursor[kThreads];
+  s_hist[tid] = 0;
+  __syncthreads();
+  const int n_chunks_ok = overflow ? 0 : n_chunks;
+  auto chunk_of = [&](int ci, int& b, int& t0, int& t1) {
+    int lo = 0, hi = p.B;  // largest b with first[b] <= ci
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
       if (first[mid] <= ci) lo = mid; else hi = mid;
     }
-    const int b = lo;
+    b = lo;
     long long t = p.context_lens[b];
     t = t > cap ? cap : t;
     const int T = (int)t;
@@ -201,10 +207,45 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     const int c = ci - first[b];
     int len = (T + n - 1) / n;                              // near-equal chunks ...
     len = ((len + stage_tok - 1) / stage_tok) * stage_tok;  // ... in whole stages
-    int t0 = c * len, t1 = t0 + len;
+    t0 = c * len;
+    t1 = t0 + len;
     if (t0 > T) t0 = T;
     if (t1 > T) t1 = T;
-    p.items[i] = make_int4(b, h, t0, t1);
+    const int stages = (t1 - t0 + stage_tok - 1) / stage_tok;
+    return kThreads - 1 - (stages < kThreads - 1 ? stages : kThreads - 1);
+  };
+  for (int ci = tid; ci < n_chunks_ok; ci += kThreads) {
+    int b, t0, t1;
+    atomicAdd(&s_hist[chunk_of(ci, b, t0, t1)], 1);
+  }
+  __syncthreads();
+  {  // exclusive scan of the histogram (bucket 0 = longest)
+    const int v = s_hist[tid];
+    int inc = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      int u = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += u;
+    }
+    if (lane == 31) s_scan[wid] = inc;
+    __syncthreads();
+    if (wid == 0) {
+      int w0 = lane < kThreads / 32 ? s_scan[lane] : 0;
+      int w = w0;
+      for (int o = 1; o < 32; o <<= 1) {
+        int u = __shfl_up_sync(0xffffffffu, w, o);
+        if (lane >= o) w += u;
+      }
+      if (lane < kThreads / 32) s_scan[lane] = w - w0;
+    }
+    __syncthreads();
+    s_cursor[tid] = s_scan[wid] + inc - v;
+  }
+  __syncthreads();
+  for (int ci = tid; ci < n_chunks_ok; ci += kThreads) {
+    int b, t0, t1;
+    const int r = chunk_of(ci, b, t0, t1);
+    const long long pos = atomicAdd(&s_cursor[r], 1);
+    for (int h = 0; h < p.Hkv; ++h) p.items[pos * p.Hkv + h] = make_int4(b, ci * p.Hkv + h, t0, t1);
   }
   // sequences without context produce zeros
   const int row = p.Hq * p.D;
@@ -414,7 +455,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
       int4 nd = make_int4(0, 0, 0, 0);
       int blk_nxt_item = 0;
-      const int b = d.x, h = d.y, t0 = d.z, t1 = d.w;
+      const int b = d.x, slot_id = d.y, h = d.y % p.Hkv, t0 = d.z, t1 = d.w;
       const int nstage_item = (t1 - t0 + kStageTok - 1) / kStageTok;
       const int32_t* row = p.block_table + (size_t)b * p.MB;
       for (int s = 0; s < nstage_item; ++s, ++it) {
@@ -436,7 +477,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const uint32_t full = s_full + 8 * slot;
         if (lane == 0) {
           const int flags = (s == 0 ? 1 : 0) | (s == nstage_item - 1 ? 2 : 0);
-          g_meta[slot] = make_int4(item, b, h, ntok | (flags << 16));
+          g_meta[slot] = make_int4(slot_id, b, h, ntok | (flags << 16));
           uint32_t bytes = 2u * nbox * box_bytes;
           if (s == 0) bytes += (uint32_t)p.G * D * 2;
           mbar_arrive_expect_tx(full, bytes);

@@ -438,7 +438,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   tl_events_between_kernels = pe != nullptr;
   if (pe) cudaEventRecord(pe[0], st);
   const size_t first_bytes = ((size_t)p.B + 1) * 4;
-  const int first_in_smem = first_bytes <= 40 * 1024;
+  const int first_in_smem = first_bytes <= 32 * 1024;  // static + dynamic shared memory stay under 48 KiB
   AppendParams ap;
   memset(&ap, 0, sizeof ap);
   if (append) ap = *append;
