@@ -288,9 +288,7 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * fit); 2 CTAs per SM {1..4}; 3 / 4 minimum / maximum split-KV chunk in tokens (multiples
  * of 128); 5 target work items per CTA; 6 non-zero = one TMA copy per 64-dim half;
  * 7 16-token tiles per consumer warp and stage {1,2}; 8 non-zero = launch the attention and
- * merge kernels with programmatic dependent launch (their prologues overlap the predecessor);
- * 9 non-zero = bandwidth-ceiling probe: K / V tiles are streamed but the arithmetic is skipped
- * and `out` is meaningless.
+ * merge kernels with programmatic dependent launch (their prologues overlap the predecessor).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.
  */

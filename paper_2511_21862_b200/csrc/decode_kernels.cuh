@@ -50,7 +50,6 @@ struct DecodeParams {
   int32_t nstages;
   int32_t grid_main;      // CTAs of the attention kernel (first items are assigned statically)
   int32_t chunk_min, chunk_max, items_per_cta;
-  int32_t probe_skip_math;  // bandwidth-ceiling probe: tiles are fetched but not used (output meaningless)
   float scale_log2e;
 };
 
@@ -617,7 +616,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       }
     }
     const int valid = ntok - r0;  // this warp's rows [0, valid) of 16 * TPW hold tokens of the chunk
-    if (valid > 0 && !p.probe_skip_math) {
+    if (valid > 0) {
       const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;
       const uint32_t vst = kst + L::kTileBytes;
       if (valid >= 16 * TPW)

@@ -18,8 +18,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobProbeSkipMath, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {0}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}};
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
 static thread_local int tl_last_launches = 0;
@@ -418,7 +418,6 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
   p.items_per_cta = g_knobs[kKnobItemsPerCta].load();
   p.scale_log2e = scale * 1.4426950408889634f;
-  p.probe_skip_math = g_knobs[kKnobProbeSkipMath].load();
 
   CUtensorMap tk, tv;
   bool five_d = s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
