@@ -27,8 +27,7 @@ struct WsHeader {  // first 256 bytes of the workspace
   int32_t n_items;
   int32_t next_item;
   int32_t chunk_tokens;
-  int32_t n_split_seqs;
-  int32_t pad[59];
+  int32_t pad[60];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
@@ -40,7 +39,6 @@ struct DecodeParams {
   WsHeader* hdr;
   int4* items;            // [max_items] {b, partial slot = chunk index * Hkv + h, t0, t1}, longest first
   int32_t* seq_first;     // [B + 1] first chunk index of each sequence (exclusive scan)
-  int32_t* split_list;    // [B] sequences that were split into more than one chunk
   float* part_o;          // [max_items, G, D] normalised partial outputs
   float* part_lse;        // [max_items, G] log2-domain log-sum-exp of each partial
   int32_t B, Hq, Hkv, G, D, bs, MB;
@@ -101,7 +99,6 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     return;
   }
   __shared__ long long s_red[kThreads / 32];
-  __shared__ int s_nsplit;
   __shared__ int s_scan[kThreads / 32];
   __shared__ long long s_total;
   __shared__ int s_run;
@@ -121,7 +118,6 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     for (int i = 0; i < kThreads / 32; ++i) t += s_red[i];
     s_total = t;
     s_run = 0;
-    s_nsplit = 0;
   }
   __syncthreads();
   // chunk length: about items_per_cta items per CTA, within [chunk_min, chunk_max]
@@ -162,7 +158,6 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
       const int f = run + s_scan[wid] + inc - n;
       p.seq_first[b] = f;
       if (first_in_smem) s_first[b] = f;
-      if (n > 1) p.split_list[atomicAdd(&s_nsplit, 1)] = b;
     }
     __syncthreads();
     if (tid == kThreads - 1) s_run = run + s_scan[wid] + inc;
@@ -183,7 +178,6 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     p.hdr->n_items = (int)n_items;
     p.hdr->next_item = p.grid_main;
     p.hdr->chunk_tokens = chunk;
-    p.hdr->n_split_seqs = overflow ? 0 : s_nsplit;
   }
   // Items in order of decreasing length (longest first keeps the tail of the dynamic schedule
   // short): counting sort of the chunks by length in stages.  An item carries its partial-result
@@ -709,21 +703,34 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------ merge
-// LSE merge of the partial results of split sequences.  One warp per (split sequence, query
-// head): lanes own D / 32 consecutive dims; chunks are taken 32 at a time (one lse per lane),
+// LSE merge of the partial results of split sequences.  One warp per (sequence, query head);
+// warps of unsplit sequences have nothing to do.  Of a split sequence: lanes own D / 32 consecutive dims; chunks are taken 32 at a time (one lse per lane),
 //   out = sum_c 2^(lse_c - M) o_c / sum_c 2^(lse_c - M),  M = max_c lse_c.
 template <int D>
 __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
   constexpr int V = D / 32;  // dims per lane
   const int lane = threadIdx.x & 31;
-  grid_dep_wait();
   const int warps_total = gridDim.x * (blockDim.x >> 5);
-  const int n_units = p.hdr->n_split_seqs * p.Hq;
-  for (int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); u < n_units; u += warps_total) {
-    const int b = p.split_list[u / p.Hq], hq = u % p.Hq;
+  const int n_units = p.B * p.Hq;
+  int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  // The chunk scan was written by the plan kernel, which had completed before the attention grid
+  // (the grid this launch depends on) passed its own dependency wait, so it may be read before
+  // the wait below; only the partial results need the attention grid to be complete.
+  int first = 0, n = 0;
+  if (p.hdr->status & kStatusPlanOverflow) return;  // no work list, no partials (status is reported)
+  if (u < n_units) {
+    first = p.seq_first[u / p.Hq];
+    n = p.seq_first[u / p.Hq + 1] - first;
+  }
+  grid_dep_wait();
+  for (; u < n_units; u += warps_total, first = -1) {
+    const int b = u / p.Hq, hq = u % p.Hq;
     const int h = hq / p.G, head = hq % p.G;
-    const int first = p.seq_first[b];
-    const int n = p.seq_first[b + 1] - first;
+    if (first < 0) {
+      first = p.seq_first[b];
+      n = p.seq_first[b + 1] - first;
+    }
+    if (n <= 1) continue;  // unsplit (or empty) sequence: the attention kernel wrote the row itself
     float M = -INFINITY, den = 0.f, acc[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) acc[i] = 0.f;

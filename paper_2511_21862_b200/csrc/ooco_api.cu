@@ -97,7 +97,7 @@ static int validate_shape(const ooco_shape_t* s) {
 
 // Workspace carve-up (all offsets multiples of 256 bytes).
 struct WsLayout {
-  size_t off_first, off_split, off_items, off_lse, off_o, total;
+  size_t off_first, off_items, off_lse, off_o, total;
   int max_items;
 };
 static WsLayout ws_layout(const ooco_shape_t* s) {
@@ -112,8 +112,7 @@ static WsLayout ws_layout(const ooco_shape_t* s) {
   WsLayout w;
   w.max_items = (int)(max_items > INT32_MAX ? INT32_MAX : max_items);
   w.off_first = 256;
-  w.off_split = w.off_first + up(((size_t)s->batch + 1) * 4);
-  w.off_items = w.off_split + up((size_t)s->batch * 4);
+  w.off_items = w.off_first + up(((size_t)s->batch + 1) * 4);
   w.off_lse = w.off_items + up((size_t)w.max_items * 16);
   w.off_o = w.off_lse + up((size_t)w.max_items * G * 4);
   w.total = w.off_o + up((size_t)w.max_items * G * s->head_dim * 4);
@@ -398,7 +397,6 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.context_lens = context_lens;
   p.hdr = (WsHeader*)ws;
   p.seq_first = (int32_t*)(ws + w.off_first);
-  p.split_list = (int32_t*)(ws + w.off_split);
   p.items = (int4*)(ws + w.off_items);
   p.part_lse = (float*)(ws + w.off_lse);
   p.part_o = (float*)(ws + w.off_o);
