@@ -92,7 +92,11 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams a) {
 template <int kThreads>
 __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stage_tok, int first_in_smem,
                                                         const AppendParams ap) {
-  extern __shared__ int s_first[];  // copy of seq_first when it fits (first_in_smem)
+  extern __shared__ int s_first[];  // when they fit (first_in_smem): seq_first [B + 1], then clamped lengths [B]
+  // Launched programmatically: nothing of the caller's buffers or of the workspace may be touched
+  // before the preceding work in the stream (which may still read the workspace, or still
+  // produce this call's inputs) is complete.
+  grid_dep_wait();
   grid_dep_launch();
   if (blockIdx.x > 0) {
     kv_append_body(ap, blockIdx.x - 1, gridDim.x - 1);
@@ -105,10 +109,18 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const long long cap = (long long)p.MB * p.bs;
 
+  int* s_len = s_first + p.B + 1;
+  auto len_of = [&](int b) -> long long {  // context length clamped to [0, table capacity]
+    if (first_in_smem) return s_len[b];
+    const long long t = p.context_lens[b];
+    return t < 0 ? 0 : (t > cap ? cap : t);
+  };
   long long acc = 0;
   for (int b = tid; b < p.B; b += kThreads) {
     long long t = p.context_lens[b];
-    acc += t < 0 ? 0 : (t > cap ? cap : t);
+    t = t < 0 ? 0 : (t > cap ? cap : t);
+    if (first_in_smem) s_len[b] = (int)t;
+    acc += t;
   }
   for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
   if (lane == 0) s_red[wid] = acc;
@@ -131,11 +143,7 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
   for (int base = 0; base < p.B; base += kThreads) {
     const int b = base + tid;
     int n = 0;
-    if (b < p.B) {
-      long long t = p.context_lens[b];
-      t = t < 0 ? 0 : (t > cap ? cap : t);
-      n = (int)((t + chunk - 1) / chunk);
-    }
+    if (b < p.B) n = (int)((len_of(b) + chunk - 1) / chunk);
     int inc = n;
     for (int o = 1; o < 32; o <<= 1) {
       int v = __shfl_up_sync(0xffffffffu, inc, o);
@@ -194,9 +202,7 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
       if (first[mid] <= ci) lo = mid; else hi = mid;
     }
     b = lo;
-    long long t = p.context_lens[b];
-    t = t > cap ? cap : t;
-    const int T = (int)t;
+    const int T = (int)len_of(b);
     const int n = first[b + 1] - first[b];
     const int c = ci - first[b];
     int len = (T + n - 1) / n;                              // near-equal chunks ...
@@ -244,7 +250,7 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
   // sequences without context produce zeros
   const int row = p.Hq * p.D;
   for (int b = wid; b < p.B; b += kThreads / 32) {
-    if (p.context_lens[b] > 0) continue;
+    if (len_of(b) > 0) continue;
     for (int i = lane; i < row; i += 32) p.out[(size_t)b * row + i] = __float2bfloat16(0.f);
   }
 }
@@ -717,6 +723,7 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
   // (the grid this launch depends on) passed its own dependency wait, so it may be read before
   // the wait below; only the partial results need the attention grid to be complete.
   int first = 0, n = 0;
+  grid_dep_launch();  // a programmatically launched successor may start its own prologue
   if (p.hdr->status & kStatusPlanOverflow) return;  // no work list, no partials (status is reported)
   if (u < n_units) {
     first = p.seq_first[u / p.Hq];

@@ -435,14 +435,16 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   }
   tl_events_between_kernels = pe != nullptr;
   if (pe) cudaEventRecord(pe[0], st);
-  const size_t first_bytes = ((size_t)p.B + 1) * 4;
-  const int first_in_smem = first_bytes <= 32 * 1024;  // static + dynamic shared memory stay under 48 KiB
+  const size_t first_bytes = (2 * (size_t)p.B + 1) * 4;  // chunk scan + clamped lengths
+  const int first_in_smem = first_bytes <= 32 * 1024;    // static + dynamic shared memory stay under 48 KiB
   AppendParams ap;
   memset(&ap, 0, sizeof ap);
   if (append) ap = *append;
   const int plan_grid = 1 + (append ? append_blocks(s, 1024) : 0);
-  plan_kernel<1024><<<plan_grid, 1024, first_in_smem ? first_bytes : 0, st>>>(p, stage_tok, first_in_smem, ap);
-  cudaError_t e = cudaGetLastError();
+  const bool pdl_on = g_knobs[kKnobPdl].load() != 0 && !pe;
+  cudaError_t e = launch_ex(plan_kernel<1024>, dim3(plan_grid), dim3(1024), first_in_smem ? first_bytes : 0, st,
+                            pdl_on, p, stage_tok, first_in_smem, ap);
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
   if (pe) cudaEventRecord(pe[1], st);
