@@ -205,6 +205,43 @@ int ooco_decode_attention_static(const ooco_shape_t* shape, const void* q, const
                                  void* cuda_stream);
 
 /*
+ * Paged KV block movement (section 3.4.3 "Offline Request Migration": an offline request's KV
+ * cache is transferred from a latency-relaxed to a latency-strict instance; section 3.4.1: space
+ * is freed on a latency-strict instance by evicting offline requests; section 4: the KV cache is
+ * what travels between instances).  The transport wants one contiguous buffer per transfer, the
+ * pool is non-contiguous, so a migration is gather (sender) -> transfer -> scatter (receiver).
+ *
+ * ooco_kv_gather_blocks   packs the n listed pool blocks, in list order, into
+ *                         k_packed / v_packed, bf16 [n, Hkv, block_size, head_dim] contiguous.
+ * ooco_kv_scatter_blocks  is the inverse: block i of the packed buffers is written to pool
+ *                         block block_ids[i].
+ * ooco_kv_copy_blocks     copies pool block src_ids[i] to pool block dst_ids[i] (pool
+ *                         compaction, copy-on-write of a shared prefix block).
+ * All copy 16-bit words verbatim; every word of a listed destination block is written, nothing
+ * else is.
+ *
+ *   shape            the pool's shape (num_kv_heads, head_dim, block_size, num_blocks and the three
+ *                    strides are used; the other fields must merely be valid)
+ *   block_ids, src_ids, dst_ids   device, int32 [n]; n = 0 is legal and launches nothing
+ *   k_packed, v_packed            device, 16-byte aligned, n * Hkv * block_size * head_dim words each
+ *   status           device int32, may be NULL.  Bits are OR-ed in, never cleared: 4 = an id was
+ *                    outside [0, num_blocks) (that list entry is skipped), 2 = a bounded wait in
+ *                    the kernel gave up.  The caller zeroes it and reads it back when it wants to.
+ * Destination ids must be distinct, and in ooco_kv_copy_blocks no block may be both a source and
+ * a destination.  One launch, asynchronous on `cuda_stream`.  The tuned case is a pool whose
+ * (block, kv head) tiles are contiguous (kv_token_stride = head_dim); other strides are moved
+ * row by row.
+ */
+int ooco_kv_gather_blocks(const ooco_shape_t* shape, const void* k_cache, const void* v_cache,
+                          const int32_t* block_ids, int32_t n, void* k_packed, void* v_packed,
+                          int32_t* status, void* cuda_stream);
+int ooco_kv_scatter_blocks(const ooco_shape_t* shape, const void* k_packed, const void* v_packed,
+                           const int32_t* block_ids, int32_t n, void* k_cache, void* v_cache,
+                           int32_t* status, void* cuda_stream);
+int ooco_kv_copy_blocks(const ooco_shape_t* shape, void* k_cache, void* v_cache, const int32_t* src_ids,
+                        const int32_t* dst_ids, int32_t n, int32_t* status, void* cuda_stream);
+
+/*
  * Reads back the device-side status word an earlier ooco_decode_attention /
  * ooco_decode_step_host call left in `workspace`.  SYNCHRONISES `cuda_stream`.
  * *status_host is 0 when every kernel ran to completion, otherwise a bit mask
@@ -288,7 +325,8 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * fit); 2 CTAs per SM {1..4}; 3 / 4 minimum / maximum split-KV chunk in tokens (multiples
  * of 128); 5 target work items per CTA; 6 non-zero = one TMA copy per 64-dim half;
  * 7 16-token tiles per consumer warp and stage {1,2}; 8 non-zero = launch the attention and
- * merge kernels with programmatic dependent launch (their prologues overlap the predecessor).
+ * merge kernels with programmatic dependent launch (their prologues overlap the predecessor);
+ * 9 CTAs per SM of the block-movement kernel {1..3}.
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.
  */

@@ -20,6 +20,7 @@ EXPORTS = (
     "ooco_decode_bytes_model", "ooco_step_staging_bytes", "ooco_decode_step_host", "ooco_decode_step",
     "ooco_last_launch_count", "ooco_last_error_detail", "ooco_set_tuning", "ooco_status_string", "ooco_version",
     "ooco_profile_enable", "ooco_profile_read", "ooco_decode_attention_static",
+    "ooco_kv_gather_blocks", "ooco_kv_scatter_blocks", "ooco_kv_copy_blocks",
 )
 
 
@@ -67,6 +68,12 @@ def lib() -> ctypes.CDLL:
                                        ctypes.c_size_t, vp]
         L.ooco_decode_attention_static.restype = ctypes.c_int
         L.ooco_decode_attention_static.argtypes = [sp, vp, vp, vp, i32p, i32p, ctypes.c_float, vp, vp]
+        L.ooco_kv_gather_blocks.restype = ctypes.c_int
+        L.ooco_kv_gather_blocks.argtypes = [sp, vp, vp, i32p, ctypes.c_int32, vp, vp, i32p, vp]
+        L.ooco_kv_scatter_blocks.restype = ctypes.c_int
+        L.ooco_kv_scatter_blocks.argtypes = [sp, vp, vp, i32p, ctypes.c_int32, vp, vp, i32p, vp]
+        L.ooco_kv_copy_blocks.restype = ctypes.c_int
+        L.ooco_kv_copy_blocks.argtypes = [sp, vp, vp, i32p, i32p, ctypes.c_int32, i32p, vp]
         L.ooco_workspace_status.restype = ctypes.c_int
         L.ooco_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.ooco_decode_bytes_model.restype = ctypes.c_int
@@ -120,7 +127,7 @@ class Shape:
 
 
 KNOBS = {"warps": 0, "stages": 1, "ctas_per_sm": 2, "chunk_min": 3, "chunk_max": 4, "items_per_cta": 5,
-         "split_halves": 6, "tiles_per_warp": 7, "pdl": 8}
+         "split_halves": 6, "tiles_per_warp": 7, "pdl": 8, "copy_ctas_per_sm": 9}
 
 
 def set_tuning(**kw):
@@ -194,6 +201,42 @@ def decode_attention_static(shape: Shape, q, k_cache, v_cache, block_table, cont
         ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_cache, torch.bfloat16),
         _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
         float(scale), _dev(out, torch.bfloat16), _stream_ptr(stream)), "ooco_decode_attention_static")
+
+
+def _opt_dev(t, dtype=None):
+    return None if t is None else _dev(t, dtype)
+
+
+def kv_gather_blocks(shape: Shape, k_cache, v_cache, block_ids, k_packed, v_packed, status=None, stream=None):
+    """Pack the listed pool blocks, in list order, into `k_packed` / `v_packed` [n, Hkv, bs, D]."""
+    n = block_ids.numel()
+    need = n * shape.num_kv_heads * shape.block_size * shape.head_dim
+    assert k_packed.numel() >= need and v_packed.numel() >= need
+    _check(lib().ooco_kv_gather_blocks(
+        ctypes.byref(shape.c()), _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16),
+        _dev(block_ids, torch.int32), n, _dev(k_packed, torch.bfloat16), _dev(v_packed, torch.bfloat16),
+        _opt_dev(status, torch.int32), _stream_ptr(stream)), "ooco_kv_gather_blocks")
+
+
+def kv_scatter_blocks(shape: Shape, k_packed, v_packed, block_ids, k_cache, v_cache, status=None, stream=None):
+    """Write block i of the packed buffers to pool block `block_ids[i]`."""
+    n = block_ids.numel()
+    need = n * shape.num_kv_heads * shape.block_size * shape.head_dim
+    assert k_packed.numel() >= need and v_packed.numel() >= need
+    _check(lib().ooco_kv_scatter_blocks(
+        ctypes.byref(shape.c()), _dev(k_packed, torch.bfloat16), _dev(v_packed, torch.bfloat16),
+        _dev(block_ids, torch.int32), n, _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16),
+        _opt_dev(status, torch.int32), _stream_ptr(stream)), "ooco_kv_scatter_blocks")
+
+
+def kv_copy_blocks(shape: Shape, k_cache, v_cache, src_ids, dst_ids, status=None, stream=None):
+    """Copy pool block `src_ids[i]` to pool block `dst_ids[i]`."""
+    n = src_ids.numel()
+    assert dst_ids.numel() == n
+    _check(lib().ooco_kv_copy_blocks(
+        ctypes.byref(shape.c()), _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16),
+        _dev(src_ids, torch.int32), _dev(dst_ids, torch.int32), n, _opt_dev(status, torch.int32),
+        _stream_ptr(stream)), "ooco_kv_copy_blocks")
 
 
 def workspace_status(workspace, stream=None) -> int:

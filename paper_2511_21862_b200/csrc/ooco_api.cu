@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "../../include/ooco.h"
+#include "block_copy_kernels.cuh"
 #include "decode_kernels.cuh"
 
 namespace ooco {
@@ -18,8 +19,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {3}};
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
 static thread_local int tl_last_launches = 0;
@@ -279,6 +280,74 @@ static int static_scratch_ptr(void** ptr_out) {
 
 static int current_device(int* dev) { return cudaGetDevice(dev) == cudaSuccess ? OOCO_OK : OOCO_E_CUDA; }
 
+// Largest contiguous run of a side: 0 = whole block, 1 = one kv head of a block, 2 = one token row.
+static int run_level(int64_t hstr, int64_t tstr, int bs, int D) {
+  if (tstr != D) return 2;
+  return hstr == (int64_t)bs * D ? 0 : 1;
+}
+
+static BlockSide pool_side(const ooco_shape_t* s, const void* k, const void* v, const int32_t* ids) {
+  BlockSide b;
+  b.k = (uint16_t*)k;
+  b.v = (uint16_t*)v;
+  b.ids = ids;
+  b.bstr = s->kv_block_stride;
+  b.hstr = s->kv_head_stride;
+  b.tstr = s->kv_token_stride;
+  b.nb = s->num_blocks;
+  return b;
+}
+
+static BlockSide packed_side(const ooco_shape_t* s, const void* k, const void* v, int n) {
+  BlockSide b;
+  b.k = (uint16_t*)k;
+  b.v = (uint16_t*)v;
+  b.ids = nullptr;
+  b.tstr = s->head_dim;
+  b.hstr = (int64_t)s->block_size * s->head_dim;
+  b.bstr = b.hstr * s->num_kv_heads;
+  b.nb = n;
+  return b;
+}
+
+// Moves n listed blocks from `src` to `dst` (K and V) with the bulk-copy kernel.
+static int launch_block_copy(const ooco_shape_t* s, const BlockSide& src, const BlockSide& dst, int n,
+                             int32_t* status, void* cuda_stream) {
+  if (n == 0) return OOCO_OK;
+  int dev = 0, rc;
+  if ((rc = current_device(&dev))) return rc;
+  const DeviceInfo di = device_info(dev);
+  if (di.sm_count <= 0) return OOCO_E_CUDA;
+  BlockCopyParams p;
+  memset(&p, 0, sizeof p);
+  p.src = src;
+  p.dst = dst;
+  p.n = n;
+  p.Hkv = s->num_kv_heads;
+  p.bs = s->block_size;
+  p.D = s->head_dim;
+  const int ls = run_level(src.hstr, src.tstr, p.bs, p.D), ld = run_level(dst.hstr, dst.tstr, p.bs, p.D);
+  p.run_level = ls > ld ? ls : ld;
+  p.runs_per_block = p.run_level == 0 ? 1 : (p.run_level == 1 ? p.Hkv : p.Hkv * p.bs);
+  p.run_bytes = 2 * p.Hkv * p.bs * p.D / p.runs_per_block;
+  p.pieces_per_run = (p.run_bytes + kCopyPieceBytes - 1) / kCopyPieceBytes;
+  p.status = status;
+  const long long total = (long long)n * p.runs_per_block * p.pieces_per_run * 2;
+  const long long cap = (long long)di.sm_count * g_knobs[kKnobCopyCtasPerSm].load();
+  const int grid = (int)(total < cap ? total : cap);
+  const size_t smem = (size_t)kCopyStages * kCopyPieceBytes + 128;
+  static std::atomic<int> configured[64];
+  if (dev < 0 || dev >= 64 || !configured[dev].load()) {
+    cudaError_t e = cudaFuncSetAttribute(block_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(block copy smem)", (long)e);
+    if (dev >= 0 && dev < 64) configured[dev].store(1);
+  }
+  cudaError_t e = launch_ex(block_copy_kernel, dim3(grid), dim3(32), smem, (cudaStream_t)cuda_stream,
+                            g_knobs[kKnobPdl].load() != 0, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the block copy kernel", (long)e);
+}
+
 }  // namespace ooco
 
 using namespace ooco;
@@ -345,6 +414,7 @@ int ooco_set_tuning(int knob, int value) {
     return OOCO_E_SHAPE;
   if (knob == kKnobItemsPerCta && (value < 1 || value > 64)) return OOCO_E_SHAPE;
   if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
+  if (knob == kKnobCopyCtasPerSm && (value < 1 || value > 3)) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
   return OOCO_OK;
 }
@@ -508,6 +578,42 @@ int ooco_decode_attention_static(const ooco_shape_t* s, const void* q, const voi
   if ((rc = static_scratch_ptr(&scratch))) return rc;
   return ooco_decode_attention(s, q, k_cache, v_cache, block_table, context_lens, scale, out, scratch,
                                (size_t)OOCO_STATIC_SCRATCH_BYTES, cuda_stream);
+}
+
+static int check_block_args(const ooco_shape_t* s, int32_t n, const void* a, const void* b, const void* c,
+                            const void* d, bool ids_ok) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  if (n < 0) return OOCO_E_SHAPE;
+  if (!a || !b || !c || !d || (!ids_ok && n > 0)) return OOCO_E_NULLPTR;
+  if (((uintptr_t)a | (uintptr_t)b | (uintptr_t)c | (uintptr_t)d) & 15) return OOCO_E_UNSUPPORTED;
+  return OOCO_OK;
+}
+
+int ooco_kv_gather_blocks(const ooco_shape_t* s, const void* k_cache, const void* v_cache,
+                          const int32_t* block_ids, int32_t n, void* k_packed, void* v_packed, int32_t* status,
+                          void* cuda_stream) {
+  int rc = check_block_args(s, n, k_cache, v_cache, k_packed, v_packed, block_ids != nullptr);
+  if (rc) return rc;
+  return launch_block_copy(s, pool_side(s, k_cache, v_cache, block_ids), packed_side(s, k_packed, v_packed, n), n,
+                           status, cuda_stream);
+}
+
+int ooco_kv_scatter_blocks(const ooco_shape_t* s, const void* k_packed, const void* v_packed,
+                           const int32_t* block_ids, int32_t n, void* k_cache, void* v_cache, int32_t* status,
+                           void* cuda_stream) {
+  int rc = check_block_args(s, n, k_cache, v_cache, k_packed, v_packed, block_ids != nullptr);
+  if (rc) return rc;
+  return launch_block_copy(s, packed_side(s, k_packed, v_packed, n), pool_side(s, k_cache, v_cache, block_ids), n,
+                           status, cuda_stream);
+}
+
+int ooco_kv_copy_blocks(const ooco_shape_t* s, void* k_cache, void* v_cache, const int32_t* src_ids,
+                        const int32_t* dst_ids, int32_t n, int32_t* status, void* cuda_stream) {
+  int rc = check_block_args(s, n, k_cache, v_cache, k_cache, v_cache, src_ids && dst_ids);
+  if (rc) return rc;
+  return launch_block_copy(s, pool_side(s, k_cache, v_cache, src_ids), pool_side(s, k_cache, v_cache, dst_ids), n,
+                           status, cuda_stream);
 }
 
 int ooco_workspace_status(const void* workspace, void* cuda_stream, int32_t* status_host) {

@@ -51,7 +51,7 @@ class DecodeConfig:
         return 1.0 / math.sqrt(self.head_dim)
 
 
-# The five workloads of the build's baseline file, in its order.
+# The five benchmark workloads.
 CONFIGS = {
     "cfg0": DecodeConfig(
         "cfg0", 8, 2, 64, 16, (LengthGroup(4, 17, 256, "fixed", (17, 64, 130, 256)),), seed=0,
