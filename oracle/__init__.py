@@ -137,3 +137,59 @@ def bytes_model(context_lens, *, num_q_heads, num_kv_heads, head_dim, block_size
     if rc != 0:
         raise ValueError(f"oracle_bytes_model failed with {rc}")
     return {k: int(v) for k, v in zip(COST_FIELDS, cost)}
+
+
+# --------------------------------------------------------------------------- paged block movement
+# Migration of an offline request moves its KV cache between instances (section 3.4.3 of the
+# paper, "Offline Request Migration"; section 4: the KV cache is what is transmitted); on a paged
+# pool that is: pack the request's blocks, transfer, unpack into the receiver's free blocks.  These
+# three are exact by definition (16-bit words copied verbatim), written with numpy indexing.
+
+def _block_view(cache: np.ndarray, strides, num_kv_heads, block_size, head_dim) -> np.ndarray:
+    """[NB, Hkv, bs, D] strided view of a uint16 pool addressed by (block, head, token) strides."""
+    assert cache.dtype == np.uint16 and cache.flags.c_contiguous
+    bstr, hstr, tstr = (int(s) for s in strides)
+    nb = cache.size // bstr
+    return np.lib.stride_tricks.as_strided(
+        cache.reshape(-1), shape=(nb, num_kv_heads, block_size, head_dim),
+        strides=(2 * bstr, 2 * hstr, 2 * tstr, 2), writeable=cache.flags.writeable)
+
+
+def _valid(ids, nb):
+    ids = np.asarray(ids, dtype=np.int64)
+    return ids, (ids >= 0) & (ids < nb)
+
+
+def gather_blocks(k_cache, v_cache, block_ids, *, num_kv_heads, block_size, head_dim, strides,
+                  k_packed=None, v_packed=None):
+    """Packed copies [n, Hkv, bs, D] of the listed pool blocks, in list order.  An id outside the
+    pool leaves its packed block as it was (zeros when the buffers are created here)."""
+    kv, vv = (_block_view(c, strides, num_kv_heads, block_size, head_dim) for c in (k_cache, v_cache))
+    ids, ok = _valid(block_ids, kv.shape[0])
+    shape = (ids.size, num_kv_heads, block_size, head_dim)
+    k_packed = np.zeros(shape, np.uint16) if k_packed is None else k_packed
+    v_packed = np.zeros(shape, np.uint16) if v_packed is None else v_packed
+    k_packed[ok] = kv[ids[ok]]
+    v_packed[ok] = vv[ids[ok]]
+    return k_packed, v_packed
+
+
+def scatter_blocks(k_packed, v_packed, block_ids, k_cache, v_cache, *, num_kv_heads, block_size, head_dim,
+                   strides) -> None:
+    """In place: pool block block_ids[i] <- packed block i (ids outside the pool are skipped)."""
+    kv, vv = (_block_view(c, strides, num_kv_heads, block_size, head_dim) for c in (k_cache, v_cache))
+    ids, ok = _valid(block_ids, kv.shape[0])
+    kv[ids[ok]] = np.asarray(k_packed).reshape(ids.size, num_kv_heads, block_size, head_dim)[ok]
+    vv[ids[ok]] = np.asarray(v_packed).reshape(ids.size, num_kv_heads, block_size, head_dim)[ok]
+
+
+def copy_blocks(k_cache, v_cache, src_ids, dst_ids, *, num_kv_heads, block_size, head_dim, strides) -> None:
+    """In place: pool block dst_ids[i] <- pool block src_ids[i]; every source is read before any
+    destination is written (sources and destinations are disjoint by contract)."""
+    kv, vv = (_block_view(c, strides, num_kv_heads, block_size, head_dim) for c in (k_cache, v_cache))
+    src, oks = _valid(src_ids, kv.shape[0])
+    dst, okd = _valid(dst_ids, kv.shape[0])
+    ok = oks & okd
+    ksrc, vsrc = kv[src[ok]].copy(), vv[src[ok]].copy()
+    kv[dst[ok]] = ksrc
+    vv[dst[ok]] = vsrc
