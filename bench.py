@@ -360,6 +360,87 @@ def run_ours(args, rank, local_rank, world):
     print(json.dumps(line))
 
 
+def run_block_moves(args, rank, local_rank, world):
+    """Secondary measurement: paged KV block movement (the data movement of a request migration).
+
+    One step packs the blocks of `--move-seqs` sequences of the workload (longest first) into a
+    contiguous buffer and unpacks them into free blocks of a second pool; gather and scatter are also
+    timed alone.  Successive steps use other pool replicas / packed buffers (working set >> L2)."""
+    from paper_2511_21862_b200 import binding, build
+    build.build()
+    binding.lib()
+    for kv in args.knob:
+        name, val = kv.split("=")
+        binding.set_tuning(**{name: int(val)})
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    cfg = inputs.CONFIGS[args.workload]
+    batch = inputs.make_batch(cfg, dev, poison=False)
+    sh = binding.shape_of(batch)
+    lens, table = batch.context_lens.cpu(), batch.block_table.cpu()
+    order = torch.argsort(lens, descending=True)[: args.move_seqs].tolist()
+    bs = cfg.block_size
+    ids = torch.cat([table[b, : (int(lens[b]) + bs - 1) // bs] for b in order]).contiguous()
+    n = ids.numel()
+    block_bytes = 2 * cfg.num_kv_heads * bs * cfg.head_dim * 2             # K + V words of one block
+    moved = n * block_bytes
+    R = max(2, min(8, -(-(1 << 30) // moved)))
+    gen = torch.Generator().manual_seed(cfg.seed + 9)
+    dst_ids = [torch.randperm(batch.num_blocks, generator=gen)[:n].to(torch.int32).to(dev) for _ in range(R)]
+    ids_d = ids.to(dev)
+    words = n * cfg.num_kv_heads * bs * cfg.head_dim
+    packs = [(torch.empty(words, dtype=torch.bfloat16, device=dev), torch.empty(words, dtype=torch.bfloat16, device=dev))
+             for _ in range(R)]
+    pool2 = (torch.empty_like(batch.k_cache), torch.empty_like(batch.v_cache))
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def gather(i):
+        binding.kv_gather_blocks(sh, batch.k_cache, batch.v_cache, ids_d, *packs[i % R], status, stream)
+
+    def scatter(i):
+        binding.kv_scatter_blocks(sh, *packs[i % R], dst_ids[i % R], *pool2, status, stream)
+
+    def timed(fn, steps):
+        for i in range(args.warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t0 = time.perf_counter()
+    ms_g = timed(gather, args.steps)
+    ms_s = timed(scatter, args.steps)
+    ms_both = timed(lambda i: (gather(i), scatter(i)), args.steps)
+    t1 = time.perf_counter()
+    sampler.stop()
+    assert int(status.item()) == 0
+    peak, peak_kind = measured_peak()
+    gbs = lambda ms: 2 * moved / (ms * 1e-3) / 1e9                          # bytes read + bytes written
+    line = {
+        "metric": "paged KV block movement GB/s (read + written)", "value": gbs(ms_both / 2), "unit": "GB/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_both, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: migrate the {len(order)} longest sequences", "blocks": n,
+                   "bytes_moved": moved, "step": "ooco_kv_gather_blocks then ooco_kv_scatter_blocks",
+                   "l2": f"inputs larger than L2: {R} packed buffers / destination lists rotated"},
+        "kernel_ms": {"gather": ms_g, "scatter": ms_s, "gather_then_scatter": ms_both},
+        "roofline": {"bound": "hbm", "achieved": gbs(ms_g), "peak": peak, "unit": "GB/s", "frac": gbs(ms_g) / peak,
+                     "peak_kind": f"of {peak_kind}", "kernel": "block_copy_kernel (gather)",
+                     "algorithmic_bytes_per_launch": 2 * moved, "traffic": None,
+                     "scatter": {"achieved": gbs(ms_s), "frac": gbs(ms_s) / peak}},
+        "gpu_launches": 2 * args.steps, "clocks": sampler.summary(t0, t1),
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -372,8 +453,17 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--ref-token-heads", type=int, default=400000,
                     help="reference arm: (tokens x q heads) of oracle work per step")
+    ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate"],
+                    help="decode_step: the decode hot path (default); kv_migrate: paged block gather + scatter")
+    ap.add_argument("--move-seqs", type=int, default=64, help="kv_migrate: sequences whose blocks are moved")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
+    if args.op == "kv_migrate":
+        if rank == 0:
+            args.steps = args.steps if args.steps is not None else 200
+            args.warmup = max(3, args.warmup if args.warmup is not None else 10)
+            run_block_moves(args, rank, local_rank, world)
+        return
     if args.impl == "reference":
         args.steps = args.steps if args.steps is not None else 5
         args.warmup = args.warmup if args.warmup is not None else 1
