@@ -19,9 +19,13 @@ def _built():
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "ooco.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(ooco_[a-z_0-9]+)\s*\(", text)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        if fn.endswith(".h"):
+            text = re.sub(r"/\*.*?\*/", "", open(os.path.join(inc, fn)).read(), flags=re.S)
+            names |= set(re.findall(r"\b(ooco_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported():
@@ -30,7 +34,8 @@ def test_every_declared_symbol_is_exported():
     L = binding.lib()
     for n in names:
         assert hasattr(L, n), n
-    assert set(names) == set(binding.EXPORTS)
+    from paper_2511_21862_b200 import sched
+    assert set(names) == set(binding.EXPORTS) | set(sched.SCHED_EXPORTS)
     assert L.ooco_version() == 1
     assert binding.status_string(0) == "ok" and "unknown" in binding.status_string(-99)
 
