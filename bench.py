@@ -441,6 +441,70 @@ def run_block_moves(args, rank, local_rank, world):
     print(json.dumps(line))
 
 
+def run_model_fit(args, local_rank):
+    """Secondary measurement: the attention term of the Roofline latency model against this kernel.
+
+    Profiling set: decode steps on reduced copies of the workloads (fewer sequences, shorter contexts).
+    ooco_fit_bandwidth turns (model bytes, measured seconds) into the achievable bandwidth M_a and a
+    static overhead; the fitted line then predicts the four full-size workloads, whose measured step
+    times give the prediction error (the paper reports about 5 % for its whole-model predictor)."""
+    from paper_2511_21862_b200 import binding, build, sched
+    build.build()
+    binding.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream()
+
+    def measure(cfg, steps):
+        batch = inputs.make_batch(cfg, dev, poison=False)
+        sh = binding.shape_of(batch)
+        cost = binding.decode_bytes_model(sh, batch.context_lens.cpu().contiguous())
+        pool_bytes = 2 * batch.k_cache.numel() * 2
+        free, _ = torch.cuda.mem_get_info(dev)
+        R = replica_count(pool_bytes, free)
+        pools = [(batch.k_cache, batch.v_cache)] + [(batch.k_cache.clone(), batch.v_cache.clone()) for _ in range(R - 1)]
+        ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device=dev)
+        out = torch.empty_like(batch.q)
+        lens1 = (batch.context_lens + 1).contiguous()
+
+        def step(i):
+            k, v = pools[i % R]
+            binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, k, v, batch.block_table, batch.context_lens,
+                                lens1, cfg.scale, out, ws, stream)
+        for i in range(max(3, args.warmup)):
+            step(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            step(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        assert binding.workspace_status(ws) == 0
+        return cost, e0.elapsed_time(e1) / steps * 1e-3
+
+    train, test = [], []
+    for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+        base = inputs.CONFIGS[name]
+        for bdiv, ldiv in ((4, 4), (2, 2), (4, 1)):
+            cfg = inputs.scaled_config(base, batch_div=bdiv, len_div=ldiv)
+            cost, sec = measure(cfg, 200)
+            train.append({"workload": cfg.name, "bytes": cost["bytes_paper"], "tokens": cost["total_tokens"], "seconds": sec})
+    M_a, O = sched.fit_bandwidth([r["bytes"] for r in train], [r["seconds"] for r in train])
+    errs = []
+    for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+        cost, sec = measure(inputs.CONFIGS[name], 100 if name in ("cfg2", "cfg4") else 400)
+        pred = O + cost["bytes_paper"] / M_a
+        errs.append(abs(pred - sec) / sec)
+        test.append({"workload": name, "bytes": cost["bytes_paper"], "tokens": cost["total_tokens"], "seconds": sec,
+                     "predicted": pred, "abs_rel_err": errs[-1]})
+    line = {"metric": "Roofline attention-latency model: mean abs relative error on the full workloads",
+            "value": sum(errs) / len(errs), "unit": "fraction", "higher_is_better": False, "n_gpus": 1,
+            "M_a_GBps": M_a / 1e9, "overhead_us": O * 1e6, "profiling_set": train, "validation": test,
+            "data": "synthetic", "dtype": "bf16"}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -453,11 +517,17 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--ref-token-heads", type=int, default=400000,
                     help="reference arm: (tokens x q heads) of oracle work per step")
-    ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate"],
-                    help="decode_step: the decode hot path (default); kv_migrate: paged block gather + scatter")
+    ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate", "model_fit"],
+                    help="decode_step: the decode hot path (default); kv_migrate: paged block gather + scatter; "
+                         "model_fit: fit and validate the attention term of the latency model")
     ap.add_argument("--move-seqs", type=int, default=64, help="kv_migrate: sequences whose blocks are moved")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
+    if args.op == "model_fit":
+        if rank == 0:
+            args.warmup = args.warmup if args.warmup is not None else 5
+            run_model_fit(args, local_rank)
+        return
     if args.op == "kv_migrate":
         if rank == 0:
             args.steps = args.steps if args.steps is not None else 200
