@@ -19,8 +19,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}};
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
 static thread_local int tl_last_launches = 0;
@@ -279,6 +279,47 @@ static int static_scratch_ptr(void** ptr_out) {
 }
 
 static int current_device(int* dev) { return cudaGetDevice(dev) == cudaSuccess ? OOCO_OK : OOCO_E_CUDA; }
+
+// Host -> device staging of a step's small inputs in ONE launch: the kernel reads page-locked host
+// buffers through their device mapping (16-byte loads over the host link) instead of one copy-engine
+// transfer per buffer, each of which costs several microseconds of fixed latency.
+constexpr int kStageBuffers = 6;
+struct HostStageParams {
+  const uint8_t* src[kStageBuffers];  // device-visible addresses of page-locked host buffers
+  uint8_t* dst[kStageBuffers];        // 256-byte aligned device buffers
+  uint32_t bytes[kStageBuffers];      // multiples of 4
+};
+__global__ void __launch_bounds__(256) host_stage_kernel(const HostStageParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
+  const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nthr = gridDim.x * blockDim.x;
+#pragma unroll 1
+  for (int k = 0; k < kStageBuffers; ++k) {
+    const uint32_t n = p.bytes[k];
+    if (((uintptr_t)p.src[k] & 15) == 0) {
+      const uint32_t n16 = n / 16;
+      for (uint32_t i = tid; i < n16; i += nthr)
+        reinterpret_cast<uint4*>(p.dst[k])[i] = reinterpret_cast<const uint4*>(p.src[k])[i];
+      for (uint32_t i = n16 * 4 + tid; i < n / 4; i += nthr)
+        reinterpret_cast<uint32_t*>(p.dst[k])[i] = reinterpret_cast<const uint32_t*>(p.src[k])[i];
+    } else {
+      for (uint32_t i = tid; i < n / 4; i += nthr)
+        reinterpret_cast<uint32_t*>(p.dst[k])[i] = reinterpret_cast<const uint32_t*>(p.src[k])[i];
+    }
+  }
+}
+
+// Device-visible address of a page-locked (pinned / registered) host buffer on the current device,
+// or nullptr when `host` is ordinary pageable memory (which a kernel must never be given).
+static void* mapped_host_pointer(const void* host) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  if (a.type != cudaMemoryTypeHost || !a.devicePointer) return nullptr;
+  return a.devicePointer;
+}
 
 // Largest contiguous run of a side: 0 = whole block, 1 = one kv head of a block, 2 = one token row.
 static int run_level(int64_t hstr, int64_t tstr, int bs, int D) {
@@ -684,20 +725,47 @@ int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void*
   uint8_t* d_tab = d_vn + up(kb);
   uint8_t* d_pos = d_tab + up(tb);
   uint8_t* d_len = d_pos + up(lb);
-  bool ok = true;
-  ok &= cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_kn, k_new_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_vn, v_new_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_tab, block_table_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_pos, positions_host, lb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_len, context_lens_host, lb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (!ok) return OOCO_E_CUDA;
+  const void* hsrc[kStageBuffers] = {q_host, k_new_host, v_new_host, block_table_host, positions_host,
+                                     context_lens_host};
+  uint8_t* ddst[kStageBuffers] = {d_q, d_kn, d_vn, d_tab, d_pos, d_len};
+  const size_t nbytes[kStageBuffers] = {qb, kb, kb, tb, lb, lb};
+  // Page-locked inputs (all six, each under 4 GiB): one staging kernel reads them through their device
+  // mapping.  Otherwise one copy per buffer.
+  HostStageParams hp;
+  bool mapped = g_knobs[kKnobHostStageKernel].load() != 0;
+  for (int k = 0; k < kStageBuffers && mapped; ++k) {
+    hp.src[k] = (const uint8_t*)mapped_host_pointer(hsrc[k]);
+    hp.dst[k] = ddst[k];
+    hp.bytes[k] = (uint32_t)nbytes[k];
+    mapped = hp.src[k] != nullptr && nbytes[k] < ((size_t)1 << 32) && ((uintptr_t)hp.src[k] & 3) == 0;
+  }
+  int launches = 0;
+  if (mapped) {
+    size_t total = 0;
+    for (int k = 0; k < kStageBuffers; ++k) total += nbytes[k];
+    int blocks = (int)((total / 16 + 255) / 256);
+    blocks = blocks < 1 ? 1 : (blocks > 592 ? 592 : blocks);
+    cudaError_t e = launch_ex(host_stage_kernel, dim3(blocks), dim3(256), 0, st, g_knobs[kKnobPdl].load() != 0, hp);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) return fail_cuda("launch of the host staging kernel", (long)e);
+    launches = 1;
+  } else {
+    bool ok = true;
+    for (int k = 0; k < kStageBuffers; ++k)
+      ok &= cudaMemcpyAsync(ddst[k], hsrc[k], nbytes[k], cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) return fail_cuda("cudaMemcpyAsync(host to device)", -1);
+  }
+  // A page-locked result buffer is written by the kernels themselves, through its device mapping.
+  void* out_mapped = g_knobs[kKnobHostStageKernel].load() != 0 ? mapped_host_pointer(out_host) : nullptr;
+  if (out_mapped && ((uintptr_t)out_mapped & 15)) out_mapped = nullptr;
   if ((rc = ooco_decode_step(s, d_q, d_kn, d_vn, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_pos,
-                             (const int32_t*)d_len, scale, d_out, workspace, workspace_bytes, st)))
+                             (const int32_t*)d_len, scale, out_mapped ? out_mapped : (void*)d_out, workspace,
+                             workspace_bytes, st)))
     return rc;
-  if (cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return OOCO_E_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return OOCO_E_CUDA;
-  tl_last_launches = 3;
+  if (!out_mapped && cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return fail_cuda("cudaMemcpyAsync(device to host)", -1);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return fail_cuda("cudaStreamSynchronize", -1);
+  tl_last_launches += launches;
   return OOCO_OK;
 }
 

@@ -161,15 +161,18 @@ def test_kv_append_skips_bad_positions():
     assert np.array_equal(inputs.as_u16(batch.k_cache), k_ref) and np.array_equal(inputs.as_u16(batch.v_cache), v_ref)
 
 
-def test_serving_step_from_host_buffers():
-    """append at T then attend T + 1 through the host-buffer entry point."""
-    cfg = C("step", 32, 8, 128, 16, (G(9, 1, 700),), seed=50, pool_fill=0.8)
+@pytest.mark.parametrize("pinned,launches", [(True, 4), (False, 3)], ids=["page-locked", "pageable"])
+def test_serving_step_from_host_buffers(pinned, launches):
+    """append at T then attend T + 1 through the host-buffer entry point: page-locked buffers are read
+    by one staging kernel and the result is written to the host directly; pageable ones are copied."""
+    cfg = C("step", 32, 8, 128, 16, (G(9, 1, 2500),), seed=50, pool_fill=0.8)
     batch = inputs.make_batch(cfg, "cuda", poison=True)
     sh = binding.shape_of(batch)
-    pin = lambda t: t.cpu().contiguous().pin_memory()
+    pin = (lambda t: t.cpu().contiguous().pin_memory()) if pinned else (lambda t: t.cpu().contiguous().clone())
     pos = pin(batch.context_lens)
     lens1 = pin(batch.context_lens + 1)
-    out_h = torch.empty(batch.q.shape, dtype=torch.bfloat16).pin_memory()
+    out_h = torch.full(batch.q.shape, float("nan"), dtype=torch.bfloat16)
+    out_h = out_h.pin_memory() if pinned else out_h
     ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device="cuda")
     stg = torch.empty(binding.step_staging_bytes(sh), dtype=torch.uint8, device="cuda")
     k_ref, v_ref = inputs.as_u16(batch.k_cache).copy(), inputs.as_u16(batch.v_cache).copy()
@@ -182,7 +185,7 @@ def test_serving_step_from_host_buffers():
     ref = oracle.decode_attention(inputs.as_u16(batch.q), k_ref, v_ref, batch.block_table.cpu().numpy(),
                                   lens1.numpy(), cfg.scale, num_kv_heads=8, block_size=16, strides=batch.strides)
     assert_parity(out_h, ref.out, what="host step")
-    assert binding.last_launch_count() == 3
+    assert binding.last_launch_count() == launches
 
 
 def test_fused_step_on_device_buffers():
