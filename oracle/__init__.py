@@ -15,17 +15,17 @@ from dataclasses import dataclass
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "ooco_oracle.c")
+_SRCS = [os.path.join(_HERE, "ooco_oracle.c"), os.path.join(_HERE, "ooco_oracle_fp8.c")]
 _LIB_PATH = os.path.join(_HERE, "libooco_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile ooco_oracle.c with gcc (OpenMP, no fast-math) next to its source."""
-    stale = (not os.path.exists(_LIB_PATH)) or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC)
+    stale = (not os.path.exists(_LIB_PATH)) or any(os.path.getmtime(_LIB_PATH) < os.path.getmtime(s) for s in _SRCS)
     if force or stale:
         cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fno-fast-math", "-shared", "-fPIC",
-               "-o", _LIB_PATH, _SRC, "-lm"]
+               "-o", _LIB_PATH] + _SRCS + ["-lm"]
         subprocess.run(cmd, check=True)
     return _LIB_PATH
 
@@ -42,6 +42,15 @@ def _load():
         lib.oracle_bytes_model.restype = ctypes.c_int
         lib.oracle_bytes_model.argtypes = [i32] * 5 + [vp, i32, vp]
         lib.oracle_num_threads.restype = ctypes.c_int
+        f32, u8 = ctypes.c_float, ctypes.c_uint8
+        lib.oracle_e4m3_decode.restype = f64
+        lib.oracle_e4m3_decode.argtypes = [u8]
+        lib.oracle_e4m3_encode.restype = u8
+        lib.oracle_e4m3_encode.argtypes = [f32]
+        lib.oracle_decode_attention_fp8.restype = ctypes.c_int
+        lib.oracle_decode_attention_fp8.argtypes = [i32] * 7 + [i64] * 3 + [vp] * 5 + [f64, f32, f32, vp, i64, vp, vp, vp]
+        lib.oracle_kv_append_fp8.restype = i64
+        lib.oracle_kv_append_fp8.argtypes = [i32] * 6 + [i64] * 3 + [vp] * 6 + [f32, f32]
         _lib = lib
     return _lib
 
@@ -122,6 +131,72 @@ def kv_append(k_new, v_new, k_cache, v_cache, block_table, positions, *, block_s
     return int(lib.oracle_kv_append(B, Hkv, D, block_size, num_blocks, MB, bstr, hstr, tstr,
                                     _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
                                     _ptr(block_table), _ptr(positions)))
+
+
+# --------------------------------------------------------------------------- 8-bit (E4M3) KV cache
+def e4m3_decode(codes) -> np.ndarray:
+    """float64 values of E4M3 codes (uint8), from the format's definition."""
+    lib = _load()
+    codes = np.asarray(codes, dtype=np.uint8)
+    return np.array([lib.oracle_e4m3_decode(int(c)) for c in codes.reshape(-1)], dtype=np.float64).reshape(codes.shape)
+
+
+def e4m3_encode(values) -> np.ndarray:
+    """Nearest-even, saturating E4M3 codes of float32 values."""
+    lib = _load()
+    values = np.asarray(values, dtype=np.float32)
+    return np.array([lib.oracle_e4m3_encode(float(x)) for x in values.reshape(-1)], dtype=np.uint8).reshape(values.shape)
+
+
+def _u8(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint8, a.dtype
+    return a
+
+
+def decode_attention_fp8(q, k_cache, v_cache, block_table, context_lens, scale, k_scale, v_scale, *, num_kv_heads,
+                         block_size, strides, pairs=None) -> AttentionResult:
+    """decode_attention over uint8 E4M3 pools; a stored code stands for decode(code) * k_scale (v_scale)."""
+    lib = _load()
+    q = _u16(q)
+    B, Hq, D = q.shape
+    k_cache, v_cache = _u8(k_cache), _u8(v_cache)
+    block_table, context_lens = _i32(block_table), _i32(context_lens)
+    MB = block_table.shape[1]
+    bstr, hstr, tstr = (int(s) for s in strides)
+    num_blocks = k_cache.size // bstr
+    out = np.full((B, Hq, D), np.nan, dtype=np.float64)
+    lse = np.full((B, Hq), np.nan, dtype=np.float64)
+    wsum = np.full((B, Hq), np.nan, dtype=np.float64)
+    if pairs is not None:
+        pairs = _i32(pairs).reshape(-1, 2)
+        pp, npairs = _ptr(pairs), pairs.shape[0]
+    else:
+        pp, npairs = None, 0
+    rc = lib.oracle_decode_attention_fp8(B, Hq, num_kv_heads, D, block_size, num_blocks, MB, bstr, hstr, tstr,
+                                         _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+                                         _ptr(context_lens), float(scale), float(k_scale), float(v_scale), pp,
+                                         npairs, _ptr(out), _ptr(lse), _ptr(wsum))
+    if rc != 0:
+        raise ValueError(f"oracle_decode_attention_fp8 failed with {rc}")
+    return AttentionResult(out, lse, wsum)
+
+
+def kv_append_fp8(k_new, v_new, k_cache, v_cache, block_table, positions, k_scale, v_scale, *, block_size,
+                  strides) -> int:
+    """In-place quantising append of bf16 rows (uint16 bits) into uint8 E4M3 pools."""
+    lib = _load()
+    k_new, v_new = _u16(k_new), _u16(v_new)
+    B, Hkv, D = k_new.shape
+    assert k_cache.dtype == np.uint8 and v_cache.dtype == np.uint8
+    assert k_cache.flags.c_contiguous and v_cache.flags.c_contiguous and k_cache.flags.writeable
+    block_table, positions = _i32(block_table), _i32(positions)
+    MB = block_table.shape[1]
+    bstr, hstr, tstr = (int(s) for s in strides)
+    num_blocks = k_cache.size // bstr
+    return int(lib.oracle_kv_append_fp8(B, Hkv, D, block_size, num_blocks, MB, bstr, hstr, tstr, _ptr(k_new),
+                                        _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+                                        _ptr(positions), float(k_scale), float(v_scale)))
 
 
 COST_FIELDS = ("flops", "bytes_q", "bytes_out", "bytes_kv", "bytes_index", "bytes_paper", "total_tokens")
