@@ -168,6 +168,35 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The same three operations over an 8-bit KV cache (the operator model's d, "byte per value", set
+ * to 1 for K and V: Table "Symbol definitions"; decode attention is memory-bound, section 3.3.3, so
+ * halving the stored bytes halves its time).  k_cache / v_cache hold OCP E4M3 codes (1 sign, 4
+ * exponent bits with bias 7, 3 mantissa bits, no infinities, S.1111.111 = NaN, largest finite 448),
+ * one byte per value, same four-index layout with the strides of `shape` counted in bytes; a code
+ * stands for decode(code) * k_scale (v_scale), one positive fp32 scale per tensor.  q, k_new,
+ * v_new and out stay bf16.
+ *   ooco_kv_append_fp8        stores e4m3(x / scale) for every new value x: one fp32 division,
+ *                             round to nearest even, magnitudes beyond 448 saturate to 448.
+ *   ooco_decode_attention_fp8 attention as ooco_decode_attention with K = decode(code) * k_scale,
+ *                             V = decode(code) * v_scale; codes are widened exactly to f16, q and
+ *                             the softmax weights are rounded to f16, accumulation is fp32.
+ *   ooco_decode_step_fp8      the fused append + attention step, as ooco_decode_step.
+ * Restrictions beyond ooco_shape_t's: head_dim = 128, strides multiples of 16 bytes.  Workspace,
+ * status word, launches, ownership and errors as for the bf16 entry points.
+ */
+int ooco_kv_append_fp8(const ooco_shape_t* shape, const void* k_new, const void* v_new, void* k_cache,
+                       void* v_cache, const int32_t* block_table, const int32_t* positions, float k_scale,
+                       float v_scale, void* cuda_stream);
+int ooco_decode_attention_fp8(const ooco_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* block_table, const int32_t* context_lens, float scale,
+                              float k_scale, float v_scale, void* out, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream);
+int ooco_decode_step_fp8(const ooco_shape_t* shape, const void* q, const void* k_new, const void* v_new,
+                         void* k_cache, void* v_cache, const int32_t* block_table, const int32_t* positions,
+                         const int32_t* context_lens, float scale, float k_scale, float v_scale, void* out,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Paged decode attention for callers that cannot allocate device memory.  (The paper has no
  * counterpart; this is a packaging variant of ooco_decode_attention.)
  *

@@ -21,6 +21,7 @@ EXPORTS = (
     "ooco_last_launch_count", "ooco_last_error_detail", "ooco_set_tuning", "ooco_status_string", "ooco_version",
     "ooco_profile_enable", "ooco_profile_read", "ooco_decode_attention_static",
     "ooco_kv_gather_blocks", "ooco_kv_scatter_blocks", "ooco_kv_copy_blocks",
+    "ooco_kv_append_fp8", "ooco_decode_attention_fp8", "ooco_decode_step_fp8",
 )
 
 
@@ -68,6 +69,14 @@ def lib() -> ctypes.CDLL:
                                        ctypes.c_size_t, vp]
         L.ooco_decode_attention_static.restype = ctypes.c_int
         L.ooco_decode_attention_static.argtypes = [sp, vp, vp, vp, i32p, i32p, ctypes.c_float, vp, vp]
+        f32 = ctypes.c_float
+        L.ooco_kv_append_fp8.restype = ctypes.c_int
+        L.ooco_kv_append_fp8.argtypes = [sp, vp, vp, vp, vp, i32p, i32p, f32, f32, vp]
+        L.ooco_decode_attention_fp8.restype = ctypes.c_int
+        L.ooco_decode_attention_fp8.argtypes = [sp, vp, vp, vp, i32p, i32p, f32, f32, f32, vp, vp, ctypes.c_size_t, vp]
+        L.ooco_decode_step_fp8.restype = ctypes.c_int
+        L.ooco_decode_step_fp8.argtypes = [sp, vp, vp, vp, vp, vp, i32p, i32p, i32p, f32, f32, f32, vp, vp,
+                                           ctypes.c_size_t, vp]
         L.ooco_kv_gather_blocks.restype = ctypes.c_int
         L.ooco_kv_gather_blocks.argtypes = [sp, vp, vp, i32p, ctypes.c_int32, vp, vp, i32p, vp]
         L.ooco_kv_scatter_blocks.restype = ctypes.c_int
@@ -186,6 +195,36 @@ def decode_step(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table, po
         _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32),
         _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), _dev(out, torch.bfloat16),
         _dev(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step")
+
+
+def kv_append_fp8(shape: Shape, k_new, v_new, k_cache, v_cache, block_table, positions, k_scale, v_scale,
+                  stream=None):
+    """Quantising append into uint8 (E4M3) caches."""
+    _check(lib().ooco_kv_append_fp8(
+        ctypes.byref(shape.c()), _dev(k_new, torch.bfloat16), _dev(v_new, torch.bfloat16),
+        _dev(k_cache, torch.uint8), _dev(v_cache, torch.uint8), _dev(block_table, torch.int32),
+        _dev(positions, torch.int32), float(k_scale), float(v_scale), _stream_ptr(stream)), "ooco_kv_append_fp8")
+
+
+def decode_attention_fp8(shape: Shape, q, k_cache, v_cache, block_table, context_lens, scale, k_scale, v_scale, out,
+                         workspace, stream=None):
+    """Decode attention over uint8 (E4M3) caches; q / out bf16."""
+    _check(lib().ooco_decode_attention_fp8(
+        ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_cache, torch.uint8), _dev(v_cache, torch.uint8),
+        _dev(block_table, torch.int32), _dev(context_lens, torch.int32), float(scale), float(k_scale),
+        float(v_scale), _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        _stream_ptr(stream)), "ooco_decode_attention_fp8")
+
+
+def decode_step_fp8(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table, positions, context_lens, scale,
+                    k_scale, v_scale, out, workspace, stream=None):
+    """Fused quantising append + attention over uint8 (E4M3) caches."""
+    _check(lib().ooco_decode_step_fp8(
+        ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_new, torch.bfloat16), _dev(v_new, torch.bfloat16),
+        _dev(k_cache, torch.uint8), _dev(v_cache, torch.uint8), _dev(block_table, torch.int32),
+        _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), float(k_scale), float(v_scale),
+        _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        _stream_ptr(stream)), "ooco_decode_step_fp8")
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

@@ -11,6 +11,8 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -48,7 +50,8 @@ struct DecodeParams {
   int32_t nstages;
   int32_t grid_main;      // CTAs of the attention kernel (first items are assigned statically)
   int32_t chunk_min, chunk_max, items_per_cta;
-  float scale_log2e;
+  float scale_log2e;        // softmax scale * log2(e) (* the K tensor scale of an 8-bit cache)
+  float v_scale;            // V tensor scale of an 8-bit cache (1 for bf16)
 };
 
 // ------------------------------------------------------------------------------------ append
@@ -61,7 +64,25 @@ struct AppendParams {
   const int32_t* positions;
   int32_t B, Hkv, D, bs, NB, MB;
   int64_t bstr, hstr, tstr;
+  int32_t kv8;              // 1: the caches hold 8-bit E4M3 codes (k_cache / v_cache are byte arrays)
+  float k_scale, v_scale;   // tensor scales of an 8-bit cache: stored code = e4m3(x / scale)
 };
+
+// Eight bf16 values -> eight E4M3 codes: one IEEE fp32 division by the tensor scale, then round to
+// nearest even, saturating at the largest finite code.
+__device__ __forceinline__ uint2 quantize_e4m3x8(const uint4 w, float scale) {
+  const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+  uint32_t out[2] = {0u, 0u};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float lo = __fdiv_rn(__uint_as_float(in[i] << 16), scale);
+    const float hi = __fdiv_rn(__uint_as_float(in[i] & 0xffff0000u), scale);
+    const uint32_t c = (uint32_t)__nv_cvt_float_to_fp8(lo, __NV_SATFINITE, __NV_E4M3) |
+                       ((uint32_t)__nv_cvt_float_to_fp8(hi, __NV_SATFINITE, __NV_E4M3) << 8);
+    out[i >> 1] |= c << (16 * (i & 1));
+  }
+  return make_uint2(out[0], out[1]);
+}
 
 // Copies the new K / V rows into their slots, one thread per 16-byte vector; `block` of
 // `nblocks` CTAs cooperate grid-stride.
@@ -77,8 +98,13 @@ __device__ __forceinline__ void kv_append_body(const AppendParams& a, int block,
     const int blk = a.block_table[(size_t)b * a.MB + pos / a.bs];
     if (blk < 0 || blk >= a.NB) continue;
     const int64_t dst = (int64_t)blk * a.bstr + (int64_t)h * a.hstr + (int64_t)(pos % a.bs) * a.tstr + 8 * v;
-    *reinterpret_cast<uint4*>(a.k_cache + dst) = a.k_new[i];
-    *reinterpret_cast<uint4*>(a.v_cache + dst) = a.v_new[i];
+    if (a.kv8) {
+      *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(a.k_cache) + dst) = quantize_e4m3x8(a.k_new[i], a.k_scale);
+      *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(a.v_cache) + dst) = quantize_e4m3x8(a.v_new[i], a.v_scale);
+    } else {
+      *reinterpret_cast<uint4*>(a.k_cache + dst) = a.k_new[i];
+      *reinterpret_cast<uint4*>(a.v_cache + dst) = a.v_new[i];
+    }
   }
 }
 
@@ -263,10 +289,10 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
 // ------------------------------------------------------------------------------------ main
 // Shared-memory carve-up, shared by host (sizing) and device.  TPW = 16-token tiles each
 // consumer warp owns per stage.
-template <int D, int NCW, int NT, int TPW>
+template <int D, int NCW, int NT, int TPW, bool KV8 = false>
 struct SmemLayout {
   static constexpr int kStageTok = 16 * NCW * TPW;
-  static constexpr int kTileBytes = kStageTok * D * 2;      // K (or V) bytes of one stage
+  static constexpr int kTileBytes = kStageTok * D * (KV8 ? 1 : 2);  // K (or V) bytes of one stage
   static constexpr int kStageBytes = 2 * kTileBytes;
   static constexpr int kHeads = NT * 8;
   static constexpr int kOStride = 64 + 4;                    // floats per head row of one 64-dim pass
@@ -390,11 +416,122 @@ __device__ __forceinline__ void consume_tiles(uint32_t kst, uint32_t vst, const 
   }
 }
 
-template <int D, int NCW, int NT, int TPW>
+// ---- 8-bit (E4M3) cache: one consumer warp's work on its 16-token tile of a stage.
+// A token row is D = 128 bytes.  The codes are widened to f16 in registers (exact) and both
+// contractions run as f16 MMAs; the tensor scales are applied outside (K's is folded into the softmax
+// scale, V's multiplies the output).  Fragment bookkeeping:
+//   scores  ldmatrix (16-bit units) hands lane (g, t) the four codes of dims 4t .. 4t+3 of a 16-dim
+//           chunk; they fill the MMA's k slots (2t, 2t+1) and (2t+8, 2t+9).  The contraction does not
+//           care about the order of k as long as Q uses the same one (it does: see the q fragments).
+//   values  ldmatrix.trans hands lane (g, t) dims (2g, 2g+1) of tokens (2t, 2t+1); a byte permute
+//           regroups them per dim, so MMA row g is dim 2g and row g + 8 is dim 2g + 1 of the chunk
+//           (the epilogue writes the accumulators back in that order).
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
+  const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(two_codes & 0xffffu), __NV_E4M3);
+  return (uint32_t)h.x | ((uint32_t)h.y << 16);
+}
+__device__ __forceinline__ float f16_lo(uint32_t x) { return __half2float(__ushort_as_half((unsigned short)(x & 0xffffu))); }
+__device__ __forceinline__ float f16_hi(uint32_t x) { return __half2float(__ushort_as_half((unsigned short)(x >> 16))); }
+
+template <int D, int NT, bool kTail>
+__device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uint32_t tile_off,
+                                                 const uint32_t (&pat)[D / 16], const uint32_t (&qf)[NT][D / 16][2],
+                                                 float (&m_run)[NT][2], float (&l_run)[NT][2],
+                                                 float (&o_acc)[NT][D / 16][4], float scale_log2e, int valid,
+                                                 int g, int t) {
+  constexpr int KS = D / 16;  // 16-dim chunks
+  float sc[NT][2][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sc[nt][a][e] = 0.f;
+#pragma unroll
+  for (int j = 0; j < KS / 2; ++j) {
+    uint32_t r0, r1, r2, r3;  // (tokens 0-7, chunk 2j) (tokens 8-15, 2j) (tokens 0-7, 2j+1) (tokens 8-15, 2j+1)
+    ldmatrix_x4(kst + tile_off + pat[j], r0, r1, r2, r3);
+    const uint32_t a0 = e4m3x2_to_f16x2(r0), a2 = e4m3x2_to_f16x2(r0 >> 16);
+    const uint32_t a1 = e4m3x2_to_f16x2(r1), a3 = e4m3x2_to_f16x2(r1 >> 16);
+    const uint32_t c0 = e4m3x2_to_f16x2(r2), c2 = e4m3x2_to_f16x2(r2 >> 16);
+    const uint32_t c1 = e4m3x2_to_f16x2(r3), c3 = e4m3x2_to_f16x2(r3 >> 16);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      mma_f16(sc[nt][0], a0, a1, a2, a3, qf[nt][2 * j][0], qf[nt][2 * j][1]);
+      mma_f16(sc[nt][1], c0, c1, c2, c3, qf[nt][2 * j + 1][0], qf[nt][2 * j + 1][1]);
+    }
+  }
+  uint32_t pb[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    float s[4];  // (token g, head 2t) (token g, head 2t+1) (token g+8, 2t) (token g+8, 2t+1)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) s[e] = (sc[nt][0][e] + sc[nt][1][e]) * scale_log2e;
+    if (kTail) {
+      if (g >= valid) s[0] = s[1] = -INFINITY;
+      if (g + 8 >= valid) s[2] = s[3] = -INFINITY;
+    }
+    float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+    }
+    const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
+    const float al0 = ex2(m_run[nt][0] - mn0), al1 = ex2(m_run[nt][1] - mn1);
+    m_run[nt][0] = mn0;
+    m_run[nt][1] = mn1;
+    const uint32_t p01 = pack_f16x2(ex2(s[0] - mn0), ex2(s[1] - mn1));  // token g
+    const uint32_t p23 = pack_f16x2(ex2(s[2] - mn0), ex2(s[3] - mn1));  // token g+8
+    // sums use the rounded weights, so numerator and denominator agree exactly
+    l_run[nt][0] = l_run[nt][0] * al0 + f16_lo(p01) + f16_lo(p23);
+    l_run[nt][1] = l_run[nt][1] * al1 + f16_hi(p01) + f16_hi(p23);
+    pb[nt][0] = movmatrix_trans(p01);  // tokens 2t,2t+1 of head g
+    pb[nt][1] = movmatrix_trans(p23);  // tokens 2t+8,2t+9 of head g
+    if (__any_sync(0xffffffffu, (al0 != 1.f) | (al1 != 1.f))) {
+#pragma unroll
+      for (int k = 0; k < KS; ++k) {
+        o_acc[nt][k][0] *= al0;
+        o_acc[nt][k][1] *= al1;
+        o_acc[nt][k][2] *= al0;
+        o_acc[nt][k][3] *= al1;
+      }
+    }
+  }
+  uint32_t mk01 = 0xffffffffu, mk23 = 0xffffffffu;
+  if (kTail) {
+    mk01 = (2 * t < valid ? 0x0000ffffu : 0u) | (2 * t + 1 < valid ? 0xffff0000u : 0u);
+    mk23 = (2 * t + 8 < valid ? 0x0000ffffu : 0u) | (2 * t + 9 < valid ? 0xffff0000u : 0u);
+  }
+#pragma unroll
+  for (int j = 0; j < KS / 2; ++j) {
+    uint32_t r0, r1, r2, r3;  // transposed: lane (g, t) holds dims (2g, 2g+1) x tokens (2t, 2t+1) of each matrix
+    ldmatrix_x4_trans(vst + tile_off + pat[j], r0, r1, r2, r3);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const uint32_t lo = half ? r2 : r0, hi = half ? r3 : r1;  // tokens 0-7 / 8-15 of chunk 2j + half
+      uint32_t a0 = e4m3x2_to_f16x2(__byte_perm(lo, 0, 0x4420));  // dim 2g,   tokens 2t, 2t+1
+      uint32_t a1 = e4m3x2_to_f16x2(__byte_perm(lo, 0, 0x4431));  // dim 2g+1, tokens 2t, 2t+1
+      uint32_t a2 = e4m3x2_to_f16x2(__byte_perm(hi, 0, 0x4420));  // dim 2g,   tokens 2t+8, 2t+9
+      uint32_t a3 = e4m3x2_to_f16x2(__byte_perm(hi, 0, 0x4431));  // dim 2g+1, tokens 2t+8, 2t+9
+      if (kTail) {
+        a0 &= mk01;
+        a1 &= mk01;
+        a2 &= mk23;
+        a3 &= mk23;
+      }
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) mma_f16(o_acc[nt][2 * j + half], a0, a1, a2, a3, pb[nt][0], pb[nt][1]);
+    }
+  }
+}
+
+template <int D, int NCW, int NT, int TPW, bool KV8 = false>
 __global__ void __launch_bounds__((NCW + 1) * 32, 1)
 decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const DecodeParams p) {
-  using L = SmemLayout<D, NCW, NT, TPW>;
+  using L = SmemLayout<D, NCW, NT, TPW, KV8>;
+  static_assert(!KV8 || (D == 128 && TPW == 1), "the 8-bit path is built for head_dim 128, one tile per warp");
   constexpr int kStageTok = L::kStageTok;
   constexpr int KS = D / 16;  // k-steps of the score MMA = m-tiles of the value MMA
   extern __shared__ uint8_t smem_raw[];
@@ -439,7 +576,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       prefetch_tmap(&tm_v);
     }
     const int boxes_per_stage = kStageTok / p.tile_rows;
-    const uint32_t box_bytes = (uint32_t)p.tile_rows * D * 2;
+    const uint32_t box_bytes = (uint32_t)p.tile_rows * D * (KV8 ? 1 : 2);
     int it = 0;
     int item = blockIdx.x;
     int4 d = make_int4(0, 0, 0, 0);
@@ -488,7 +625,10 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           const int c_tok = tb % p.bs;
           const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + lane * box_bytes;
           const uint32_t dv = dk + L::kTileBytes;
-          if (D == 128 && !p.split_halves) {
+          if (KV8) {  // a token row is one 128-byte swizzle row: one 4-d copy per box
+            tma_load_4d(dk, &tm_k, full, 0, c_tok, h, blk_cur);
+            tma_load_4d(dv, &tm_v, full, 0, c_tok, h, blk_cur);
+          } else if (D == 128 && !p.split_halves) {
             tma_load_5d(dk, &tm_k, full, 0, c_tok, 0, h, blk_cur);
             tma_load_5d(dv, &tm_v, full, 0, c_tok, 0, h, blk_cur);
           } else {
@@ -563,10 +703,11 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   // Per-lane byte offsets of the ldmatrix rows inside a stage's K / V tile.  A box holds
   // [D/64 halves][tile_rows][64 dims] with the 128-byte swizzle (16-byte chunk ^= row & 7).
   const int r0 = 16 * TPW * warp;  // first token row of this warp inside a stage
-  const uint32_t box_bytes = (uint32_t)p.tile_rows * D * 2;
+  const uint32_t box_bytes = (uint32_t)p.tile_rows * D * (KV8 ? 1 : 2);
   const uint32_t half_bytes = (uint32_t)p.tile_rows * 128;
   const int lr_k = (lane & 7) + ((lane >> 3) & 1) * 8, cs_k = lane >> 4;
-  const int lr_v = (lane & 7) + (lane >> 4) * 8, cs_v = (lane >> 3) & 1;
+  // 8-bit tiles are read with the K pattern for V too (matrices: tokens 0-7 / 8-15 of chunk c, then c + 1)
+  const int lr_v = KV8 ? lr_k : (lane & 7) + (lane >> 4) * 8, cs_v = KV8 ? cs_k : (lane >> 3) & 1;
   uint32_t tile_k[TPW], tile_v[TPW], kpat[KS], vpat[KS];
 #pragma unroll
   for (int u = 0; u < TPW; ++u) {
@@ -606,9 +747,15 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           o_acc[nt][k][0] = o_acc[nt][k][1] = o_acc[nt][k][2] = o_acc[nt][k][3] = 0.f;
           uint32_t v0 = 0u, v1 = 0u;
           if (head < p.G) {
-            const uint8_t* src = qs + ((size_t)head * D + 16 * k + 2 * t) * 2;
-            v0 = *reinterpret_cast<const uint32_t*>(src);
-            v1 = *reinterpret_cast<const uint32_t*>(src + 16);
+            if (KV8) {  // dims 16k + 4t .. + 3 as two f16 pairs (the k order of the 8-bit score MMA)
+              const uint2 w = *reinterpret_cast<const uint2*>(qs + ((size_t)head * D + 16 * k + 4 * t) * 2);
+              v0 = pack_f16x2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u));
+              v1 = pack_f16x2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xffff0000u));
+            } else {
+              const uint8_t* src = qs + ((size_t)head * D + 16 * k + 2 * t) * 2;
+              v0 = *reinterpret_cast<const uint32_t*>(src);
+              v1 = *reinterpret_cast<const uint32_t*>(src + 16);
+            }
           }
           qf[nt][k][0] = v0;
           qf[nt][k][1] = v1;
@@ -619,7 +766,12 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (valid > 0) {
       const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;
       const uint32_t vst = kst + L::kTileBytes;
-      if (valid >= 16 * TPW)
+      if (KV8) {
+        if (valid >= 16)
+          consume_tile_kv8<D, NT, false>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t);
+        else
+          consume_tile_kv8<D, NT, true>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t);
+      } else if (valid >= 16 * TPW)
         consume_tiles<D, NT, TPW, false>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
                                          p.scale_log2e, valid, g, t);
       else
@@ -669,10 +821,12 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
             const int k = 4 * pass + kk;
-            mo[(size_t)h0 * L::kOStride + 16 * kk + g] = o_acc[nt][k][0];
-            mo[(size_t)(h0 + 1) * L::kOStride + 16 * kk + g] = o_acc[nt][k][1];
-            mo[(size_t)h0 * L::kOStride + 16 * kk + g + 8] = o_acc[nt][k][2];
-            mo[(size_t)(h0 + 1) * L::kOStride + 16 * kk + g + 8] = o_acc[nt][k][3];
+            // accumulator rows g / g + 8 hold dims g / g + 8 of the chunk (bf16) or 2g / 2g + 1 (8-bit)
+            const int d_lo = 16 * kk + (KV8 ? 2 * g : g), d_hi = 16 * kk + (KV8 ? 2 * g + 1 : g + 8);
+            mo[(size_t)h0 * L::kOStride + d_lo] = o_acc[nt][k][0];
+            mo[(size_t)(h0 + 1) * L::kOStride + d_lo] = o_acc[nt][k][1];
+            mo[(size_t)h0 * L::kOStride + d_hi] = o_acc[nt][k][2];
+            mo[(size_t)(h0 + 1) * L::kOStride + d_hi] = o_acc[nt][k][3];
           }
         }
         mbar_arrive(s_mbar);
@@ -693,7 +847,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             den += sw * all_m[(w * L::kHeads + head) * 2 + 1];
             num += sw * g_merge[((size_t)w * L::kHeads + head) * L::kOStride + dl];
           }
-          const float o = num / den;
+          const float o = KV8 ? num / den * p.v_scale : num / den;
           if (n_chunks == 1) {
             p.out[((size_t)b * p.Hq + (size_t)h * p.G + head) * D + dim] = __float2bfloat16_rn(o);
           } else {

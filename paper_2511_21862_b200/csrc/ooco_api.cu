@@ -150,11 +150,27 @@ static int encode_kv_map(CUtensorMap* tm, const ooco_shape_t* s, const void* bas
   return r == CUDA_SUCCESS ? OOCO_OK : fail_cuda(five_d ? "cuTensorMapEncodeTiled(5d)" : "cuTensorMapEncodeTiled(4d)", (long)r);
 }
 
-template <int D, int NCW, int NT, int TPW>
+// 8-bit pool: (128 bytes of a token row, token, head, block), one box = [tile_rows][128 B].
+static int encode_kv8_map(CUtensorMap* tm, const ooco_shape_t* s, const void* base, int tile_rows) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return fail_cuda("cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)", -1);
+  cuuint64_t dims[4] = {(cuuint64_t)s->head_dim, (cuuint64_t)s->block_size, (cuuint64_t)s->num_kv_heads,
+                        (cuuint64_t)s->num_blocks};
+  cuuint64_t strides[3] = {(cuuint64_t)s->kv_token_stride, (cuuint64_t)s->kv_head_stride,
+                           (cuuint64_t)s->kv_block_stride};
+  cuuint32_t box[4] = {(cuuint32_t)s->head_dim, (cuuint32_t)tile_rows, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? OOCO_OK : fail_cuda("cuTensorMapEncodeTiled(8-bit)", (long)r);
+}
+
+template <int D, int NCW, int NT, int TPW, bool KV8 = false>
 static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                        int ctas_per_sm, int want_stages, cudaStream_t st, int dev) {
-  using L = SmemLayout<D, NCW, NT, TPW>;
-  auto kern = decode_main_kernel<D, NCW, NT, TPW>;
+  using L = SmemLayout<D, NCW, NT, TPW, KV8>;
+  auto kern = decode_main_kernel<D, NCW, NT, TPW, KV8>;
   // the opt-in limit covers static + dynamic shared memory of the kernel
   static std::atomic<int> static_smem{-1};
   if (static_smem.load() < 0) {
@@ -189,6 +205,23 @@ static int launch_main_nt(const CUtensorMap& tk, const CUtensorMap& tv, DecodePa
                           int cps, int stages, cudaStream_t st, int dev) {
   if (p.G <= 8) return launch_main<D, NCW, 1, TPW>(tk, tv, p, di, cps, stages, st, dev);
   return launch_main<D, NCW, 2, TPW>(tk, tv, p, di, cps, stages, st, dev);
+}
+
+// 8-bit cache: head_dim 128, one tile per warp.
+static int launch_main_kv8(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
+                           const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev) {
+  const bool wide = p.G > 8;
+  switch (ncw) {
+    case 2:
+      return wide ? launch_main<128, 2, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev)
+                  : launch_main<128, 2, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev);
+    case 8:
+      return wide ? launch_main<128, 8, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev)
+                  : launch_main<128, 8, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev);
+    default:
+      return wide ? launch_main<128, 4, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev)
+                  : launch_main<128, 4, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev);
+  }
 }
 
 template <int D>
@@ -244,6 +277,8 @@ static AppendParams make_append_params(const ooco_shape_t* s, const void* k_new,
   a.bstr = s->kv_block_stride;
   a.hstr = s->kv_head_stride;
   a.tstr = s->kv_token_stride;
+  a.kv8 = 0;
+  a.k_scale = a.v_scale = 1.f;
   return a;
 }
 
@@ -479,11 +514,25 @@ size_t ooco_decode_workspace_bytes(const ooco_shape_t* s) {
 }
 
 // Plan (+ optional fused append) -> split-KV attention -> LSE merge on `cuda_stream`.
+struct Kv8Scales {  // present: the caches hold E4M3 codes, a code stands for decode(code) * scale
+  float k_scale, v_scale;
+};
+
+static int validate_kv8(const ooco_shape_t* s, const Kv8Scales* kv8) {
+  if (!kv8) return OOCO_OK;
+  if (!(kv8->k_scale > 0.f) || !(kv8->v_scale > 0.f)) return OOCO_E_SHAPE;
+  if (s->head_dim != 128) return OOCO_E_UNSUPPORTED;
+  if ((s->kv_block_stride | s->kv_head_stride | s->kv_token_stride) & 15) return OOCO_E_UNSUPPORTED;
+  return OOCO_OK;
+}
+
 static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
                        const int32_t* block_table, const int32_t* context_lens, float scale, void* out,
-                       void* workspace, size_t workspace_bytes, void* cuda_stream, const AppendParams* append) {
+                       void* workspace, size_t workspace_bytes, void* cuda_stream, const AppendParams* append,
+                       const Kv8Scales* kv8 = nullptr) {
   int rc = validate_shape(s);
   if (rc) return rc;
+  if ((rc = validate_kv8(s, kv8))) return rc;
   if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
   if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q) & 15) return OOCO_E_UNSUPPORTED;
   const WsLayout w = ws_layout(s);
@@ -497,7 +546,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   const int ncw = g_knobs[kKnobWarps].load();
   const int cps = g_knobs[kKnobCtasPerSm].load();
   int tpw = g_knobs[kKnobTilesPerWarp].load();
-  if (ncw == 8) tpw = 1;
+  if (ncw == 8 || kv8) tpw = 1;
   const int stage_tok = 16 * ncw * tpw;
   DecodeParams p;
   memset(&p, 0, sizeof p);
@@ -526,12 +575,16 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.chunk_max = g_knobs[kKnobChunkMax].load();
   if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
   p.items_per_cta = g_knobs[kKnobItemsPerCta].load();
-  p.scale_log2e = scale * 1.4426950408889634f;
+  p.scale_log2e = scale * 1.4426950408889634f * (kv8 ? kv8->k_scale : 1.f);
+  p.v_scale = kv8 ? kv8->v_scale : 1.f;
 
   CUtensorMap tk, tv;
-  bool five_d = s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
+  bool five_d = !kv8 && s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
   if (five_d && encode_kv_map(&tk, s, k_cache, p.tile_rows, true) != OOCO_OK) five_d = false;
-  if (five_d) {
+  if (kv8) {
+    if ((rc = encode_kv8_map(&tk, s, k_cache, p.tile_rows))) return rc;
+    if ((rc = encode_kv8_map(&tv, s, v_cache, p.tile_rows))) return rc;
+  } else if (five_d) {
     if ((rc = encode_kv_map(&tv, s, v_cache, p.tile_rows, true))) return rc;
   } else {
     if ((rc = encode_kv_map(&tk, s, k_cache, p.tile_rows, false))) return rc;
@@ -559,7 +612,9 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
   if (pe) cudaEventRecord(pe[1], st);
-  if (s->head_dim == 128)
+  if (kv8)
+    rc = launch_main_kv8(ncw, tk, tv, p, di, cps, stages, st, dev);
+  else if (s->head_dim == 128)
     rc = launch_main_ncw<128>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);
   else
     rc = launch_main_ncw<64>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);
@@ -601,6 +656,53 @@ int ooco_decode_step(const ooco_shape_t* s, const void* q, const void* k_new, co
   const AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
   return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
                      cuda_stream, &ap);
+}
+
+int ooco_kv_append_fp8(const ooco_shape_t* s, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                       const int32_t* block_table, const int32_t* positions, float k_scale, float v_scale,
+                       void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  const Kv8Scales sc = {k_scale, v_scale};
+  if ((rc = validate_kv8(s, &sc))) return rc;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
+    return OOCO_E_UNSUPPORTED;
+  AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
+  ap.kv8 = 1;
+  ap.k_scale = k_scale;
+  ap.v_scale = v_scale;
+  kv_append_kernel<<<append_blocks(s, 256), 256, 0, (cudaStream_t)cuda_stream>>>(ap);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the append kernel", (long)e);
+}
+
+int ooco_decode_attention_fp8(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* block_table, const int32_t* context_lens, float scale, float k_scale,
+                              float v_scale, void* out, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream) {
+  const Kv8Scales sc = {k_scale, v_scale};
+  return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                     cuda_stream, nullptr, &sc);
+}
+
+int ooco_decode_step_fp8(const ooco_shape_t* s, const void* q, const void* k_new, const void* v_new, void* k_cache,
+                         void* v_cache, const int32_t* block_table, const int32_t* positions,
+                         const int32_t* context_lens, float scale, float k_scale, float v_scale, void* out,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  const Kv8Scales sc = {k_scale, v_scale};
+  if ((rc = validate_kv8(s, &sc))) return rc;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
+    return OOCO_E_UNSUPPORTED;
+  AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
+  ap.kv8 = 1;
+  ap.k_scale = k_scale;
+  ap.v_scale = v_scale;
+  return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                     cuda_stream, &ap, &sc);
 }
 
 int ooco_decode_attention_static(const ooco_shape_t* s, const void* q, const void* k_cache,

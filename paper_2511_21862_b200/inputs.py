@@ -210,3 +210,26 @@ def make_batch(cfg: DecodeConfig, device="cpu", *, poison: bool = True, table_pa
 def as_u16(t: torch.Tensor):
     """Raw bit patterns of a bf16 tensor as a numpy uint16 array (host copy)."""
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view("uint16")
+
+
+def to_e4m3_pool(batch: DecodeBatch, k_scale: float, v_scale: float, *, poison: bool = True) -> DecodeBatch:
+    """The same batch with 8-bit (E4M3) caches: code = nearest E4M3 of value / scale, made with the
+    library dtype cast (this only synthesises stored data; both the CUDA path and the oracle read the
+    codes).  Values beyond the format's range are clamped first.  With `poison`, every slot that held
+    NaN (slots at or beyond T_b, unused blocks) holds the NaN code."""
+    def conv(x, s):
+        out = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        step = max(1, (1 << 26) // max(1, x[0].numel()))
+        for a in range(0, x.shape[0], step):
+            y = x[a:a + step].float() / s
+            nan = torch.isnan(y)
+            c = y.clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+            out[a:a + step] = torch.where(nan, torch.full_like(c, 0x7F if poison else 0), c)
+        return out
+    return replace(batch, k_cache=conv(batch.k_cache, k_scale), v_cache=conv(batch.v_cache, v_scale),
+                   extras=dict(batch.extras, k_scale=float(k_scale), v_scale=float(v_scale)))
+
+
+def as_u8(t: torch.Tensor):
+    """Host numpy uint8 copy of a uint8 tensor."""
+    return t.detach().cpu().contiguous().numpy()
