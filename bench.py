@@ -238,14 +238,22 @@ def run_ours(args, rank, local_rank, world):
         dist.init_process_group("nccl", device_id=dev)
     cfg = inputs.replace(inputs.CONFIGS[args.workload], seed=inputs.CONFIGS[args.workload].seed + 100 * rank)
     batch = inputs.make_batch(cfg, dev, poison=False)
+    fp8 = args.kv == "fp8"
+    K_SCALE, V_SCALE = 1.0 / 32, 1.0 / 32                                 # N(0, sigma) values sit well inside +-448
+    if fp8:
+        batch = inputs.to_e4m3_pool(batch, K_SCALE, V_SCALE, poison=False)
     sh = binding.shape_of(batch)
     B = sh.batch
     lens_host = batch.context_lens.cpu().contiguous()
     cost = binding.decode_bytes_model(sh, lens_host)
-    append_bytes = 2 * 2 * B * cfg.num_kv_heads * cfg.head_dim * 2        # K and V rows, read + written
+    if fp8:                                                               # K / V stored with d = 1, q / out with d = 2
+        cost = dict(cost, bytes_kv=binding.decode_bytes_model(sh, lens_host, 1)["bytes_kv"])
+        cost["bytes_paper"] = cost["bytes_q"] + cost["bytes_out"] + cost["bytes_kv"]
+    kv_b = 1 if fp8 else 2
+    append_bytes = 2 * B * cfg.num_kv_heads * cfg.head_dim * (2 + kv_b)   # K and V rows: bf16 read, cache written
     step_bytes = cost["bytes_paper"] + append_bytes
 
-    pool_bytes = 2 * batch.k_cache.numel() * 2
+    pool_bytes = 2 * batch.k_cache.numel() * batch.k_cache.element_size()
     free, _ = torch.cuda.mem_get_info(dev)
     R = replica_count(pool_bytes, free)
     pools = [(batch.k_cache, batch.v_cache)] + [(batch.k_cache.clone(), batch.v_cache.clone()) for _ in range(R - 1)]
@@ -257,8 +265,12 @@ def run_ours(args, rank, local_rank, world):
 
     def step(i):
         k, v = pools[i % R]
-        binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, k, v, batch.block_table, positions, lens1,
-                            cfg.scale, out, ws, stream)
+        if fp8:
+            binding.decode_step_fp8(sh, batch.q, batch.k_new, batch.v_new, k, v, batch.block_table, positions, lens1,
+                                    cfg.scale, K_SCALE, V_SCALE, out, ws, stream)
+        else:
+            binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, k, v, batch.block_table, positions, lens1,
+                                cfg.scale, out, ws, stream)
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -294,6 +306,8 @@ def run_ours(args, rank, local_rank, world):
     binding.profile_enable(0)
 
     # ---- end to end through the host-buffer entry point (pinned inputs in, result out, every step)
+    if fp8:
+        return finish_fp8(args, world, cfg, B, cost, step_bytes, ms_local, recs, clocks, R, pool_bytes, sampler)
     pin = lambda t: t.cpu().contiguous().pin_memory()
     hq, hk, hv, ht = pin(batch.q), pin(batch.k_new), pin(batch.v_new), pin(batch.block_table)
     hp, hl = pin(positions), pin(lens1)
@@ -505,6 +519,31 @@ def run_model_fit(args, local_rank):
     print(json.dumps(line))
 
 
+def finish_fp8(args, world, cfg, B, cost, step_bytes, ms, recs, clocks, R, pool_bytes, sampler):
+    """JSON line of the 8-bit-cache variant (single GPU; device-resident inputs only)."""
+    sampler.stop()
+    peak, peak_kind = measured_peak()
+    attn = sorted(r[1] for r in recs)
+    attn_avg = sum(attn) / len(attn)
+    achieved = cost["bytes_paper"] / (attn_avg * 1e-3) / 1e9
+    line = {
+        "metric": METRIC + " (8-bit E4M3 KV cache)", "value": step_bytes / (ms * 1e-3) / 1e12, "unit": "TB/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16 (e4m3 codes widened)", "data": "synthetic",
+        "config": {"workload": cfg.name + " with an 8-bit KV cache", "description": cfg.description, "batch": B,
+                   "total_tokens": cost["total_tokens"], "step": "ooco_decode_step_fp8, one layer",
+                   "l2": f"inputs larger than L2: steps rotate over {R} pool replicas ({R * pool_bytes / 2**30:.2f} GiB)"},
+        "decode_tokens_per_s": B / (ms * 1e-3), "step_bytes": step_bytes,
+        "kernel_ms": {"plan": sum(r[0] for r in recs) / len(recs), "attention": attn_avg,
+                      "merge": sum(r[2] for r in recs) / len(recs)},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "kernel": "decode_main_kernel (8-bit cache)",
+                     "algorithmic_bytes_per_launch": cost["bytes_paper"], "traffic": None},
+        "gpu_launches": args.steps * 3, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -520,6 +559,8 @@ def main():
     ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate", "model_fit"],
                     help="decode_step: the decode hot path (default); kv_migrate: paged block gather + scatter; "
                          "model_fit: fit and validate the attention term of the latency model")
+    ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
+                    help="decode_step: KV cache element type (fp8 = E4M3 codes; a secondary measurement)")
     ap.add_argument("--move-seqs", type=int, default=64, help="kv_migrate: sequences whose blocks are moved")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()

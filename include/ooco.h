@@ -181,7 +181,8 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  *                             V = decode(code) * v_scale; codes are widened exactly to f16, q and
  *                             the softmax weights are rounded to f16, accumulation is fp32.
  *   ooco_decode_step_fp8      the fused append + attention step, as ooco_decode_step.
- * Restrictions beyond ooco_shape_t's: head_dim = 128, strides multiples of 16 bytes.  Workspace,
+ * Restrictions beyond ooco_shape_t's: head_dim = 128, strides multiples of 16 bytes; a NaN code
+ * inside the attended range is not propagated as NaN (it reads as a finite value).  Workspace,
  * status word, launches, ownership and errors as for the bf16 entry points.
  */
 int ooco_kv_append_fp8(const ooco_shape_t* shape, const void* k_new, const void* v_new, void* k_cache,

@@ -417,19 +417,32 @@ __device__ __forceinline__ void consume_tiles(uint32_t kst, uint32_t vst, const 
 }
 
 // ---- 8-bit (E4M3) cache: one consumer warp's work on its 16-token tile of a stage.
-// A token row is D = 128 bytes.  The codes are widened to f16 in registers (exact) and both
-// contractions run as f16 MMAs; the tensor scales are applied outside (K's is folded into the softmax
-// scale, V's multiplies the output).  Fragment bookkeeping:
+// A token row is D = 128 bytes.  The codes are widened to f16 in registers (exactly, up to the fixed
+// factor 2^-8: see e4m3x2_to_f16x2) and both contractions run as f16 MMAs; the tensor scales and
+// that factor are applied outside (K's is folded into the softmax scale, V's multiplies the output).
+// (The 8-bit mma.sync shapes were measured slower than widening plus f16 MMAs on this part.)
+// Fragment bookkeeping:
 //   scores  ldmatrix (16-bit units) hands lane (g, t) the four codes of dims 4t .. 4t+3 of a 16-dim
 //           chunk; they fill the MMA's k slots (2t, 2t+1) and (2t+8, 2t+9).  The contraction does not
 //           care about the order of k as long as Q uses the same one (it does: see the q fragments).
 //   values  ldmatrix.trans hands lane (g, t) dims (2g, 2g+1) of tokens (2t, 2t+1); a byte permute
 //           regroups them per dim, so MMA row g is dim 2g and row g + 8 is dim 2g + 1 of the chunk
 //           (the epilogue writes the accumulators back in that order).
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
-  const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(two_codes & 0xffffu), __NV_E4M3);
-  return (uint32_t)h.x | ((uint32_t)h.y << 16);
+// Two E4M3 codes (bytes of `x` picked by the byte-permute selector `sel`, which must also zero the
+// upper byte of each 16-bit lane) -> f16x2 holding their values / 256, exactly, with integer
+// operations only (the conversion instruction runs on the slow special-function pipe): with the code
+// c in the low byte of a lane, (c + (c & 0x80)) << 7 moves the sign to bit 15 and the 7 magnitude bits
+// to bits 7..13, i.e. exponent and mantissa land in the f16 fields with the exponent read against
+// bias 15 instead of 7 (hence the factor 2^-8; subnormal codes become f16 subnormals of the same
+// relative value).  The NaN codes come out as the finite +-480 / 256.
+template <uint32_t sel>
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
+  const uint32_t c = __byte_perm(x, 0u, sel);
+  return (c + (c & 0x00800080u)) << 7;
 }
+constexpr uint32_t kSelB0B1 = 0x4140, kSelB2B3 = 0x4342;  // consecutive codes (score operand)
+constexpr uint32_t kSelB0B2 = 0x4240, kSelB1B3 = 0x4341;  // codes two apart (value operand: regroup per dim)
+constexpr float kE4m3WidenFactor = 256.f;                  // what the widened values must be multiplied by
 __device__ __forceinline__ float f16_lo(uint32_t x) { return __half2float(__ushort_as_half((unsigned short)(x & 0xffffu))); }
 __device__ __forceinline__ float f16_hi(uint32_t x) { return __half2float(__ushort_as_half((unsigned short)(x >> 16))); }
 
@@ -451,10 +464,10 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
   for (int j = 0; j < KS / 2; ++j) {
     uint32_t r0, r1, r2, r3;  // (tokens 0-7, chunk 2j) (tokens 8-15, 2j) (tokens 0-7, 2j+1) (tokens 8-15, 2j+1)
     ldmatrix_x4(kst + tile_off + pat[j], r0, r1, r2, r3);
-    const uint32_t a0 = e4m3x2_to_f16x2(r0), a2 = e4m3x2_to_f16x2(r0 >> 16);
-    const uint32_t a1 = e4m3x2_to_f16x2(r1), a3 = e4m3x2_to_f16x2(r1 >> 16);
-    const uint32_t c0 = e4m3x2_to_f16x2(r2), c2 = e4m3x2_to_f16x2(r2 >> 16);
-    const uint32_t c1 = e4m3x2_to_f16x2(r3), c3 = e4m3x2_to_f16x2(r3 >> 16);
+    const uint32_t a0 = e4m3x2_to_f16x2<kSelB0B1>(r0), a2 = e4m3x2_to_f16x2<kSelB2B3>(r0);
+    const uint32_t a1 = e4m3x2_to_f16x2<kSelB0B1>(r1), a3 = e4m3x2_to_f16x2<kSelB2B3>(r1);
+    const uint32_t c0 = e4m3x2_to_f16x2<kSelB0B1>(r2), c2 = e4m3x2_to_f16x2<kSelB2B3>(r2);
+    const uint32_t c1 = e4m3x2_to_f16x2<kSelB0B1>(r3), c3 = e4m3x2_to_f16x2<kSelB2B3>(r3);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       mma_f16(sc[nt][0], a0, a1, a2, a3, qf[nt][2 * j][0], qf[nt][2 * j][1]);
@@ -510,10 +523,10 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const uint32_t lo = half ? r2 : r0, hi = half ? r3 : r1;  // tokens 0-7 / 8-15 of chunk 2j + half
-      uint32_t a0 = e4m3x2_to_f16x2(__byte_perm(lo, 0, 0x4420));  // dim 2g,   tokens 2t, 2t+1
-      uint32_t a1 = e4m3x2_to_f16x2(__byte_perm(lo, 0, 0x4431));  // dim 2g+1, tokens 2t, 2t+1
-      uint32_t a2 = e4m3x2_to_f16x2(__byte_perm(hi, 0, 0x4420));  // dim 2g,   tokens 2t+8, 2t+9
-      uint32_t a3 = e4m3x2_to_f16x2(__byte_perm(hi, 0, 0x4431));  // dim 2g+1, tokens 2t+8, 2t+9
+      uint32_t a0 = e4m3x2_to_f16x2<kSelB0B2>(lo);  // dim 2g,   tokens 2t, 2t+1
+      uint32_t a1 = e4m3x2_to_f16x2<kSelB1B3>(lo);  // dim 2g+1, tokens 2t, 2t+1
+      uint32_t a2 = e4m3x2_to_f16x2<kSelB0B2>(hi);  // dim 2g,   tokens 2t+8, 2t+9
+      uint32_t a3 = e4m3x2_to_f16x2<kSelB1B3>(hi);  // dim 2g+1, tokens 2t+8, 2t+9
       if (kTail) {
         a0 &= mk01;
         a1 &= mk01;
@@ -526,8 +539,10 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
   }
 }
 
+// The 8-bit path is bound by the consumer warps' instruction latency, not by HBM, so its 8-warp shape
+// is compiled for two CTAs per SM (16 consumer warps), which caps it at 112 registers per thread.
 template <int D, int NCW, int NT, int TPW, bool KV8 = false>
-__global__ void __launch_bounds__((NCW + 1) * 32, 1)
+__global__ void __launch_bounds__((NCW + 1) * 32, (KV8 && NCW == 8 && NT == 1) ? 2 : 1)
 decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const DecodeParams p) {
   using L = SmemLayout<D, NCW, NT, TPW, KV8>;
@@ -725,9 +740,12 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   uint32_t mphase = 0;  // parity of the next merge-barrier phase to wait for
   bool merge_pending_read = false;
 
+  int slot = -1;
+  uint32_t full_phase = 1u;  // slot / phase of stage `it` without dividing by the runtime stage count
   for (int it = 0;; ++it) {
-    const int slot = it % nst;
-    if (!warp_wait(s_full + 8 * slot, (uint32_t)(it / nst) & 1u, s_abort)) {
+    if (++slot == nst) slot = 0;
+    if (slot == 0) full_phase ^= 1u;
+    if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
       if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
       return;
     }

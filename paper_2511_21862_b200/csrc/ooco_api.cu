@@ -21,6 +21,7 @@ namespace ooco {
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
             kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobCount };
 static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}};
+static std::atomic<int> g_warps_overridden{0};  // ooco_set_tuning(0, ..) was called
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
 static thread_local int tl_last_launches = 0;
@@ -492,6 +493,7 @@ int ooco_set_tuning(int knob, int value) {
   if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
   if (knob == kKnobCopyCtasPerSm && (value < 1 || value > 3)) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
+  if (knob == kKnobWarps) g_warps_overridden.store(1);
   return OOCO_OK;
 }
 
@@ -543,7 +545,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (di.sm_count <= 0) return OOCO_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
-  const int ncw = g_knobs[kKnobWarps].load();
+  // the 8-bit path wants 16 consumer warps per SM (it is latency-bound): 8 per CTA unless overridden
+  const int ncw = kv8 && !g_warps_overridden.load() ? 8 : g_knobs[kKnobWarps].load();
   const int cps = g_knobs[kKnobCtasPerSm].load();
   int tpw = g_knobs[kKnobTilesPerWarp].load();
   if (ncw == 8 || kv8) tpw = 1;
@@ -575,8 +578,9 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.chunk_max = g_knobs[kKnobChunkMax].load();
   if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
   p.items_per_cta = g_knobs[kKnobItemsPerCta].load();
-  p.scale_log2e = scale * 1.4426950408889634f * (kv8 ? kv8->k_scale : 1.f);
-  p.v_scale = kv8 ? kv8->v_scale : 1.f;
+  // the 8-bit path widens codes to value / 256 (kE4m3WidenFactor): both scales carry the factor back
+  p.scale_log2e = scale * 1.4426950408889634f * (kv8 ? kv8->k_scale * kE4m3WidenFactor : 1.f);
+  p.v_scale = kv8 ? kv8->v_scale * kE4m3WidenFactor : 1.f;
 
   CUtensorMap tk, tv;
   bool five_d = !kv8 && s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
