@@ -73,3 +73,36 @@ def test_large_config_sampled_sequences(name):
         out1 = gpu_attention(batch, context_lens=lens1)
         ref1 = oracle_attention(batch, context_lens=lens1, seqs=seqs[:4])
         assert_parity(out1, ref1.out, rows=seqs[:4], what="cfg4 after append")
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg3"])
+def test_fp8_cache_full_size_sampled_sequences(name):
+    """The 8-bit cache path at benchmark size and launch shape: fused step, sampled whole sequences."""
+    cfg = inputs.CONFIGS[name]
+    ks, vs = 1.0 / 32, 1.0 / 32
+    batch = inputs.to_e4m3_pool(inputs.make_batch(cfg, "cuda", poison=True), ks, vs)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(batch.q, float("nan"))
+    lens1 = (batch.context_lens + 1).contiguous()
+    binding.decode_step_fp8(sh, batch.q, batch.k_new, batch.v_new, batch.k_cache, batch.v_cache, batch.block_table,
+                            batch.context_lens, lens1, cfg.scale, ks, vs, out, ws)
+    assert binding.workspace_status(ws) == 0
+    assert torch.isfinite(out.float()).all()
+    seqs = sample_sequences(batch.context_lens, n_each=2)
+    # oracle on a compacted host copy of just the sampled sequences' blocks (after the append)
+    lens, table = lens1.cpu(), batch.block_table.cpu()
+    bs = cfg.block_size
+    new_table, ids = table.clone(), []
+    for b in seqs:
+        n = (int(lens[b]) + bs - 1) // bs
+        new_table[b, :n] = torch.arange(len(ids), len(ids) + n, dtype=torch.int32)
+        ids.extend(table[b, :n].tolist())
+    idx = torch.tensor(ids, dtype=torch.long, device="cuda")
+    pairs = np.array([(b, h) for b in seqs for h in range(cfg.num_q_heads)], dtype=np.int32)
+    ref = oracle.decode_attention_fp8(inputs.as_u16(batch.q), inputs.as_u8(batch.k_cache.index_select(0, idx)),
+                                      inputs.as_u8(batch.v_cache.index_select(0, idx)), new_table.numpy(), lens.numpy(),
+                                      cfg.scale, ks, vs, num_kv_heads=cfg.num_kv_heads, block_size=bs,
+                                      strides=batch.strides, pairs=pairs)
+    mx, mean = assert_parity(out, ref.out, rows=seqs, what=name + " fp8")
+    print(f"{name} fp8 sampled {len(seqs)} sequences: max abs {mx:.3e} mean abs {mean:.3e}")
