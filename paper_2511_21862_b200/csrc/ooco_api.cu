@@ -21,7 +21,7 @@ namespace ooco {
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
             kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobCount };
 static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}};
-static std::atomic<int> g_warps_overridden{0};  // ooco_set_tuning(0, ..) was called
+static std::atomic<int> g_overridden[kKnobCount];  // knob set through ooco_set_tuning
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
 static thread_local int tl_last_launches = 0;
@@ -493,7 +493,7 @@ int ooco_set_tuning(int knob, int value) {
   if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
   if (knob == kKnobCopyCtasPerSm && (value < 1 || value > 3)) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
-  if (knob == kKnobWarps) g_warps_overridden.store(1);
+  g_overridden[knob].store(1);
   return OOCO_OK;
 }
 
@@ -545,9 +545,13 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (di.sm_count <= 0) return OOCO_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
-  // the 8-bit path wants 16 consumer warps per SM (it is latency-bound): 8 per CTA unless overridden
-  const int ncw = kv8 && !g_warps_overridden.load() ? 8 : g_knobs[kKnobWarps].load();
-  const int cps = g_knobs[kKnobCtasPerSm].load();
+  // Launch shape: 4 consumer warps x 2 CTAs per SM; the 8-bit path wants 16 consumer warps per SM (it is
+  // latency-bound): 8 x 2; groups of more than 8 query heads need two MMA column tiles and too many
+  // registers for two CTAs of any shape: 8 x 1.  A knob set by the caller wins.
+  const int G_ = s->num_q_heads / s->num_kv_heads;
+  int ncw = g_knobs[kKnobWarps].load(), cps = g_knobs[kKnobCtasPerSm].load();
+  if (!g_overridden[kKnobWarps].load() && (kv8 || G_ > 8)) ncw = 8;
+  if (!g_overridden[kKnobCtasPerSm].load() && G_ > 8) cps = 1;
   int tpw = g_knobs[kKnobTilesPerWarp].load();
   if (ncw == 8 || kv8) tpw = 1;
   const int stage_tok = 16 * ncw * tpw;
