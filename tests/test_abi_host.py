@@ -125,3 +125,24 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libooco.so")
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_block_movement_and_fp8_argument_validation_needs_no_device():
+    """Bad arguments are refused on the host before any CUDA call (this runs without a GPU)."""
+    L = binding.lib()
+    sh = binding.Shape(1, 8, 8, 128, 16, 10, 1, 8 * 16 * 128, 16 * 128, 128).c()
+    p = ctypes.c_void_p
+    buf = (ctypes.c_uint8 * 64)()
+    a = ctypes.addressof(buf)
+    a16 = (a + 15) & ~15
+    assert L.ooco_kv_gather_blocks(ctypes.byref(sh), None, p(a16), p(a16), 1, p(a16), p(a16), None, None) == -1
+    assert L.ooco_kv_gather_blocks(ctypes.byref(sh), p(a16), p(a16), p(a16), -1, p(a16), p(a16), None, None) == -2
+    assert L.ooco_kv_scatter_blocks(ctypes.byref(sh), p(a16 + 2), p(a16), p(a16), 1, p(a16), p(a16), None, None) == -3
+    assert L.ooco_kv_copy_blocks(ctypes.byref(sh), p(a16), p(a16), None, p(a16), 1, None, None) == -1
+    assert L.ooco_kv_gather_blocks(ctypes.byref(sh), p(a16), p(a16), None, 0, p(a16), p(a16), None, None) == 0   # n = 0
+    bad = binding.Shape(1, 8, 8, 64, 16, 10, 1, 8 * 16 * 64, 16 * 64, 64).c()
+    f = ctypes.c_float
+    assert L.ooco_kv_append_fp8(ctypes.byref(bad), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), f(1), f(1), None) == -3
+    assert L.ooco_kv_append_fp8(ctypes.byref(sh), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), f(-1), f(1), None) == -2
+    assert L.ooco_decode_attention_fp8(ctypes.byref(sh), p(a16), p(a16), p(a16), p(a16), p(a16), f(1), f(1), f(0),
+                                       p(a16), p(a16), 0, None) == -2

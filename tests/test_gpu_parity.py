@@ -215,3 +215,37 @@ def test_many_sequences_plan_scan():
     cfg = C("many", 8, 2, 64, 16, (G(2500, 0, 40), G(3, 600, 900)), seed=51)
     batch = inputs.make_batch(cfg, "cuda", poison=True)
     assert_parity(gpu_attention(batch), oracle_attention(batch).out, what="many")
+
+
+def test_step_replays_from_a_cuda_graph():
+    """The three launches of ooco_decode_step (programmatic dependent launches included) are captured
+    into a CUDA graph once and replayed: same bits as the direct call, also after the inputs change."""
+    cfg = C("graph", 32, 8, 128, 16, (G(12, 1, 3000),), seed=55, pool_fill=0.9)
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device="cuda")
+    lens1 = (batch.context_lens + 1).contiguous()
+    out_direct, out_graph = torch.empty_like(batch.q), torch.full_like(batch.q, float("nan"))
+    binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, batch.k_cache, batch.v_cache, batch.block_table,
+                        batch.context_lens, lens1, cfg.scale, out_direct, ws)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, batch.k_cache, batch.v_cache, batch.block_table,
+                            batch.context_lens, lens1, cfg.scale, out_graph, ws, side)
+        graph.capture_end()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    assert torch.equal(out_direct.view(torch.int16), out_graph.view(torch.int16))
+    # new query values in the same buffers: the replay picks them up
+    batch.q.copy_(torch.randn_like(batch.q.float()).to(torch.bfloat16))
+    binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, batch.k_cache, batch.v_cache, batch.block_table,
+                        batch.context_lens, lens1, cfg.scale, out_direct, ws)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out_direct.view(torch.int16), out_graph.view(torch.int16))
+    ref = oracle_attention(batch, context_lens=lens1)
+    assert_parity(out_graph, ref.out, what="graph replay")
