@@ -117,6 +117,25 @@ def decode_attention(q, k_cache, v_cache, block_table, context_lens, scale, *, n
     return AttentionResult(out, lse, wsum)
 
 
+def decode_attention_mq(q, k_cache, v_cache, block_table, context_lens, scale, *, num_kv_heads, block_size,
+                        strides) -> AttentionResult:
+    """Several query tokens per sequence (the operator table's S_q > 1: multi-token decode, a chunk of
+    a prefill): q is uint16 [B, Sq, Hq, D], the Sq query tokens are the LAST Sq tokens of the sequence,
+    context_lens[b] counts them, and query i sees tokens [0, T_b - Sq + i + 1) -- causal attention over the
+    cache.  By definition this is the one-query operator on B * Sq rows with those lengths, which is how
+    it is computed.  Results are shaped [B, Sq, Hq, ...]; a query without visible tokens gives zeros."""
+    q = _u16(q)
+    B, Sq, Hq, D = q.shape
+    lens = _i32(context_lens)
+    table = _i32(block_table)
+    lens_x = (lens[:, None] - Sq + 1 + np.arange(Sq, dtype=np.int32)[None, :]).reshape(-1)
+    lens_x = np.where(np.repeat(lens, Sq) <= 0, 0, np.maximum(lens_x, 0)).astype(np.int32)
+    table_x = np.repeat(table, Sq, axis=0)
+    r = decode_attention(q.reshape(B * Sq, Hq, D), k_cache, v_cache, table_x, lens_x, scale,
+                         num_kv_heads=num_kv_heads, block_size=block_size, strides=strides)
+    return AttentionResult(r.out.reshape(B, Sq, Hq, D), r.lse.reshape(B, Sq, Hq), r.wsum.reshape(B, Sq, Hq))
+
+
 def kv_append(k_new, v_new, k_cache, v_cache, block_table, positions, *, block_size, strides) -> int:
     """In-place append of k_new / v_new uint16 [B, Hkv, D] into the uint16 pools. Returns rows written."""
     lib = _load()

@@ -268,3 +268,33 @@ def test_append_then_attend_context_one_more():
                                 strides=batch.strides)
     vnew = bf16_to_f64(inputs.as_u16(batch.v_new))[0, 0]
     np.testing.assert_allclose(r.out[0, 0], vnew, rtol=0, atol=1e-9)
+
+
+def test_multi_query_oracle_is_bottom_right_causal_attention():
+    """S_q > 1: against a library softmax attention in fp64 with an explicit causal mask aligned to the
+    end of the sequence, on gathered contiguous K / V with heads repeated."""
+    rng = np.random.default_rng(11)
+    B, Sq, Hq, Hkv, D, bs, NB = 3, 3, 4, 2, 8, 4, 12
+    lens = np.array([9, 3, 14], dtype=np.int32)                 # the second sequence is nothing but its queries
+    table = np.stack([rng.permutation(NB)[:4] for _ in range(B)]).astype(np.int32)
+    to_bits = lambda x: torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    from_bits = lambda u: torch.from_numpy(u.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64)
+    k = to_bits(rng.standard_normal((NB, Hkv, bs, D)))
+    v = to_bits(rng.standard_normal((NB, Hkv, bs, D)))
+    q = to_bits(rng.standard_normal((B, Sq, Hq, D)))
+    got = oracle.decode_attention_mq(q, k, v, table, lens, 0.4, num_kv_heads=Hkv, block_size=bs,
+                                     strides=(Hkv * bs * D, bs * D, D))
+    kf, vf, qf = from_bits(k), from_bits(v), from_bits(q)
+    for b in range(B):
+        T = int(lens[b])
+        blocks = torch.from_numpy(table[b, :(T + bs - 1) // bs].astype(np.int64))
+        kk = kf[blocks].permute(1, 0, 2, 3).reshape(Hkv, -1, D)[:, :T].repeat_interleave(Hq // Hkv, 0)   # [Hq, T, D]
+        vv = vf[blocks].permute(1, 0, 2, 3).reshape(Hkv, -1, D)[:, :T].repeat_interleave(Hq // Hkv, 0)
+        mask = torch.ones(Sq, T, dtype=torch.bool).tril(diagonal=T - Sq)                                # query i sees t <= T - Sq + i
+        want = torch.nn.functional.scaled_dot_product_attention(qf[b].permute(1, 0, 2), kk, vv, attn_mask=mask, scale=0.4)
+        assert np.allclose(got.out[b], want.permute(1, 0, 2).numpy(), atol=1e-12)
+    assert np.allclose(got.wsum, 1.0, atol=1e-12)
+    # S_q = 1 is the one-query operator itself
+    one = oracle.decode_attention_mq(q[:, -1:], k, v, table, lens, 0.4, num_kv_heads=Hkv, block_size=bs,
+                                     strides=(Hkv * bs * D, bs * D, D))
+    assert np.array_equal(one.out[:, 0], got.out[:, -1])
