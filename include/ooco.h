@@ -168,6 +168,30 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Several query tokens per sequence (the attention row of Table "Operator Modeling" with S_q > 1:
+ * multi-token decode, or a short chunk of a prefill running next to decodes).  The q_len query
+ * tokens of sequence b are the LAST q_len tokens of its context: their K / V must already be in the
+ * cache (ooco_kv_append_mq writes them), context_lens[b] counts them, and query token i attends to
+ * tokens [0, T_b - q_len + i + 1) -- causal attention over the cache.  A query token that sees no
+ * token at all (T_b - q_len + i + 1 <= 0) gives a zero row.
+ *   q, out          device, bf16 [B, q_len, Hq, head_dim], contiguous
+ *   k_new, v_new    device, bf16 [B, q_len, Hkv, head_dim]; token i of sequence b is written at
+ *                   position positions[b] + i (ooco_kv_append_mq); positions beyond the block table
+ *                   are skipped, as in ooco_kv_append
+ *   workspace       >= ooco_decode_workspace_bytes_mq(shape, q_len)
+ * Supported: (Hq / Hkv) * q_len <= 16; bf16 caches.  q_len = 1 is ooco_decode_attention /
+ * ooco_kv_append exactly.  Everything else as for those two.
+ */
+size_t ooco_decode_workspace_bytes_mq(const ooco_shape_t* shape, int32_t q_len);
+int ooco_decode_attention_mq(const ooco_shape_t* shape, int32_t q_len, const void* q, const void* k_cache,
+                             const void* v_cache, const int32_t* block_table, const int32_t* context_lens,
+                             float scale, void* out, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream);
+int ooco_kv_append_mq(const ooco_shape_t* shape, int32_t q_len, const void* k_new, const void* v_new,
+                      void* k_cache, void* v_cache, const int32_t* block_table, const int32_t* positions,
+                      void* cuda_stream);
+
+/*
  * The same three operations over an 8-bit KV cache (the operator model's d, "byte per value", set
  * to 1 for K and V: Table "Symbol definitions"; decode attention is memory-bound, section 3.3.3, so
  * halving the stored bytes halves its time).  k_cache / v_cache hold OCP E4M3 codes (1 sign, 4

@@ -22,6 +22,7 @@ EXPORTS = (
     "ooco_profile_enable", "ooco_profile_read", "ooco_decode_attention_static",
     "ooco_kv_gather_blocks", "ooco_kv_scatter_blocks", "ooco_kv_copy_blocks",
     "ooco_kv_append_fp8", "ooco_decode_attention_fp8", "ooco_decode_step_fp8",
+    "ooco_decode_workspace_bytes_mq", "ooco_decode_attention_mq", "ooco_kv_append_mq",
 )
 
 
@@ -77,6 +78,13 @@ def lib() -> ctypes.CDLL:
         L.ooco_decode_step_fp8.restype = ctypes.c_int
         L.ooco_decode_step_fp8.argtypes = [sp, vp, vp, vp, vp, vp, i32p, i32p, i32p, f32, f32, f32, vp, vp,
                                            ctypes.c_size_t, vp]
+        L.ooco_decode_workspace_bytes_mq.restype = ctypes.c_size_t
+        L.ooco_decode_workspace_bytes_mq.argtypes = [sp, ctypes.c_int32]
+        L.ooco_decode_attention_mq.restype = ctypes.c_int
+        L.ooco_decode_attention_mq.argtypes = [sp, ctypes.c_int32, vp, vp, vp, i32p, i32p, ctypes.c_float, vp, vp,
+                                               ctypes.c_size_t, vp]
+        L.ooco_kv_append_mq.restype = ctypes.c_int
+        L.ooco_kv_append_mq.argtypes = [sp, ctypes.c_int32, vp, vp, vp, vp, i32p, i32p, vp]
         L.ooco_kv_gather_blocks.restype = ctypes.c_int
         L.ooco_kv_gather_blocks.argtypes = [sp, vp, vp, i32p, ctypes.c_int32, vp, vp, i32p, vp]
         L.ooco_kv_scatter_blocks.restype = ctypes.c_int
@@ -225,6 +233,33 @@ def decode_step_fp8(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table
         _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), float(k_scale), float(v_scale),
         _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_step_fp8")
+
+
+def workspace_bytes_mq(shape: Shape, q_len: int) -> int:
+    n = lib().ooco_decode_workspace_bytes_mq(ctypes.byref(shape.c()), int(q_len))
+    if n == 0:
+        raise OocoError(-3, "ooco_decode_workspace_bytes_mq")
+    return int(n)
+
+
+def decode_attention_mq(shape: Shape, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace,
+                        stream=None):
+    """q, out: bf16 [B, q_len, Hq, D]; the query tokens are the last q_len tokens of each context."""
+    assert q.dim() == 4 and q.shape == out.shape
+    _check(lib().ooco_decode_attention_mq(
+        ctypes.byref(shape.c()), int(q.shape[1]), _dev(q, torch.bfloat16), _dev(k_cache, torch.bfloat16),
+        _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
+        float(scale), _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        _stream_ptr(stream)), "ooco_decode_attention_mq")
+
+
+def kv_append_mq(shape: Shape, k_new, v_new, k_cache, v_cache, block_table, positions, stream=None):
+    """k_new, v_new: bf16 [B, q_len, Hkv, D]; token i of sequence b goes to position positions[b] + i."""
+    assert k_new.dim() == 4 and k_new.shape == v_new.shape
+    _check(lib().ooco_kv_append_mq(
+        ctypes.byref(shape.c()), int(k_new.shape[1]), _dev(k_new, torch.bfloat16), _dev(v_new, torch.bfloat16),
+        _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32),
+        _dev(positions, torch.int32), _stream_ptr(stream)), "ooco_kv_append_mq")
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

@@ -41,9 +41,11 @@ struct DecodeParams {
   WsHeader* hdr;
   int4* items;            // [max_items] {b, partial slot = chunk index * Hkv + h, t0, t1}, longest first
   int32_t* seq_first;     // [B + 1] first chunk index of each sequence (exclusive scan)
-  float* part_o;          // [max_items, G, D] normalised partial outputs
-  float* part_lse;        // [max_items, G] log2-domain log-sum-exp of each partial
+  float* part_o;          // [max_items, GQ, D] normalised partial outputs
+  float* part_lse;        // [max_items, GQ] log2-domain log-sum-exp of each partial
   int32_t B, Hq, Hkv, G, D, bs, MB;
+  int32_t Sq;             // query tokens per sequence (the last Sq tokens of its context); 1 = decode
+  int32_t GQ;             // G * Sq: score columns of one (sequence, kv head), column = query * G + head
   int32_t max_items;
   int32_t tile_rows;      // token rows per TMA box = min(bs, stage tokens)
   int32_t split_halves;   // 1: one 4-d TMA per 64-dim half; 0: one 5-d TMA per box
@@ -63,6 +65,7 @@ struct AppendParams {
   const int32_t* block_table;
   const int32_t* positions;
   int32_t B, Hkv, D, bs, NB, MB;
+  int32_t Sq;               // new tokens per sequence: k_new / v_new are [B, Sq, Hkv, D], token i goes to positions[b] + i
   int64_t bstr, hstr, tstr;
   int32_t kv8;              // 1: the caches hold 8-bit E4M3 codes (k_cache / v_cache are byte arrays)
   float k_scale, v_scale;   // tensor scales of an 8-bit cache: stored code = e4m3(x / scale)
@@ -88,12 +91,14 @@ __device__ __forceinline__ uint2 quantize_e4m3x8(const uint4 w, float scale) {
 // `nblocks` CTAs cooperate grid-stride.
 __device__ __forceinline__ void kv_append_body(const AppendParams& a, int block, int nblocks) {
   const int vec_per_row = a.D / 8;
-  const long long n = (long long)a.B * a.Hkv * vec_per_row;
+  const long long n = (long long)a.B * a.Sq * a.Hkv * vec_per_row;
   for (long long i = block * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)nblocks * blockDim.x) {
     const int v = (int)(i % vec_per_row);
     const int h = (int)((i / vec_per_row) % a.Hkv);
-    const int b = (int)(i / ((long long)vec_per_row * a.Hkv));
-    const int pos = a.positions[b];
+    const long long tok = i / ((long long)vec_per_row * a.Hkv);  // (sequence, new token) index
+    const int b = (int)(tok / a.Sq);
+    const long long pos64 = (long long)a.positions[b] + (tok % a.Sq);
+    const int pos = pos64 > 0x7fffffffLL ? -1 : (int)pos64;
     if (pos < 0 || (long long)pos >= (long long)a.MB * a.bs) continue;
     const int blk = a.block_table[(size_t)b * a.MB + pos / a.bs];
     if (blk < 0 || blk >= a.NB) continue;
@@ -274,7 +279,7 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     for (int h = 0; h < p.Hkv; ++h) p.items[pos * p.Hkv + h] = make_int4(b, ci * p.Hkv + h, t0, t1);
   }
   // sequences without context produce zeros
-  const int row = p.Hq * p.D;
+  const int row = p.Sq * p.Hq * p.D;
   for (int b = wid; b < p.B; b += kThreads / 32) {
     if (len_of(b) > 0) continue;
     for (int i = lane; i < row; i += 32) p.out[(size_t)b * row + i] = __float2bfloat16(0.f);
@@ -313,7 +318,10 @@ __device__ __forceinline__ void consume_tiles(uint32_t kst, uint32_t vst, const 
                                               const uint32_t (&vpat)[D / 16],
                                               const uint32_t (&qf)[NT][D / 16][2], float (&m_run)[NT][2],
                                               float (&l_run)[NT][2], float (&o_acc)[NT][D / 16][4],
-                                              float scale_log2e, int valid, int g, int t) {
+                                              float scale_log2e, int valid, int g, int t, int lim_w = 0,
+                                              const int (*qi_col)[2] = nullptr) {
+  // kTail only: lim_w = rows of this warp the first query token may see (causal limit, several query
+  // tokens per sequence), qi_col[nt][c] = query token of the lane's score column c of tile nt.
   constexpr int KS = D / 16;
   constexpr int NACC = TPW == 1 ? 2 : 1;  // a lone tile splits its k-steps over two accumulators
   // ---- scores: S = K_tile x Q^T
@@ -352,8 +360,11 @@ __device__ __forceinline__ void consume_tiles(uint32_t kst, uint32_t vst, const 
         s[u][e] = v * scale_log2e;
       }
       if (kTail) {
-        if (16 * u + g >= valid) s[u][0] = s[u][1] = -INFINITY;
-        if (16 * u + g + 8 >= valid) s[u][2] = s[u][3] = -INFINITY;
+        const int l0 = min(valid, lim_w + qi_col[nt][0]), l1 = min(valid, lim_w + qi_col[nt][1]);
+        if (16 * u + g >= l0) s[u][0] = -INFINITY;
+        if (16 * u + g >= l1) s[u][1] = -INFINITY;
+        if (16 * u + g + 8 >= l0) s[u][2] = -INFINITY;
+        if (16 * u + g + 8 >= l1) s[u][3] = -INFINITY;
       }
       mx0 = fmaxf(mx0, fmaxf(s[u][0], s[u][2]));
       mx1 = fmaxf(mx1, fmaxf(s[u][1], s[u][3]));
@@ -363,10 +374,15 @@ __device__ __forceinline__ void consume_tiles(uint32_t kst, uint32_t vst, const 
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
     }
-    const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
-    const float al0 = ex2(m_run[nt][0] - mn0), al1 = ex2(m_run[nt][1] - mn1);
+    const float mo0 = m_run[nt][0], mo1 = m_run[nt][1];
+    float mn0 = fmaxf(mo0, mx0), mn1 = fmaxf(mo1, mx1);
     m_run[nt][0] = mn0;
     m_run[nt][1] = mn1;
+    if (kTail) {  // a column that has seen nothing yet (causal limit): keep the exponents finite
+      mn0 = mn0 == -INFINITY ? 0.f : mn0;
+      mn1 = mn1 == -INFINITY ? 0.f : mn1;
+    }
+    const float al0 = ex2(mo0 - mn0), al1 = ex2(mo1 - mn1);
     float add0 = 0.f, add1 = 0.f;
 #pragma unroll
     for (int u = 0; u < TPW; ++u) {
@@ -555,7 +571,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const int nst = p.nstages;
-  const int qslot = L::q_slot_bytes(p.G);
+  const int qslot = L::q_slot_bytes(p.GQ);
   const uint32_t s_stage = base;
   const uint32_t s_q = s_stage + (uint32_t)nst * L::kStageBytes;
   const uint32_t s_merge = s_q + (uint32_t)nst * qslot;
@@ -596,17 +612,24 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     int item = blockIdx.x;
     int4 d = make_int4(0, 0, 0, 0);
     int blk_cur = 0;
+    int T_cur = 0;  // context length of the item's sequence (only read when there are several query tokens)
+    const long long cap_tokens = (long long)p.MB * p.bs;
+    auto seq_len = [&](int b) {
+      const long long T = p.context_lens[b];
+      return (int)(T < 0 ? 0 : (T > cap_tokens ? cap_tokens : T));
+    };
     if (item < n_items) {
       d = p.items[item];
       const int tb = d.z + lane * p.tile_rows;
       if (lane < boxes_per_stage && tb < d.w) blk_cur = p.block_table[(size_t)d.x * p.MB + tb / p.bs];
+      if (p.Sq > 1) T_cur = seq_len(d.x);
     }
     bool ok = true;
     while (item < n_items && ok) {
       int nxt = 0;
       if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
       int4 nd = make_int4(0, 0, 0, 0);
-      int blk_nxt_item = 0;
+      int blk_nxt_item = 0, T_nxt = 0;
       const int b = d.x, slot_id = d.y, h = d.y % p.Hkv, t0 = d.z, t1 = d.w;
       const int nstage_item = (t1 - t0 + kStageTok - 1) / kStageTok;
       const int32_t* row = p.block_table + (size_t)b * p.MB;
@@ -629,9 +652,16 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const uint32_t full = s_full + 8 * slot;
         if (lane == 0) {
           const int flags = (s == 0 ? 1 : 0) | (s == nstage_item - 1 ? 2 : 0);
-          g_meta[slot] = make_int4(slot_id, b, h, ntok | (flags << 16));
+          // rows of this stage the first query token may see, biased by 16 and clipped to 10 bits
+          // (one query token: everything)
+          int cm = 1023;
+          if (p.Sq > 1) {
+            const long long lim0 = (long long)T_cur - p.Sq + 1 - tok0 + 16;
+            cm = lim0 < 0 ? 0 : (lim0 > 1023 ? 1023 : (int)lim0);
+          }
+          g_meta[slot] = make_int4(slot_id, b, h, ntok | (flags << 16) | (cm << 18));
           uint32_t bytes = 2u * nbox * box_bytes;
-          if (s == 0) bytes += (uint32_t)p.G * D * 2;
+          if (s == 0) bytes += (uint32_t)p.GQ * D * 2;
           mbar_arrive_expect_tx(full, bytes);
         }
         __syncwarp();
@@ -654,9 +684,9 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             }
           }
         }
-        if (s == 0 && lane == 0)
-          bulk_g2s(s_q + (uint32_t)slot * qslot, p.q + ((size_t)b * p.Hq + (size_t)h * p.G) * D,
-                   (uint32_t)p.G * D * 2, full);
+        if (s == 0 && lane < p.Sq)  // one run of G heads per query token, side by side: [query][head][D]
+          bulk_g2s(s_q + (uint32_t)slot * qslot + (uint32_t)lane * p.G * D * 2,
+                   p.q + (((size_t)b * p.Sq + lane) * p.Hq + (size_t)h * p.G) * D, (uint32_t)p.G * D * 2, full);
         // look ahead to the next item: its descriptor, then its first table entries
         if (s == 0) {
           nxt = __shfl_sync(0xffffffffu, nxt, 0);
@@ -665,6 +695,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         if (s == (nstage_item > 1 ? 1 : 0) && nxt < n_items) {
           const int tb = nd.z + lane * p.tile_rows;
           if (lane < boxes_per_stage && tb < nd.w) blk_nxt_item = p.block_table[(size_t)nd.x * p.MB + tb / p.bs];
+          if (p.Sq > 1) T_nxt = seq_len(nd.x);
         }
         blk_cur = blk_n;
       }
@@ -672,6 +703,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       item = nxt;
       d = nd;
       blk_cur = blk_nxt_item;
+      T_cur = T_nxt;
     }
     // end marker (one stage, seen by every consumer warp)
     if (ok) {
@@ -737,6 +769,12 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     kpat[k] = (uint32_t)(ck >> 3) * half_bytes + (uint32_t)(((ck & 7) ^ (lr_k & 7)) << 4);
     vpat[k] = (uint32_t)(cv >> 3) * half_bytes + (uint32_t)(((cv & 7) ^ (lr_v & 7)) << 4);
   }
+  int qi_col[NT][2];  // query token of this lane's score columns 8 nt + 2t, + 1 (column = query * G + head)
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    qi_col[nt][0] = p.Sq > 1 ? (8 * nt + 2 * t) / p.G : 0;
+    qi_col[nt][1] = p.Sq > 1 ? (8 * nt + 2 * t + 1) / p.G : 0;
+  }
   uint32_t mphase = 0;  // parity of the next merge-barrier phase to wait for
   bool merge_pending_read = false;
 
@@ -764,7 +802,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         for (int k = 0; k < KS; ++k) {
           o_acc[nt][k][0] = o_acc[nt][k][1] = o_acc[nt][k][2] = o_acc[nt][k][3] = 0.f;
           uint32_t v0 = 0u, v1 = 0u;
-          if (head < p.G) {
+          if (head < p.GQ) {
             if (KV8) {  // dims 16k + 4t .. + 3 as two f16 pairs (the k order of the 8-bit score MMA)
               const uint2 w = *reinterpret_cast<const uint2*>(qs + ((size_t)head * D + 16 * k + 4 * t) * 2);
               v0 = pack_f16x2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u));
@@ -789,12 +827,16 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           consume_tile_kv8<D, NT, false>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t);
         else
           consume_tile_kv8<D, NT, true>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t);
-      } else if (valid >= 16 * TPW)
-        consume_tiles<D, NT, TPW, false>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
-                                         p.scale_log2e, valid, g, t);
-      else
-        consume_tiles<D, NT, TPW, true>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
-                                        p.scale_log2e, valid, g, t);
+      } else {
+        // rows of this warp the first query token may see; with one query token that is all of them
+        const int lim_w = ((meta.w >> 18) & 1023) - 16 - r0;
+        if (valid >= 16 * TPW && lim_w >= 16 * TPW)
+          consume_tiles<D, NT, TPW, false>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
+                                           p.scale_log2e, valid, g, t);
+        else
+          consume_tiles<D, NT, TPW, true>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
+                                          p.scale_log2e, valid, g, t, lim_w, qi_col);
+      }
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(s_empty + 8 * slot);
@@ -853,24 +895,27 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           return;
         }
         mphase ^= 1u;
-        for (int idx = threadIdx.x; idx < p.G * 64; idx += NCW * 32) {
-          const int head = idx >> 6, dl = idx & 63, dim = 64 * pass + dl;
+        for (int idx = threadIdx.x; idx < p.GQ * 64; idx += NCW * 32) {
+          const int col = idx >> 6, dl = idx & 63, dim = 64 * pass + dl;  // column = query * G + head
           float M = -INFINITY;
 #pragma unroll
-          for (int w = 0; w < NCW; ++w) M = fmaxf(M, all_m[(w * L::kHeads + head) * 2]);
+          for (int w = 0; w < NCW; ++w) M = fmaxf(M, all_m[(w * L::kHeads + col) * 2]);
+          const float Ms = M == -INFINITY ? 0.f : M;  // a query that saw nothing of this chunk (causal limit)
           float den = 0.f, num = 0.f;
 #pragma unroll
           for (int w = 0; w < NCW; ++w) {
-            const float sw = ex2(all_m[(w * L::kHeads + head) * 2] - M);
-            den += sw * all_m[(w * L::kHeads + head) * 2 + 1];
-            num += sw * g_merge[((size_t)w * L::kHeads + head) * L::kOStride + dl];
+            const float sw = ex2(all_m[(w * L::kHeads + col) * 2] - Ms);
+            den += sw * all_m[(w * L::kHeads + col) * 2 + 1];
+            num += sw * g_merge[((size_t)w * L::kHeads + col) * L::kOStride + dl];
           }
-          const float o = KV8 ? num / den * p.v_scale : num / den;
+          float o = den > 0.f ? num / den : 0.f;
+          if (KV8) o *= p.v_scale;
           if (n_chunks == 1) {
-            p.out[((size_t)b * p.Hq + (size_t)h * p.G + head) * D + dim] = __float2bfloat16_rn(o);
+            const int qi = p.Sq > 1 ? col / p.G : 0, head = col - qi * p.G;
+            p.out[(((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D + dim] = __float2bfloat16_rn(o);
           } else {
-            p.part_o[((size_t)item * p.G + head) * D + dim] = o;
-            if (dim == 0) p.part_lse[(size_t)item * p.G + head] = M + lg2(den);
+            p.part_o[((size_t)item * p.GQ + col) * D + dim] = o;
+            if (dim == 0) p.part_lse[(size_t)item * p.GQ + col] = den > 0.f ? M + lg2(den) : -INFINITY;
           }
         }
         mbar_arrive(s_mbar);
@@ -889,7 +934,8 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
   constexpr int V = D / 32;  // dims per lane
   const int lane = threadIdx.x & 31;
   const int warps_total = gridDim.x * (blockDim.x >> 5);
-  const int n_units = p.B * p.Hq;
+  const int per_seq = p.Sq * p.Hq;  // (query token, query head) rows of one sequence
+  const int n_units = p.B * per_seq;
   int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   // The chunk scan was written by the plan kernel, which had completed before the attention grid
   // (the grid this launch depends on) passed its own dependency wait, so it may be read before
@@ -898,13 +944,14 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
   grid_dep_launch();  // a programmatically launched successor may start its own prologue
   if (p.hdr->status & kStatusPlanOverflow) return;  // no work list, no partials (status is reported)
   if (u < n_units) {
-    first = p.seq_first[u / p.Hq];
-    n = p.seq_first[u / p.Hq + 1] - first;
+    first = p.seq_first[u / per_seq];
+    n = p.seq_first[u / per_seq + 1] - first;
   }
   grid_dep_wait();
   for (; u < n_units; u += warps_total, first = -1) {
-    const int b = u / p.Hq, hq = u % p.Hq;
-    const int h = hq / p.G, head = hq % p.G;
+    const int b = u / per_seq, rem = u % per_seq;
+    const int qi = rem / p.Hq, hq = rem % p.Hq;
+    const int h = hq / p.G, head = qi * p.G + hq % p.G;  // `head` = score column of (query, head) in its group
     if (first < 0) {
       first = p.seq_first[b];
       n = p.seq_first[b + 1] - first;
@@ -916,22 +963,23 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
     for (int c0 = 0; c0 < n; c0 += 32) {
       const int cnt = min(32, n - c0);
       float lse = -INFINITY;
-      if (lane < cnt) lse = p.part_lse[((size_t)(first + c0 + lane) * p.Hkv + h) * p.G + head];
+      if (lane < cnt) lse = p.part_lse[((size_t)(first + c0 + lane) * p.Hkv + h) * p.GQ + head];
       float gm = lse;
 #pragma unroll
       for (int o = 16; o; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
       const float Mn = fmaxf(M, gm);
-      const float resc = exp2f(M - Mn);
+      const float Ms = Mn == -INFINITY ? 0.f : Mn;  // nothing seen so far (causal limit): keep exponents finite
+      const float resc = exp2f(M - Ms);
       M = Mn;
-      const float w_lane = exp2f(lse - M);  // 0 for lanes beyond cnt
+      const float w_lane = exp2f(lse - Ms);  // 0 for lanes beyond cnt
       float ws = w_lane;
 #pragma unroll
       for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
       den = den * resc + ws;
 #pragma unroll
       for (int i = 0; i < V; ++i) acc[i] *= resc;
-      const float* src = p.part_o + (((size_t)(first + c0) * p.Hkv + h) * p.G + head) * D + lane * V;
-      const size_t cstride = (size_t)p.Hkv * p.G * D;
+      const float* src = p.part_o + (((size_t)(first + c0) * p.Hkv + h) * p.GQ + head) * D + lane * V;
+      const size_t cstride = (size_t)p.Hkv * p.GQ * D;
 #pragma unroll 8
       for (int j = 0; j < cnt; ++j) {
         const float w = __shfl_sync(0xffffffffu, w_lane, j);
@@ -944,8 +992,8 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
         }
       }
     }
-    __nv_bfloat16* dst = p.out + ((size_t)b * p.Hq + hq) * D + lane * V;
-    const float inv = 1.f / den;
+    __nv_bfloat16* dst = p.out + (((size_t)b * p.Sq + qi) * p.Hq + hq) * D + lane * V;
+    const float inv = den > 0.f ? 1.f / den : 0.f;  // den = 0: the query saw no token at all
 #pragma unroll
     for (int i = 0; i < V; i += 2)
       *reinterpret_cast<__nv_bfloat162*>(dst + i) = __floats2bfloat162_rn(acc[i] * inv, acc[i + 1] * inv);

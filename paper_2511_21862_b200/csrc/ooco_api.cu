@@ -102,8 +102,8 @@ struct WsLayout {
   size_t off_first, off_items, off_lse, off_o, total;
   int max_items;
 };
-static WsLayout ws_layout(const ooco_shape_t* s) {
-  const int G = s->num_q_heads / s->num_kv_heads;
+static WsLayout ws_layout(const ooco_shape_t* s, int q_len = 1) {
+  const int G = s->num_q_heads / s->num_kv_heads * q_len;  // score columns per (sequence, kv head)
   const int64_t cmax = g_knobs[kKnobChunkMax].load();
   const int64_t ipc = g_knobs[kKnobItemsPerCta].load();
   const int64_t per_seq = ((int64_t)s->max_blocks_per_seq * s->block_size + cmax - 1) / cmax;
@@ -185,10 +185,10 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
   const size_t budget = ctas_per_sm > 1 ? ((size_t)di.smem_optin + 1024) / ctas_per_sm - 1024 - static_smem.load()
                                         : dyn_max;
   int nst = want_stages > 0 ? want_stages : 32;
-  while (nst > 2 && L::total(nst, p.G) > budget) --nst;
-  if (L::total(nst, p.G) > dyn_max) return OOCO_E_UNSUPPORTED;
+  while (nst > 2 && L::total(nst, p.GQ) > budget) --nst;
+  if (L::total(nst, p.GQ) > dyn_max) return OOCO_E_UNSUPPORTED;
   p.nstages = nst;
-  const size_t smem = L::total(nst, p.G);
+  const size_t smem = L::total(nst, p.GQ);
   static std::atomic<size_t> configured[64];
   if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max);
@@ -204,14 +204,14 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
 template <int D, int NCW, int TPW>
 static int launch_main_nt(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                           int cps, int stages, cudaStream_t st, int dev) {
-  if (p.G <= 8) return launch_main<D, NCW, 1, TPW>(tk, tv, p, di, cps, stages, st, dev);
+  if (p.GQ <= 8) return launch_main<D, NCW, 1, TPW>(tk, tv, p, di, cps, stages, st, dev);
   return launch_main<D, NCW, 2, TPW>(tk, tv, p, di, cps, stages, st, dev);
 }
 
 // 8-bit cache: head_dim 128, one tile per warp.
 static int launch_main_kv8(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
                            const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev) {
-  const bool wide = p.G > 8;
+  const bool wide = p.GQ > 8;
   switch (ncw) {
     case 2:
       return wide ? launch_main<128, 2, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev)
@@ -278,13 +278,14 @@ static AppendParams make_append_params(const ooco_shape_t* s, const void* k_new,
   a.bstr = s->kv_block_stride;
   a.hstr = s->kv_head_stride;
   a.tstr = s->kv_token_stride;
+  a.Sq = 1;
   a.kv8 = 0;
   a.k_scale = a.v_scale = 1.f;
   return a;
 }
 
-static int append_blocks(const ooco_shape_t* s, int threads) {
-  const long long n = (long long)s->batch * s->num_kv_heads * (s->head_dim / 8);
+static int append_blocks(const ooco_shape_t* s, int threads, int q_len = 1) {
+  const long long n = (long long)s->batch * q_len * s->num_kv_heads * (s->head_dim / 8);
   long long blocks = (n + threads - 1) / threads;
   return (int)(blocks > 2048 ? 2048 : blocks);
 }
@@ -516,6 +517,15 @@ size_t ooco_decode_workspace_bytes(const ooco_shape_t* s) {
 }
 
 // Plan (+ optional fused append) -> split-KV attention -> LSE merge on `cuda_stream`.
+// Query tokens per sequence: the score columns of a (sequence, kv head) pair, G * q_len, must fit the
+// two 8-column MMA tiles of the kernel; the 8-bit path is built for one query token.
+static int validate_q_len(const ooco_shape_t* s, int q_len, bool kv8) {
+  if (q_len < 1) return OOCO_E_SHAPE;
+  if (q_len == 1) return OOCO_OK;
+  if (kv8 || (long long)(s->num_q_heads / s->num_kv_heads) * q_len > 16) return OOCO_E_UNSUPPORTED;
+  return OOCO_OK;
+}
+
 struct Kv8Scales {  // present: the caches hold E4M3 codes, a code stands for decode(code) * scale
   float k_scale, v_scale;
 };
@@ -531,13 +541,14 @@ static int validate_kv8(const ooco_shape_t* s, const Kv8Scales* kv8) {
 static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
                        const int32_t* block_table, const int32_t* context_lens, float scale, void* out,
                        void* workspace, size_t workspace_bytes, void* cuda_stream, const AppendParams* append,
-                       const Kv8Scales* kv8 = nullptr) {
+                       const Kv8Scales* kv8 = nullptr, int q_len = 1) {
   int rc = validate_shape(s);
   if (rc) return rc;
   if ((rc = validate_kv8(s, kv8))) return rc;
+  if ((rc = validate_q_len(s, q_len, kv8 != nullptr))) return rc;
   if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
   if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q) & 15) return OOCO_E_UNSUPPORTED;
-  const WsLayout w = ws_layout(s);
+  const WsLayout w = ws_layout(s, q_len);
   if (workspace_bytes < w.total || ((uintptr_t)workspace & 255)) return OOCO_E_WORKSPACE;
   int dev = 0;
   if ((rc = current_device(&dev))) return rc;
@@ -548,7 +559,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // Launch shape: 4 consumer warps x 2 CTAs per SM; the 8-bit path wants 16 consumer warps per SM (it is
   // latency-bound): 8 x 2; groups of more than 8 query heads need two MMA column tiles and too many
   // registers for two CTAs of any shape: 8 x 1.  A knob set by the caller wins.
-  const int G_ = s->num_q_heads / s->num_kv_heads;
+  const int G_ = s->num_q_heads / s->num_kv_heads * q_len;
   int ncw = g_knobs[kKnobWarps].load(), cps = g_knobs[kKnobCtasPerSm].load();
   if (!g_overridden[kKnobWarps].load() && (kv8 || G_ > 8)) ncw = 8;
   if (!g_overridden[kKnobCtasPerSm].load() && G_ > 8) cps = 1;
@@ -571,6 +582,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.Hq = s->num_q_heads;
   p.Hkv = s->num_kv_heads;
   p.G = p.Hq / p.Hkv;
+  p.Sq = q_len;
+  p.GQ = p.G * q_len;
   p.D = s->head_dim;
   p.bs = s->block_size;
   p.MB = s->max_blocks_per_seq;
@@ -612,7 +625,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   AppendParams ap;
   memset(&ap, 0, sizeof ap);
   if (append) ap = *append;
-  const int plan_grid = 1 + (append ? append_blocks(s, 1024) : 0);
+  const int plan_grid = 1 + (append ? append_blocks(s, 1024, append->Sq) : 0);
   const bool pdl_on = g_knobs[kKnobPdl].load() != 0 && !pe;
   cudaError_t e = launch_ex(plan_kernel<1024>, dim3(plan_grid), dim3(1024), first_in_smem ? first_bytes : 0, st,
                             pdl_on, p, stage_tok, first_in_smem, ap);
@@ -629,7 +642,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (rc) return rc;
   if (pe) cudaEventRecord(pe[2], st);
   {
-    long long warps = (long long)p.B * p.Hq;  // upper bound on (split sequence, query head) units
+    long long warps = (long long)p.B * p.Sq * p.Hq;  // (sequence, query token, query head) units
     int blocks = (int)((warps + 7) / 8);
     if (blocks > di.sm_count * 8) blocks = di.sm_count * 8;
     const bool pdl = g_knobs[kKnobPdl].load() != 0 && !pe;
@@ -711,6 +724,33 @@ int ooco_decode_step_fp8(const ooco_shape_t* s, const void* q, const void* k_new
   ap.v_scale = v_scale;
   return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
                      cuda_stream, &ap, &sc);
+}
+
+size_t ooco_decode_workspace_bytes_mq(const ooco_shape_t* s, int32_t q_len) {
+  if (validate_shape(s) || validate_q_len(s, q_len, false)) return 0;
+  return ws_layout(s, q_len).total;
+}
+
+int ooco_decode_attention_mq(const ooco_shape_t* s, int32_t q_len, const void* q, const void* k_cache,
+                             const void* v_cache, const int32_t* block_table, const int32_t* context_lens,
+                             float scale, void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                     cuda_stream, nullptr, nullptr, q_len);
+}
+
+int ooco_kv_append_mq(const ooco_shape_t* s, int32_t q_len, const void* k_new, const void* v_new, void* k_cache,
+                      void* v_cache, const int32_t* block_table, const int32_t* positions, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  if (q_len < 1) return OOCO_E_SHAPE;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
+    return OOCO_E_UNSUPPORTED;
+  AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
+  ap.Sq = q_len;
+  kv_append_kernel<<<append_blocks(s, 256, q_len), 256, 0, (cudaStream_t)cuda_stream>>>(ap);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the append kernel", (long)e);
 }
 
 int ooco_decode_attention_static(const ooco_shape_t* s, const void* q, const void* k_cache,

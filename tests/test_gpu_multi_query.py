@@ -1,0 +1,116 @@
+"""Several query tokens per sequence (S_q > 1) on the GPU vs the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_21862_b200 import binding, build, inputs
+from util import assert_parity
+
+pytestmark = pytest.mark.gpu
+G = inputs.LengthGroup
+C = inputs.DecodeConfig
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    binding.lib()
+
+
+def fixed(*vals):
+    return (G(len(vals), min(vals), max(vals), "fixed", tuple(vals)),)
+
+
+def run_case(cfg, Sq, seed):
+    batch = inputs.make_batch(cfg, "cuda", poison=True, table_pad=2**31 - 1)
+    B, Hq, D = cfg.batch, cfg.num_q_heads, cfg.head_dim
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    q = (torch.randn((B, Sq, Hq, D), generator=g, device="cuda") * cfg.sigma).to(torch.bfloat16)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_attention_mq(sh, q, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens,
+                                cfg.scale, out, ws)
+    assert binding.workspace_status(ws) == 0
+    ref = oracle.decode_attention_mq(inputs.as_u16(q), inputs.as_u16(batch.k_cache), inputs.as_u16(batch.v_cache),
+                                     batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                     num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size, strides=batch.strides)
+    assert_parity(out.reshape(B * Sq, Hq, D), ref.out.reshape(B * Sq, Hq, D), what=f"{cfg.name} Sq={Sq}")
+    return batch, q, out, ref
+
+
+CASES = [
+    # lengths around tile / stage / block boundaries; some contexts hold nothing but (part of) the queries
+    (C("mq-edges-g4", 32, 8, 128, 16, fixed(0, 1, 2, 3, 4, 15, 16, 17, 18, 19, 63, 64, 65, 66, 67, 127, 128, 129, 130, 300),
+       seed=81, pool_fill=0.7, shuffle_batch=False), 4),
+    (C("mq-g4-sq2", 32, 8, 128, 16, (G(8, 1, 600),), seed=82), 2),
+    (C("mq-g1-sq16", 8, 8, 128, 16, (G(6, 1, 500),), seed=83), 16),
+    (C("mq-g8-sq2-bs32", 64, 8, 128, 32, (G(5, 1, 900),), seed=84, sigma=0.5), 2),
+    (C("mq-g5-sq3", 40, 8, 128, 32, (G(6, 1, 700),), seed=85), 3),
+    (C("mq-d64-g4-sq3", 8, 2, 64, 16, (G(6, 1, 400),), seed=86), 3),
+    (C("mq-token-major", 32, 8, 128, 16, (G(6, 1, 500),), seed=87, layout="token_major"), 4),
+    # split into several chunks; chunk boundaries fall inside the last few tokens for some
+    (C("mq-split", 32, 8, 128, 16, fixed(5000, 37, 2049, 2050, 2051, 1025, 300, 9999), seed=88, pool_fill=0.9,
+       shuffle_batch=False), 4),
+    (C("mq-split-g2-sq8", 16, 8, 128, 16, fixed(7000, 129, 4097, 4100, 64), seed=89, shuffle_batch=False), 8),
+]
+
+
+@pytest.mark.parametrize("cfg,Sq", CASES, ids=lambda v: getattr(v, "name", str(v)))
+def test_multi_query_matches_oracle(cfg, Sq):
+    run_case(cfg, Sq, seed=cfg.seed)
+
+
+def test_last_query_token_equals_single_query_call():
+    """The last query token sees the whole context: the same result as ooco_decode_attention on that
+    token, up to the rounding of a different summation order (the launch shape depends on the number
+    of score columns)."""
+    cfg = C("mq-vs-single", 32, 8, 128, 16, (G(10, 3, 200),), seed=90)
+    batch, q, out, _ = run_case(cfg, 3, seed=1)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device="cuda")
+    q1 = q[:, -1].contiguous()
+    out1 = torch.empty_like(q1)
+    binding.decode_attention(sh, q1, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens, cfg.scale,
+                             out1, ws)
+    torch.cuda.synchronize()
+    assert float((out[:, -1].float() - out1.float()).abs().max()) <= 4e-3            # a bf16 ulp or two at |x| < 1
+
+
+def test_append_mq_bit_exact_then_attend():
+    cfg = C("mq-append", 32, 8, 128, 16, (G(20, 1, 700),), seed=91, pool_fill=0.8)
+    Sq = 4
+    # room for Sq new tokens: draw the batch with contexts Sq - 1 longer, then treat the tail as not yet written
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    lens = batch.context_lens
+    short = torch.clamp(lens - (Sq - 1), min=0).contiguous()             # positions of the first new token
+    ok = (lens >= Sq - 1)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    k_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    v_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    positions = torch.where(ok, short, torch.full_like(short, -100)).contiguous()   # too-short sequences: skipped
+    sh = binding.shape_of(batch)
+    k_ref, v_ref = inputs.as_u16(batch.k_cache).copy(), inputs.as_u16(batch.v_cache).copy()
+    table = batch.block_table.cpu().numpy()
+    for i in range(Sq):                                                    # oracle: one token at a time
+        oracle.kv_append(inputs.as_u16(k_new[:, i].contiguous()), inputs.as_u16(v_new[:, i].contiguous()), k_ref, v_ref,
+                         table, (positions + i).cpu().numpy() * ok.cpu().numpy() - 100 * (~ok).cpu().numpy(),
+                         block_size=16, strides=batch.strides)
+    binding.kv_append_mq(sh, k_new, v_new, batch.k_cache, batch.v_cache, batch.block_table, positions)
+    torch.cuda.synchronize()
+    assert np.array_equal(inputs.as_u16(batch.k_cache), k_ref) and np.array_equal(inputs.as_u16(batch.v_cache), v_ref)
+
+
+def test_unsupported_shapes_are_refused():
+    cfg = C("mq-too-wide", 64, 8, 128, 16, fixed(50), seed=92)
+    batch = inputs.make_batch(cfg, "cuda", poison=False)
+    sh = binding.shape_of(batch)
+    with pytest.raises(binding.OocoError):
+        binding.workspace_bytes_mq(sh, 3)                                  # 8 heads x 3 tokens > 16 columns
+    ws = torch.empty(binding.workspace_bytes_mq(sh, 2), dtype=torch.uint8, device="cuda")
+    q = torch.zeros((1, 3, 64, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.OocoError) as e:
+        binding.decode_attention_mq(sh, q, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens, 1.0,
+                                    torch.empty_like(q), ws)
+    assert e.value.status == -3
