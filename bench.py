@@ -455,6 +455,84 @@ def run_block_moves(args, rank, local_rank, world):
     print(json.dumps(line))
 
 
+def run_multi_query(args, local_rank):
+    """Secondary measurement: several query tokens per sequence (multi-token decode).  One step appends
+    q_len new tokens per sequence (ooco_kv_append_mq) and attends with causal masking over the cache
+    (ooco_decode_attention_mq).  Bytes follow the operator table with S_q = q_len."""
+    from paper_2511_21862_b200 import binding, build
+    build.build()
+    binding.lib()
+    for kv in args.knob:
+        name, val = kv.split("=")
+        binding.set_tuning(**{name: int(val)})
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream()
+    Sq = args.q_len
+    base = inputs.CONFIGS[args.workload]
+    cfg = inputs.replace(base, groups=tuple(inputs.replace(g, lo=g.lo + Sq, hi=g.hi + Sq) if g.dist != "fixed" else g
+                                            for g in base.groups))
+    batch = inputs.make_batch(cfg, dev, poison=False)
+    sh = binding.shape_of(batch)
+    B = sh.batch
+    gen = torch.Generator(device=dev).manual_seed(cfg.seed + 7)
+    q = (torch.randn((B, Sq, cfg.num_q_heads, cfg.head_dim), generator=gen, device=dev) * cfg.sigma).to(torch.bfloat16)
+    k_new = (torch.randn((B, Sq, cfg.num_kv_heads, cfg.head_dim), generator=gen, device=dev) * cfg.sigma).to(torch.bfloat16)
+    v_new = (torch.randn((B, Sq, cfg.num_kv_heads, cfg.head_dim), generator=gen, device=dev) * cfg.sigma).to(torch.bfloat16)
+    positions = (batch.context_lens - Sq).contiguous()                   # the new tokens are the last q_len of each context
+    lens_host = batch.context_lens.cpu().contiguous()
+    cost = binding.decode_bytes_model(sh, lens_host)
+    nbytes = cost["bytes_kv"] + Sq * (cost["bytes_q"] + cost["bytes_out"])      # table row with S_q = q_len
+    pool_bytes = 2 * batch.k_cache.numel() * 2
+    free, _ = torch.cuda.mem_get_info(dev)
+    R = replica_count(pool_bytes, free)
+    pools = [(batch.k_cache, batch.v_cache)] + [(batch.k_cache.clone(), batch.v_cache.clone()) for _ in range(R - 1)]
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device=dev)
+    out = torch.empty_like(q)
+
+    def step(i):
+        k, v = pools[i % R]
+        binding.kv_append_mq(sh, k_new, v_new, k, v, batch.block_table, positions, stream)
+        binding.decode_attention_mq(sh, q, k, v, batch.block_table, batch.context_lens, cfg.scale, out, ws, stream)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    binding.profile_enable(args.steps)
+    for i in range(args.steps):
+        step(i)
+    recs = binding.profile_read(args.steps)
+    binding.profile_enable(0)
+    attn = sum(r[1] for r in recs) / len(recs)
+    peak, peak_kind = measured_peak()
+    achieved = nbytes / (attn * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC + f" ({Sq} query tokens per sequence)", "value": nbytes / (ms * 1e-3) / 1e12, "unit": "TB/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}, {Sq} query tokens per sequence", "batch": B,
+                   "total_tokens": cost["total_tokens"], "step": "ooco_kv_append_mq + ooco_decode_attention_mq, one layer",
+                   "l2": f"inputs larger than L2: steps rotate over {R} pool replicas"},
+        "query_tokens_per_s": B * Sq / (ms * 1e-3),
+        "kernel_ms": {"plan": sum(r[0] for r in recs) / len(recs), "attention": attn, "merge": sum(r[2] for r in recs) / len(recs)},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "kernel": "decode_main_kernel", "algorithmic_bytes_per_launch": nbytes,
+                     "traffic": None},
+        "gpu_launches": 4 * args.steps, "clocks": sampler.summary(t0, t1)}))
+
+
 def run_model_fit(args, local_rank):
     """Secondary measurement: the attention term of the Roofline latency model against this kernel.
 
@@ -556,14 +634,22 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--ref-token-heads", type=int, default=400000,
                     help="reference arm: (tokens x q heads) of oracle work per step")
-    ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate", "model_fit"],
+    ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate", "model_fit", "decode_mq"],
                     help="decode_step: the decode hot path (default); kv_migrate: paged block gather + scatter; "
-                         "model_fit: fit and validate the attention term of the latency model")
+                         "model_fit: fit and validate the attention term of the latency model; "
+                         "decode_mq: --q-len query tokens per sequence")
+    ap.add_argument("--q-len", type=int, default=4, help="decode_mq: query tokens per sequence")
     ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
                     help="decode_step: KV cache element type (fp8 = E4M3 codes; a secondary measurement)")
     ap.add_argument("--move-seqs", type=int, default=64, help="kv_migrate: sequences whose blocks are moved")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
+    if args.op == "decode_mq":
+        if rank == 0:
+            args.steps = args.steps if args.steps is not None else 300
+            args.warmup = max(3, args.warmup if args.warmup is not None else 10)
+            run_multi_query(args, local_rank)
+        return
     if args.op == "model_fit":
         if rank == 0:
             args.warmup = args.warmup if args.warmup is not None else 5
