@@ -293,6 +293,7 @@ def run_ours(args, rank, local_rank, world):
         dist.barrier()
     t_end = time.perf_counter()
     ms_local = e0.elapsed_time(e1) / args.steps
+    launches_per_step = binding.last_launch_count()                       # kernels of one timed step
     assert binding.workspace_status(ws) == 0
     clocks = sampler.summary(t_begin, t_end)
 
@@ -363,7 +364,7 @@ def run_ours(args, rank, local_rank, world):
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
         "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e12, "unit": "TB/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
-        "gpu_launches": args.steps * binding.last_launch_count(),
+        "gpu_launches": args.steps * launches_per_step,
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:
