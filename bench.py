@@ -482,8 +482,8 @@ def run_multi_query(args, local_rank):
     v_new = (torch.randn((B, Sq, cfg.num_kv_heads, cfg.head_dim), generator=gen, device=dev) * cfg.sigma).to(torch.bfloat16)
     positions = (batch.context_lens - Sq).contiguous()                   # the new tokens are the last q_len of each context
     lens_host = batch.context_lens.cpu().contiguous()
-    cost = binding.decode_bytes_model(sh, lens_host)
-    nbytes = cost["bytes_kv"] + Sq * (cost["bytes_q"] + cost["bytes_out"])      # table row with S_q = q_len
+    cost = binding.attention_bytes_model(sh, Sq, lens_host)                     # table row with S_q = q_len
+    nbytes = cost["bytes_paper"]
     pool_bytes = 2 * batch.k_cache.numel() * 2
     free, _ = torch.cuda.mem_get_info(dev)
     R = replica_count(pool_bytes, free)

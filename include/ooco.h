@@ -324,6 +324,14 @@ int ooco_decode_bytes_model(const ooco_shape_t* shape, const int32_t* context_le
                             int32_t bytes_per_value, ooco_cost_t* cost_out);
 
 /*
+ * The same row of Table "Operator Modeling" with S_q = q_len query tokens per sequence, as printed
+ * (no causal discount): flops = sum_b 4 D_h q_len T_b; bytes_q = bytes_out = d q_len D_h per
+ * sequence; the K / V and index terms do not depend on q_len.  q_len = 1 is ooco_decode_bytes_model.
+ */
+int ooco_attention_bytes_model(const ooco_shape_t* shape, int32_t q_len, const int32_t* context_lens_host,
+                               int32_t bytes_per_value, ooco_cost_t* cost_out);
+
+/*
  * Bytes of device staging memory ooco_decode_step_host needs for `shape`
  * (0 for an invalid shape).  Host arithmetic only.
  */

@@ -22,7 +22,7 @@ EXPORTS = (
     "ooco_profile_enable", "ooco_profile_read", "ooco_decode_attention_static",
     "ooco_kv_gather_blocks", "ooco_kv_scatter_blocks", "ooco_kv_copy_blocks",
     "ooco_kv_append_fp8", "ooco_decode_attention_fp8", "ooco_decode_step_fp8",
-    "ooco_decode_workspace_bytes_mq", "ooco_decode_attention_mq", "ooco_kv_append_mq",
+    "ooco_decode_workspace_bytes_mq", "ooco_decode_attention_mq", "ooco_kv_append_mq", "ooco_attention_bytes_model",
 )
 
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.ooco_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.ooco_decode_bytes_model.restype = ctypes.c_int
         L.ooco_decode_bytes_model.argtypes = [sp, i32p, ctypes.c_int32, ctypes.POINTER(ooco_cost_t)]
+        L.ooco_attention_bytes_model.restype = ctypes.c_int
+        L.ooco_attention_bytes_model.argtypes = [sp, ctypes.c_int32, i32p, ctypes.c_int32, ctypes.POINTER(ooco_cost_t)]
         L.ooco_step_staging_bytes.restype = ctypes.c_size_t
         L.ooco_step_staging_bytes.argtypes = [sp]
         L.ooco_decode_step_host.restype = ctypes.c_int
@@ -329,6 +331,16 @@ def decode_bytes_model(shape: Shape, context_lens_host, bytes_per_value: int = 2
     c = ooco_cost_t()
     _check(lib().ooco_decode_bytes_model(ctypes.byref(shape.c()), t.data_ptr(), bytes_per_value,
                                          ctypes.byref(c)), "ooco_decode_bytes_model")
+    return {n: int(getattr(c, n)) for n, _ in ooco_cost_t._fields_}
+
+
+def attention_bytes_model(shape: Shape, q_len: int, context_lens_host, bytes_per_value: int = 2) -> dict:
+    """Host-only: the operator table's attention row with S_q = q_len."""
+    t = context_lens_host
+    assert not t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()
+    c = ooco_cost_t()
+    _check(lib().ooco_attention_bytes_model(ctypes.byref(shape.c()), int(q_len), t.data_ptr(), bytes_per_value,
+                                            ctypes.byref(c)), "ooco_attention_bytes_model")
     return {n: int(getattr(c, n)) for n, _ in ooco_cost_t._fields_}
 
 

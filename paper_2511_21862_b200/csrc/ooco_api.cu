@@ -819,9 +819,14 @@ int ooco_workspace_status(const void* workspace, void* cuda_stream, int32_t* sta
 
 int ooco_decode_bytes_model(const ooco_shape_t* s, const int32_t* context_lens_host, int32_t bytes_per_value,
                             ooco_cost_t* c) {
+  return ooco_attention_bytes_model(s, 1, context_lens_host, bytes_per_value, c);
+}
+
+int ooco_attention_bytes_model(const ooco_shape_t* s, int32_t q_len, const int32_t* context_lens_host,
+                               int32_t bytes_per_value, ooco_cost_t* c) {
   if (!s || !context_lens_host || !c) return OOCO_E_NULLPTR;
   if (s->batch <= 0 || s->num_q_heads <= 0 || s->num_kv_heads <= 0 || s->head_dim <= 0 || s->block_size <= 0 ||
-      bytes_per_value <= 0 || s->num_q_heads % s->num_kv_heads)
+      bytes_per_value <= 0 || s->num_q_heads % s->num_kv_heads || q_len < 1)
     return OOCO_E_SHAPE;
   const int64_t d = bytes_per_value;
   const int64_t q_row = (int64_t)s->num_q_heads * s->head_dim;     // D_h of the operator table
@@ -833,8 +838,8 @@ int ooco_decode_bytes_model(const ooco_shape_t* s, const int32_t* context_lens_h
     blocks += (t + s->block_size - 1) / s->block_size;
   }
   c->total_tokens = tokens;
-  c->flops = 4 * q_row * tokens;
-  c->bytes_q = d * s->batch * q_row;
+  c->flops = 4 * q_row * q_len * tokens;          // 4 D_h S_q S_kv
+  c->bytes_q = d * s->batch * q_len * q_row;      // d S_q D_h per sequence
   c->bytes_out = c->bytes_q;
   c->bytes_kv = 2 * d * kv_row * tokens;
   c->bytes_index = 4 * ((int64_t)s->batch + blocks);

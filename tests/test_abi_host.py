@@ -146,3 +146,21 @@ def test_block_movement_and_fp8_argument_validation_needs_no_device():
     assert L.ooco_kv_append_fp8(ctypes.byref(sh), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), f(-1), f(1), None) == -2
     assert L.ooco_decode_attention_fp8(ctypes.byref(sh), p(a16), p(a16), p(a16), p(a16), p(a16), f(1), f(1), f(0),
                                        p(a16), p(a16), 0, None) == -2
+
+
+def test_attention_bytes_model_with_several_query_tokens():
+    """Against the scheduling oracle's literal table row, summed over the batch; q_len = 1 is the decode model."""
+    from oracle import sched_oracle as so
+    rng = np.random.default_rng(4)
+    for Hq, Hkv, D, d, Sq in [(32, 8, 128, 2, 1), (32, 8, 128, 2, 4), (40, 8, 128, 1, 3), (8, 8, 64, 2, 16)]:
+        lens = rng.integers(0, 9000, 23).astype(np.int32)
+        sh = binding.Shape(len(lens), Hq, Hkv, D, 16, 1, 1, Hkv * 16 * D, 16 * D, D)
+        got = binding.attention_bytes_model(sh, Sq, torch.from_numpy(lens), d)
+        fl = by = 0
+        for T in lens:
+            f, b = so.attention_cost(Hq * D, Sq, int(T), Hq, Hkv, d)
+            fl, by = fl + f, by + b
+        assert (got["flops"], got["bytes_paper"]) == (fl, by)
+        assert got["bytes_q"] == got["bytes_out"] == d * Sq * Hq * D * len(lens)
+        if Sq == 1:
+            assert got == binding.decode_bytes_model(sh, torch.from_numpy(lens), d)

@@ -106,3 +106,21 @@ def test_fp8_cache_full_size_sampled_sequences(name):
                                       strides=batch.strides, pairs=pairs)
     mx, mean = assert_parity(out, ref.out, rows=seqs, what=name + " fp8")
     print(f"{name} fp8 sampled {len(seqs)} sequences: max abs {mx:.3e} mean abs {mean:.3e}")
+
+
+def test_very_long_context_next_to_very_short_ones():
+    """One 400 K-token sequence (50 chunks per kv head at the largest chunk size, two rounds of the
+    merge's 32-chunk batches for nobody, but a deep partial list) beside sequences of 1 and 40 tokens."""
+    cfg = inputs.DecodeConfig("long", 32, 8, 128, 16, (inputs.LengthGroup(3, 1, 400_000, "fixed", (400_000, 1, 40)),),
+                              seed=95, shuffle_batch=False)
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    out = gpu_attention(batch)
+    assert torch.isfinite(out.float()).all()
+    pairs = np.array([(0, 0), (0, 13), (0, 31), (1, 5), (2, 0), (2, 31)], dtype=np.int32)
+    ref = oracle.decode_attention(inputs.as_u16(batch.q), inputs.as_u16(batch.k_cache), inputs.as_u16(batch.v_cache),
+                                  batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                  num_kv_heads=8, block_size=16, strides=batch.strides, pairs=pairs)
+    got = out.cpu().double().numpy()
+    for b, h in pairs:
+        err = np.abs(got[b, h] - ref.out[b, h])
+        assert err.max() <= 1e-2 and err.mean() <= 1e-3, (b, h, err.max())
