@@ -15,6 +15,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -548,8 +549,8 @@ def run_model_fit(args, local_rank):
     dev = torch.device("cuda", local_rank)
     stream = torch.cuda.current_stream()
 
-    def measure(cfg, steps):
-        batch = inputs.make_batch(cfg, dev, poison=False)
+    def measure(cfg, steps, context_lens=None):
+        batch = inputs.make_batch(cfg, dev, poison=False, context_lens=context_lens)
         sh = binding.shape_of(batch)
         cost = binding.decode_bytes_model(sh, batch.context_lens.cpu().contiguous())
         pool_bytes = 2 * batch.k_cache.numel() * 2
@@ -591,9 +592,36 @@ def run_model_fit(args, local_rank):
         errs.append(abs(pred - sec) / sec)
         test.append({"workload": name, "bytes": cost["bytes_paper"], "tokens": cost["total_tokens"], "seconds": sec,
                      "predicted": pred, "abs_rel_err": errs[-1]})
+    # ---- closing the loop: Algorithm "Mix Decoding Selection" driven by the fitted predictor.  An
+    # attention-only instance (one layer, GEMM terms switched off by unbounded F_g / M_g) gets a TPOT
+    # bound S; the selection picks offline requests next to all online ones; the selected batch is
+    # then actually run and its measured step time compared with S and with the prediction.
+    base = inputs.CONFIGS["cfg2"]
+    model = sched.Model(1, base.num_q_heads * base.head_dim, base.num_q_heads, base.num_kv_heads, base.head_dim,
+                        base.head_dim, base.head_dim)
+    big = 1e30
+    hw = sched.Hw(big, big, big, big, M_a, 0.0, O, big)
+    gen = torch.Generator().manual_seed(123)
+    online = torch.randint(512, 4097, (32,), generator=gen).tolist()
+    u = torch.rand(600, generator=gen, dtype=torch.float64)
+    offline = torch.exp(math.log(4096) + u * (math.log(32768) - math.log(4096))).round().to(torch.int64).tolist()
+    slo = []
+    for S in (0.4e-3, 0.8e-3, 1.6e-3):
+        K = 16
+        probes = torch.randperm(len(offline), generator=gen)[:K].tolist()
+        margin = 0.97                                                    # the predictor is good to a few percent
+        sel, pred, over = sched.mix_decoding_select(model, hw, online, offline, S * margin, probes, K)
+        lens = online + [t for t, m in zip(offline, sel) if m]
+        cfg = inputs.replace(base, name=f"slo-{S * 1e3:.1f}ms", seed=77)
+        batch_lens = torch.tensor(lens, dtype=torch.int32)
+        cost, sec = measure(cfg, 100, context_lens=batch_lens)
+        slo.append({"slo_ms": S * 1e3, "online": len(online), "offline_selected": int(sel.sum()), "margin": margin, "batch": len(lens),
+                    "tokens": cost["total_tokens"], "predicted_ms": pred * 1e3, "measured_ms": sec * 1e3,
+                    "within_slo": bool(sec <= S), "headroom": 1.0 - sec / S})
     line = {"metric": "Roofline attention-latency model: mean abs relative error on the full workloads",
             "value": sum(errs) / len(errs), "unit": "fraction", "higher_is_better": False, "n_gpus": 1,
             "M_a_GBps": M_a / 1e9, "overhead_us": O * 1e6, "profiling_set": train, "validation": test,
+            "mix_decoding_selection": slo,
             "data": "synthetic", "dtype": "bf16"}
     print(json.dumps(line))
 
