@@ -81,6 +81,16 @@ int ooco_predict_decode_latency(const ooco_model_t* model, const ooco_hw_params_
                                 int64_t total_tokens, ooco_latency_t* out);
 
 /*
+ * Latency of a prefill iteration over the given prompts (sections 3.3.1 / 3.3.2; host pointer
+ * prompt_lens [n], non-positive lengths are ignored): the linear layers see all prompt tokens
+ * (N = their sum), the attention operator of a layer is one fused operator over the requests with
+ * S_q = S_kv = the prompt length (the table's row as printed, no causal discount), timed against
+ * F_ap and M_a, only the last token of each request passes through the LM head, plus O_p.
+ */
+int ooco_predict_prefill_latency(const ooco_model_t* model, const ooco_hw_params_t* hw, const int32_t* prompt_lens,
+                                 int32_t n, ooco_latency_t* out);
+
+/*
  * bs_sat of Algorithm "Offline Request Migration Decision": the smallest decode batch size at
  * which the GEMM operators of an iteration are compute-bound as a whole (summed FLOP time >=
  * summed byte time).  The paper takes the threshold as given; this derives it from the same

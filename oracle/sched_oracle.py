@@ -110,6 +110,50 @@ def L(model, hw, lens) -> float:
     return predict_decode_latency(model, hw, lens)["total"]
 
 
+def prefill_operators(model: Model, prompt_lens):
+    """Every operator of one prefill iteration over the given prompts, in execution order.  Linear
+    layers see all prompt tokens (N = their sum); the attention operator of a layer is one fused
+    operator over the requests with S_q = S_kv = the prompt length (the table has no causal discount);
+    only the last token of each request goes through the LM head."""
+    m, d, tp = model, model.bytes_per_value, model.tp
+    lens = [int(t) for t in prompt_lens if int(t) > 0]
+    ops = []
+    if not lens:
+        return ops
+    N = sum(lens)
+    hq, hkv = m.num_q_heads // tp, m.num_kv_heads // tp
+    D_h = hq * m.head_dim
+    for _ in range(m.num_layers):
+        ops.append(("gemm",) + gemm_cost(N, m.hidden, (hq + 2 * hkv) * m.head_dim, d))
+        fl = by = 0
+        for S in lens:
+            f, b = attention_cost(D_h, S, S, hq, hkv, d)
+            fl, by = fl + f, by + b
+        ops.append(("attention", fl, by))
+        ops.append(("gemm",) + gemm_cost(N, D_h, m.hidden, d))
+        if tp > 1:
+            ops.append(("comm", 0, N * m.hidden * d))
+        ops.append(("gemm",) + gemm_cost(N, m.hidden, (2 if m.gated_mlp else 1) * m.intermediate // tp, d))
+        ops.append(("gemm",) + gemm_cost(N, m.intermediate // tp, m.hidden, d))
+        if tp > 1:
+            ops.append(("comm", 0, N * m.hidden * d))
+    ops.append(("gemm",) + gemm_cost(len(lens), m.hidden, m.vocab // tp, d))
+    return ops
+
+
+def predict_prefill_latency(model: Model, hw: Hw, prompt_lens) -> dict:
+    """Latency of a prefill iteration: operator latencies (attention against F_ap) plus O_p."""
+    parts = {"gemm": 0.0, "attention": 0.0, "comm": 0.0}
+    for kind, fl, by in prefill_operators(model, prompt_lens):
+        if kind == "gemm":
+            parts["gemm"] += op_latency(fl, by, hw.F_g, hw.M_g)
+        elif kind == "attention":
+            parts["attention"] += op_latency(fl, by, hw.F_ap, hw.M_a)
+        else:
+            parts["comm"] += by / hw.B_c
+    return dict(parts, overhead=hw.O_p, total=parts["gemm"] + parts["attention"] + parts["comm"] + hw.O_p)
+
+
 def compute_saturated_batch(model: Model, hw: Hw, limit=1 << 20) -> int:
     """Smallest N whose GEMMs are compute-bound as a whole (linear scan)."""
     for N in range(1, limit):

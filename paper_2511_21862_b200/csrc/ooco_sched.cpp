@@ -93,6 +93,44 @@ int ooco_predict_decode_latency(const ooco_model_t* model, const ooco_hw_params_
   return OOCO_OK;
 }
 
+int ooco_predict_prefill_latency(const ooco_model_t* model, const ooco_hw_params_t* hw, const int32_t* prompt_lens,
+                                 int32_t n, ooco_latency_t* out) {
+  if (!model || !hw || !out || (n > 0 && !prompt_lens)) return OOCO_E_NULLPTR;
+  Predictor p;
+  if (!p.init(model, hw) || n < 0 || !(hw->F_ap > 0) || !(hw->O_p >= 0)) return OOCO_E_SHAPE;
+  const ooco_model_t* m = model;
+  double N = 0.0, sq = 0.0, reqs = 0.0;  // prompt tokens, sum of squared prompt lengths, requests
+  for (int32_t i = 0; i < n; ++i) {
+    if (prompt_lens[i] <= 0) continue;
+    N += prompt_lens[i];
+    sq += (double)prompt_lens[i] * prompt_lens[i];
+    reqs += 1.0;
+  }
+  out->gemm = out->attention = out->comm = 0.0;
+  out->overhead = hw->O_p;
+  out->gemm_compute_bound = out->attention_compute_bound = 0;
+  if (reqs > 0) {
+    const double d = m->bytes_per_value;
+    double layer = 0.0, fl = 0.0, by = 0.0;
+    p.gemm(N, m->hidden, (double)(p.hq + 2 * p.hkv) * m->head_dim, layer, fl, by);
+    p.gemm(N, (double)p.D_h, m->hidden, layer, fl, by);
+    p.gemm(N, m->hidden, (double)(m->gated_mlp ? 2 : 1) * m->intermediate / m->tp, layer, fl, by);
+    p.gemm(N, (double)m->intermediate / m->tp, m->hidden, layer, fl, by);
+    double head = 0.0, hfl = 0.0, hby = 0.0;
+    p.gemm(reqs, m->hidden, (double)m->vocab / m->tp, head, hfl, hby);  // last token of each request only
+    out->gemm = layer * m->num_layers + head;
+    out->gemm_compute_bound = fl * m->num_layers + hfl >= by * m->num_layers + hby;
+    // attention row with S_q = S_kv = prompt length, summed over the requests (one fused operator)
+    const double a_fl = 4.0 * (double)p.D_h * sq / hw->F_ap;
+    const double a_by = 2.0 * d * (N * p.D_h + N * (double)(p.hkv * m->head_dim)) / hw->M_a;
+    out->attention = std::max(a_fl, a_by) * m->num_layers;
+    out->attention_compute_bound = a_fl >= a_by;
+    if (m->tp > 1) out->comm = 2.0 * m->num_layers * (N * m->hidden * d / hw->B_c);
+  }
+  out->total = out->gemm + out->attention + out->comm + out->overhead;
+  return OOCO_OK;
+}
+
 int64_t ooco_compute_saturated_batch(const ooco_model_t* model, const ooco_hw_params_t* hw) {
   Predictor p;
   if (!p.init(model, hw)) return 0;

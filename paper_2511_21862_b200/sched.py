@@ -11,7 +11,7 @@ from .binding import OocoError, lib
 SCHED_EXPORTS = (
     "ooco_predict_decode_latency", "ooco_compute_saturated_batch", "ooco_mix_decoding_select",
     "ooco_migration_length_preference", "ooco_select_closest_to_preference", "ooco_select_evictions",
-    "ooco_fit_bandwidth",
+    "ooco_fit_bandwidth", "ooco_predict_prefill_latency",
 )
 
 
@@ -73,6 +73,8 @@ def _lib():
         vp, i32, i64, f64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_double
         L.ooco_predict_decode_latency.restype = ctypes.c_int
         L.ooco_predict_decode_latency.argtypes = [mp, hp, i64, i64, ctypes.POINTER(ooco_latency_t)]
+        L.ooco_predict_prefill_latency.restype = ctypes.c_int
+        L.ooco_predict_prefill_latency.argtypes = [mp, hp, vp, i32, ctypes.POINTER(ooco_latency_t)]
         L.ooco_compute_saturated_batch.restype = i64
         L.ooco_compute_saturated_batch.argtypes = [mp, hp]
         L.ooco_mix_decoding_select.restype = ctypes.c_int
@@ -108,6 +110,14 @@ def predict_decode_latency(model: Model, hw: Hw, batch_size: int, total_tokens: 
     out = ooco_latency_t()
     _check(_lib().ooco_predict_decode_latency(ctypes.byref(model.c()), ctypes.byref(hw.c()), int(batch_size),
                                               int(total_tokens), ctypes.byref(out)), "ooco_predict_decode_latency")
+    return {n: getattr(out, n) for n, _ in ooco_latency_t._fields_}
+
+
+def predict_prefill_latency(model: Model, hw: Hw, prompt_lens) -> dict:
+    lens = _i32(prompt_lens)
+    out = ooco_latency_t()
+    _check(_lib().ooco_predict_prefill_latency(ctypes.byref(model.c()), ctypes.byref(hw.c()), _p(lens), lens.size,
+                                               ctypes.byref(out)), "ooco_predict_prefill_latency")
     return {n: getattr(out, n) for n, _ in ooco_latency_t._fields_}
 
 

@@ -159,3 +159,21 @@ def test_closest_evictions_and_fit():
     slope, icpt = np.polyfit(xs, ys, 1)
     M, O = so.fit_bandwidth(xs, ys)
     assert M == pytest.approx(1 / slope, rel=1e-9) and O == pytest.approx(icpt, rel=1e-6)
+
+
+def test_prefill_latency_hand_example_and_compute_saturation():
+    """Hand-worked: layers 1, hidden 4, Hq 2, Hkv 1, head_dim 2, intermediate 6 (gated), vocab 8, d 2; prompts 3
+    and 5 (N = 8).  QKV 8x4->8: 512 FLOP, 2(32+32+64) = 256 B; attention D_h = 4: 4*4*(9+25) = 544 FLOP,
+    2*2*(3*4 + 3*2) + 2*2*(5*4 + 5*2) = 72 + 120 = 192 B; O 4->4: 256 FLOP, 2(32+16+32) = 160 B; up 4->12: 768 FLOP,
+    2(32+48+96) = 352 B; down 6->4: 384 FLOP, 2(48+24+32) = 208 B; head (2 last tokens) 4->8: 128 FLOP, 2(8+32+16) = 112 B.
+    F_g 64, M_g 32, F_ap 16, M_a 16, O_p 0.25: gemm max(8,8)+max(4,5)+max(12,11)+max(6,6.5)+max(2,3.5) = 35;
+    attention max(34, 12) = 34."""
+    m = so.Model(1, 4, 2, 1, 2, 6, 8)
+    hw = so.Hw(F_g=64, F_ap=16, F_ad=1, M_g=32, M_a=16, O_p=0.25, O_d=9, B_c=1)
+    r = so.predict_prefill_latency(m, hw, [3, 5])
+    assert (r["gemm"], r["attention"], r["comm"], r["total"]) == pytest.approx((35.0, 34.0, 0.0, 69.25), rel=1e-14)
+    assert so.predict_prefill_latency(m, hw, [])["total"] == 0.25
+    # section 3.3.3: beyond a few hundred tokens prefill is compute-bound (GEMM time proportional to tokens)
+    g = lambda S: so.predict_prefill_latency(QWEN7B, HW, [S])["gemm"]
+    assert g(4096) / g(2048) == pytest.approx(2.0, rel=0.02)
+    assert g(16) / g(8) < 1.1

@@ -123,3 +123,15 @@ def test_closest_evictions_fit_and_argument_errors():
         sched.predict_decode_latency(lm, sched.Hw(0, 1, 1, 1, 1, 0, 0, 1), 1, 1)       # F_g = 0
     with pytest.raises(Exception):
         sched.fit_bandwidth([1.0, 1.0], [2.0, 3.0])                                     # one distinct x
+
+
+@pytest.mark.parametrize("mname,hname", PAIRS)
+def test_prefill_latency_predictor(mname, hname):
+    (om, oh), (lm, lh) = both(mname, hname)
+    rng = np.random.default_rng(4 + hash((mname, hname)) % 2**32)
+    for n in [0, 1, 3, 17]:
+        lens = rng.integers(1, 6000, n).tolist() + ([0, -3] if n == 3 else [])
+        want = so.predict_prefill_latency(om, oh, lens)
+        got = sched.predict_prefill_latency(lm, lh, lens)
+        for k in ("total", "gemm", "attention", "comm", "overhead"):
+            assert got[k] == pytest.approx(want[k], rel=REL, abs=0), (k, n)
