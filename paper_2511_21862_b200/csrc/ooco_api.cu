@@ -563,6 +563,10 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   int ncw = g_knobs[kKnobWarps].load(), cps = g_knobs[kKnobCtasPerSm].load();
   if (!g_overridden[kKnobWarps].load() && (kv8 || G_ > 8)) ncw = 8;
   if (!g_overridden[kKnobCtasPerSm].load() && G_ > 8) cps = 1;
+  // head_dim 64 halves the bytes per token, not the per-token work of the consumers: four smaller CTAs per
+  // SM (16 consumer warps) keep up with HBM where two do not (4.9 -> 6.8 TB/s)
+  if (!g_overridden[kKnobCtasPerSm].load() && !g_overridden[kKnobWarps].load() && G_ <= 8 && s->head_dim == 64)
+    cps = 4;
   int tpw = g_knobs[kKnobTilesPerWarp].load();
   if (ncw == 8 || kv8) tpw = 1;
   const int stage_tok = 16 * ncw * tpw;
