@@ -47,6 +47,9 @@ SMALL = [
     # long enough to be split into several chunks (several stages, ragged last chunk)
     C("split", 32, 8, 128, 16, fixed(5000, 37, 2049, 1025, 300, 9999), seed=42, pool_fill=0.9, shuffle_batch=False),
     C("split-g8-bs32", 64, 8, 128, 32, fixed(20000, 129, 4097, 64), seed=43, sigma=0.5, shuffle_batch=False),
+    # more sequences than the plan keeps in shared memory (its global-memory path), many of them empty or tiny
+    C("batch-5000", 8, 2, 128, 16, (G(5000, 0, 40),), seed=44, pool_fill=0.9),
+    C("batch-4200-d64", 8, 2, 64, 16, (G(4200, 0, 70),), seed=45),
 ]
 
 
