@@ -926,77 +926,115 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------ merge
-// LSE merge of the partial results of split sequences.  One warp per (sequence, query head);
-// warps of unsplit sequences have nothing to do.  Of a split sequence: lanes own D / 32 consecutive dims; chunks are taken 32 at a time (one lse per lane),
-//   out = sum_c 2^(lse_c - M) o_c / sum_c 2^(lse_c - M),  M = max_c lse_c.
+// LSE merge of the partial results of split sequences.  `wpu` warps (1, 2, 4 or 8, all in one CTA)
+// share a (sequence, query token, query head) unit: each takes a contiguous share of the unit's
+// chunks, 32 chunks at a time (one lse per lane), lanes own D / 32 consecutive dims,
+//   out = sum_c 2^(lse_c - M) o_c / sum_c 2^(lse_c - M),  M = max_c lse_c,
+// and the first warp of the unit combines the shares through shared memory.  Units of unsplit
+// sequences have nothing to do.  The host picks wpu > 1 when there are too few units to fill the GPU
+// (a handful of very long sequences).
 template <int D>
-__global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, const int wpu) {
   constexpr int V = D / 32;  // dims per lane
-  const int lane = threadIdx.x & 31;
-  const int warps_total = gridDim.x * (blockDim.x >> 5);
+  __shared__ float s_part[8][D + 2];  // per warp: its share's accumulator, running maximum, denominator
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int units_per_block = 8 / wpu, sub = warp % wpu;
   const int per_seq = p.Sq * p.Hq;  // (query token, query head) rows of one sequence
   const int n_units = p.B * per_seq;
-  int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   // The chunk scan was written by the plan kernel, which had completed before the attention grid
   // (the grid this launch depends on) passed its own dependency wait, so it may be read before
   // the wait below; only the partial results need the attention grid to be complete.
   int first = 0, n = 0;
   grid_dep_launch();  // a programmatically launched successor may start its own prologue
   if (p.hdr->status & kStatusPlanOverflow) return;  // no work list, no partials (status is reported)
-  if (u < n_units) {
-    first = p.seq_first[u / per_seq];
-    n = p.seq_first[u / per_seq + 1] - first;
+  {
+    const int u = blockIdx.x * units_per_block + warp / wpu;
+    if (u < n_units) {
+      first = p.seq_first[u / per_seq];
+      n = p.seq_first[u / per_seq + 1] - first;
+    }
   }
   grid_dep_wait();
-  for (; u < n_units; u += warps_total, first = -1) {
-    const int b = u / per_seq, rem = u % per_seq;
+  for (int ub = blockIdx.x * units_per_block; ub < n_units; ub += gridDim.x * units_per_block, first = -1) {
+    const int u = ub + warp / wpu;
+    const bool live = u < n_units;
+    const int b = live ? u / per_seq : 0, rem = live ? u % per_seq : 0;
     const int qi = rem / p.Hq, hq = rem % p.Hq;
     const int h = hq / p.G, head = qi * p.G + hq % p.G;  // `head` = score column of (query, head) in its group
-    if (first < 0) {
+    if (live && first < 0) {
       first = p.seq_first[b];
       n = p.seq_first[b + 1] - first;
     }
-    if (n <= 1) continue;  // unsplit (or empty) sequence: the attention kernel wrote the row itself
+    const bool work = live && n > 1;  // unsplit (or empty) sequence: the attention kernel wrote the row itself
     float M = -INFINITY, den = 0.f, acc[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) acc[i] = 0.f;
-    for (int c0 = 0; c0 < n; c0 += 32) {
-      const int cnt = min(32, n - c0);
-      float lse = -INFINITY;
-      if (lane < cnt) lse = p.part_lse[((size_t)(first + c0 + lane) * p.Hkv + h) * p.GQ + head];
-      float gm = lse;
+    if (work) {
+      const int c_lo = (int)((long long)n * sub / wpu), c_hi = (int)((long long)n * (sub + 1) / wpu);
+      for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
+        const int cnt = min(32, c_hi - c0);
+        float lse = -INFINITY;
+        if (lane < cnt) lse = p.part_lse[((size_t)(first + c0 + lane) * p.Hkv + h) * p.GQ + head];
+        float gm = lse;
 #pragma unroll
-      for (int o = 16; o; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
-      const float Mn = fmaxf(M, gm);
-      const float Ms = Mn == -INFINITY ? 0.f : Mn;  // nothing seen so far (causal limit): keep exponents finite
-      const float resc = exp2f(M - Ms);
-      M = Mn;
-      const float w_lane = exp2f(lse - Ms);  // 0 for lanes beyond cnt
-      float ws = w_lane;
+        for (int o = 16; o; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
+        const float Mn = fmaxf(M, gm);
+        const float Ms = Mn == -INFINITY ? 0.f : Mn;  // nothing seen so far (causal limit): keep exponents finite
+        const float resc = exp2f(M - Ms);
+        M = Mn;
+        const float w_lane = exp2f(lse - Ms);  // 0 for lanes beyond cnt
+        float ws = w_lane;
 #pragma unroll
-      for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
-      den = den * resc + ws;
+        for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
+        den = den * resc + ws;
 #pragma unroll
-      for (int i = 0; i < V; ++i) acc[i] *= resc;
-      const float* src = p.part_o + (((size_t)(first + c0) * p.Hkv + h) * p.GQ + head) * D + lane * V;
-      const size_t cstride = (size_t)p.Hkv * p.GQ * D;
+        for (int i = 0; i < V; ++i) acc[i] *= resc;
+        const float* src = p.part_o + (((size_t)(first + c0) * p.Hkv + h) * p.GQ + head) * D + lane * V;
+        const size_t cstride = (size_t)p.Hkv * p.GQ * D;
 #pragma unroll 8
-      for (int j = 0; j < cnt; ++j) {
-        const float w = __shfl_sync(0xffffffffu, w_lane, j);
-        if (V == 4) {
-          const float4 o = *reinterpret_cast<const float4*>(src + j * cstride);
-          acc[0] += w * o.x; acc[1] += w * o.y; acc[2] += w * o.z; acc[V - 1] += w * o.w;
-        } else {
-          const float2 o = *reinterpret_cast<const float2*>(src + j * cstride);
-          acc[0] += w * o.x; acc[V - 1] += w * o.y;
+        for (int j = 0; j < cnt; ++j) {
+          const float w = __shfl_sync(0xffffffffu, w_lane, j);
+          if (V == 4) {
+            const float4 o = *reinterpret_cast<const float4*>(src + j * cstride);
+            acc[0] += w * o.x; acc[1] += w * o.y; acc[2] += w * o.z; acc[V - 1] += w * o.w;
+          } else {
+            const float2 o = *reinterpret_cast<const float2*>(src + j * cstride);
+            acc[0] += w * o.x; acc[V - 1] += w * o.y;
+          }
         }
       }
     }
-    __nv_bfloat16* dst = p.out + (((size_t)b * p.Sq + qi) * p.Hq + hq) * D + lane * V;
-    const float inv = den > 0.f ? 1.f / den : 0.f;  // den = 0: the query saw no token at all
+    if (wpu > 1) {  // the unit's first warp folds in the other shares (block-uniform control flow)
+      if (sub != 0) {
 #pragma unroll
-    for (int i = 0; i < V; i += 2)
-      *reinterpret_cast<__nv_bfloat162*>(dst + i) = __floats2bfloat162_rn(acc[i] * inv, acc[i + 1] * inv);
+        for (int i = 0; i < V; ++i) s_part[warp][lane * V + i] = acc[i];
+        if (lane == 0) {
+          s_part[warp][D] = M;
+          s_part[warp][D + 1] = den;
+        }
+      }
+      __syncthreads();
+      if (work && sub == 0) {
+        for (int w = 1; w < wpu; ++w) {
+          const float Mw = s_part[warp + w][D], dw = s_part[warp + w][D + 1];
+          const float Mn = fmaxf(M, Mw);
+          const float Ms = Mn == -INFINITY ? 0.f : Mn;
+          const float ra = exp2f(M - Ms), rb = exp2f(Mw - Ms);
+          M = Mn;
+          den = den * ra + dw * rb;
+#pragma unroll
+          for (int i = 0; i < V; ++i) acc[i] = acc[i] * ra + s_part[warp + w][lane * V + i] * rb;
+        }
+      }
+      __syncthreads();  // the shares are consumed before the next round overwrites them
+    }
+    if (work && sub == 0) {
+      __nv_bfloat16* dst = p.out + (((size_t)b * p.Sq + qi) * p.Hq + hq) * D + lane * V;
+      const float inv = den > 0.f ? 1.f / den : 0.f;  // den = 0: the query saw no token at all
+#pragma unroll
+      for (int i = 0; i < V; i += 2)
+        *reinterpret_cast<__nv_bfloat162*>(dst + i) = __floats2bfloat162_rn(acc[i] * inv, acc[i + 1] * inv);
+    }
   }
 }
 

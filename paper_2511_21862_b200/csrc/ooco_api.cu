@@ -646,14 +646,16 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (rc) return rc;
   if (pe) cudaEventRecord(pe[2], st);
   {
-    long long warps = (long long)p.B * p.Sq * p.Hq;  // (sequence, query token, query head) units
-    int blocks = (int)((warps + 7) / 8);
-    if (blocks > di.sm_count * 8) blocks = di.sm_count * 8;
+    const long long units = (long long)p.B * p.Sq * p.Hq;  // (sequence, query token, query head)
+    int wpu = 1;  // warps per unit: more when the units alone cannot fill the SMs (few, very long sequences)
+    while (wpu < 8 && units * wpu * 2 <= (long long)di.sm_count * 8) wpu *= 2;
+    const long long need = (units * wpu + 7) / 8;
+    const int blocks = (int)(need < (long long)di.sm_count * 8 ? need : (long long)di.sm_count * 8);
     const bool pdl = g_knobs[kKnobPdl].load() != 0 && !pe;
     if (s->head_dim == 128)
-      e = launch_ex(lse_merge_kernel<128>, dim3(blocks), dim3(256), 0, st, pdl, p);
+      e = launch_ex(lse_merge_kernel<128>, dim3(blocks), dim3(256), 0, st, pdl, p, wpu);
     else
-      e = launch_ex(lse_merge_kernel<64>, dim3(blocks), dim3(256), 0, st, pdl, p);
+      e = launch_ex(lse_merge_kernel<64>, dim3(blocks), dim3(256), 0, st, pdl, p, wpu);
   }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the merge kernel", (long)e);
