@@ -345,10 +345,12 @@ size_t ooco_step_staging_bytes(const ooco_shape_t* shape);
  * `cuda_stream` in that order and the call returns after the stream has been
  * SYNCHRONISED, so out_host is valid on return.
  *
- * When all six input buffers are page-locked (cudaHostAlloc / cudaHostRegister, e.g. torch pinned
- * memory) one staging kernel reads them through their device mapping, and a page-locked out_host is
- * written by the attention kernels directly; pageable buffers are detected and go through one
- * cudaMemcpyAsync each.  The results are the same.
+ * When all six input buffers are page-locked and 16-byte aligned (cudaHostAlloc / cudaHostRegister,
+ * e.g. torch pinned memory) the step's first launch reads them through their device mapping (the
+ * planning and append CTAs directly, extra CTAs staging q and the block table for the attention
+ * kernel), and a page-locked out_host is written by the attention kernels directly: three launches,
+ * no copy-engine transfer.  Pageable buffers are detected and go through one cudaMemcpyAsync each.
+ * The results are the same.
  *
  *   q_host, k_new_host, v_new_host   HOST (pinned for full copy speed), bf16
  *                                    [B,Hq,D], [B,Hkv,D], [B,Hkv,D]
@@ -394,7 +396,7 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * 7 16-token tiles per consumer warp and stage {1,2}; 8 non-zero = launch the attention and
  * merge kernels with programmatic dependent launch (their prologues overlap the predecessor);
  * 9 CTAs per SM of the block-movement kernel {1..3}; 10 non-zero = ooco_decode_step_host reads
- * page-locked inputs with one staging kernel and lets the kernels write a page-locked result
+ * page-locked inputs through their device mapping and lets the kernels write a page-locked result
  * directly (zero = always one copy per buffer).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.

@@ -117,12 +117,43 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams a) {
   kv_append_body(a, blockIdx.x, gridDim.x);
 }
 
+// ------------------------------------------------------------------------------------ host staging
+// Host -> device staging of inputs that live in page-locked host memory: the CTAs read the host
+// buffers through their device mapping (16-byte loads over the host link) instead of one copy-engine
+// transfer per buffer, each of which costs several microseconds of fixed latency.
+constexpr int kStageBuffers = 3;
+struct HostStageParams {
+  const uint8_t* src[kStageBuffers];  // device-visible addresses of page-locked host buffers
+  uint8_t* dst[kStageBuffers];        // 256-byte aligned device buffers
+  uint32_t bytes[kStageBuffers];      // multiples of 4; 0 = unused
+};
+__device__ __forceinline__ void host_stage_body(const HostStageParams& p, int block, int nblocks) {
+  const uint32_t tid = block * blockDim.x + threadIdx.x, nthr = nblocks * blockDim.x;
+#pragma unroll 1
+  for (int k = 0; k < kStageBuffers; ++k) {
+    const uint32_t n = p.bytes[k];
+    if (((uintptr_t)p.src[k] & 15) == 0) {
+      const uint32_t n16 = n / 16;
+      for (uint32_t i = tid; i < n16; i += nthr)
+        reinterpret_cast<uint4*>(p.dst[k])[i] = reinterpret_cast<const uint4*>(p.src[k])[i];
+      for (uint32_t i = n16 * 4 + tid; i < n / 4; i += nthr)
+        reinterpret_cast<uint32_t*>(p.dst[k])[i] = reinterpret_cast<const uint32_t*>(p.src[k])[i];
+    } else {
+      for (uint32_t i = tid; i < n / 4; i += nthr)
+        reinterpret_cast<uint32_t*>(p.dst[k])[i] = reinterpret_cast<const uint32_t*>(p.src[k])[i];
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------ plan
-// CTA 0 plans; CTAs 1.. (present only in the fused step) do the KV append.  The plan chooses the chunk length from the total work, splits every sequence into
-// near-equal chunks that are multiples of `stage_tok`, and writes the item list.
+// CTA 0 plans; CTAs 1 .. n_append (present only in the fused step) do the KV append; any further CTAs
+// (host-buffer step only) stage the inputs the attention kernel reads.  The plan chooses the chunk
+// length from the total work, splits every sequence into near-equal chunks that are multiples of
+// `stage_tok`, and writes the item list.
 template <int kThreads>
 __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stage_tok, int first_in_smem,
-                                                        const AppendParams ap) {
+                                                        const AppendParams ap, int n_append,
+                                                        const HostStageParams hs) {
   extern __shared__ int s_first[];  // when they fit (first_in_smem): seq_first [B + 1], then clamped lengths [B]
   // Launched programmatically: nothing of the caller's buffers or of the workspace may be touched
   // before the preceding work in the stream (which may still read the workspace, or still
@@ -130,7 +161,10 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
   grid_dep_wait();
   grid_dep_launch();
   if (blockIdx.x > 0) {
-    kv_append_body(ap, blockIdx.x - 1, gridDim.x - 1);
+    if ((int)blockIdx.x <= n_append)
+      kv_append_body(ap, blockIdx.x - 1, n_append);
+    else
+      host_stage_body(hs, blockIdx.x - 1 - n_append, gridDim.x - 1 - n_append);
     return;
   }
   __shared__ long long s_red[kThreads / 32];

@@ -317,35 +317,6 @@ static int static_scratch_ptr(void** ptr_out) {
 
 static int current_device(int* dev) { return cudaGetDevice(dev) == cudaSuccess ? OOCO_OK : OOCO_E_CUDA; }
 
-// Host -> device staging of a step's small inputs in ONE launch: the kernel reads page-locked host
-// buffers through their device mapping (16-byte loads over the host link) instead of one copy-engine
-// transfer per buffer, each of which costs several microseconds of fixed latency.
-constexpr int kStageBuffers = 6;
-struct HostStageParams {
-  const uint8_t* src[kStageBuffers];  // device-visible addresses of page-locked host buffers
-  uint8_t* dst[kStageBuffers];        // 256-byte aligned device buffers
-  uint32_t bytes[kStageBuffers];      // multiples of 4
-};
-__global__ void __launch_bounds__(256) host_stage_kernel(const HostStageParams p) {
-  grid_dep_wait();
-  grid_dep_launch();
-  const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nthr = gridDim.x * blockDim.x;
-#pragma unroll 1
-  for (int k = 0; k < kStageBuffers; ++k) {
-    const uint32_t n = p.bytes[k];
-    if (((uintptr_t)p.src[k] & 15) == 0) {
-      const uint32_t n16 = n / 16;
-      for (uint32_t i = tid; i < n16; i += nthr)
-        reinterpret_cast<uint4*>(p.dst[k])[i] = reinterpret_cast<const uint4*>(p.src[k])[i];
-      for (uint32_t i = n16 * 4 + tid; i < n / 4; i += nthr)
-        reinterpret_cast<uint32_t*>(p.dst[k])[i] = reinterpret_cast<const uint32_t*>(p.src[k])[i];
-    } else {
-      for (uint32_t i = tid; i < n / 4; i += nthr)
-        reinterpret_cast<uint32_t*>(p.dst[k])[i] = reinterpret_cast<const uint32_t*>(p.src[k])[i];
-    }
-  }
-}
-
 // Device-visible address of a page-locked (pinned / registered) host buffer on the current device,
 // or nullptr when `host` is ordinary pageable memory (which a kernel must never be given).
 static void* mapped_host_pointer(const void* host) {
@@ -541,7 +512,11 @@ static int validate_kv8(const ooco_shape_t* s, const Kv8Scales* kv8) {
 static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache, const void* v_cache,
                        const int32_t* block_table, const int32_t* context_lens, float scale, void* out,
                        void* workspace, size_t workspace_bytes, void* cuda_stream, const AppendParams* append,
-                       const Kv8Scales* kv8 = nullptr, int q_len = 1) {
+                       const Kv8Scales* kv8 = nullptr, int q_len = 1, const HostStageParams* host_stage = nullptr,
+                       const int32_t* plan_context_lens = nullptr) {
+  // host_stage / plan_context_lens (host-buffer step): extra CTAs of the first launch stage q and the
+  // block table for the attention kernel while its planning CTA reads the lengths, and its append CTAs
+  // the new rows, straight from the mapped host buffers.
   int rc = validate_shape(s);
   if (rc) return rc;
   if ((rc = validate_kv8(s, kv8))) return rc;
@@ -629,10 +604,23 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   AppendParams ap;
   memset(&ap, 0, sizeof ap);
   if (append) ap = *append;
-  const int plan_grid = 1 + (append ? append_blocks(s, 1024, append->Sq) : 0);
+  const int n_append = append ? append_blocks(s, 1024, append->Sq) : 0;
+  HostStageParams hs;
+  memset(&hs, 0, sizeof hs);
+  int n_stage = 0;
+  if (host_stage) {
+    hs = *host_stage;
+    size_t total = 0;
+    for (int k = 0; k < kStageBuffers; ++k) total += hs.bytes[k];
+    n_stage = (int)((total / 16 + 1023) / 1024);
+    n_stage = n_stage < 1 ? 1 : (n_stage > 256 ? 256 : n_stage);
+  }
   const bool pdl_on = g_knobs[kKnobPdl].load() != 0 && !pe;
-  cudaError_t e = launch_ex(plan_kernel<1024>, dim3(plan_grid), dim3(1024), first_in_smem ? first_bytes : 0, st,
-                            pdl_on, p, stage_tok, first_in_smem, ap);
+  DecodeParams pp = p;  // the planning CTA may read the lengths from another (host-mapped) copy
+  if (plan_context_lens) pp.context_lens = plan_context_lens;
+  cudaError_t e = launch_ex(plan_kernel<1024>, dim3(1 + n_append + n_stage), dim3(1024),
+                            first_in_smem ? first_bytes : 0, st, pdl_on, pp, stage_tok, first_in_smem, ap, n_append,
+                            hs);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
@@ -886,47 +874,49 @@ int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void*
   uint8_t* d_tab = d_vn + up(kb);
   uint8_t* d_pos = d_tab + up(tb);
   uint8_t* d_len = d_pos + up(lb);
-  const void* hsrc[kStageBuffers] = {q_host, k_new_host, v_new_host, block_table_host, positions_host,
-                                     context_lens_host};
-  uint8_t* ddst[kStageBuffers] = {d_q, d_kn, d_vn, d_tab, d_pos, d_len};
-  const size_t nbytes[kStageBuffers] = {qb, kb, kb, tb, lb, lb};
-  // Page-locked inputs (all six, each under 4 GiB): one staging kernel reads them through their device
-  // mapping.  Otherwise one copy per buffer.
-  HostStageParams hp;
+  const void* hsrc[6] = {q_host, k_new_host, v_new_host, block_table_host, positions_host, context_lens_host};
+  uint8_t* ddst[6] = {d_q, d_kn, d_vn, d_tab, d_pos, d_len};
+  const size_t nbytes[6] = {qb, kb, kb, tb, lb, lb};
+  // Page-locked inputs (all six, each under 4 GiB) are read through their device mapping inside the
+  // step's first launch: the planning CTA reads the lengths, the append CTAs the new rows, positions and
+  // table entries, and extra CTAs stage q, the block table and the lengths for the attention kernel.
+  // Otherwise one copy per buffer.
+  const void* msrc[6];
   bool mapped = g_knobs[kKnobHostStageKernel].load() != 0;
-  for (int k = 0; k < kStageBuffers && mapped; ++k) {
-    hp.src[k] = (const uint8_t*)mapped_host_pointer(hsrc[k]);
-    hp.dst[k] = ddst[k];
-    hp.bytes[k] = (uint32_t)nbytes[k];
-    mapped = hp.src[k] != nullptr && nbytes[k] < ((size_t)1 << 32) && ((uintptr_t)hp.src[k] & 3) == 0;
-  }
-  int launches = 0;
-  if (mapped) {
-    size_t total = 0;
-    for (int k = 0; k < kStageBuffers; ++k) total += nbytes[k];
-    int blocks = (int)((total / 16 + 255) / 256);
-    blocks = blocks < 1 ? 1 : (blocks > 592 ? 592 : blocks);
-    cudaError_t e = launch_ex(host_stage_kernel, dim3(blocks), dim3(256), 0, st, g_knobs[kKnobPdl].load() != 0, hp);
-    if (e == cudaSuccess) e = cudaGetLastError();
-    if (e != cudaSuccess) return fail_cuda("launch of the host staging kernel", (long)e);
-    launches = 1;
-  } else {
-    bool ok = true;
-    for (int k = 0; k < kStageBuffers; ++k)
-      ok &= cudaMemcpyAsync(ddst[k], hsrc[k], nbytes[k], cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!ok) return fail_cuda("cudaMemcpyAsync(host to device)", -1);
+  for (int k = 0; k < 6 && mapped; ++k) {
+    msrc[k] = mapped_host_pointer(hsrc[k]);
+    mapped = msrc[k] != nullptr && nbytes[k] < ((size_t)1 << 32) && ((uintptr_t)msrc[k] & 15) == 0;
   }
   // A page-locked result buffer is written by the kernels themselves, through its device mapping.
   void* out_mapped = g_knobs[kKnobHostStageKernel].load() != 0 ? mapped_host_pointer(out_host) : nullptr;
   if (out_mapped && ((uintptr_t)out_mapped & 15)) out_mapped = nullptr;
-  if ((rc = ooco_decode_step(s, d_q, d_kn, d_vn, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_pos,
-                             (const int32_t*)d_len, scale, out_mapped ? out_mapped : (void*)d_out, workspace,
-                             workspace_bytes, st)))
-    return rc;
+  void* out_dev = out_mapped ? out_mapped : (void*)d_out;
+  if (mapped) {
+    HostStageParams hs;
+    memset(&hs, 0, sizeof hs);
+    const int pick[kStageBuffers] = {0, 3, 5};  // q, block table, lengths
+    for (int k = 0; k < kStageBuffers; ++k) {
+      hs.src[k] = (const uint8_t*)msrc[pick[k]];
+      hs.dst[k] = ddst[pick[k]];
+      hs.bytes[k] = (uint32_t)nbytes[pick[k]];
+    }
+    const AppendParams ap = make_append_params(s, msrc[1], msrc[2], k_cache, v_cache, (const int32_t*)msrc[3],
+                                               (const int32_t*)msrc[4]);
+    if ((rc = decode_core(s, d_q, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_len, scale, out_dev,
+                          workspace, workspace_bytes, st, &ap, nullptr, 1, &hs, (const int32_t*)msrc[5])))
+      return rc;
+  } else {
+    bool ok = true;
+    for (int k = 0; k < 6; ++k)
+      ok &= cudaMemcpyAsync(ddst[k], hsrc[k], nbytes[k], cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) return fail_cuda("cudaMemcpyAsync(host to device)", -1);
+    if ((rc = ooco_decode_step(s, d_q, d_kn, d_vn, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_pos,
+                               (const int32_t*)d_len, scale, out_dev, workspace, workspace_bytes, st)))
+      return rc;
+  }
   if (!out_mapped && cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return fail_cuda("cudaMemcpyAsync(device to host)", -1);
   if (cudaStreamSynchronize(st) != cudaSuccess) return fail_cuda("cudaStreamSynchronize", -1);
-  tl_last_launches += launches;
   return OOCO_OK;
 }
 
