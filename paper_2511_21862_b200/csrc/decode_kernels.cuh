@@ -968,11 +968,11 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 // sequences have nothing to do.  The host picks wpu > 1 when there are too few units to fill the GPU
 // (a handful of very long sequences).
 template <int D>
-__global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, const int wpu) {
+__global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, const int wpu_log2) {
   constexpr int V = D / 32;  // dims per lane
   __shared__ float s_part[8][D + 2];  // per warp: its share's accumulator, running maximum, denominator
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int units_per_block = 8 / wpu, sub = warp % wpu;
+  const int wpu = 1 << wpu_log2, units_per_block = 8 >> wpu_log2, sub = warp & (wpu - 1);
   const int per_seq = p.Sq * p.Hq;  // (query token, query head) rows of one sequence
   const int n_units = p.B * per_seq;
   // The chunk scan was written by the plan kernel, which had completed before the attention grid
@@ -982,7 +982,7 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, co
   grid_dep_launch();  // a programmatically launched successor may start its own prologue
   if (p.hdr->status & kStatusPlanOverflow) return;  // no work list, no partials (status is reported)
   {
-    const int u = blockIdx.x * units_per_block + warp / wpu;
+    const int u = blockIdx.x * units_per_block + (warp >> wpu_log2);
     if (u < n_units) {
       first = p.seq_first[u / per_seq];
       n = p.seq_first[u / per_seq + 1] - first;
@@ -990,7 +990,7 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, co
   }
   grid_dep_wait();
   for (int ub = blockIdx.x * units_per_block; ub < n_units; ub += gridDim.x * units_per_block, first = -1) {
-    const int u = ub + warp / wpu;
+    const int u = ub + (warp >> wpu_log2);
     const bool live = u < n_units;
     const int b = live ? u / per_seq : 0, rem = live ? u % per_seq : 0;
     const int qi = rem / p.Hq, hq = rem % p.Hq;
@@ -1004,7 +1004,7 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, co
 #pragma unroll
     for (int i = 0; i < V; ++i) acc[i] = 0.f;
     if (work) {
-      const int c_lo = (int)((long long)n * sub / wpu), c_hi = (int)((long long)n * (sub + 1) / wpu);
+      const int c_lo = (int)(((long long)n * sub) >> wpu_log2), c_hi = (int)(((long long)n * (sub + 1)) >> wpu_log2);
       for (int c0 = c_lo; c0 < c_hi; c0 += 32) {
         const int cnt = min(32, c_hi - c0);
         float lse = -INFINITY;

@@ -635,15 +635,15 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (pe) cudaEventRecord(pe[2], st);
   {
     const long long units = (long long)p.B * p.Sq * p.Hq;  // (sequence, query token, query head)
-    int wpu = 1;  // warps per unit: more when the units alone cannot fill the SMs (few, very long sequences)
-    while (wpu < 8 && units * wpu * 2 <= (long long)di.sm_count * 8) wpu *= 2;
-    const long long need = (units * wpu + 7) / 8;
+    int wpu_log2 = 0;  // warps per unit: more when the units alone cannot fill the SMs (few, very long sequences)
+    while (wpu_log2 < 3 && (units << (wpu_log2 + 1)) <= (long long)di.sm_count * 8) ++wpu_log2;
+    const long long need = ((units << wpu_log2) + 7) / 8;
     const int blocks = (int)(need < (long long)di.sm_count * 8 ? need : (long long)di.sm_count * 8);
     const bool pdl = g_knobs[kKnobPdl].load() != 0 && !pe;
     if (s->head_dim == 128)
-      e = launch_ex(lse_merge_kernel<128>, dim3(blocks), dim3(256), 0, st, pdl, p, wpu);
+      e = launch_ex(lse_merge_kernel<128>, dim3(blocks), dim3(256), 0, st, pdl, p, wpu_log2);
     else
-      e = launch_ex(lse_merge_kernel<64>, dim3(blocks), dim3(256), 0, st, pdl, p, wpu);
+      e = launch_ex(lse_merge_kernel<64>, dim3(blocks), dim3(256), 0, st, pdl, p, wpu_log2);
   }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the merge kernel", (long)e);
