@@ -253,3 +253,23 @@ def test_step_replays_from_a_cuda_graph():
     assert torch.equal(out_direct.view(torch.int16), out_graph.view(torch.int16))
     ref = oracle_attention(batch, context_lens=lens1)
     assert_parity(out_graph, ref.out, what="graph replay")
+
+
+def test_kv_head_sharding_needs_no_exchange():
+    """Tensor-parallel layout: each of two ranks holds half of the kv heads of the pool and the
+    matching query heads; their outputs, side by side on the head axis, are the unsharded result."""
+    cfg = C("tp2", 32, 8, 128, 16, (G(9, 1, 2500),), seed=57, pool_fill=0.8)
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    ref = oracle_attention(batch)
+    outs = []
+    for rank in range(2):
+        k = batch.k_cache[:, 4 * rank:4 * rank + 4].contiguous()             # [NB, Hkv / 2, bs, D]
+        v = batch.v_cache[:, 4 * rank:4 * rank + 4].contiguous()
+        q = batch.q[:, 16 * rank:16 * rank + 16].contiguous()
+        sh = binding.Shape(cfg.batch, 16, 4, 128, 16, batch.num_blocks, batch.max_blocks_per_seq, 4 * 16 * 128, 16 * 128, 128)
+        ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device="cuda")
+        out = torch.full_like(q, float("nan"))
+        binding.decode_attention(sh, q, k, v, batch.block_table, batch.context_lens, cfg.scale, out, ws)
+        assert binding.workspace_status(ws) == 0
+        outs.append(out)
+    assert_parity(torch.cat(outs, dim=1), ref.out, what="kv-head sharding")
