@@ -535,6 +535,197 @@ def run_multi_query(args, local_rank):
         "gpu_launches": 4 * args.steps, "clocks": sampler.summary(t0, t1)}))
 
 
+def run_serve_loop(args, local_rank):
+    """Secondary measurement: the step-level scheduling of a latency-strict instance driving the kernels.
+
+    An attention-only instance (one layer) decodes all its online requests every step and, beside them, the
+    offline requests Algorithm "Mix Decoding Selection" admits under the TPOT bound S; after each step
+    Algorithm "Offline Request Migration Decision" may pull offline requests of the preferred length from a
+    pool of candidates (a latency-relaxed instance), online requests arrive and leave, and when the KV pool
+    is full offline requests are evicted by the rule of section 3.4.1.  Every step is one
+    ooco_decode_step_host call (block tables, lengths and new rows come from host memory); its wall time
+    is what is compared with S.  The latency predictor uses M_a and the overhead fitted on a few
+    host-step measurements taken first; the bound handed to the algorithms carries a 3 % margin and a running
+    measured / predicted correction."""
+    import numpy as np
+    from paper_2511_21862_b200 import binding, build, sched
+    build.build()
+    binding.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream()
+    rng = np.random.default_rng(2024)
+    Hq, Hkv, D, bs = 40, 8, 128, 16                                        # the cfg2 shape
+    scale = 1.0 / math.sqrt(D)
+    cap_tokens = args.pool_tokens
+    NB = cap_tokens // bs
+    MB = (32768 + 2048) // bs
+    Bmax = 640
+    g = torch.Generator(device=dev).manual_seed(9)
+    k_cache = (torch.randn((NB, Hkv, bs, D), generator=g, device=dev)).to(torch.bfloat16)
+    v_cache = (torch.randn((NB, Hkv, bs, D), generator=g, device=dev)).to(torch.bfloat16)
+    pin = lambda t: t.pin_memory()
+    hq = pin(torch.randn((Bmax, Hq, D)).to(torch.bfloat16))
+    hk = pin(torch.randn((Bmax, Hkv, D)).to(torch.bfloat16))
+    hv = pin(torch.randn((Bmax, Hkv, D)).to(torch.bfloat16))
+    htab = pin(torch.zeros((Bmax, MB), dtype=torch.int32))
+    hpos = pin(torch.zeros(Bmax, dtype=torch.int32))
+    hlen = pin(torch.zeros(Bmax, dtype=torch.int32))
+    hout = pin(torch.empty((Bmax, Hq, D), dtype=torch.bfloat16))
+    free_blocks = list(rng.permutation(NB))
+
+    class Req:
+        __slots__ = ("len", "left", "blocks", "online")
+
+        def __init__(self, length, left, online):
+            self.len, self.left, self.online, self.blocks = int(length), int(left), online, []
+
+    def reserve(r, tokens):                                                # blocks for `tokens` cached tokens
+        need = -(-tokens // bs) - len(r.blocks)
+        if need > len(free_blocks):
+            return False
+        for _ in range(max(0, need)):
+            r.blocks.append(free_blocks.pop())
+        return True
+
+    def release(r):
+        free_blocks.extend(r.blocks)
+        r.blocks = []
+
+    def run_step(batch):
+        B = len(batch)
+        tab = htab.numpy()
+        for i, r in enumerate(batch):
+            tab[i, :len(r.blocks)] = r.blocks
+            hpos[i] = r.len
+            hlen[i] = r.len + 1
+        sh = binding.Shape(B, Hq, Hkv, D, bs, NB, MB, Hkv * bs * D, bs * D, D)
+        ws = ws_all[: binding.workspace_bytes(sh)]
+        stg = stg_all[: binding.step_staging_bytes(sh)]
+        t0 = time.perf_counter()
+        binding.decode_step_host(sh, hq[:B], hk[:B], hv[:B], htab[:B], hpos[:B], hlen[:B], k_cache, v_cache, scale,
+                                 hout[:B], stg, ws, stream)
+        return time.perf_counter() - t0
+
+    sh_max = binding.Shape(Bmax, Hq, Hkv, D, bs, NB, MB, Hkv * bs * D, bs * D, D)
+    ws_all = torch.empty(binding.workspace_bytes(sh_max), dtype=torch.uint8, device=dev)
+    stg_all = torch.empty(binding.step_staging_bytes(sh_max), dtype=torch.uint8, device=dev)
+
+    # ---- profiling data for the predictor: a few batches through the same host-step call
+    xs, ys = [], []
+    for nreq, lo, hi in ((32, 512, 4096), (96, 2048, 8192), (160, 4096, 16384), (64, 8192, 32768), (256, 4096, 12000),
+                         (48, 512, 2048), (128, 1024, 6000)):
+        reqs = [Req(rng.integers(lo, hi), 1, False) for _ in range(nreq)]
+        while sum(r.len + bs for r in reqs) > 0.9 * cap_tokens:           # a small pool: fewer requests
+            reqs.pop()
+        assert all(reserve(r, r.len + 1) for r in reqs)
+        nreq = len(reqs)
+        for _ in range(3):
+            run_step(reqs)
+        t = min(run_step(reqs) for _ in range(10))
+        sh = binding.Shape(nreq, Hq, Hkv, D, bs, NB, MB, Hkv * bs * D, bs * D, D)
+        cost = binding.decode_bytes_model(sh, torch.tensor([r.len + 1 for r in reqs], dtype=torch.int32))
+        xs.append(cost["bytes_paper"]); ys.append(t)
+        for r in reqs:
+            release(r)
+    M_a, O = sched.fit_bandwidth(xs, ys)
+    model = sched.Model(1, Hq * D, Hq, Hkv, D, D, D)
+    big = 1e30
+    hw = sched.Hw(big, big, big, big, M_a, 0.0, O, big)
+    bs_sat = 256                                                           # an instance parameter (compute-saturated batch)
+
+    # ---- the instance
+    S = args.slo_ms * 1e-3
+    margin = 0.97
+    corr = 1.0                                                             # running measured / predicted ratio
+    online = [Req(rng.integers(512, 4097), rng.integers(50, 300), True) for _ in range(32)]
+    for r in online:
+        assert reserve(r, r.len + 1)
+    offline = []
+    new_offline = lambda: Req(int(np.exp(rng.uniform(np.log(4096), np.log(32768)))), rng.integers(100, 1000), False)
+    relaxed_pool = [new_offline() for _ in range(400)]
+    stats = {"steps": 0, "within": 0, "batch": 0, "offline_tokens": 0, "evicted": 0, "migrated": 0, "worst_ms": 0.0,
+             "sum_ms": 0.0, "online_tokens": 0, "pred_err": 0.0}
+    t_begin = time.perf_counter()
+    for step_i in range(args.steps):
+        on_lens = [r.len + 1 for r in online]
+        off_lens = [r.len + 1 for r in offline]
+        K = 8
+        probes = rng.permutation(len(offline))[:K].tolist() if offline else []
+        sel, pred, over = sched.mix_decoding_select(model, hw, on_lens, off_lens, S * margin / corr, probes, len(probes))
+        chosen = [r for r, m in zip(offline, sel) if m]
+        batch = online + chosen
+        # room for the token of this step; when the pool runs dry, offline requests are evicted by the rule
+        # of section 3.4.1 (they go back to the latency-relaxed side and leave this step's batch)
+        while True:
+            short = sum(1 for r in batch if len(r.blocks) * bs < r.len + 1) - len(free_blocks)
+            if short <= 0:
+                break
+            ev, freed = sched.select_evictions([x.len for x in offline], (short + 32) * bs, len(batch) >= bs_sat)
+            assert ev.any(), "KV pool exhausted by online requests alone"
+            for x, e in zip(list(offline), ev):
+                if e:
+                    release(x); offline.remove(x); relaxed_pool.append(x); stats["evicted"] += 1
+                    if x in chosen:
+                        chosen.remove(x)
+            batch = online + chosen
+        for r in batch:
+            assert reserve(r, r.len + 1)
+        sec = run_step(batch)
+        stats["steps"] += 1
+        stats["within"] += sec <= S
+        stats["batch"] += len(batch)
+        stats["sum_ms"] += sec * 1e3
+        stats["worst_ms"] = max(stats["worst_ms"], sec * 1e3)
+        stats["pred_err"] += abs(pred - sec) / sec
+        corr = 0.9 * corr + 0.1 * min(1.5, max(0.67, sec / pred))         # feedback on the predictor's bias
+        stats["offline_tokens"] += len(chosen)
+        stats["online_tokens"] += len(online)
+        for r in batch:
+            r.len += 1
+            r.left -= 1
+        for r in [r for r in online if r.left <= 0]:                       # finished online requests leave, new ones arrive
+            release(r); online.remove(r)
+            n = Req(rng.integers(512, 4097), rng.integers(50, 300), True)
+            need = -(-(n.len + 1) // bs)
+            if need > len(free_blocks):                                    # section 3.4.1: evict offline requests to make room
+                ev, freed = sched.select_evictions([x.len for x in offline], (need - len(free_blocks)) * bs,
+                                                   len(batch) >= bs_sat)
+                for x, e in zip(list(offline), ev):
+                    if e:
+                        release(x); offline.remove(x); relaxed_pool.append(x); stats["evicted"] += 1
+            assert reserve(n, n.len + 1)
+            online.append(n)
+        for r in [r for r in offline if r.left <= 0]:
+            release(r); offline.remove(r); relaxed_pool.append(new_offline())
+        # migration decision (pull model): only when everything on the instance already decodes
+        tokens = sum(r.len for r in batch)
+        pref = sched.migration_length_preference(model, hw, len(batch), tokens, len(chosen) == len(offline), S * margin / corr,
+                                                 bs_sat, cap_tokens - 64 * bs, 4096, 32768)
+        if pref >= 0 and relaxed_pool:
+            picks = sched.select_closest_to_preference([r.len for r in relaxed_pool], pref, 4)
+            for idx in sorted(picks, reverse=True):
+                r = relaxed_pool[idx]
+                headroom = 2 * (len(batch) + 4)                            # blocks the residents will need soon
+                if -(-(r.len + 1) // bs) + headroom <= len(free_blocks) and reserve(r, r.len + 1):
+                    offline.append(relaxed_pool.pop(idx)); stats["migrated"] += 1
+    wall = time.perf_counter() - t_begin
+    n = stats["steps"]
+    print(json.dumps({
+        "metric": "latency-strict instance loop: share of decode steps within the TPOT bound", "value": stats["within"] / n,
+        "unit": "fraction", "higher_is_better": True, "n_gpus": 1, "steps": n, "data": "synthetic", "dtype": "bf16",
+        "config": {"workload": "32 online requests U[512,4096] + offline requests log-uniform [4096,32768] pulled by "
+                               "the migration decision; cfg2 head shape; one layer", "slo_ms": args.slo_ms,
+                   "margin": margin, "pool_tokens": cap_tokens, "bs_sat": bs_sat},
+        "fitted": {"M_a_GBps": M_a / 1e9, "overhead_us": O * 1e6},
+        "mean_step_ms": stats["sum_ms"] / n, "worst_step_ms": stats["worst_ms"], "mean_batch": stats["batch"] / n,
+        "mean_abs_prediction_error": stats["pred_err"] / n,
+        "offline_tokens_per_s_of_gpu_time": stats["offline_tokens"] / (stats["sum_ms"] * 1e-3),
+        "online_tokens_per_s_of_gpu_time": stats["online_tokens"] / (stats["sum_ms"] * 1e-3),
+        "slo_utilisation": stats["sum_ms"] / n / args.slo_ms, "migrated": stats["migrated"], "evicted": stats["evicted"],
+        "offline_resident_at_end": len(offline), "host_loop_wall_s": wall}))
+
+
 def run_model_fit(args, local_rank):
     """Secondary measurement: the attention term of the Roofline latency model against this kernel.
 
@@ -663,16 +854,23 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--ref-token-heads", type=int, default=400000,
                     help="reference arm: (tokens x q heads) of oracle work per step")
-    ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate", "model_fit", "decode_mq"],
+    ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate", "model_fit", "decode_mq", "serve_loop"],
                     help="decode_step: the decode hot path (default); kv_migrate: paged block gather + scatter; "
                          "model_fit: fit and validate the attention term of the latency model; "
-                         "decode_mq: --q-len query tokens per sequence")
+                         "decode_mq: --q-len query tokens per sequence; serve_loop: scheduler-driven decode loop")
+    ap.add_argument("--slo-ms", type=float, default=1.0, help="serve_loop: TPOT bound of the one-layer instance")
+    ap.add_argument("--pool-tokens", type=int, default=3_000_000, help="serve_loop: KV pool capacity in tokens")
     ap.add_argument("--q-len", type=int, default=4, help="decode_mq: query tokens per sequence")
     ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
                     help="decode_step: KV cache element type (fp8 = E4M3 codes; a secondary measurement)")
     ap.add_argument("--move-seqs", type=int, default=64, help="kv_migrate: sequences whose blocks are moved")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
+    if args.op == "serve_loop":
+        if rank == 0:
+            args.steps = args.steps if args.steps is not None else 600
+            run_serve_loop(args, local_rank)
+        return
     if args.op == "decode_mq":
         if rank == 0:
             args.steps = args.steps if args.steps is not None else 300
