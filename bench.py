@@ -459,8 +459,7 @@ def run_block_moves(args, rank, local_rank, world):
 
 def run_multi_query(args, local_rank):
     """Secondary measurement: several query tokens per sequence (multi-token decode).  One step appends
-    q_len new tokens per sequence (ooco_kv_append_mq) and attends with causal masking over the cache
-    (ooco_decode_attention_mq).  Bytes follow the operator table with S_q = q_len."""
+    q_len new tokens per sequence and attends with causal masking over the cache (ooco_decode_step_mq).  Bytes follow the operator table with S_q = q_len."""
     from paper_2511_21862_b200 import binding, build
     build.build()
     binding.lib()
@@ -494,8 +493,8 @@ def run_multi_query(args, local_rank):
 
     def step(i):
         k, v = pools[i % R]
-        binding.kv_append_mq(sh, k_new, v_new, k, v, batch.block_table, positions, stream)
-        binding.decode_attention_mq(sh, q, k, v, batch.block_table, batch.context_lens, cfg.scale, out, ws, stream)
+        binding.decode_step_mq(sh, q, k_new, v_new, k, v, batch.block_table, positions, batch.context_lens, cfg.scale,
+                               out, ws, stream)
     sampler = ClockSampler(local_rank)
     sampler.start()
     for i in range(args.warmup):
@@ -525,14 +524,14 @@ def run_multi_query(args, local_rank):
         "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{cfg.name}, {Sq} query tokens per sequence", "batch": B,
-                   "total_tokens": cost["total_tokens"], "step": "ooco_kv_append_mq + ooco_decode_attention_mq, one layer",
+                   "total_tokens": cost["total_tokens"], "step": "ooco_decode_step_mq, one layer",
                    "l2": f"inputs larger than L2: steps rotate over {R} pool replicas"},
         "query_tokens_per_s": B * Sq / (ms * 1e-3),
         "kernel_ms": {"plan": sum(r[0] for r in recs) / len(recs), "attention": attn, "merge": sum(r[2] for r in recs) / len(recs)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "kernel": "decode_main_kernel", "algorithmic_bytes_per_launch": nbytes,
                      "traffic": None},
-        "gpu_launches": 4 * args.steps, "clocks": sampler.summary(t0, t1)}))
+        "gpu_launches": 3 * args.steps, "clocks": sampler.summary(t0, t1)}))
 
 
 def run_serve_loop(args, local_rank):

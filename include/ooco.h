@@ -190,6 +190,12 @@ int ooco_decode_attention_mq(const ooco_shape_t* shape, int32_t q_len, const voi
 int ooco_kv_append_mq(const ooco_shape_t* shape, int32_t q_len, const void* k_new, const void* v_new,
                       void* k_cache, void* v_cache, const int32_t* block_table, const int32_t* positions,
                       void* cuda_stream);
+/* ooco_kv_append_mq fused into the first launch of ooco_decode_attention_mq (three launches), as
+ * ooco_decode_step does for one token; a serving step passes context_lens = positions + q_len. */
+int ooco_decode_step_mq(const ooco_shape_t* shape, int32_t q_len, const void* q, const void* k_new,
+                        const void* v_new, void* k_cache, void* v_cache, const int32_t* block_table,
+                        const int32_t* positions, const int32_t* context_lens, float scale, void* out,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * The same three operations over an 8-bit KV cache (the operator model's d, "byte per value", set

@@ -747,6 +747,22 @@ int ooco_kv_append_mq(const ooco_shape_t* s, int32_t q_len, const void* k_new, c
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the append kernel", (long)e);
 }
 
+int ooco_decode_step_mq(const ooco_shape_t* s, int32_t q_len, const void* q, const void* k_new, const void* v_new,
+                        void* k_cache, void* v_cache, const int32_t* block_table, const int32_t* positions,
+                        const int32_t* context_lens, float scale, void* out, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  if ((rc = validate_q_len(s, q_len, false))) return rc;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
+    return OOCO_E_UNSUPPORTED;
+  AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
+  ap.Sq = q_len;
+  return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                     cuda_stream, &ap, nullptr, q_len);
+}
+
 int ooco_decode_attention_static(const ooco_shape_t* s, const void* q, const void* k_cache,
                                  const void* v_cache, const int32_t* block_table,
                                  const int32_t* context_lens, float scale, void* out, void* cuda_stream) {
