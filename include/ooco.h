@@ -179,7 +179,7 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  *                   position positions[b] + i (ooco_kv_append_mq); positions beyond the block table
  *                   are skipped, as in ooco_kv_append
  *   workspace       >= ooco_decode_workspace_bytes_mq(shape, q_len)
- * Supported: (Hq / Hkv) * q_len <= 16; bf16 caches.  q_len = 1 is ooco_decode_attention /
+ * Supported: (Hq / Hkv) * q_len <= 16.  q_len = 1 is ooco_decode_attention /
  * ooco_kv_append exactly.  Everything else as for those two.
  */
 size_t ooco_decode_workspace_bytes_mq(const ooco_shape_t* shape, int32_t q_len);
@@ -226,6 +226,18 @@ int ooco_decode_step_fp8(const ooco_shape_t* shape, const void* q, const void* k
                          void* k_cache, void* v_cache, const int32_t* block_table, const int32_t* positions,
                          const int32_t* context_lens, float scale, float k_scale, float v_scale, void* out,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Both variants at once: q_len query tokens per sequence over an 8-bit cache.  With k_new and v_new
+ * (bf16 [B, q_len, Hkv, head_dim]) the quantising append of the q_len new tokens at positions[b] + i
+ * is fused into the first launch, as in ooco_decode_step_mq; with both NULL (positions may be NULL
+ * too) only the attention runs.  Restrictions: those of the two variants together.
+ */
+int ooco_decode_step_mq_fp8(const ooco_shape_t* shape, int32_t q_len, const void* q, const void* k_new,
+                            const void* v_new, void* k_cache, void* v_cache, const int32_t* block_table,
+                            const int32_t* positions, const int32_t* context_lens, float scale, float k_scale,
+                            float v_scale, void* out, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream);
 
 /*
  * Paged decode attention for callers that cannot allocate device memory.  (The paper has no

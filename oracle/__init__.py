@@ -201,6 +201,20 @@ def decode_attention_fp8(q, k_cache, v_cache, block_table, context_lens, scale, 
     return AttentionResult(out, lse, wsum)
 
 
+def decode_attention_mq_fp8(q, k_cache, v_cache, block_table, context_lens, scale, k_scale, v_scale, *, num_kv_heads,
+                            block_size, strides) -> AttentionResult:
+    """decode_attention_mq over uint8 E4M3 pools: the one-query 8-bit operator on B * Sq rows."""
+    q = _u16(q)
+    B, Sq, Hq, D = q.shape
+    lens = _i32(context_lens)
+    lens_x = (lens[:, None] - Sq + 1 + np.arange(Sq, dtype=np.int32)[None, :]).reshape(-1)
+    lens_x = np.where(np.repeat(lens, Sq) <= 0, 0, np.maximum(lens_x, 0)).astype(np.int32)
+    r = decode_attention_fp8(q.reshape(B * Sq, Hq, D), k_cache, v_cache, np.repeat(_i32(block_table), Sq, axis=0),
+                             lens_x, scale, k_scale, v_scale, num_kv_heads=num_kv_heads, block_size=block_size,
+                             strides=strides)
+    return AttentionResult(r.out.reshape(B, Sq, Hq, D), r.lse.reshape(B, Sq, Hq), r.wsum.reshape(B, Sq, Hq))
+
+
 def kv_append_fp8(k_new, v_new, k_cache, v_cache, block_table, positions, k_scale, v_scale, *, block_size,
                   strides) -> int:
     """In-place quantising append of bf16 rows (uint16 bits) into uint8 E4M3 pools."""

@@ -23,7 +23,7 @@ EXPORTS = (
     "ooco_kv_gather_blocks", "ooco_kv_scatter_blocks", "ooco_kv_copy_blocks",
     "ooco_kv_append_fp8", "ooco_decode_attention_fp8", "ooco_decode_step_fp8",
     "ooco_decode_workspace_bytes_mq", "ooco_decode_attention_mq", "ooco_kv_append_mq", "ooco_attention_bytes_model",
-    "ooco_decode_step_mq",
+    "ooco_decode_step_mq", "ooco_decode_step_mq_fp8",
 )
 
 
@@ -87,6 +87,9 @@ def lib() -> ctypes.CDLL:
         L.ooco_decode_step_mq.restype = ctypes.c_int
         L.ooco_decode_step_mq.argtypes = [sp, ctypes.c_int32, vp, vp, vp, vp, vp, i32p, i32p, i32p, ctypes.c_float, vp,
                                           vp, ctypes.c_size_t, vp]
+        L.ooco_decode_step_mq_fp8.restype = ctypes.c_int
+        L.ooco_decode_step_mq_fp8.argtypes = [sp, ctypes.c_int32, vp, vp, vp, vp, vp, i32p, i32p, i32p, ctypes.c_float,
+                                              ctypes.c_float, ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
         L.ooco_kv_append_mq.restype = ctypes.c_int
         L.ooco_kv_append_mq.argtypes = [sp, ctypes.c_int32, vp, vp, vp, vp, i32p, i32p, vp]
         L.ooco_kv_gather_blocks.restype = ctypes.c_int
@@ -269,6 +272,18 @@ def decode_step_mq(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table,
         _dev(block_table, torch.int32), _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale),
         _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_step_mq")
+
+
+def decode_step_mq_fp8(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table, positions, context_lens, scale,
+                       k_scale, v_scale, out, workspace, stream=None):
+    """Several query tokens over uint8 (E4M3) caches; k_new = v_new = None runs the attention only."""
+    assert q.dim() == 4 and q.shape == out.shape
+    _check(lib().ooco_decode_step_mq_fp8(
+        ctypes.byref(shape.c()), int(q.shape[1]), _dev(q, torch.bfloat16), _opt_dev(k_new, torch.bfloat16),
+        _opt_dev(v_new, torch.bfloat16), _dev(k_cache, torch.uint8), _dev(v_cache, torch.uint8),
+        _dev(block_table, torch.int32), _opt_dev(positions, torch.int32), _dev(context_lens, torch.int32),
+        float(scale), float(k_scale), float(v_scale), _dev(out, torch.bfloat16), _dev(workspace),
+        workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step_mq_fp8")
 
 
 def kv_append_mq(shape: Shape, k_new, v_new, k_cache, v_cache, block_table, positions, stream=None):

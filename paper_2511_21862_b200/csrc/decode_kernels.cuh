@@ -501,7 +501,8 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
                                                  const uint32_t (&pat)[D / 16], const uint32_t (&qf)[NT][D / 16][2],
                                                  float (&m_run)[NT][2], float (&l_run)[NT][2],
                                                  float (&o_acc)[NT][D / 16][4], float scale_log2e, int valid,
-                                                 int g, int t) {
+                                                 int g, int t, int lim_w = 0, const int (*qi_col)[2] = nullptr) {
+  // kTail only: lim_w / qi_col carry the causal limit of several query tokens, as in consume_tiles
   constexpr int KS = D / 16;  // 16-dim chunks
   float sc[NT][2][4];
 #pragma unroll
@@ -531,8 +532,11 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
 #pragma unroll
     for (int e = 0; e < 4; ++e) s[e] = (sc[nt][0][e] + sc[nt][1][e]) * scale_log2e;
     if (kTail) {
-      if (g >= valid) s[0] = s[1] = -INFINITY;
-      if (g + 8 >= valid) s[2] = s[3] = -INFINITY;
+      const int l0 = min(valid, lim_w + qi_col[nt][0]), l1 = min(valid, lim_w + qi_col[nt][1]);
+      if (g >= l0) s[0] = -INFINITY;
+      if (g >= l1) s[1] = -INFINITY;
+      if (g + 8 >= l0) s[2] = -INFINITY;
+      if (g + 8 >= l1) s[3] = -INFINITY;
     }
     float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
 #pragma unroll
@@ -540,10 +544,15 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
     }
-    const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
-    const float al0 = ex2(m_run[nt][0] - mn0), al1 = ex2(m_run[nt][1] - mn1);
+    const float mo0 = m_run[nt][0], mo1 = m_run[nt][1];
+    float mn0 = fmaxf(mo0, mx0), mn1 = fmaxf(mo1, mx1);
     m_run[nt][0] = mn0;
     m_run[nt][1] = mn1;
+    if (kTail) {  // a column that has seen nothing yet (causal limit): keep the exponents finite
+      mn0 = mn0 == -INFINITY ? 0.f : mn0;
+      mn1 = mn1 == -INFINITY ? 0.f : mn1;
+    }
+    const float al0 = ex2(mo0 - mn0), al1 = ex2(mo1 - mn1);
     const uint32_t p01 = pack_f16x2(ex2(s[0] - mn0), ex2(s[1] - mn1));  // token g
     const uint32_t p23 = pack_f16x2(ex2(s[2] - mn0), ex2(s[3] - mn1));  // token g+8
     // sums use the rounded weights, so numerator and denominator agree exactly
@@ -856,14 +865,15 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (valid > 0) {
       const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;
       const uint32_t vst = kst + L::kTileBytes;
+      // rows of this warp the first query token may see; with one query token that is all of them
+      const int lim_w = ((meta.w >> 18) & 1023) - 16 - r0;
       if (KV8) {
-        if (valid >= 16)
+        if (valid >= 16 && lim_w >= 16)
           consume_tile_kv8<D, NT, false>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t);
         else
-          consume_tile_kv8<D, NT, true>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t);
+          consume_tile_kv8<D, NT, true>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t,
+                                        lim_w, qi_col);
       } else {
-        // rows of this warp the first query token may see; with one query token that is all of them
-        const int lim_w = ((meta.w >> 18) & 1023) - 16 - r0;
         if (valid >= 16 * TPW && lim_w >= 16 * TPW)
           consume_tiles<D, NT, TPW, false>(kst, vst, tile_k, tile_v, kpat, vpat, qf, m_run, l_run, o_acc,
                                            p.scale_log2e, valid, g, t);

@@ -489,11 +489,11 @@ size_t ooco_decode_workspace_bytes(const ooco_shape_t* s) {
 
 // Plan (+ optional fused append) -> split-KV attention -> LSE merge on `cuda_stream`.
 // Query tokens per sequence: the score columns of a (sequence, kv head) pair, G * q_len, must fit the
-// two 8-column MMA tiles of the kernel; the 8-bit path is built for one query token.
-static int validate_q_len(const ooco_shape_t* s, int q_len, bool kv8) {
+// two 8-column MMA tiles of the kernel.
+static int validate_q_len(const ooco_shape_t* s, int q_len) {
   if (q_len < 1) return OOCO_E_SHAPE;
   if (q_len == 1) return OOCO_OK;
-  if (kv8 || (long long)(s->num_q_heads / s->num_kv_heads) * q_len > 16) return OOCO_E_UNSUPPORTED;
+  if ((long long)(s->num_q_heads / s->num_kv_heads) * q_len > 16) return OOCO_E_UNSUPPORTED;
   return OOCO_OK;
 }
 
@@ -520,7 +520,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   int rc = validate_shape(s);
   if (rc) return rc;
   if ((rc = validate_kv8(s, kv8))) return rc;
-  if ((rc = validate_q_len(s, q_len, kv8 != nullptr))) return rc;
+  if ((rc = validate_q_len(s, q_len))) return rc;
   if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
   if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q) & 15) return OOCO_E_UNSUPPORTED;
   const WsLayout w = ws_layout(s, q_len);
@@ -721,7 +721,7 @@ int ooco_decode_step_fp8(const ooco_shape_t* s, const void* q, const void* k_new
 }
 
 size_t ooco_decode_workspace_bytes_mq(const ooco_shape_t* s, int32_t q_len) {
-  if (validate_shape(s) || validate_q_len(s, q_len, false)) return 0;
+  if (validate_shape(s) || validate_q_len(s, q_len)) return 0;
   return ws_layout(s, q_len).total;
 }
 
@@ -753,7 +753,7 @@ int ooco_decode_step_mq(const ooco_shape_t* s, int32_t q_len, const void* q, con
                         size_t workspace_bytes, void* cuda_stream) {
   int rc = validate_shape(s);
   if (rc) return rc;
-  if ((rc = validate_q_len(s, q_len, false))) return rc;
+  if ((rc = validate_q_len(s, q_len))) return rc;
   if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !positions) return OOCO_E_NULLPTR;
   if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
     return OOCO_E_UNSUPPORTED;
@@ -761,6 +761,31 @@ int ooco_decode_step_mq(const ooco_shape_t* s, int32_t q_len, const void* q, con
   ap.Sq = q_len;
   return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
                      cuda_stream, &ap, nullptr, q_len);
+}
+
+int ooco_decode_step_mq_fp8(const ooco_shape_t* s, int32_t q_len, const void* q, const void* k_new,
+                            const void* v_new, void* k_cache, void* v_cache, const int32_t* block_table,
+                            const int32_t* positions, const int32_t* context_lens, float scale, float k_scale,
+                            float v_scale, void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_shape(s);
+  if (rc) return rc;
+  const Kv8Scales sc = {k_scale, v_scale};
+  if ((rc = validate_kv8(s, &sc))) return rc;
+  if ((rc = validate_q_len(s, q_len))) return rc;
+  if (!k_cache || !v_cache || !block_table) return OOCO_E_NULLPTR;
+  if (!k_new && !v_new)  // attention only
+    return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                       cuda_stream, nullptr, &sc, q_len);
+  if (!k_new || !v_new || !positions) return OOCO_E_NULLPTR;
+  if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)
+    return OOCO_E_UNSUPPORTED;
+  AppendParams ap = make_append_params(s, k_new, v_new, k_cache, v_cache, block_table, positions);
+  ap.Sq = q_len;
+  ap.kv8 = 1;
+  ap.k_scale = k_scale;
+  ap.v_scale = v_scale;
+  return decode_core(s, q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, workspace_bytes,
+                     cuda_stream, &ap, &sc, q_len);
 }
 
 int ooco_decode_attention_static(const ooco_shape_t* s, const void* q, const void* k_cache,

@@ -142,3 +142,56 @@ def test_fused_step_mq():
     ref = oracle.decode_attention_mq(inputs.as_u16(q), k_ref, v_ref, table, lens.cpu().numpy(), cfg.scale,
                                      num_kv_heads=8, block_size=16, strides=batch.strides)
     assert_parity(out.reshape(-1, 32, 128), ref.out.reshape(-1, 32, 128), what="fused mq step")
+
+
+@pytest.mark.parametrize("cfg,Sq", [
+    (C("mq8-edges", 32, 8, 128, 16, fixed(0, 1, 2, 3, 4, 15, 16, 17, 18, 63, 64, 65, 66, 127, 129, 300), seed=94,
+       pool_fill=0.7, shuffle_batch=False), 4),
+    (C("mq8-g8-sq2", 64, 8, 128, 32, (G(5, 1, 900),), seed=95, sigma=0.5), 2),
+    (C("mq8-split", 32, 8, 128, 16, fixed(5000, 37, 2049, 2050, 2051, 300), seed=96, shuffle_batch=False), 3),
+], ids=lambda v: getattr(v, "name", str(v)))
+def test_multi_query_over_8bit_cache(cfg, Sq):
+    ks, vs = 1.0 / 32, 0.04
+    b16 = inputs.make_batch(cfg, "cuda", poison=True, table_pad=2**31 - 1)
+    batch = inputs.to_e4m3_pool(b16, ks, vs)
+    B, Hq, D = cfg.batch, cfg.num_q_heads, cfg.head_dim
+    g = torch.Generator(device="cuda").manual_seed(cfg.seed)
+    q = (torch.randn((B, Sq, Hq, D), generator=g, device="cuda") * cfg.sigma).to(torch.bfloat16)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_step_mq_fp8(sh, q, None, None, batch.k_cache, batch.v_cache, batch.block_table, None,
+                               batch.context_lens, cfg.scale, ks, vs, out, ws)
+    assert binding.workspace_status(ws) == 0
+    ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), inputs.as_u8(batch.k_cache), inputs.as_u8(batch.v_cache),
+                                         batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                         ks, vs, num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size,
+                                         strides=batch.strides)
+    assert_parity(out.reshape(B * Sq, Hq, D), ref.out.reshape(B * Sq, Hq, D), what=f"{cfg.name} Sq={Sq}")
+
+
+def test_fused_step_mq_over_8bit_cache():
+    cfg = C("mq8-step", 32, 8, 128, 16, (G(12, 4, 2600),), seed=97, pool_fill=0.85)
+    Sq, ks, vs = 4, 1.0 / 32, 1.0 / 32
+    batch = inputs.to_e4m3_pool(inputs.make_batch(cfg, "cuda", poison=True), ks, vs)
+    sh = binding.shape_of(batch)
+    g = torch.Generator(device="cuda").manual_seed(8)
+    q = torch.randn((cfg.batch, Sq, 32, 128), generator=g, device="cuda").to(torch.bfloat16)
+    k_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    v_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    lens = batch.context_lens
+    positions = (lens - Sq).contiguous()
+    k_ref, v_ref = inputs.as_u8(batch.k_cache).copy(), inputs.as_u8(batch.v_cache).copy()
+    table = batch.block_table.cpu().numpy()
+    for i in range(Sq):
+        oracle.kv_append_fp8(inputs.as_u16(k_new[:, i].contiguous()), inputs.as_u16(v_new[:, i].contiguous()), k_ref,
+                             v_ref, table, (positions + i).cpu().numpy(), ks, vs, block_size=16, strides=batch.strides)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_step_mq_fp8(sh, q, k_new, v_new, batch.k_cache, batch.v_cache, batch.block_table, positions, lens,
+                               cfg.scale, ks, vs, out, ws)
+    assert binding.workspace_status(ws) == 0
+    assert np.array_equal(inputs.as_u8(batch.k_cache), k_ref) and np.array_equal(inputs.as_u8(batch.v_cache), v_ref)
+    ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), k_ref, v_ref, table, lens.cpu().numpy(), cfg.scale, ks, vs,
+                                         num_kv_heads=8, block_size=16, strides=batch.strides)
+    assert_parity(out.reshape(-1, 32, 128), ref.out.reshape(-1, 32, 128), what="fused mq step, 8-bit cache")
