@@ -54,6 +54,8 @@ def draw_case(seed):
             mode = "bf16"
         else:
             Sq = int(rng.choice(choices))
+            if D == 128 and rng.random() < 0.4:
+                mode = "mq8"
     cfg = inputs.DecodeConfig(f"fuzz{seed}", Hkv * G, Hkv, D, bs,
                               (inputs.LengthGroup(B, int(lens.min()), int(lens.max()), "fixed", tuple(int(x) for x in lens)),),
                               seed=2000 + seed, pool_fill=float(rng.choice([1.0, 0.9, 0.6])), layout=layout,
@@ -61,7 +63,7 @@ def draw_case(seed):
     return cfg, mode, Sq
 
 
-@pytest.mark.parametrize("seed", range(48))
+@pytest.mark.parametrize("seed", range(64))
 def test_random_case(seed):
     cfg, mode, Sq = draw_case(seed)
     batch = inputs.make_batch(cfg, "cuda", poison=True, table_pad=-7)
@@ -77,6 +79,19 @@ def test_random_case(seed):
                                      out, ws)
         ref = oracle.decode_attention_fp8(inputs.as_u16(b8.q), inputs.as_u8(b8.k_cache), inputs.as_u8(b8.v_cache), table,
                                           lens, cfg.scale, ks, vs, **kw).out
+    elif mode == "mq8":
+        ks, vs = 1.0 / 16, 1.0 / 64
+        b8 = inputs.to_e4m3_pool(batch, ks, vs)
+        g = torch.Generator(device="cuda").manual_seed(seed)
+        q = torch.randn((cfg.batch, Sq, cfg.num_q_heads, cfg.head_dim), generator=g, device="cuda").to(torch.bfloat16)
+        sh = binding.shape_of(b8)
+        ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+        out = torch.full_like(q, float("nan"))
+        binding.decode_step_mq_fp8(sh, q, None, None, b8.k_cache, b8.v_cache, b8.block_table, None, b8.context_lens,
+                                   cfg.scale, ks, vs, out, ws)
+        ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), inputs.as_u8(b8.k_cache), inputs.as_u8(b8.v_cache), table,
+                                             lens, cfg.scale, ks, vs, **kw).out
+        out, ref = out.reshape(-1, cfg.num_q_heads, cfg.head_dim), ref.reshape(-1, cfg.num_q_heads, cfg.head_dim)
     elif mode == "mq":
         g = torch.Generator(device="cuda").manual_seed(seed)
         q = torch.randn((cfg.batch, Sq, cfg.num_q_heads, cfg.head_dim), generator=g, device="cuda").to(torch.bfloat16)
