@@ -50,7 +50,8 @@ struct DecodeParams {
   int32_t tile_rows;      // token rows per TMA box = min(bs, stage tokens)
   int32_t split_halves;   // 1: one 4-d TMA per 64-dim half; 0: one 5-d TMA per box
   int32_t nstages;
-  int32_t grid_main;      // CTAs of the attention kernel (first items are assigned statically)
+  int32_t grid_main;      // CTAs the plan sizes the chunks for
+  int32_t next_item_init; // start of the dynamic work counter = CTAs of the attention grid (they take the first units statically)
   int32_t chunk_min, chunk_max, items_per_cta;
   float scale_log2e;        // softmax scale * log2(e) (* the K tensor scale of an 8-bit cache)
   float v_scale;            // V tensor scale of an 8-bit cache (1 for bf16)
@@ -249,7 +250,7 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
   if (tid == 0) {
     p.hdr->status = overflow ? kStatusPlanOverflow : 0;
     p.hdr->n_items = (int)n_items;
-    p.hdr->next_item = p.grid_main;
+    p.hdr->next_item = p.next_item_init;
     p.hdr->chunk_tokens = chunk;
   }
   // Items in order of decreasing length (longest first keeps the tail of the dynamic schedule

@@ -12,6 +12,7 @@
 
 #include "../../include/ooco.h"
 #include "block_copy_kernels.cuh"
+#include "chunk_kernels.cuh"
 #include "decode_kernels.cuh"
 
 namespace ooco {
@@ -97,6 +98,13 @@ static int validate_shape(const ooco_shape_t* s) {
   return OOCO_OK;
 }
 
+// More than 16 score columns per (sequence, kv head) go to the prefill-chunk kernel; consumer warps of
+// its CTA (16 columns each) for a given number of columns.
+constexpr int kDecodeMaxColumns = 16;
+constexpr int kMaxQLen = 8192;
+static int chunk_warps(int columns) { return columns <= 32 ? 2 : (columns <= 64 ? 4 : 8); }
+static int chunk_row_tiles(int columns) { return (columns + 16 * chunk_warps(columns) - 1) / (16 * chunk_warps(columns)); }
+
 // Workspace carve-up (all offsets multiples of 256 bytes).
 struct WsLayout {
   size_t off_first, off_items, off_lse, off_o, total;
@@ -108,7 +116,10 @@ static WsLayout ws_layout(const ooco_shape_t* s, int q_len = 1) {
   const int64_t ipc = g_knobs[kKnobItemsPerCta].load();
   const int64_t per_seq = ((int64_t)s->max_blocks_per_seq * s->block_size + cmax - 1) / cmax;
   int64_t extra = (int64_t)s->num_kv_heads * s->batch * per_seq;
-  if (extra < kGridCap * ipc) extra = kGridCap * ipc;
+  // the plan cuts the sequences into about (CTAs it sizes for) x ipc items; the chunk path sizes for the
+  // CTAs divided by the row tiles of an item, since every item is worked on once per row tile
+  const int64_t sized_ctas = G > kDecodeMaxColumns ? (kGridCap + chunk_row_tiles(G) - 1) / chunk_row_tiles(G) : kGridCap;
+  if (extra < sized_ctas * ipc) extra = sized_ctas * ipc;
   const int64_t max_items = (int64_t)s->num_kv_heads * s->batch + extra + 64;
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
   WsLayout w;
@@ -195,7 +206,7 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
     if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
-  cudaError_t e = launch_ex(kern, dim3(p.grid_main), dim3((NCW + 1) * 32), smem, st,
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + 1) * 32), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the attention kernel", (long)e);
@@ -238,6 +249,49 @@ static int launch_main_ncw(int ncw, int tpw, const CUtensorMap& tk, const CUtens
     case 2: return launch_main_nt<D, 2, 1>(tk, tv, p, di, cps, stages, st, dev);
     case 8: return launch_main_nt<D, 8, 1>(tk, tv, p, di, cps, stages, st, dev);
     default: return launch_main_nt<D, 4, 1>(tk, tv, p, di, cps, stages, st, dev);
+  }
+}
+
+// Prefill-chunk kernel: as many 64-token stages as the CTA's share of shared memory holds (at most 8).
+template <int D, int NCW>
+static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
+                        int ctas_per_sm, cudaStream_t st, int dev) {
+  using L = ChunkSmem<D>;
+  auto kern = chunk_main_kernel<D, NCW>;
+  static std::atomic<int> static_smem{-1};
+  if (static_smem.load() < 0) {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncGetAttributes", (long)e);
+    static_smem.store((int)fa.sharedSizeBytes);
+  }
+  const size_t dyn_max = (size_t)di.smem_optin - (size_t)static_smem.load();
+  const size_t budget = ctas_per_sm > 1 ? ((size_t)di.smem_optin + 1024) / ctas_per_sm - 1024 - static_smem.load()
+                                        : dyn_max;
+  int nst = 8;
+  while (nst > 2 && L::total(nst) > budget) --nst;
+  if (L::total(nst) > dyn_max) return OOCO_E_UNSUPPORTED;
+  p.nstages = nst;
+  const size_t smem = L::total(nst);
+  static std::atomic<size_t> configured[64];
+  if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
+    if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
+  }
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + 1) * 32), smem, st,
+                            g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the chunk attention kernel", (long)e);
+}
+
+template <int D>
+static int launch_chunk_ncw(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
+                            const DeviceInfo& di, int cps, cudaStream_t st, int dev) {
+  switch (ncw) {
+    case 2: return launch_chunk<D, 2>(tk, tv, p, di, cps, st, dev);
+    case 4: return launch_chunk<D, 4>(tk, tv, p, di, cps, st, dev);
+    default: return launch_chunk<D, 8>(tk, tv, p, di, cps, st, dev);
   }
 }
 
@@ -490,10 +544,12 @@ size_t ooco_decode_workspace_bytes(const ooco_shape_t* s) {
 // Plan (+ optional fused append) -> split-KV attention -> LSE merge on `cuda_stream`.
 // Query tokens per sequence: the score columns of a (sequence, kv head) pair, G * q_len, must fit the
 // two 8-column MMA tiles of the kernel.
-static int validate_q_len(const ooco_shape_t* s, int q_len) {
+static int validate_q_len(const ooco_shape_t* s, int q_len, bool kv8 = false) {
   if (q_len < 1) return OOCO_E_SHAPE;
   if (q_len == 1) return OOCO_OK;
-  if ((long long)(s->num_q_heads / s->num_kv_heads) * q_len > 16) return OOCO_E_UNSUPPORTED;
+  if (q_len > kMaxQLen) return OOCO_E_UNSUPPORTED;
+  // the 8-bit cache has the decode kernel only
+  if (kv8 && (long long)(s->num_q_heads / s->num_kv_heads) * q_len > kDecodeMaxColumns) return OOCO_E_UNSUPPORTED;
   return OOCO_OK;
 }
 
@@ -520,7 +576,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   int rc = validate_shape(s);
   if (rc) return rc;
   if ((rc = validate_kv8(s, kv8))) return rc;
-  if ((rc = validate_q_len(s, q_len))) return rc;
+  if ((rc = validate_q_len(s, q_len, kv8 != nullptr))) return rc;
   if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
   if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q) & 15) return OOCO_E_UNSUPPORTED;
   const WsLayout w = ws_layout(s, q_len);
@@ -544,7 +600,13 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
     cps = 4;
   int tpw = g_knobs[kKnobTilesPerWarp].load();
   if (ncw == 8 || kv8) tpw = 1;
-  const int stage_tok = 16 * ncw * tpw;
+  // prefill chunk: 64-token stages; 8 warps (128 columns) x 1 CTA per SM, fewer columns: smaller CTAs x 2
+  const bool chunk = G_ > kDecodeMaxColumns;
+  if (chunk) {
+    ncw = chunk_warps(G_);
+    cps = ncw == 8 ? 1 : 2;
+  }
+  const int stage_tok = chunk ? kChunkStageTok : 16 * ncw * tpw;
   DecodeParams p;
   memset(&p, 0, sizeof p);
   uint8_t* ws = (uint8_t*)workspace;
@@ -570,6 +632,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.tile_rows = s->block_size < stage_tok ? s->block_size : stage_tok;
   p.grid_main = di.sm_count * cps;
   if (p.grid_main > kGridCap) p.grid_main = kGridCap;
+  p.next_item_init = p.grid_main;
+  if (chunk) p.grid_main = (p.grid_main + chunk_row_tiles(G_) - 1) / chunk_row_tiles(G_);
   p.chunk_min = g_knobs[kKnobChunkMin].load();
   p.chunk_max = g_knobs[kKnobChunkMax].load();
   if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
@@ -579,7 +643,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.v_scale = kv8 ? kv8->v_scale * kE4m3WidenFactor : 1.f;
 
   CUtensorMap tk, tv;
-  bool five_d = !kv8 && s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
+  bool five_d = !kv8 && !chunk && s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
   if (five_d && encode_kv_map(&tk, s, k_cache, p.tile_rows, true) != OOCO_OK) five_d = false;
   if (kv8) {
     if ((rc = encode_kv8_map(&tk, s, k_cache, p.tile_rows))) return rc;
@@ -625,7 +689,10 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
   if (pe) cudaEventRecord(pe[1], st);
-  if (kv8)
+  if (chunk)
+    rc = s->head_dim == 128 ? launch_chunk_ncw<128>(ncw, tk, tv, p, di, cps, st, dev)
+                            : launch_chunk_ncw<64>(ncw, tk, tv, p, di, cps, st, dev);
+  else if (kv8)
     rc = launch_main_kv8(ncw, tk, tv, p, di, cps, stages, st, dev);
   else if (s->head_dim == 128)
     rc = launch_main_ncw<128>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);

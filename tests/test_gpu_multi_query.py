@@ -62,6 +62,45 @@ def test_multi_query_matches_oracle(cfg, Sq):
     run_case(cfg, Sq, seed=cfg.seed)
 
 
+# More than 16 score columns per (sequence, kv head): the prefill-chunk kernel (row tiles of 32 / 64 / 128
+# columns).  Contexts shorter than, equal to and just above the chunk; ragged last row tile; every block size.
+CHUNK_CASES = [
+    (C("ck-g4-sq5", 32, 8, 128, 16, fixed(0, 1, 4, 5, 6, 63, 64, 65, 129, 700), seed=101, pool_fill=0.7,
+       shuffle_batch=False), 5),                                              # 20 columns: 2-warp CTAs
+    (C("ck-g4-sq16", 32, 8, 128, 16, fixed(3, 16, 17, 64, 100, 1000), seed=102, shuffle_batch=False), 16),   # 64 columns
+    (C("ck-g4-sq33", 32, 8, 128, 16, fixed(33, 34, 200, 1500), seed=103, shuffle_batch=False), 33),          # 132: ragged tile
+    (C("ck-g4-sq128-fresh", 32, 8, 128, 16, fixed(128, 128, 500, 1290), seed=104, shuffle_batch=False), 128),  # T = S_q: a whole prompt
+    (C("ck-g5-sq7-bs32", 40, 8, 128, 32, (G(5, 7, 900),), seed=105), 7),
+    (C("ck-g8-sq64-bs64", 64, 8, 128, 64, (G(3, 64, 1200),), seed=106, sigma=0.5), 64),
+    (C("ck-g1-sq100-bs128", 8, 8, 128, 128, (G(4, 100, 800),), seed=107), 100),
+    (C("ck-d64-g4-sq40", 8, 2, 64, 16, (G(6, 1, 900),), seed=108), 40),
+    (C("ck-token-major", 32, 8, 128, 16, (G(4, 50, 600),), seed=109, layout="token_major"), 24),
+    # split into several chunks (few long sequences)
+    (C("ck-split", 32, 8, 128, 16, fixed(9000, 2049, 70), seed=110, pool_fill=0.9, shuffle_batch=False), 48),
+    (C("ck-split-g2", 16, 8, 128, 16, fixed(20000, 4100), seed=111, shuffle_batch=False), 9),
+]
+
+
+@pytest.mark.parametrize("cfg,Sq", CHUNK_CASES, ids=lambda v: getattr(v, "name", str(v)))
+def test_prefill_chunk_matches_oracle(cfg, Sq):
+    run_case(cfg, Sq, seed=cfg.seed)
+
+
+def test_chunk_rows_agree_with_decode_rows():
+    """A chunk of 8 query tokens (32 columns: chunk kernel) and two calls of 4 (16 columns: decode kernel)
+    over the same cache compute the same rows, up to the rounding of a different summation order."""
+    cfg = C("ck-vs-mq", 32, 8, 128, 16, (G(6, 8, 900),), seed=112)
+    batch, q, out, _ = run_case(cfg, 8, seed=2)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, 4), dtype=torch.uint8, device="cuda")
+    q_hi = q[:, 4:].contiguous()
+    out_hi = torch.empty_like(q_hi)
+    binding.decode_attention_mq(sh, q_hi, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens,
+                                cfg.scale, out_hi, ws)
+    torch.cuda.synchronize()
+    assert float((out[:, 4:].float() - out_hi.float()).abs().max()) <= 4e-3
+
+
 def test_last_query_token_equals_single_query_call():
     """The last query token sees the whole context: the same result as ooco_decode_attention on that
     token, up to the rounding of a different summation order (the launch shape depends on the number
@@ -104,16 +143,25 @@ def test_append_mq_bit_exact_then_attend():
 
 def test_unsupported_shapes_are_refused():
     cfg = C("mq-too-wide", 64, 8, 128, 16, fixed(50), seed=92)
-    batch = inputs.make_batch(cfg, "cuda", poison=False)
+    batch = inputs.to_e4m3_pool(inputs.make_batch(cfg, "cuda", poison=False), 1.0, 1.0)
     sh = binding.shape_of(batch)
     with pytest.raises(binding.OocoError):
-        binding.workspace_bytes_mq(sh, 3)                                  # 8 heads x 3 tokens > 16 columns
-    ws = torch.empty(binding.workspace_bytes_mq(sh, 2), dtype=torch.uint8, device="cuda")
+        binding.workspace_bytes_mq(sh, 8193)                               # beyond the largest chunk
+    # the 8-bit cache has no prefill-chunk kernel: 8 heads x 3 tokens > 16 columns
+    ws = torch.empty(binding.workspace_bytes_mq(sh, 3), dtype=torch.uint8, device="cuda")
     q = torch.zeros((1, 3, 64, 128), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(binding.OocoError) as e:
-        binding.decode_attention_mq(sh, q, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens, 1.0,
-                                    torch.empty_like(q), ws)
+        binding.decode_step_mq_fp8(sh, q, None, None, batch.k_cache, batch.v_cache, batch.block_table, None,
+                                   batch.context_lens, 1.0, 1.0, 1.0, torch.empty_like(q), ws)
     assert e.value.status == -3
+    # a workspace sized for fewer query tokens is refused
+    b16 = inputs.make_batch(cfg, "cuda", poison=False)
+    sh16 = binding.shape_of(b16)
+    small = torch.empty(binding.workspace_bytes_mq(sh16, 2), dtype=torch.uint8, device="cuda")
+    q = torch.zeros((1, 64, 64, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.OocoError):
+        binding.decode_attention_mq(sh16, q, b16.k_cache, b16.v_cache, b16.block_table, b16.context_lens, 1.0,
+                                    torch.empty_like(q), small)
 
 
 def test_fused_step_mq():
