@@ -174,7 +174,7 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
 
 /*
  * Several query tokens per sequence (the attention row of Table "Operator Modeling" with S_q > 1:
- * multi-token decode, or a short chunk of a prefill running next to decodes).  The q_len query
+ * multi-token decode, or a chunk of a prefill running next to decodes).  The q_len query
  * tokens of sequence b are the LAST q_len tokens of its context: their K / V must already be in the
  * cache (ooco_kv_append_mq writes them), context_lens[b] counts them, and query token i attends to
  * tokens [0, T_b - q_len + i + 1) -- causal attention over the cache.  A query token that sees no
@@ -184,7 +184,13 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  *                   position positions[b] + i (ooco_kv_append_mq); positions beyond the block table
  *                   are skipped, as in ooco_kv_append
  *   workspace       >= ooco_decode_workspace_bytes_mq(shape, q_len)
- * Supported: (Hq / Hkv) * q_len <= 16.  q_len = 1 is ooco_decode_attention /
+ * Supported: 1 <= q_len <= 8192 (OOCO_E_UNSUPPORTED beyond).  Up to 16 score columns per
+ * (sequence, kv head), (Hq / Hkv) * q_len <= 16, run the decode kernel (HBM-bound: the cache is
+ * read once); more columns run the prefill-chunk kernel, which cuts the columns into row tiles of
+ * up to 128, reads the cache once per row tile (the repeats hit L2) and never loads tokens a tile
+ * cannot see; it becomes bound by the tensor pipe from about 64 columns on.  The 8-bit cache
+ * (ooco_decode_step_mq_fp8) has the decode kernel only.  The workspace grows with q_len: one fp32
+ * partial row per (split item, score column).  q_len = 1 is ooco_decode_attention /
  * ooco_kv_append exactly.  Everything else as for those two.
  */
 size_t ooco_decode_workspace_bytes_mq(const ooco_shape_t* shape, int32_t q_len);

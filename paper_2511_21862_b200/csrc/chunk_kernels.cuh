@@ -47,14 +47,17 @@ __device__ __forceinline__ void chunk_consume(uint32_t kst, uint32_t vst, const 
   // ---- scores: two k-steps (32 dims) per ldmatrix
 #pragma unroll
   for (int kp = 0; kp < KS / 2; ++kp) {
+    const uint32_t ka = kst + (uint32_t)(kp >> 1) * ChunkSmem<D>::kHalfBytes + k_off[kp & 1];
 #pragma unroll
-    for (int j = 0; j < NS; ++j) {
+    for (int j = 0; j < NS; j += 2) {  // two token tiles at a time: their MMAs do not depend on each other
       if (kTail && 8 * j >= ntok) continue;
-      uint32_t b0, b1, b2, b3;
-      ldmatrix_x4(kst + (uint32_t)(kp >> 1) * ChunkSmem<D>::kHalfBytes + (uint32_t)j * 1024 + k_off[kp & 1], b0, b1, b2,
-                  b3);
+      uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
+      ldmatrix_x4(ka + (uint32_t)j * 1024, b0, b1, b2, b3);
+      ldmatrix_x4(ka + (uint32_t)(j + 1) * 1024, c0, c1, c2, c3);
       mma_bf16(s[j], qf[2 * kp][0], qf[2 * kp][1], qf[2 * kp][2], qf[2 * kp][3], b0, b1);
+      mma_bf16(s[j + 1], qf[2 * kp][0], qf[2 * kp][1], qf[2 * kp][2], qf[2 * kp][3], c0, c1);
       mma_bf16(s[j], qf[2 * kp + 1][0], qf[2 * kp + 1][1], qf[2 * kp + 1][2], qf[2 * kp + 1][3], b2, b3);
+      mma_bf16(s[j + 1], qf[2 * kp + 1][0], qf[2 * kp + 1][1], qf[2 * kp + 1][2], qf[2 * kp + 1][3], c2, c3);
     }
   }
   // ---- online softmax; lane (g, t) holds tokens 8j + 2t, + 1 of rows g (s[j][0..1]) and g + 8 (s[j][2..3])
