@@ -530,7 +530,7 @@ def run_multi_query(args, local_rank):
     peak, peak_kind = measured_peak()
     achieved = nbytes / (attn * 1e-3) / 1e9
     columns = Sq * (cfg.num_q_heads // cfg.num_kv_heads)
-    kernel = "chunk_main_kernel" if columns > 16 else "decode_main_kernel"
+    kernel = "chunk_main_kernel" if columns > 16 else ("row16_main_kernel" if columns > 8 else "decode_main_kernel")
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "kernel": kernel, "algorithmic_bytes_per_launch": nbytes,
                 "traffic": None}

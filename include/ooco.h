@@ -426,7 +426,9 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * merge kernels with programmatic dependent launch (their prologues overlap the predecessor);
  * 9 CTAs per SM of the block-movement kernel {1..3}; 10 non-zero = ooco_decode_step_host reads
  * page-locked inputs through their device mapping and lets the kernels write a page-locked result
- * directly (zero = always one copy per buffer).
+ * directly (zero = always one copy per buffer); 11 non-zero = 9 to 16 score columns per
+ * (sequence, kv head) run the kernel whose warps share 16 score rows and split the tokens of a
+ * stage (zero = the decode kernel with two 8-column tiles).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.
  */

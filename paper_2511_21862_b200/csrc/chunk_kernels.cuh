@@ -35,12 +35,14 @@ struct ChunkSmem {
 // One consumer warp on one stage.  kTail: some tokens of the stage are hidden from some of the warp's rows
 // (causal limit, end of the chunk) or are not there at all (`ntok` < 64: rows beyond hold stale bytes).
 //   e0 / e1   tokens [0, e) of the stage the lane's rows g / g + 8 may see
-template <int D, bool kTail>
+//   NTOK      tokens the call covers, starting at row 0 of `kst` / `vst`: a whole 64-token stage, or the
+//             16-token slice of a warp that shares its rows with the other warps (row16_main_kernel)
+template <int D, int NTOK, bool kTail>
 __device__ __forceinline__ void chunk_consume(uint32_t kst, uint32_t vst, const uint32_t (&k_off)[2],
                                               const uint32_t (&v_off)[4], const uint32_t (&qf)[D / 16][4],
                                               float (&m_run)[2], float (&l_run)[2], float (&o_acc)[D / 8][4],
                                               float scale_log2e, int ntok, int e0, int e1, int t) {
-  constexpr int KS = D / 16, NS = kChunkStageTok / 8, NO = D / 8;
+  constexpr int KS = D / 16, NS = NTOK / 8, NO = D / 8;
   float s[NS][4];
 #pragma unroll
   for (int j = 0; j < NS; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
@@ -113,7 +115,7 @@ __device__ __forceinline__ void chunk_consume(uint32_t kst, uint32_t vst, const 
   }
   // ---- values: 16 tokens per k-step, two 8-dim column tiles per ldmatrix
 #pragma unroll
-  for (int kk = 0; kk < kChunkStageTok / 16; ++kk) {
+  for (int kk = 0; kk < NTOK / 16; ++kk) {
     if (kTail && 16 * kk >= ntok) continue;
     uint32_t mk01 = 0xffffffffu, mk23 = 0xffffffffu;
     if (kTail) {  // rows beyond the stage's tokens may hold anything (NaN included): clear them
@@ -135,6 +137,126 @@ __device__ __forceinline__ void chunk_consume(uint32_t kst, uint32_t vst, const 
       }
       mma_bf16(o_acc[2 * np], a0, a1, a2, a3, b0, b1);
       mma_bf16(o_acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+    }
+  }
+}
+
+// The producer warp of both kernels below: walks its units of work (item, row tile of RT score columns),
+// streams the K / V stages of each through TMA and describes every stage in two int4 of `g_meta`:
+//   {partial slot, sequence, kv head, tokens | first << 16 | last << 17}  {first token, T - S_q + 1, chunk end, row tile}
+template <int D>
+__device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const DecodeParams& p,
+                                              const int RT, const int nst, const uint32_t s_stage,
+                                              const uint32_t s_full, const uint32_t s_empty, int4* g_meta,
+                                              volatile int* s_abort, const int lane) {
+  using L = ChunkSmem<D>;
+  const int nrt = (p.GQ + RT - 1) / RT;
+  const long long n_units = (long long)p.hdr->n_items * nrt;
+  // ================================================================= producer warp
+  if (lane == 0) {
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+  }
+  const int boxes_per_stage = kChunkStageTok / p.tile_rows;
+  const uint32_t box_rows_bytes = (uint32_t)p.tile_rows * 128;  // one box of one 64-dim half
+  const long long cap_tokens = (long long)p.MB * p.bs;
+  int it = 0;
+  bool ok = true;
+  long long unit = blockIdx.x;
+  // waits for stage `it`'s slot to be free; false when the wait gave up
+  auto acquire = [&](int& slot) {
+    slot = it % nst;
+    return warp_wait(s_empty + 8 * slot, (((uint32_t)(it / nst)) & 1u) ^ 1u, s_abort);
+  };
+  while (unit < n_units && ok) {
+    int nxt = 0;
+    if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
+    nxt = __shfl_sync(0xffffffffu, nxt, 0);
+    const int item = (int)(unit / nrt), rt = (int)(unit - (long long)item * nrt);
+    const int4 d = p.items[item];
+    const int b = d.x, h = d.y % p.Hkv, t0 = d.z, t1 = d.w;
+    long long T = p.context_lens[b];
+    T = T < 0 ? 0 : (T > cap_tokens ? cap_tokens : T);
+    const int lim_base = (int)T - p.Sq + 1;                       // tokens the first query token sees
+    const int col_hi = min(p.GQ, (rt + 1) * RT) - 1;
+    const int t1e = min(t1, lim_base + col_hi / p.G);              // nothing beyond is visible to this tile
+    const int nstage = t1e > t0 ? (t1e - t0 + kChunkStageTok - 1) / kChunkStageTok : 0;
+    const int32_t* row = p.block_table + (size_t)b * p.MB;
+    int blk_cur = 0;
+    {
+      const int tb = t0 + lane * p.tile_rows;
+      if (lane < boxes_per_stage && tb < t1e) blk_cur = row[tb / p.bs];
+    }
+    if (nstage == 0) {  // the tile sees nothing of this chunk: one empty stage carries the bookkeeping
+      int slot;
+      if (!acquire(slot)) {
+        ok = false;
+        break;
+      }
+      if (lane == 0) {
+        g_meta[2 * slot] = make_int4(d.y, b, h, 0 | (3 << 16));
+        g_meta[2 * slot + 1] = make_int4(t0, lim_base, t1, rt);
+        mbar_arrive(s_full + 8 * slot);
+      }
+      ++it;
+    }
+    for (int s = 0; s < nstage; ++s, ++it) {
+      const int tok0 = t0 + s * kChunkStageTok;
+      const int ntok = min(kChunkStageTok, t1e - tok0);
+      const int nbox = (ntok + p.tile_rows - 1) / p.tile_rows;
+      int blk_n = 0;  // table entries of the following stage, one stage ahead of their use
+      {
+        const int tb = tok0 + kChunkStageTok + lane * p.tile_rows;
+        if (s + 1 < nstage && lane < boxes_per_stage && tb < t1e) blk_n = row[tb / p.bs];
+      }
+      int slot;
+      if (!acquire(slot)) {
+        ok = false;
+        break;
+      }
+      const uint32_t full = s_full + 8 * slot;
+      if (lane == 0) {
+        const int flags = (s == 0 ? 1 : 0) | (s == nstage - 1 ? 2 : 0);
+        g_meta[2 * slot] = make_int4(d.y, b, h, ntok | (flags << 16));
+        g_meta[2 * slot + 1] = make_int4(tok0, lim_base, t1, rt);
+        mbar_arrive_expect_tx(full, 2u * (uint32_t)nbox * box_rows_bytes * (D / 64));
+      }
+      __syncwarp();
+      if (lane < nbox) {
+        const int tb = tok0 + lane * p.tile_rows;
+        const int c_tok = tb % p.bs;
+        const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + (uint32_t)lane * box_rows_bytes;
+        const uint32_t dv = dk + L::kTileBytes;
+#pragma unroll
+        for (int j = 0; j < D / 64; ++j) {
+          tma_load_4d(dk + j * L::kHalfBytes, &tm_k, full, 64 * j, c_tok, h, blk_cur);
+          tma_load_4d(dv + j * L::kHalfBytes, &tm_v, full, 64 * j, c_tok, h, blk_cur);
+        }
+      }
+      blk_cur = blk_n;
+    }
+    unit = nxt;
+  }
+  if (ok) {  // end marker (one stage, seen by every consumer warp)
+    int slot;
+    if (acquire(slot)) {
+      if (lane == 0) {
+        g_meta[2 * slot] = make_int4(-1, 0, 0, 0);
+        mbar_arrive(s_full + 8 * slot);
+      }
+      ++it;
+    } else {
+      ok = false;
+    }
+  }
+  if (!ok) {
+    // stop path: record it, then wait (bounded) until every copy already issued has landed
+    if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+    int dummy_abort = 0;
+    const int pending = it < nst ? it : nst;
+    for (int k = 0; k < pending; ++k) {
+      const int j = it - 1 - k;
+      mbar_wait_bounded(s_full + 8 * (j % nst), (uint32_t)(j / nst) & 1u, &dummy_abort, kWaitLimitNs / 8);
     }
   }
 }
@@ -172,117 +294,9 @@ chunk_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   __syncthreads();
   grid_dep_wait();    // the plan (and a fused append) must have completed
   grid_dep_launch();  // the merge kernel may queue up behind this grid
-  const int nrt = (p.GQ + RT - 1) / RT;
-  const long long n_units = (long long)p.hdr->n_items * nrt;
 
   if (warp == NCW) {
-    // ================================================================= producer warp
-    if (lane == 0) {
-      prefetch_tmap(&tm_k);
-      prefetch_tmap(&tm_v);
-    }
-    const int boxes_per_stage = kChunkStageTok / p.tile_rows;
-    const uint32_t box_rows_bytes = (uint32_t)p.tile_rows * 128;  // one box of one 64-dim half
-    const long long cap_tokens = (long long)p.MB * p.bs;
-    int it = 0;
-    bool ok = true;
-    long long unit = blockIdx.x;
-    // waits for stage `it`'s slot to be free; false when the wait gave up
-    auto acquire = [&](int& slot) {
-      slot = it % nst;
-      return warp_wait(s_empty + 8 * slot, (((uint32_t)(it / nst)) & 1u) ^ 1u, s_abort);
-    };
-    while (unit < n_units && ok) {
-      int nxt = 0;
-      if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
-      nxt = __shfl_sync(0xffffffffu, nxt, 0);
-      const int item = (int)(unit / nrt), rt = (int)(unit - (long long)item * nrt);
-      const int4 d = p.items[item];
-      const int b = d.x, h = d.y % p.Hkv, t0 = d.z, t1 = d.w;
-      long long T = p.context_lens[b];
-      T = T < 0 ? 0 : (T > cap_tokens ? cap_tokens : T);
-      const int lim_base = (int)T - p.Sq + 1;                       // tokens the first query token sees
-      const int col_hi = min(p.GQ, (rt + 1) * RT) - 1;
-      const int t1e = min(t1, lim_base + col_hi / p.G);              // nothing beyond is visible to this tile
-      const int nstage = t1e > t0 ? (t1e - t0 + kChunkStageTok - 1) / kChunkStageTok : 0;
-      const int32_t* row = p.block_table + (size_t)b * p.MB;
-      int blk_cur = 0;
-      {
-        const int tb = t0 + lane * p.tile_rows;
-        if (lane < boxes_per_stage && tb < t1e) blk_cur = row[tb / p.bs];
-      }
-      if (nstage == 0) {  // the tile sees nothing of this chunk: one empty stage carries the bookkeeping
-        int slot;
-        if (!acquire(slot)) {
-          ok = false;
-          break;
-        }
-        if (lane == 0) {
-          g_meta[2 * slot] = make_int4(d.y, b, h, 0 | (3 << 16));
-          g_meta[2 * slot + 1] = make_int4(t0, lim_base, t1, rt);
-          mbar_arrive(s_full + 8 * slot);
-        }
-        ++it;
-      }
-      for (int s = 0; s < nstage; ++s, ++it) {
-        const int tok0 = t0 + s * kChunkStageTok;
-        const int ntok = min(kChunkStageTok, t1e - tok0);
-        const int nbox = (ntok + p.tile_rows - 1) / p.tile_rows;
-        int blk_n = 0;  // table entries of the following stage, one stage ahead of their use
-        {
-          const int tb = tok0 + kChunkStageTok + lane * p.tile_rows;
-          if (s + 1 < nstage && lane < boxes_per_stage && tb < t1e) blk_n = row[tb / p.bs];
-        }
-        int slot;
-        if (!acquire(slot)) {
-          ok = false;
-          break;
-        }
-        const uint32_t full = s_full + 8 * slot;
-        if (lane == 0) {
-          const int flags = (s == 0 ? 1 : 0) | (s == nstage - 1 ? 2 : 0);
-          g_meta[2 * slot] = make_int4(d.y, b, h, ntok | (flags << 16));
-          g_meta[2 * slot + 1] = make_int4(tok0, lim_base, t1, rt);
-          mbar_arrive_expect_tx(full, 2u * (uint32_t)nbox * box_rows_bytes * (D / 64));
-        }
-        __syncwarp();
-        if (lane < nbox) {
-          const int tb = tok0 + lane * p.tile_rows;
-          const int c_tok = tb % p.bs;
-          const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + (uint32_t)lane * box_rows_bytes;
-          const uint32_t dv = dk + L::kTileBytes;
-#pragma unroll
-          for (int j = 0; j < D / 64; ++j) {
-            tma_load_4d(dk + j * L::kHalfBytes, &tm_k, full, 64 * j, c_tok, h, blk_cur);
-            tma_load_4d(dv + j * L::kHalfBytes, &tm_v, full, 64 * j, c_tok, h, blk_cur);
-          }
-        }
-        blk_cur = blk_n;
-      }
-      unit = nxt;
-    }
-    if (ok) {  // end marker (one stage, seen by every consumer warp)
-      int slot;
-      if (acquire(slot)) {
-        if (lane == 0) {
-          g_meta[2 * slot] = make_int4(-1, 0, 0, 0);
-          mbar_arrive(s_full + 8 * slot);
-        }
-        ++it;
-      } else {
-        ok = false;
-      }
-    }
-    if (!ok) {
-      // stop path: record it, then wait (bounded) until every copy already issued has landed
-      if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
-      int dummy_abort = 0;
-      const int pending = it < nst ? it : nst;
-      for (int k = 0; k < pending; ++k) {
-        const int j = it - 1 - k;
-        mbar_wait_bounded(s_full + 8 * (j % nst), (uint32_t)(j / nst) & 1u, &dummy_abort, kWaitLimitNs / 8);
-      }
-    }
+    chunk_produce<D>(tm_k, tm_v, p, RT, nst, s_stage, s_full, s_empty, g_meta, s_abort, lane);
     return;
   }
 
@@ -359,9 +373,9 @@ chunk_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;
         const uint32_t vst = kst + L::kTileBytes;
         if (e_first >= kChunkStageTok)
-          chunk_consume<D, false>(kst, vst, k_off, v_off, qf, m_run, l_run, o_acc, p.scale_log2e, ntok, e0, e1, t);
+          chunk_consume<D, kChunkStageTok, false>(kst, vst, k_off, v_off, qf, m_run, l_run, o_acc, p.scale_log2e, ntok, e0, e1, t);
         else
-          chunk_consume<D, true>(kst, vst, k_off, v_off, qf, m_run, l_run, o_acc, p.scale_log2e, ntok, e0, e1, t);
+          chunk_consume<D, kChunkStageTok, true>(kst, vst, k_off, v_off, qf, m_run, l_run, o_acc, p.scale_log2e, ntok, e0, e1, t);
       }
     }
     __syncwarp();
@@ -398,6 +412,227 @@ chunk_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
           if (t == 0) p.part_lse[(size_t)slot_id * p.GQ + col] = l > 0.f ? m + lg2(l) : -INFINITY;
         }
       }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ 9 .. 16 score columns
+// Up to 16 score columns (one 16-row tile), too few to give every warp rows of its own: the NCW consumer
+// warps share the tile's rows and split the TOKENS of each 64-token stage, 16 per warp, in the row layout
+// above (the decode kernel's column layout needs a second 8-column MMA tile and a transposition per tile
+// for more than 8 columns).  Each warp keeps its own running maximum, sum and O[16 x D]; when an item ends
+// the warps combine through shared memory and write the rows.  The scratch for that is the item's last
+// stage itself: the K / V rows a warp alone reads (its 16-token slices) are exactly as large as its fp32
+// O tile, so it overwrites them right after its last MMA, one mbarrier phase later every warp reads all
+// four tiles, and only then is the stage handed back to the producer.
+template <int NCW>
+struct Row16Smem {
+  static constexpr int kStatBytes = 2 * NCW * 16 * 2 * 4;  // running maximum and sum per (warp, row), two item parities
+  template <int D>
+  __host__ __device__ static size_t total(int nstages) {
+    return 1024 + (size_t)nstages * (ChunkSmem<D>::kStageBytes + 32 + 16) + kStatBytes + 64;
+  }
+};
+
+template <int D, int NCW>
+__global__ void __launch_bounds__((NCW + 1) * 32, 2)
+row16_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                  const DecodeParams p) {
+  static_assert(NCW * 16 == kChunkStageTok, "one 16-token slice of a stage per consumer warp");
+  using L = ChunkSmem<D>;
+  using M = Row16Smem<NCW>;
+  constexpr int KS = D / 16, NO = D / 8;
+  constexpr int kRowBytes = D * 4;                // one fp32 row of a warp's O tile
+  constexpr int kRowsPerPiece = 2048 / kRowBytes; // a warp's slice of one 64-dim half of K or V is 2 KiB
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const int nst = p.nstages;
+  const uint32_t s_stage = base;
+  const uint32_t s_merge = s_stage + (uint32_t)nst * L::kStageBytes;
+  const uint32_t s_meta = s_merge + M::kStatBytes;
+  const uint32_t s_full = s_meta + (uint32_t)nst * 32;
+  const uint32_t s_empty = s_full + (uint32_t)nst * 8;
+  const uint32_t s_mbar = s_empty + (uint32_t)nst * 8;
+  float* g_stat = reinterpret_cast<float*>(gen + (s_merge - base));
+  int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
+  volatile int* s_abort = reinterpret_cast<volatile int*>(gen + (s_mbar + 8 - base));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    *s_abort = 0;
+    for (int i = 0; i < nst; ++i) {
+      mbar_init(s_full + 8 * i, 1);
+      mbar_init(s_empty + 8 * i, NCW);
+    }
+    mbar_init(s_mbar, NCW * 32);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  grid_dep_wait();    // the plan (and a fused append) must have completed
+  grid_dep_launch();  // the merge kernel may queue up behind this grid
+
+  if (warp == NCW) {
+    chunk_produce<D>(tm_k, tm_v, p, 16, nst, s_stage, s_full, s_empty, g_meta, s_abort, lane);
+    return;
+  }
+
+  // =================================================================== consumer warps
+  const int g = lane >> 2, t = lane & 3;
+  const int lane_row = lane & 7, mi = lane >> 3;
+  uint32_t k_off[2], v_off[4];
+  {
+    const uint32_t pat = (uint32_t)((mi ^ lane_row) << 4);
+    k_off[0] = (uint32_t)lane_row * 128 + pat;
+    k_off[1] = (uint32_t)lane_row * 128 + (pat ^ 64u);
+    const uint32_t vrow = (uint32_t)((mi & 1) * 8 + lane_row) * 128;
+    const uint32_t vx = (uint32_t)(((mi >> 1) ^ lane_row) << 4);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v_off[i] = vrow + (((uint32_t)i * 32u) ^ vx);
+  }
+  const uint32_t slice = (uint32_t)warp * 16 * 128;  // this warp's 16 token rows inside a 64-dim half
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  float o_acc[NO][4];
+  uint32_t qf[KS][4];
+#pragma unroll
+  for (int n = 0; n < NO; ++n) o_acc[n][0] = o_acc[n][1] = o_acc[n][2] = o_acc[n][3] = 0.f;
+#pragma unroll
+  for (int k = 0; k < KS; ++k) qf[k][0] = qf[k][1] = qf[k][2] = qf[k][3] = 0u;
+  int lim_row0 = 0, lim_row1 = 0;
+  uint32_t mphase = 0;  // parity of the next combine-barrier phase to wait for = parity of the item count
+
+  int slot = -1;
+  uint32_t full_phase = 1u;
+  for (;;) {
+    if (++slot == nst) slot = 0;
+    if (slot == 0) full_phase ^= 1u;
+    if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
+      if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+      return;
+    }
+    const int4 meta = g_meta[2 * slot], meta2 = g_meta[2 * slot + 1];
+    if (meta.x < 0) break;
+    const int ntok = meta.w & 0xffff;
+    const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+    const int b = meta.y, h = meta.z, lim_base = meta2.y;
+    if (first) {
+      m_run[0] = m_run[1] = -INFINITY;
+      l_run[0] = l_run[1] = 0.f;
+#pragma unroll
+      for (int n = 0; n < NO; ++n) o_acc[n][0] = o_acc[n][1] = o_acc[n][2] = o_acc[n][3] = 0.f;
+      const int c0 = g, c1 = g + 8;
+      const int qi0 = c0 / p.G, qi1 = c1 / p.G;
+      lim_row0 = lim_base + qi0;
+      lim_row1 = lim_base + qi1;
+      const __nv_bfloat16* q0 = p.q + (((size_t)b * p.Sq + qi0) * p.Hq + (size_t)h * p.G + (c0 - qi0 * p.G)) * D;
+      const __nv_bfloat16* q1 = p.q + (((size_t)b * p.Sq + qi1) * p.Hq + (size_t)h * p.G + (c1 - qi1 * p.G)) * D;
+      const bool ok0 = c0 < p.GQ, ok1 = c1 < p.GQ;
+#pragma unroll
+      for (int k = 0; k < KS; ++k) {
+        qf[k][0] = ok0 ? *reinterpret_cast<const uint32_t*>(q0 + 16 * k + 2 * t) : 0u;
+        qf[k][1] = ok1 ? *reinterpret_cast<const uint32_t*>(q1 + 16 * k + 2 * t) : 0u;
+        qf[k][2] = ok0 ? *reinterpret_cast<const uint32_t*>(q0 + 16 * k + 8 + 2 * t) : 0u;
+        qf[k][3] = ok1 ? *reinterpret_cast<const uint32_t*>(q1 + 16 * k + 8 + 2 * t) : 0u;
+      }
+    }
+    const int nslice = ntok - 16 * warp;  // tokens of this warp's slice that exist
+    if (nslice > 0) {
+      const int tokw = meta2.x + 16 * warp, t1 = meta2.z;
+      const int e0 = min(t1, lim_row0) - tokw, e1 = min(t1, lim_row1) - tokw;
+      const int e_first = min(t1, lim_base) - tokw;                       // row 0 sees the fewest tokens
+      const int e_last = min(t1, lim_base + (p.GQ - 1) / p.G) - tokw;     // the last real row the most
+      if (e_last > 0) {
+        const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes + slice;
+        const uint32_t vst = kst + L::kTileBytes;
+        if (e_first >= 16)
+          chunk_consume<D, 16, false>(kst, vst, k_off, v_off, qf, m_run, l_run, o_acc, p.scale_log2e, nslice, e0, e1, t);
+        else
+          chunk_consume<D, 16, true>(kst, vst, k_off, v_off, qf, m_run, l_run, o_acc, p.scale_log2e, nslice, e0, e1, t);
+      }
+    }
+    __syncwarp();
+    if (!last) {
+      if (lane == 0) mbar_arrive(s_empty + 8 * slot);
+      continue;
+    }
+    // ---- the item is complete: combine the NCW warps' running states through this stage's memory
+    {
+      const int slot_id = meta.x;
+      const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
+      float l0 = l_run[0], l1 = l_run[1];
+#pragma unroll
+      for (int o = 1; o < 4; o <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, o);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+      }
+      // O tile of warp w: row r lives in piece r / kRowsPerPiece (the warp's 2 KiB slices of K half 0, K half 1,
+      // V half 0, V half 1, 8 KiB apart), 16-byte chunk c of a row at position c ^ (r & 7) (bank spreading)
+      uint8_t* stage_gen = gen + (size_t)slot * L::kStageBytes;
+      auto tile_row = [&](int w, int r) {
+        return stage_gen + (size_t)(r / kRowsPerPiece) * L::kHalfBytes + (size_t)w * 2048 +
+               (size_t)(r % kRowsPerPiece) * kRowBytes;
+      };
+      float* all_m = g_stat + (size_t)mphase * (NCW * 16 * 2);
+      if (t == 0) {
+        float* mm = all_m + ((size_t)warp * 16 + g) * 2;
+        mm[0] = m_run[0];
+        mm[1] = l0;
+        mm[16] = m_run[1];
+        mm[17] = l1;
+      }
+      {
+        uint8_t* r0 = tile_row(warp, g);
+        uint8_t* r1 = tile_row(warp, g + 8);
+#pragma unroll
+        for (int n = 0; n < NO; ++n) {
+          const int off = (((2 * n + (t >> 1)) ^ g) << 4) + (t & 1) * 8;  // (g + 8) & 7 = g
+          *reinterpret_cast<float2*>(r0 + off) = make_float2(o_acc[n][0], o_acc[n][1]);
+          *reinterpret_cast<float2*>(r1 + off) = make_float2(o_acc[n][2], o_acc[n][3]);
+        }
+      }
+      mbar_arrive(s_mbar);
+      if (!warp_wait(s_mbar, mphase, s_abort)) {
+        if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+        return;
+      }
+      mphase ^= 1u;
+      for (int idx = threadIdx.x; idx < p.GQ * (D / 4); idx += NCW * 32) {
+        const int col = idx / (D / 4), c = idx % (D / 4);  // four dims 4c .. 4c + 3 of score column `col`
+        float mx = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NCW; ++w) mx = fmaxf(mx, all_m[(w * 16 + col) * 2]);
+        const float ms = mx == -INFINITY ? 0.f : mx;  // a row that saw nothing of this chunk (causal limit)
+        float den = 0.f;
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < NCW; ++w) {
+          const float sw = ex2(all_m[(w * 16 + col) * 2] - ms);
+          den += sw * all_m[(w * 16 + col) * 2 + 1];
+          const float4 o = *reinterpret_cast<const float4*>(tile_row(w, col) + ((c ^ (col & 7)) << 4));
+          num.x += sw * o.x;
+          num.y += sw * o.y;
+          num.z += sw * o.z;
+          num.w += sw * o.w;
+        }
+        const float inv = den > 0.f ? 1.f / den : 0.f;
+        if (n_chunks == 1) {
+          const int qi = col / p.G, head = col - qi * p.G;
+          __nv_bfloat16* dst = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D + 4 * c;
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(num.x * inv, num.y * inv);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(num.z * inv, num.w * inv);
+          *reinterpret_cast<uint2*>(dst) =
+              make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+        } else {
+          *reinterpret_cast<float4*>(p.part_o + ((size_t)slot_id * p.GQ + col) * D + 4 * c) =
+              make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+          if (c == 0) p.part_lse[(size_t)slot_id * p.GQ + col] = den > 0.f ? mx + lg2(den) : -INFINITY;
+        }
+      }
+      // the stage was written through the generic proxy; the producer refills it through the async proxy
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_empty + 8 * slot);
     }
   }
 }

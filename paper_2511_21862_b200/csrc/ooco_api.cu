@@ -20,8 +20,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}};
 static std::atomic<int> g_overridden[kKnobCount];  // knob set through ooco_set_tuning
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
@@ -283,6 +283,40 @@ static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the chunk attention kernel", (long)e);
+}
+
+// 9 .. 16 score columns: the warps of a CTA share one 16-row tile and split the tokens of a stage.
+template <int D>
+static int launch_row16(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
+                        int ctas_per_sm, cudaStream_t st, int dev) {
+  constexpr int NCW = 4;
+  using M = Row16Smem<NCW>;
+  auto kern = row16_main_kernel<D, NCW>;
+  static std::atomic<int> static_smem{-1};
+  if (static_smem.load() < 0) {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncGetAttributes", (long)e);
+    static_smem.store((int)fa.sharedSizeBytes);
+  }
+  const size_t dyn_max = (size_t)di.smem_optin - (size_t)static_smem.load();
+  const size_t budget = ctas_per_sm > 1 ? ((size_t)di.smem_optin + 1024) / ctas_per_sm - 1024 - static_smem.load()
+                                        : dyn_max;
+  int nst = 8;
+  while (nst > 2 && M::template total<D>(nst) > budget) --nst;
+  if (M::template total<D>(nst) > dyn_max) return OOCO_E_UNSUPPORTED;
+  p.nstages = nst;
+  const size_t smem = M::template total<D>(nst);
+  static std::atomic<size_t> configured[64];
+  if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
+    if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
+  }
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + 1) * 32), smem, st,
+                            g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the 16-row attention kernel", (long)e);
 }
 
 template <int D>
@@ -602,11 +636,17 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (ncw == 8 || kv8) tpw = 1;
   // prefill chunk: 64-token stages; 8 warps (128 columns) x 1 CTA per SM, fewer columns: smaller CTAs x 2
   const bool chunk = G_ > kDecodeMaxColumns;
+  // 9 .. 16 columns: the row layout with the tokens of a stage split over 4 warps x 2 CTAs per SM (the
+  // column layout of the decode kernel needs a second MMA tile and a transposition per tile there)
+  const bool row16 = !chunk && !kv8 && G_ > 8 && g_knobs[kKnobRowLayout16].load() != 0;
   if (chunk) {
     ncw = chunk_warps(G_);
     cps = ncw == 8 ? 1 : 2;
+  } else if (row16) {
+    ncw = 4;
+    cps = 2;
   }
-  const int stage_tok = chunk ? kChunkStageTok : 16 * ncw * tpw;
+  const int stage_tok = (chunk || row16) ? kChunkStageTok : 16 * ncw * tpw;
   DecodeParams p;
   memset(&p, 0, sizeof p);
   uint8_t* ws = (uint8_t*)workspace;
@@ -643,7 +683,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.v_scale = kv8 ? kv8->v_scale * kE4m3WidenFactor : 1.f;
 
   CUtensorMap tk, tv;
-  bool five_d = !kv8 && !chunk && s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
+  bool five_d = !kv8 && !chunk && !row16 && s->head_dim == 128 && !g_knobs[kKnobSplitHalves].load();
   if (five_d && encode_kv_map(&tk, s, k_cache, p.tile_rows, true) != OOCO_OK) five_d = false;
   if (kv8) {
     if ((rc = encode_kv8_map(&tk, s, k_cache, p.tile_rows))) return rc;
@@ -692,6 +732,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (chunk)
     rc = s->head_dim == 128 ? launch_chunk_ncw<128>(ncw, tk, tv, p, di, cps, st, dev)
                             : launch_chunk_ncw<64>(ncw, tk, tv, p, di, cps, st, dev);
+  else if (row16)
+    rc = s->head_dim == 128 ? launch_row16<128>(tk, tv, p, di, cps, st, dev) : launch_row16<64>(tk, tv, p, di, cps, st, dev);
   else if (kv8)
     rc = launch_main_kv8(ncw, tk, tv, p, di, cps, stages, st, dev);
   else if (s->head_dim == 128)
