@@ -63,7 +63,8 @@ enum {
  *
  * Supported by the kernels: head_dim in {64, 128}; block_size in
  * {16, 32, 64, 128, 256}; 1 <= Hq / Hkv <= 16; every stride a multiple of 8
- * elements (16 bytes) and the cache base addresses 16-byte aligned.
+ * elements (16 bytes) and the cache, q and out base addresses 16-byte aligned
+ * (OOCO_E_UNSUPPORTED otherwise: the kernels use vector loads and stores).
  */
 typedef struct {
   int32_t batch;              /* B: sequences in the decode batch                  */

@@ -612,7 +612,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if ((rc = validate_kv8(s, kv8))) return rc;
   if ((rc = validate_q_len(s, q_len, kv8 != nullptr))) return rc;
   if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
-  if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q) & 15) return OOCO_E_UNSUPPORTED;
+  if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q | (uintptr_t)out) & 15) return OOCO_E_UNSUPPORTED;
   const WsLayout w = ws_layout(s, q_len);
   if (workspace_bytes < w.total || ((uintptr_t)workspace & 255)) return OOCO_E_WORKSPACE;
   int dev = 0;
