@@ -1,4 +1,4 @@
-"""Seeded random shapes and length mixes against the oracle: bf16, 8-bit cache and several query tokens."""
+"""Seeded random shapes and length mixes against the oracle: bf16, 8-bit cache, several query tokens, prefill chunks."""
 import numpy as np
 import pytest
 import torch
@@ -114,3 +114,50 @@ def test_random_case(seed):
     assert binding.workspace_status(ws) == 0
     assert_close(out, ref, what=f"{cfg.name} {mode} Sq={Sq} G={cfg.num_q_heads // cfg.num_kv_heads} D={cfg.head_dim} "
                                  f"bs={cfg.block_size} {cfg.layout}")
+
+
+def draw_chunk_case(seed):
+    """Random prefill chunks: more than 8 score columns per (sequence, kv head), i.e. the two row-layout
+    kernels; contexts shorter than, equal to and far longer than the chunk."""
+    rng = np.random.default_rng(5000 + seed)
+    D = int(rng.choice([64, 128, 128]))
+    Hkv = int(rng.choice([1, 2, 2, 4]))
+    G = int(rng.choice([1, 2, 3, 4, 5, 8, 16]))
+    bs = int(rng.choice([16, 16, 32, 64, 128, 256]))
+    B = int(rng.integers(1, 6))
+    Sq = int(rng.choice([2, 3, 5, 8, 16, 17, 31, 32, 33, 48, 64, 65, 80]))
+    while Sq * G <= 8:
+        Sq *= 2
+    kinds = rng.integers(0, 4, B)
+    lens = np.where(kinds == 0, rng.integers(0, Sq + 2, B),                  # shorter than / about the chunk
+                    np.where(kinds == 1, Sq + rng.integers(0, 3, B),         # a fresh prompt: context = chunk
+                             np.where(kinds == 2, rng.integers(Sq, 700, B), rng.integers(700, 6000, B))))
+    # keep the oracle's work bounded: rows x tokens
+    while B * Sq * Hkv * G * max(1, int(lens.mean())) > 6_000_000:
+        lens = np.maximum(lens // 2, 1)
+    layout = "token_major" if rng.random() < 0.25 else "head_major"
+    cfg = inputs.DecodeConfig(f"chunkfuzz{seed}", Hkv * G, Hkv, D, bs,
+                              (inputs.LengthGroup(B, int(lens.min()), int(lens.max()), "fixed", tuple(int(x) for x in lens)),),
+                              seed=6000 + seed, pool_fill=float(rng.choice([1.0, 0.8])), layout=layout,
+                              shuffle_batch=False)
+    return cfg, Sq
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_chunk_case(seed):
+    cfg, Sq = draw_chunk_case(seed)
+    batch = inputs.make_batch(cfg, "cuda", poison=True, table_pad=-7)
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    q = torch.randn((cfg.batch, Sq, cfg.num_q_heads, cfg.head_dim), generator=g, device="cuda").to(torch.bfloat16)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_attention_mq(sh, q, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens, cfg.scale,
+                                out, ws)
+    assert binding.workspace_status(ws) == 0
+    ref = oracle.decode_attention_mq(inputs.as_u16(q), inputs.as_u16(batch.k_cache), inputs.as_u16(batch.v_cache),
+                                     batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                     num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size, strides=batch.strides).out
+    assert_close(out.reshape(-1, cfg.num_q_heads, cfg.head_dim), ref.reshape(-1, cfg.num_q_heads, cfg.head_dim),
+                 what=f"{cfg.name} Sq={Sq} G={cfg.num_q_heads // cfg.num_kv_heads} D={cfg.head_dim} bs={cfg.block_size} "
+                      f"{cfg.layout} lens={batch.context_lens.cpu().tolist()}")
