@@ -35,7 +35,7 @@ FALLBACK_BF16_TFLOPS = 1590.0
 METRIC = "paged decode-attn achieved HBM TB/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one attention-kernel launch, from the
 # ncu capture summarised in profiles/ (null for workloads without a capture).
-NCU_TRAFFIC_BYTES = {"cfg1": 579_375_616 + 8_673_792}   # profiles/decode_main_kernel_cfg1_ncu_full.md
+NCU_TRAFFIC_BYTES = {"cfg1": 579_344_768 + 7_974_016}   # mean of the two launches in profiles/decode_main_kernel_cfg1_ncu_full.md
 
 
 def measured_peak():

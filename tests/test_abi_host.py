@@ -120,6 +120,27 @@ def test_argument_validation_without_a_device():
     assert L.ooco_decode_workspace_bytes(ctypes.byref(bad.c())) == 0
 
 
+def test_query_length_limits_and_workspace_growth_without_a_device():
+    """Host-side rules of the several-query-token entry points: q_len in [1, 8192]; the workspace holds one
+    fp32 partial row per (split item, score column), so it grows with q_len; q_len = 1 is the decode size;
+    a misaligned q or out pointer is refused before anything is launched."""
+    L = binding.lib()
+    sh = binding.Shape(4, 32, 8, 128, 16, 1000, 64, 8 * 16 * 128, 16 * 128, 128)
+    assert binding.workspace_bytes_mq(sh, 1) == binding.workspace_bytes(sh)
+    sizes = [binding.workspace_bytes_mq(sh, q) for q in (1, 2, 4, 5, 16, 64, 1024, 8192)]
+    assert all(a < b for a, b in zip(sizes, sizes[1:]))
+    for q in (0, -1, 8193):
+        with pytest.raises(binding.OocoError):
+            binding.workspace_bytes_mq(sh, q)
+    ok, odd = ctypes.c_void_p(256), ctypes.c_void_p(258)
+    def attn(q_len, q=ok, out=ok, ws_bytes=1 << 40):
+        return L.ooco_decode_attention_mq(ctypes.byref(sh.c()), q_len, q, ok, ok, ok, ok, 1.0, out, ok, ws_bytes, None)
+    assert attn(8193) == -3 and attn(0) == -2
+    assert attn(64, q=odd) == -3 and attn(64, out=odd) == -3
+    assert attn(64, ws_bytes=binding.workspace_bytes_mq(sh, 4)) == -4
+    assert L.ooco_set_tuning(11, 0) == 0 and L.ooco_set_tuning(11, 1) == 0 and L.ooco_set_tuning(12, 1) == -2
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libooco.so")
