@@ -172,7 +172,8 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
     int nxt = 0;
     if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
     nxt = __shfl_sync(0xffffffffu, nxt, 0);
-    const int item = (int)(unit / nrt), rt = (int)(unit - (long long)item * nrt);
+    // the last row tile of an item sees the most tokens: it goes first (longest work first)
+    const int item = (int)(unit / nrt), rt = nrt - 1 - (int)(unit - (long long)item * nrt);
     const int4 d = p.items[item];
     const int b = d.x, h = d.y % p.Hkv, t0 = d.z, t1 = d.w;
     long long T = p.context_lens[b];

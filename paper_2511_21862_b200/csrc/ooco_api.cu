@@ -120,7 +120,8 @@ static WsLayout ws_layout(const ooco_shape_t* s, int q_len = 1) {
   // CTAs divided by the row tiles of an item, since every item is worked on once per row tile
   const int64_t sized_ctas = G > kDecodeMaxColumns ? (kGridCap + chunk_row_tiles(G) - 1) / chunk_row_tiles(G) : kGridCap;
   if (extra < sized_ctas * ipc) extra = sized_ctas * ipc;
-  const int64_t max_items = (int64_t)s->num_kv_heads * s->batch + extra + 64;
+  // (the bound needs no slack; a partial row per score column makes chunk-path items large, so theirs is small)
+  const int64_t max_items = (int64_t)s->num_kv_heads * s->batch + extra + (G > kDecodeMaxColumns ? 8 : 64);
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
   WsLayout w;
   w.max_items = (int)(max_items > INT32_MAX ? INT32_MAX : max_items);
