@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libooco.so")
 SOURCES = ["ooco_api.cu", "ooco_sched.cpp"]
-HEADERS = ["decode_kernels.cuh", "chunk_kernels.cuh", "block_copy_kernels.cuh", "ptx.cuh", os.path.join("..", "..", "include", "ooco.h"),
+HEADERS = ["decode_kernels.cuh", "chunk_kernels.cuh", "chunk_tc_kernels.cuh", "block_copy_kernels.cuh", "ptx.cuh", os.path.join("..", "..", "include", "ooco.h"),
            os.path.join("..", "..", "include", "ooco_sched.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",

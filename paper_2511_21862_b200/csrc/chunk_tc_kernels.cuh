@@ -1,0 +1,322 @@
+// Prefill-chunk attention over the paged cache on the 5th-generation tensor cores (tcgen05), head_dim 128,
+// for 65 or more score columns per (sequence, kv head).  Same units of work, producer warp, stage layout and
+// meta words as chunk_main_kernel (chunk_kernels.cuh); row tiles are 128 score rows = the MMA's M.
+//
+//   warp 4      producer: TMA K / V stages of 64 tokens ([half][64 tok][64 dims], 128-byte swizzle)
+//   warp 5      owns the tensor memory; one lane issues the MMAs:
+//                 S[128 x 64]   = Q[128 x 128] . K_stage^T      8 x tcgen05.mma M128 N64 K16, both operands K-major
+//                 O[128 x 128] (+)= P[128 x 64] . V_stage        4 x tcgen05.mma M128 N128 K16, V MN-major
+//               S lives in tensor-memory columns 0..63, O in columns 64..191, for the whole unit
+//   warps 0..3  softmax: thread r owns score row r.  It reads its S row from tensor memory, masks, keeps a
+//               reference maximum that is only raised when the row maximum exceeds it by more than 8 (log2
+//               units: the weights stay below 2^8, and raising it means rescaling the row of O in tensor
+//               memory, which then happens a few times per unit instead of once per stage), writes the bf16
+//               weights as the K-major, swizzled P tile into the K half of the stage (K is dead once S is
+//               complete), and at the end of the unit normalises its O row and writes it.
+// Every wait is bounded; on a wait that gives up the CTA stops issuing, drains and releases the tensor memory.
+#pragma once
+#include "chunk_kernels.cuh"
+
+namespace ooco {
+
+constexpr int kTcRows = 128;        // score rows per row tile
+constexpr int kTcTmemCols = 256;    // allocated columns (a power of two): S 0..63, O 64..191
+constexpr int kTcColS = 0, kTcColO = 64;
+constexpr float kTcRescaleStep = 8.f;
+
+struct ChunkTcSmem {
+  static constexpr int kQBytes = kTcRows * 128 * 2;  // [2 halves][128 rows][64 dims] bf16
+  __host__ __device__ static size_t total(int nstages) {
+    return 1024 + (size_t)nstages * (ChunkSmem<128>::kStageBytes + 32 + 16) + kQBytes + 128;
+  }
+};
+
+__global__ void __launch_bounds__(192, 2)
+chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                const DecodeParams p) {
+  constexpr int D = 128;
+  using L = ChunkSmem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const int nst = p.nstages;
+  const uint32_t s_stage = base;
+  const uint32_t s_q = s_stage + (uint32_t)nst * L::kStageBytes;
+  const uint32_t s_meta = s_q + ChunkTcSmem::kQBytes;
+  const uint32_t s_full = s_meta + (uint32_t)nst * 32;
+  const uint32_t s_empty = s_full + (uint32_t)nst * 8;
+  const uint32_t s_sready = s_empty + (uint32_t)nst * 8;  // S of the stage is complete        (MMA commit)
+  const uint32_t s_pready = s_sready + 8;                 // P (and the meta words) are consumed (128 softmax threads)
+  const uint32_t s_qready = s_pready + 8;                 // Q of the unit is in shared memory  (128 softmax threads)
+  const uint32_t s_oready = s_qready + 8;                 // O of the unit is complete          (MMA commit)
+  const uint32_t s_drain = s_oready + 8;
+  const uint32_t s_slot = s_drain + 8;
+  int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
+  uint8_t* g_q = gen + (s_q - base);
+  volatile uint32_t* g_slot = reinterpret_cast<volatile uint32_t*>(gen + (s_slot - base));
+  volatile int* s_abort = reinterpret_cast<volatile int*>(gen + (s_slot + 4 - base));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    *s_abort = 0;
+    for (int i = 0; i < nst; ++i) {
+      mbar_init(s_full + 8 * i, 1);
+      mbar_init(s_empty + 8 * i, 1);
+    }
+    mbar_init(s_sready, 1);
+    mbar_init(s_pready, 128);
+    mbar_init(s_qready, 128);
+    mbar_init(s_oready, 1);
+    mbar_init(s_drain, 1);
+    fence_mbar_init();
+  }
+  if (warp == 5) tmem_alloc(s_slot, kTcTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = *g_slot;
+  grid_dep_wait();    // the plan (and a fused append) must have completed
+  grid_dep_launch();  // the merge kernel may queue up behind this grid
+
+  if (warp == 4) {
+    chunk_produce<D>(tm_k, tm_v, p, kTcRows, nst, s_stage, s_full, s_empty, g_meta, s_abort, lane);
+  } else if (warp == 5) {
+    // ================================================================= MMA warp
+    const uint32_t idesc_s = umma_idesc_bf16(kTcRows, kChunkStageTok, 0);
+    const uint32_t idesc_o = umma_idesc_bf16(kTcRows, D, 1);
+    uint32_t ph_q = 0, ph_p = 0, full_phase = 1u;
+    int slot = -1;
+    bool issued = false, ok = true;
+    for (;;) {
+      if (++slot == nst) slot = 0;
+      if (slot == 0) full_phase ^= 1u;
+      if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
+        ok = false;
+        break;
+      }
+      const int4 meta = g_meta[2 * slot];
+      if (meta.x < 0) break;
+      const int ntok = meta.w & 0xffff;
+      const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+      const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes, vst = kst + L::kTileBytes;
+      if (ntok > 0) {
+        if (first) {
+          if (!warp_wait(s_qready, ph_q, s_abort)) {
+            ok = false;
+            break;
+          }
+          ph_q ^= 1u;
+        }
+        tc_fence_after_sync();
+        if (lane == 0) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma_ss(tmem + kTcColS, umma_smem_desc(s_q + h * (kTcRows * 128) + k * 32, 0, 1024),
+                      umma_smem_desc(kst + h * L::kHalfBytes + k * 32, 0, 1024), idesc_s, (h | k) ? 1u : 0u);
+          umma_commit(s_sready);
+        }
+        __syncwarp();
+        issued = true;
+      }
+      // the softmax threads are done with this stage's meta words (and, with tokens, have written P)
+      if (!warp_wait(s_pready, ph_p, s_abort)) {
+        ok = false;
+        break;
+      }
+      ph_p ^= 1u;
+      if (ntok > 0) {
+        tc_fence_after_sync();
+        if (lane == 0) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)  // P sits where K was; 16 tokens of V are 16 rows of 128 bytes in either half
+            umma_ss(tmem + kTcColO, umma_smem_desc(kst + k * 32, 0, 1024),
+                    umma_smem_desc(vst + k * 2048, L::kHalfBytes, 1024), idesc_o, (first && k == 0) ? 0u : 1u);
+          umma_commit(s_empty + 8 * slot);
+          if (last) umma_commit(s_oready);
+        }
+        __syncwarp();
+      } else if (lane == 0) {
+        mbar_arrive(s_empty + 8 * slot);
+      }
+    }
+    if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+    if (!ok && issued) {  // the tensor memory must not be released under MMAs in flight
+      if (lane == 0) umma_commit(s_drain);
+      __syncwarp();
+      int dummy = 0;
+      mbar_wait_bounded(s_drain, 0u, &dummy, kWaitLimitNs / 8);
+    }
+  } else {
+    // ================================================================= softmax warps: thread = score row
+    const int row = threadIdx.x;
+    const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
+    float m_ref = -INFINITY, l_run = 0.f;
+    int lim_row = 0;
+    uint32_t ph_s = 0, ph_o = 0, full_phase = 1u;
+    int slot = -1;
+    for (;;) {
+      if (++slot == nst) slot = 0;
+      if (slot == 0) full_phase ^= 1u;
+      if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
+        if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+        break;
+      }
+      const int4 meta = g_meta[2 * slot], meta2 = g_meta[2 * slot + 1];
+      if (meta.x < 0) break;
+      const int ntok = meta.w & 0xffff;
+      const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+      const int b = meta.y, h = meta.z, rt = meta2.w, lim_base = meta2.y;
+      const int col = rt * kTcRows + row;
+      const int qi = col / p.G, head = col - qi * p.G;
+      const bool real_row = col < p.GQ;
+      uint8_t* stage_gen = gen + (size_t)slot * L::kStageBytes;
+      if (first) {
+        m_ref = -INFINITY;
+        l_run = 0.f;
+        lim_row = lim_base + qi;
+        if (ntok > 0) {  // this thread's Q row into the swizzled K-major tile
+          const uint4* src = reinterpret_cast<const uint4*>(
+              p.q + (((size_t)b * p.Sq + (real_row ? qi : 0)) * p.Hq + (size_t)h * p.G + (real_row ? head : 0)) * D);
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const uint4 v = real_row ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(g_q + (size_t)(c >> 3) * (kTcRows * 128) + (size_t)row * 128 +
+                                      (((c & 7) ^ (row & 7)) << 4)) = v;
+          }
+          fence_proxy_async_smem();
+          mbar_arrive(s_qready);
+        }
+      }
+      if (ntok > 0) {
+        if (!warp_wait(s_sready, ph_s, s_abort)) {
+          if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+          break;
+        }
+        ph_s ^= 1u;
+        tc_fence_after_sync();
+        uint32_t sr[2][32];
+        tmem_ld32(trow + kTcColS, sr[0]);
+        tmem_ld32(trow + kTcColS + 32, sr[1]);
+        tmem_ld_wait();
+        // tokens [0, e) of the stage are visible to this row
+        const int e = min(min(meta2.z, lim_row) - meta2.x, ntok);
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          float s = __uint_as_float(sr[j >> 5][j & 31]) * p.scale_log2e;
+          s = j < e ? s : -INFINITY;
+          sr[j >> 5][j & 31] = __float_as_uint(s);
+          mx = fmaxf(mx, s);
+        }
+        // reference maximum: raised only when the row maximum is more than kTcRescaleStep above it
+        const bool raise = m_ref != -INFINITY && mx > m_ref + kTcRescaleStep;
+        float alpha = 1.f;
+        if (m_ref == -INFINITY) {
+          m_ref = mx;  // nothing accumulated for this row so far (O row is 0 or not yet written)
+        } else if (raise) {
+          alpha = ex2(m_ref - mx);
+          m_ref = mx;
+        }
+        if (__any_sync(0xffffffffu, raise)) {  // warp-uniform: the tensor-memory accesses are warp-wide
+#pragma unroll 1
+          for (int c4 = 0; c4 < D / 32; ++c4) {
+            uint32_t o[32];
+            tmem_ld32(trow + kTcColO + 32 * c4, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+            tmem_st32(trow + kTcColO + 32 * c4, o);
+          }
+          tmem_st_wait();
+          l_run *= alpha;
+        }
+        const float mu = m_ref == -INFINITY ? 0.f : m_ref;
+        float add = 0.f;
+        uint8_t* prow = stage_gen + (size_t)row * 128;  // P tile [128 rows][64 tokens] over the stage's K
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int j = 8 * c + 2 * i;
+            w[i] = pack_bf16x2(ex2(__uint_as_float(sr[j >> 5][j & 31]) - mu),
+                               ex2(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]) - mu));
+            // sums use the rounded weights, so numerator and denominator agree exactly
+            add += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xffff0000u);
+          }
+          *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        l_run += add;
+        if (ntok < kChunkStageTok) {  // V rows beyond the stage's tokens may hold anything (NaN included): clear them
+          uint8_t* vgen = stage_gen + L::kTileBytes;
+          for (int idx = threadIdx.x; idx < (kChunkStageTok - ntok) * 16; idx += 128) {
+            const int r = ntok + (idx >> 4), c = idx & 15;
+            *reinterpret_cast<uint4*>(vgen + (size_t)(c >> 3) * L::kHalfBytes + (size_t)r * 128 + ((c & 7) << 4)) =
+                make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+        fence_proxy_async_smem();  // P and the cleared rows are read by the MMA through the async proxy
+        tc_fence_before_sync();
+        __syncwarp();
+      }
+      mbar_arrive(s_pready);
+
+      if (last) {
+        // ---- the unit is complete: normalise this row of O and write it
+        const int slot_id = meta.x;
+        const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
+        if (ntok > 0) {
+          if (!warp_wait(s_oready, ph_o, s_abort)) {
+            if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+            break;
+          }
+          ph_o ^= 1u;
+          tc_fence_after_sync();
+        }
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // l = 0: the row saw no token of this chunk
+        __nv_bfloat16* orow = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D;
+        float* prow_o = p.part_o + ((size_t)slot_id * p.GQ + col) * D;
+#pragma unroll 1
+        for (int c4 = 0; c4 < D / 32; ++c4) {
+          uint32_t o[32];
+          if (ntok > 0) {
+            tmem_ld32(trow + kTcColO + 32 * c4, o);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = 0u;
+          }
+          if (real_row && n_chunks == 1) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                w[i] = pack_bf16x2(__uint_as_float(o[8 * v + 2 * i]) * inv, __uint_as_float(o[8 * v + 2 * i + 1]) * inv);
+              *reinterpret_cast<uint4*>(orow + 32 * c4 + 8 * v) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          } else if (real_row) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+              *reinterpret_cast<float4*>(prow_o + 32 * c4 + 4 * v) =
+                  make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
+                              __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
+          }
+          __syncwarp();  // the tensor-memory loads are warp-wide: reconverge before the next one
+        }
+        if (real_row && n_chunks > 1)
+          p.part_lse[(size_t)slot_id * p.GQ + col] = l_run > 0.f ? m_ref + lg2(l_run) : -INFINITY;
+        tc_fence_before_sync();  // the next unit's first MMA overwrites O: ordered behind these reads by q-ready
+      }
+    }
+  }
+  // ---- common exit: release the tensor memory once every warp is done with it
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, kTcTmemCols);
+}
+
+}  // namespace ooco

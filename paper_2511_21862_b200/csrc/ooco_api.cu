@@ -13,6 +13,7 @@
 #include "../../include/ooco.h"
 #include "block_copy_kernels.cuh"
 #include "chunk_kernels.cuh"
+#include "chunk_tc_kernels.cuh"
 #include "decode_kernels.cuh"
 
 namespace ooco {
@@ -20,8 +21,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}};
 static std::atomic<int> g_overridden[kKnobCount];  // knob set through ooco_set_tuning
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
@@ -179,6 +180,24 @@ static int encode_kv8_map(CUtensorMap* tm, const ooco_shape_t* s, const void* ba
   return r == CUDA_SUCCESS ? OOCO_OK : fail_cuda("cuTensorMapEncodeTiled(8-bit)", (long)r);
 }
 
+// Launch with the programmatic-stream-serialization attribute (the kernel itself waits for its
+// predecessor with griddepcontrol.wait) when `pdl`, else an ordinary launch.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 template <int D, int NCW, int NT, int TPW, bool KV8 = false>
 static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                        int ctas_per_sm, int want_stages, cudaStream_t st, int dev) {
@@ -286,6 +305,37 @@ static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the chunk attention kernel", (long)e);
 }
 
+// Prefill chunk on tcgen05 (head_dim 128, more than 64 score columns): 128-row tiles, two CTAs per SM.
+static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
+                           int ctas_per_sm, cudaStream_t st, int dev) {
+  auto kern = chunk_tc_kernel;
+  static std::atomic<int> static_smem{-1};
+  if (static_smem.load() < 0) {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncGetAttributes", (long)e);
+    static_smem.store((int)fa.sharedSizeBytes);
+  }
+  const size_t dyn_max = (size_t)di.smem_optin - (size_t)static_smem.load();
+  const size_t budget = ctas_per_sm > 1 ? ((size_t)di.smem_optin + 1024) / ctas_per_sm - 1024 - static_smem.load()
+                                        : dyn_max;
+  int nst = 6;
+  while (nst > 2 && ChunkTcSmem::total(nst) > budget) --nst;
+  if (ChunkTcSmem::total(nst) > dyn_max) return OOCO_E_UNSUPPORTED;
+  p.nstages = nst;
+  const size_t smem = ChunkTcSmem::total(nst);
+  static std::atomic<size_t> configured[64];
+  if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
+    if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
+  }
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(192), smem, st,
+                            g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the tcgen05 chunk attention kernel", (long)e);
+}
+
 // 9 .. 16 score columns: the warps of a CTA share one 16-row tile and split the tokens of a stage.
 template <int D>
 static int launch_row16(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
@@ -328,24 +378,6 @@ static int launch_chunk_ncw(int ncw, const CUtensorMap& tk, const CUtensorMap& t
     case 4: return launch_chunk<D, 4>(tk, tv, p, di, cps, st, dev);
     default: return launch_chunk<D, 8>(tk, tv, p, di, cps, st, dev);
   }
-}
-
-// Launch with the programmatic-stream-serialization attribute (the kernel itself waits for its
-// predecessor with griddepcontrol.wait) when `pdl`, else an ordinary launch.
-template <typename... KArgs, typename... Args>
-static cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                             bool pdl, Args&&... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
 static AppendParams make_append_params(const ooco_shape_t* s, const void* k_new, const void* v_new,
@@ -640,9 +672,11 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // 9 .. 16 columns: the row layout with the tokens of a stage split over 4 warps x 2 CTAs per SM (the
   // column layout of the decode kernel needs a second MMA tile and a transposition per tile there)
   const bool row16 = !chunk && !kv8 && G_ > 8 && g_knobs[kKnobRowLayout16].load() != 0;
+  const bool chunk_tc = chunk && G_ > 64 && s->head_dim == 128 && g_knobs[kKnobChunkTcgen05].load() != 0;
   if (chunk) {
     ncw = chunk_warps(G_);
-    cps = ncw == 8 ? 1 : 2;
+    cps = (ncw == 8 && !chunk_tc) ? 1 : 2;
+    if (chunk_tc && g_overridden[kKnobCtasPerSm].load()) cps = g_knobs[kKnobCtasPerSm].load() > 1 ? 2 : 1;
   } else if (row16) {
     ncw = 4;
     cps = 2;
@@ -730,7 +764,9 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
   const int stages = g_knobs[kKnobStages].load();
   if (pe) cudaEventRecord(pe[1], st);
-  if (chunk)
+  if (chunk_tc)
+    rc = launch_chunk_tc(tk, tv, p, di, cps, st, dev);
+  else if (chunk)
     rc = s->head_dim == 128 ? launch_chunk_ncw<128>(ncw, tk, tv, p, di, cps, st, dev)
                             : launch_chunk_ncw<64>(ncw, tk, tv, p, di, cps, st, dev);
   else if (row16)
