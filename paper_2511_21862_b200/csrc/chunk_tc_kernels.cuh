@@ -6,7 +6,8 @@
 //   warp 5      owns the tensor memory; one lane issues the MMAs:
 //                 S[128 x 64]   = Q[128 x 128] . K_stage^T      8 x tcgen05.mma M128 N64 K16, both operands K-major
 //                 O[128 x 128] (+)= P[128 x 64] . V_stage        4 x tcgen05.mma M128 N128 K16, V MN-major
-//               S lives in tensor-memory columns 0..63, O in columns 64..191, for the whole unit
+//               two S buffers (tensor-memory columns 0..63, 64..127): the scores of the next stage are issued
+//               before this stage's P.V, so they run while the softmax threads work; O in columns 128..255
 //   warps 0..3  softmax: thread r owns score row r.  It reads its S row from tensor memory, masks, keeps a
 //               reference maximum that is only raised when the row maximum exceeds it by more than 8 (log2
 //               units: the weights stay below 2^8, and raising it means rescaling the row of O in tensor
@@ -20,8 +21,8 @@
 namespace ooco {
 
 constexpr int kTcRows = 128;        // score rows per row tile
-constexpr int kTcTmemCols = 256;    // allocated columns (a power of two): S 0..63, O 64..191
-constexpr int kTcColS = 0, kTcColO = 64;
+constexpr int kTcTmemCols = 256;    // allocated columns (a power of two): S buffers 0..63 and 64..127, O 128..255
+constexpr int kTcColS = 0, kTcColO = 128;
 constexpr float kTcRescaleStep = 8.f;
 
 struct ChunkTcSmem {
@@ -31,6 +32,9 @@ struct ChunkTcSmem {
   }
 };
 
+// Barrier bookkeeping.  Barriers that come in pairs ([2]) are used alternately by consecutive stages, and use
+// number n of a pair takes barrier n & 1 with phase parity (n >> 1) & 1: a waiter can then never be overtaken
+// by two completions of the barrier it waits on (the completion after next needs the waiter's own progress).
 __global__ void __launch_bounds__(192, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                 const DecodeParams p) {
@@ -46,11 +50,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   const uint32_t s_meta = s_q + ChunkTcSmem::kQBytes;
   const uint32_t s_full = s_meta + (uint32_t)nst * 32;
   const uint32_t s_empty = s_full + (uint32_t)nst * 8;
-  const uint32_t s_sready = s_empty + (uint32_t)nst * 8;  // S of the stage is complete        (MMA commit)
-  const uint32_t s_pready = s_sready + 8;                 // P (and the meta words) are consumed (128 softmax threads)
-  const uint32_t s_qready = s_pready + 8;                 // Q of the unit is in shared memory  (128 softmax threads)
-  const uint32_t s_oready = s_qready + 8;                 // O of the unit is complete          (MMA commit)
-  const uint32_t s_drain = s_oready + 8;
+  const uint32_t s_sready = s_empty + (uint32_t)nst * 8;  // [2] S buffer holds the stage's scores       (MMA commit)
+  const uint32_t s_sfree = s_sready + 16;                 // [2] S buffer has been read into registers  (128 softmax threads)
+  const uint32_t s_pready = s_sfree + 16;                 // [2] meta words consumed, P written         (128 softmax threads)
+  const uint32_t s_pvdone = s_pready + 16;                // [2] the stage's P.V is complete            (MMA commit)
+  const uint32_t s_qready = s_pvdone + 16;                // Q of the unit is in shared memory          (128 softmax threads)
+  const uint32_t s_drain = s_qready + 8;
   const uint32_t s_slot = s_drain + 8;
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
   uint8_t* g_q = gen + (s_q - base);
@@ -64,10 +69,13 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
       mbar_init(s_full + 8 * i, 1);
       mbar_init(s_empty + 8 * i, 1);
     }
-    mbar_init(s_sready, 1);
-    mbar_init(s_pready, 128);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(s_sready + 8 * i, 1);
+      mbar_init(s_sfree + 8 * i, 128);
+      mbar_init(s_pready + 8 * i, 128);
+      mbar_init(s_pvdone + 8 * i, 1);
+    }
     mbar_init(s_qready, 128);
-    mbar_init(s_oready, 1);
     mbar_init(s_drain, 1);
     fence_mbar_init();
   }
@@ -85,9 +93,29 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     // ================================================================= MMA warp
     const uint32_t idesc_s = umma_idesc_bf16(kTcRows, kChunkStageTok, 0);
     const uint32_t idesc_o = umma_idesc_bf16(kTcRows, D, 1);
-    uint32_t ph_q = 0, ph_p = 0, full_phase = 1u;
+    uint32_t ph_q = 0, full_phase = 1u;
+    uint32_t n_s = 0, n_p = 0, n_pv = 0;  // score MMAs issued, stages handed over by the softmax threads, P.V issued
     int slot = -1;
-    bool issued = false, ok = true;
+    bool issued = false, ok = true, s_ahead = false;  // s_ahead: this stage's scores were issued one stage early
+    // scores of the stage in `sl` into S buffer n_s & 1, once the softmax threads have emptied that buffer
+    auto issue_scores = [&](int sl) {
+      if (!warp_wait(s_sfree + 8 * (n_s & 1), ((n_s >> 1) & 1u) ^ 1u, s_abort)) return false;
+      tc_fence_after_sync();
+      if (lane == 0) {
+        const uint32_t kst = s_stage + (uint32_t)sl * L::kStageBytes;
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_ss(tmem + kTcColS + 64 * (n_s & 1), umma_smem_desc(s_q + h * (kTcRows * 128) + k * 32, 0, 1024),
+                    umma_smem_desc(kst + h * L::kHalfBytes + k * 32, 0, 1024), idesc_s, (h | k) ? 1u : 0u);
+        umma_commit(s_sready + 8 * (n_s & 1));
+      }
+      __syncwarp();
+      ++n_s;
+      issued = true;
+      return true;
+    };
     for (;;) {
       if (++slot == nst) slot = 0;
       if (slot == 0) full_phase ^= 1u;
@@ -99,45 +127,60 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
       if (meta.x < 0) break;
       const int ntok = meta.w & 0xffff;
       const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
-      const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes, vst = kst + L::kTileBytes;
       if (ntok > 0) {
-        if (first) {
-          if (!warp_wait(s_qready, ph_q, s_abort)) {
+        if (!s_ahead) {
+          if (first) {
+            if (!warp_wait(s_qready, ph_q, s_abort)) {
+              ok = false;
+              break;
+            }
+            ph_q ^= 1u;
+          }
+          if (!issue_scores(slot)) {
             ok = false;
             break;
           }
-          ph_q ^= 1u;
         }
-        tc_fence_after_sync();
-        if (lane == 0) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_ss(tmem + kTcColS, umma_smem_desc(s_q + h * (kTcRows * 128) + k * 32, 0, 1024),
-                      umma_smem_desc(kst + h * L::kHalfBytes + k * 32, 0, 1024), idesc_s, (h | k) ? 1u : 0u);
-          umma_commit(s_sready);
+        s_ahead = false;
+        if (!last) {  // the next stage belongs to the same unit: its scores run while this stage's softmax does
+          const int ns = slot + 1 == nst ? 0 : slot + 1;
+          if (!warp_wait(s_full + 8 * ns, ns == 0 ? full_phase ^ 1u : full_phase, s_abort) || !issue_scores(ns)) {
+            ok = false;
+            break;
+          }
+          s_ahead = true;
         }
+      }
+      if (ntok == 0) {
+        // a stage without tokens takes a turn of the S-buffer barriers as well, so that the softmax threads
+        // can never be more than one stage ahead of this warp (see the note on barrier pairs)
+        if (!warp_wait(s_sfree + 8 * (n_s & 1), ((n_s >> 1) & 1u) ^ 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        if (lane == 0) mbar_arrive(s_sready + 8 * (n_s & 1));
         __syncwarp();
-        issued = true;
+        ++n_s;
       }
       // the softmax threads are done with this stage's meta words (and, with tokens, have written P)
-      if (!warp_wait(s_pready, ph_p, s_abort)) {
+      if (!warp_wait(s_pready + 8 * (n_p & 1), (n_p >> 1) & 1u, s_abort)) {
         ok = false;
         break;
       }
-      ph_p ^= 1u;
+      ++n_p;
       if (ntok > 0) {
         tc_fence_after_sync();
         if (lane == 0) {
+          const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes, vst = kst + L::kTileBytes;
 #pragma unroll
           for (int k = 0; k < 4; ++k)  // P sits where K was; 16 tokens of V are 16 rows of 128 bytes in either half
             umma_ss(tmem + kTcColO, umma_smem_desc(kst + k * 32, 0, 1024),
                     umma_smem_desc(vst + k * 2048, L::kHalfBytes, 1024), idesc_o, (first && k == 0) ? 0u : 1u);
           umma_commit(s_empty + 8 * slot);
-          if (last) umma_commit(s_oready);
+          umma_commit(s_pvdone + 8 * (n_pv & 1));
         }
         __syncwarp();
+        ++n_pv;
       } else if (lane == 0) {
         mbar_arrive(s_empty + 8 * slot);
       }
@@ -153,15 +196,19 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     // ================================================================= softmax warps: thread = score row
     const int row = threadIdx.x;
     const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
-    float m_ref = -INFINITY, l_run = 0.f;
+    float m_ref = -INFINITY, l_run = 0.f;  // reference maximum (scaled, log2 domain), sum of the weights
     int lim_row = 0;
-    uint32_t ph_s = 0, ph_o = 0, full_phase = 1u;
+    uint32_t full_phase = 1u;
+    uint32_t n_s = 0, n_pv = 0;  // stages seen so far (each takes a turn of the S and P barriers), stages with tokens
     int slot = -1;
+    bool ok = true;
+    // P.V number k is complete
+    auto wait_pv = [&](uint32_t k) { return warp_wait(s_pvdone + 8 * (k & 1), (k >> 1) & 1u, s_abort); };
     for (;;) {
       if (++slot == nst) slot = 0;
       if (slot == 0) full_phase ^= 1u;
       if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
-        if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+        ok = false;
         break;
       }
       const int4 meta = g_meta[2 * slot], meta2 = g_meta[2 * slot + 1];
@@ -190,37 +237,47 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
           mbar_arrive(s_qready);
         }
       }
+      const uint32_t k_stage = n_s++;  // the stage is use k_stage of the S-buffer and P barriers
+      if (!warp_wait(s_sready + 8 * (k_stage & 1), (k_stage >> 1) & 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      if (ntok == 0) mbar_arrive(s_sfree + 8 * (k_stage & 1));
       if (ntok > 0) {
-        if (!warp_wait(s_sready, ph_s, s_abort)) {
-          if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
-          break;
-        }
-        ph_s ^= 1u;
+        const uint32_t k_pv = n_pv++;  // this stage's P.V is number k_pv
         tc_fence_after_sync();
         uint32_t sr[2][32];
-        tmem_ld32(trow + kTcColS, sr[0]);
-        tmem_ld32(trow + kTcColS + 32, sr[1]);
+        tmem_ld32(trow + kTcColS + 64 * (k_stage & 1), sr[0]);
+        tmem_ld32(trow + kTcColS + 64 * (k_stage & 1) + 32, sr[1]);
         tmem_ld_wait();
+        tc_fence_before_sync();
+        mbar_arrive(s_sfree + 8 * (k_stage & 1));  // the buffer may take the scores of the stage after next
         // tokens [0, e) of the stage are visible to this row
         const int e = min(min(meta2.z, lim_row) - meta2.x, ntok);
-        float mx = -INFINITY;
+        if (e < kChunkStageTok) {
 #pragma unroll
-        for (int j = 0; j < 64; ++j) {
-          float s = __uint_as_float(sr[j >> 5][j & 31]) * p.scale_log2e;
-          s = j < e ? s : -INFINITY;
-          sr[j >> 5][j & 31] = __float_as_uint(s);
-          mx = fmaxf(mx, s);
+          for (int j = 0; j < 64; ++j)
+            if (j >= e) sr[j >> 5][j & 31] = 0xff800000u;  // -inf
         }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains: the row is one thread's work
+#pragma unroll
+        for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sr[j >> 5][j & 31]));
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;  // the scale is positive
         // reference maximum: raised only when the row maximum is more than kTcRescaleStep above it
         const bool raise = m_ref != -INFINITY && mx > m_ref + kTcRescaleStep;
         float alpha = 1.f;
         if (m_ref == -INFINITY) {
-          m_ref = mx;  // nothing accumulated for this row so far (O row is 0 or not yet written)
+          m_ref = mx;  // nothing accumulated for this row so far (its O row is 0 or not yet written)
         } else if (raise) {
           alpha = ex2(m_ref - mx);
           m_ref = mx;
         }
         if (__any_sync(0xffffffffu, raise)) {  // warp-uniform: the tensor-memory accesses are warp-wide
+          if (!wait_pv(k_pv - 1)) {            // O must hold everything issued so far (never on a unit's first stage)
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
 #pragma unroll 1
           for (int c4 = 0; c4 < D / 32; ++c4) {
             uint32_t o[32];
@@ -233,8 +290,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
           tmem_st_wait();
           l_run *= alpha;
         }
-        const float mu = m_ref == -INFINITY ? 0.f : m_ref;
-        float add = 0.f;
+        const float neg_mu = m_ref == -INFINITY ? 0.f : -m_ref;
+        float add4[4] = {0.f, 0.f, 0.f, 0.f};
         uint8_t* prow = stage_gen + (size_t)row * 128;  // P tile [128 rows][64 tokens] over the stage's K
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -242,14 +299,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int j = 8 * c + 2 * i;
-            w[i] = pack_bf16x2(ex2(__uint_as_float(sr[j >> 5][j & 31]) - mu),
-                               ex2(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]) - mu));
-            // sums use the rounded weights, so numerator and denominator agree exactly
-            add += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xffff0000u);
+            const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2e, neg_mu));
+            const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2e, neg_mu));
+            add4[i] += p0 + p1;
+            w[i] = pack_bf16x2(p0, p1);
           }
           *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        l_run += add;
+        l_run += (add4[0] + add4[1]) + (add4[2] + add4[3]);
         if (ntok < kChunkStageTok) {  // V rows beyond the stage's tokens may hold anything (NaN included): clear them
           uint8_t* vgen = stage_gen + L::kTileBytes;
           for (int idx = threadIdx.x; idx < (kChunkStageTok - ntok) * 16; idx += 128) {
@@ -262,18 +319,17 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         tc_fence_before_sync();
         __syncwarp();
       }
-      mbar_arrive(s_pready);
+      mbar_arrive(s_pready + 8 * (k_stage & 1));
 
       if (last) {
         // ---- the unit is complete: normalise this row of O and write it
         const int slot_id = meta.x;
         const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
         if (ntok > 0) {
-          if (!warp_wait(s_oready, ph_o, s_abort)) {
-            if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+          if (!wait_pv(n_pv - 1)) {
+            ok = false;
             break;
           }
-          ph_o ^= 1u;
           tc_fence_after_sync();
         }
         const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // l = 0: the row saw no token of this chunk
@@ -309,9 +365,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         }
         if (real_row && n_chunks > 1)
           p.part_lse[(size_t)slot_id * p.GQ + col] = l_run > 0.f ? m_ref + lg2(l_run) : -INFINITY;
-        tc_fence_before_sync();  // the next unit's first MMA overwrites O: ordered behind these reads by q-ready
+        tc_fence_before_sync();  // the next unit's first P.V overwrites O: ordered behind these reads by q-ready
       }
     }
+    if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
   }
   // ---- common exit: release the tensor memory once every warp is done with it
   tc_fence_before_sync();

@@ -106,6 +106,13 @@ constexpr int kMaxQLen = 8192;
 static int chunk_warps(int columns) { return columns <= 32 ? 2 : (columns <= 64 ? 4 : 8); }
 static int chunk_row_tiles(int columns) { return (columns + 16 * chunk_warps(columns) - 1) / (16 * chunk_warps(columns)); }
 
+// Work items the plan aims at per CTA: many short ones balance the HBM-bound decode kernels; the chunk
+// kernels pay a query load, an epilogue and a partial row per score column for every item, and want few.
+static int plan_items_per_cta(int columns) {
+  if (columns > kDecodeMaxColumns && !g_overridden[kKnobItemsPerCta].load()) return 2;
+  return g_knobs[kKnobItemsPerCta].load();
+}
+
 // Workspace carve-up (all offsets multiples of 256 bytes).
 struct WsLayout {
   size_t off_first, off_items, off_lse, off_o, total;
@@ -114,7 +121,7 @@ struct WsLayout {
 static WsLayout ws_layout(const ooco_shape_t* s, int q_len = 1) {
   const int G = s->num_q_heads / s->num_kv_heads * q_len;  // score columns per (sequence, kv head)
   const int64_t cmax = g_knobs[kKnobChunkMax].load();
-  const int64_t ipc = g_knobs[kKnobItemsPerCta].load();
+  const int64_t ipc = plan_items_per_cta(G);
   const int64_t per_seq = ((int64_t)s->max_blocks_per_seq * s->block_size + cmax - 1) / cmax;
   int64_t extra = (int64_t)s->num_kv_heads * s->batch * per_seq;
   // the plan cuts the sequences into about (CTAs it sizes for) x ipc items; the chunk path sizes for the
@@ -712,7 +719,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.chunk_min = g_knobs[kKnobChunkMin].load();
   p.chunk_max = g_knobs[kKnobChunkMax].load();
   if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
-  p.items_per_cta = g_knobs[kKnobItemsPerCta].load();
+  p.items_per_cta = plan_items_per_cta(G_);
   // the 8-bit path widens codes to value / 256 (kE4m3WidenFactor): both scales carry the factor back
   p.scale_log2e = scale * 1.4426950408889634f * (kv8 ? kv8->k_scale * kE4m3WidenFactor : 1.f);
   p.v_scale = kv8 ? kv8->v_scale * kE4m3WidenFactor : 1.f;
