@@ -186,10 +186,12 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  *                   are skipped, as in ooco_kv_append
  *   workspace       >= ooco_decode_workspace_bytes_mq(shape, q_len)
  * Supported: 1 <= q_len <= 8192 (OOCO_E_UNSUPPORTED beyond).  Up to 16 score columns per
- * (sequence, kv head), (Hq / Hkv) * q_len <= 16, run the decode kernel (HBM-bound: the cache is
- * read once); more columns run the prefill-chunk kernel, which cuts the columns into row tiles of
+ * (sequence, kv head), (Hq / Hkv) * q_len <= 16, run the decode kernels (HBM-bound: the cache is
+ * read once); more columns run a prefill-chunk kernel, which cuts the columns into row tiles of
  * up to 128, reads the cache once per row tile (the repeats hit L2) and never loads tokens a tile
- * cannot see; it becomes bound by the tensor pipe from about 64 columns on.  The 8-bit cache
+ * cannot see; it becomes bound by the tensor pipe from about 64 columns on.  At head_dim 128 and
+ * more than 64 columns that kernel runs on tcgen05 (scores and output in tensor memory), otherwise
+ * on mma.sync.  The 8-bit cache
  * (ooco_decode_step_mq_fp8) has the decode kernel only.  The workspace grows with q_len: one fp32
  * partial row per (split item, score column).  q_len = 1 is ooco_decode_attention /
  * ooco_kv_append exactly.  Everything else as for those two.
@@ -429,7 +431,8 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * page-locked inputs through their device mapping and lets the kernels write a page-locked result
  * directly (zero = always one copy per buffer); 11 non-zero = 9 to 16 score columns per
  * (sequence, kv head) run the kernel whose warps share 16 score rows and split the tokens of a
- * stage (zero = the decode kernel with two 8-column tiles).
+ * stage (zero = the decode kernel with two 8-column tiles); 12 non-zero = more than 64 score columns
+ * at head_dim 128 run the tcgen05 kernel (zero = the mma.sync kernel of the prefill-chunk path).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.
  */

@@ -86,6 +86,19 @@ def test_prefill_chunk_matches_oracle(cfg, Sq):
     run_case(cfg, Sq, seed=cfg.seed)
 
 
+@pytest.mark.parametrize("cfg,Sq", [c for c in CHUNK_CASES if c[0].name in
+                                    ("ck-g4-sq33", "ck-g4-sq128-fresh", "ck-g8-sq64-bs64", "ck-split")],
+                         ids=lambda v: getattr(v, "name", str(v)))
+def test_prefill_chunk_on_the_mma_sync_kernel(cfg, Sq):
+    """head_dim 128 with more than 64 score columns runs the tcgen05 kernel by default; the mma.sync kernel
+    of the same shape stays selectable and must agree with the oracle too."""
+    binding.set_tuning(chunk_tcgen05=0)
+    try:
+        run_case(cfg, Sq, seed=cfg.seed)
+    finally:
+        binding.set_tuning(chunk_tcgen05=1)
+
+
 def test_chunk_rows_agree_with_decode_rows():
     """A chunk of 8 query tokens (32 columns: chunk kernel) and two calls of 4 (16 columns: decode kernel)
     over the same cache compute the same rows, up to the rounding of a different summation order."""
