@@ -3,17 +3,17 @@
 // meta words as chunk_main_kernel (chunk_kernels.cuh); row tiles are 128 score rows = the MMA's M.
 //
 //   warp 4      producer: TMA K / V stages of 64 tokens ([half][64 tok][64 dims], 128-byte swizzle)
-//   warp 5      owns the tensor memory; one lane issues the MMAs:
-//                 S[128 x 64]   = Q[128 x 128] . K_stage^T      8 x tcgen05.mma M128 N64 K16, both operands K-major
-//                 O[128 x 128] (+)= P[128 x 64] . V_stage        4 x tcgen05.mma M128 N128 K16, V MN-major
-//               two S buffers (tensor-memory columns 0..63, 64..127): the scores of the next stage are issued
-//               before this stage's P.V, so they run while the softmax threads work; O in columns 128..255
-//   warps 0..3  softmax: thread r owns score row r.  It reads its S row from tensor memory, masks, keeps a
-//               reference maximum that is only raised when the row maximum exceeds it by more than 8 (log2
-//               units: the weights stay below 2^8, and raising it means rescaling the row of O in tensor
-//               memory, which then happens a few times per unit instead of once per stage), writes the bf16
-//               weights as the K-major, swizzled P tile into the K half of the stage (K is dead once S is
-//               complete), and at the end of the unit normalises its O row and writes it.
+//   warp 5      owns the tensor memory; one lane issues the MMAs, whose A operands live in tensor memory:
+//                 S[128 x 64]   = Q[128 x 128] . K_stage^T      8 x tcgen05.mma M128 N64 K16, K K-major from the stage
+//                 O[128 x 128] (+)= P[128 x 64] . V_stage        4 x tcgen05.mma M128 N128 K16, V MN-major from the stage
+//               tensor-memory columns: S 0..63 (P, two bf16 per column, over its first 32 once the softmax
+//               threads have read S), O 64..191, Q 192..255 -- shared memory holds nothing but the stages
+//   warps 0..3  softmax: thread r owns score row r (tensor-memory lane r).  At the start of a unit it stores
+//               its Q row into tensor memory.  Per stage it reads its S row, masks, keeps a reference maximum
+//               that is only raised when the row maximum exceeds it by more than 8 (log2 units: the weights
+//               stay below 2^8, and raising it means rescaling the row of O in tensor memory, which then
+//               happens a few times per unit instead of once per stage), stores the bf16 weights as its P
+//               row, and at the end of the unit normalises its O row and writes it.
 // Every wait is bounded; on a wait that gives up the CTA stops issuing, drains and releases the tensor memory.
 #pragma once
 #include "chunk_kernels.cuh"
@@ -21,14 +21,13 @@
 namespace ooco {
 
 constexpr int kTcRows = 128;        // score rows per row tile
-constexpr int kTcTmemCols = 256;    // allocated columns (a power of two): S buffers 0..63 and 64..127, O 128..255
-constexpr int kTcColS = 0, kTcColO = 128;
+constexpr int kTcTmemCols = 256;    // allocated columns (a power of two)
+constexpr int kTcColS = 0, kTcColO = 64, kTcColQ = 192;
 constexpr float kTcRescaleStep = 8.f;
 
 struct ChunkTcSmem {
-  static constexpr int kQBytes = kTcRows * 128 * 2;  // [2 halves][128 rows][64 dims] bf16
   __host__ __device__ static size_t total(int nstages) {
-    return 1024 + (size_t)nstages * (ChunkSmem<128>::kStageBytes + 32 + 16) + kQBytes + 128;
+    return 1024 + (size_t)nstages * (ChunkSmem<128>::kStageBytes + 32 + 16) + 128;
   }
 };
 
@@ -46,8 +45,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   uint8_t* gen = smem_raw + (base - raw);
   const int nst = p.nstages;
   const uint32_t s_stage = base;
-  const uint32_t s_q = s_stage + (uint32_t)nst * L::kStageBytes;
-  const uint32_t s_meta = s_q + ChunkTcSmem::kQBytes;
+  const uint32_t s_meta = s_stage + (uint32_t)nst * L::kStageBytes;
   const uint32_t s_full = s_meta + (uint32_t)nst * 32;
   const uint32_t s_empty = s_full + (uint32_t)nst * 8;
   const uint32_t s_sready = s_empty + (uint32_t)nst * 8;  // [2] S buffer holds the stage's scores       (MMA commit)
@@ -58,7 +56,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   const uint32_t s_drain = s_qready + 8;
   const uint32_t s_slot = s_drain + 8;
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
-  uint8_t* g_q = gen + (s_q - base);
   volatile uint32_t* g_slot = reinterpret_cast<volatile uint32_t*>(gen + (s_slot - base));
   volatile int* s_abort = reinterpret_cast<volatile int*>(gen + (s_slot + 4 - base));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -96,8 +93,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     uint32_t ph_q = 0, full_phase = 1u;
     uint32_t n_s = 0, n_p = 0, n_pv = 0;  // score MMAs issued, stages handed over by the softmax threads, P.V issued
     int slot = -1;
-    bool issued = false, ok = true, s_ahead = false;  // s_ahead: this stage's scores were issued one stage early
-    // scores of the stage in `sl` into S buffer n_s & 1, once the softmax threads have emptied that buffer
+    bool issued = false, ok = true;
+    // scores of the stage in `sl` (S also holds the previous stage's P: the tensor pipe runs in order, so these
+    // MMAs start once the previous P.V has read it; the softmax threads have long read the previous scores)
     auto issue_scores = [&](int sl) {
       if (!warp_wait(s_sfree + 8 * (n_s & 1), ((n_s >> 1) & 1u) ^ 1u, s_abort)) return false;
       tc_fence_after_sync();
@@ -106,8 +104,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_ss(tmem + kTcColS + 64 * (n_s & 1), umma_smem_desc(s_q + h * (kTcRows * 128) + k * 32, 0, 1024),
+          for (int k = 0; k < 4; ++k)  // 16 dims of Q are 8 tensor-memory columns
+            umma_ts(tmem + kTcColS, tmem + kTcColQ + 8 * (4 * h + k),
                     umma_smem_desc(kst + h * L::kHalfBytes + k * 32, 0, 1024), idesc_s, (h | k) ? 1u : 0u);
         umma_commit(s_sready + 8 * (n_s & 1));
       }
@@ -126,29 +124,18 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
       const int4 meta = g_meta[2 * slot];
       if (meta.x < 0) break;
       const int ntok = meta.w & 0xffff;
-      const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+      const bool first = (meta.w >> 16) & 1;
       if (ntok > 0) {
-        if (!s_ahead) {
-          if (first) {
-            if (!warp_wait(s_qready, ph_q, s_abort)) {
-              ok = false;
-              break;
-            }
-            ph_q ^= 1u;
-          }
-          if (!issue_scores(slot)) {
+        if (first) {
+          if (!warp_wait(s_qready, ph_q, s_abort)) {
             ok = false;
             break;
           }
+          ph_q ^= 1u;
         }
-        s_ahead = false;
-        if (!last) {  // the next stage belongs to the same unit: its scores run while this stage's softmax does
-          const int ns = slot + 1 == nst ? 0 : slot + 1;
-          if (!warp_wait(s_full + 8 * ns, ns == 0 ? full_phase ^ 1u : full_phase, s_abort) || !issue_scores(ns)) {
-            ok = false;
-            break;
-          }
-          s_ahead = true;
+        if (!issue_scores(slot)) {
+          ok = false;
+          break;
         }
       }
       if (ntok == 0) {
@@ -173,9 +160,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         if (lane == 0) {
           const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes, vst = kst + L::kTileBytes;
 #pragma unroll
-          for (int k = 0; k < 4; ++k)  // P sits where K was; 16 tokens of V are 16 rows of 128 bytes in either half
-            umma_ss(tmem + kTcColO, umma_smem_desc(kst + k * 32, 0, 1024),
-                    umma_smem_desc(vst + k * 2048, L::kHalfBytes, 1024), idesc_o, (first && k == 0) ? 0u : 1u);
+          for (int k = 0; k < 4; ++k)  // 16 tokens: 8 columns of P, 16 rows of 128 bytes of V in either half
+            umma_ts(tmem + kTcColO, tmem + kTcColS + 8 * k, umma_smem_desc(vst + k * 2048, L::kHalfBytes, 1024), idesc_o,
+                    (first && k == 0) ? 0u : 1u);
           umma_commit(s_empty + 8 * slot);
           umma_commit(s_pvdone + 8 * (n_pv & 1));
         }
@@ -228,12 +215,20 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
           const uint4* src = reinterpret_cast<const uint4*>(
               p.q + (((size_t)b * p.Sq + (real_row ? qi : 0)) * p.Hq + (size_t)h * p.G + (real_row ? head : 0)) * D);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const uint4 v = real_row ? src[c] : make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(g_q + (size_t)(c >> 3) * (kTcRows * 128) + (size_t)row * 128 +
-                                      (((c & 7) ^ (row & 7)) << 4)) = v;
+          for (int half = 0; half < 2; ++half) {  // 64 dims = 32 columns of two bf16 each
+            uint32_t qw[32];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const uint4 v = real_row ? src[8 * half + c] : make_uint4(0u, 0u, 0u, 0u);
+              qw[4 * c] = v.x;
+              qw[4 * c + 1] = v.y;
+              qw[4 * c + 2] = v.z;
+              qw[4 * c + 3] = v.w;
+            }
+            tmem_st32(trow + kTcColQ + 32 * half, qw);
           }
-          fence_proxy_async_smem();
+          tmem_st_wait();
+          tc_fence_before_sync();
           mbar_arrive(s_qready);
         }
       }
@@ -247,11 +242,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         const uint32_t k_pv = n_pv++;  // this stage's P.V is number k_pv
         tc_fence_after_sync();
         uint32_t sr[2][32];
-        tmem_ld32(trow + kTcColS + 64 * (k_stage & 1), sr[0]);
-        tmem_ld32(trow + kTcColS + 64 * (k_stage & 1) + 32, sr[1]);
+        tmem_ld32(trow + kTcColS, sr[0]);
+        tmem_ld32(trow + kTcColS + 32, sr[1]);
         tmem_ld_wait();
         tc_fence_before_sync();
-        mbar_arrive(s_sfree + 8 * (k_stage & 1));  // the buffer may take the scores of the stage after next
+        mbar_arrive(s_sfree + 8 * (k_stage & 1));
         // tokens [0, e) of the stage are visible to this row
         const int e = min(min(meta2.z, lim_row) - meta2.x, ntok);
         if (e < kChunkStageTok) {
@@ -292,21 +287,19 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         }
         const float neg_mu = m_ref == -INFINITY ? 0.f : -m_ref;
         float add4[4] = {0.f, 0.f, 0.f, 0.f};
-        uint8_t* prow = stage_gen + (size_t)row * 128;  // P tile [128 rows][64 tokens] over the stage's K
+        uint32_t pw[32];  // this row of P: 64 weights, two bf16 per word, in token order
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          uint32_t w[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int j = 8 * c + 2 * i;
-            const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2e, neg_mu));
-            const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2e, neg_mu));
-            add4[i] += p0 + p1;
-            w[i] = pack_bf16x2(p0, p1);
-          }
-          *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int i = 0; i < 32; ++i) {
+          const int j = 2 * i;
+          const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2e, neg_mu));
+          const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2e, neg_mu));
+          add4[i & 3] += p0 + p1;
+          pw[i] = pack_bf16x2(p0, p1);
         }
         l_run += (add4[0] + add4[1]) + (add4[2] + add4[3]);
+        // over the first half of this row's scores (all of them are in registers by now)
+        tmem_st32(trow + kTcColS, pw);
+        tmem_st_wait();
         if (ntok < kChunkStageTok) {  // V rows beyond the stage's tokens may hold anything (NaN included): clear them
           uint8_t* vgen = stage_gen + L::kTileBytes;
           for (int idx = threadIdx.x; idx < (kChunkStageTok - ntok) * 16; idx += 128) {
@@ -314,8 +307,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
             *reinterpret_cast<uint4*>(vgen + (size_t)(c >> 3) * L::kHalfBytes + (size_t)r * 128 + ((c & 7) << 4)) =
                 make_uint4(0u, 0u, 0u, 0u);
           }
+          fence_proxy_async_smem();  // the cleared rows are read by the MMA through the async proxy
         }
-        fence_proxy_async_smem();  // P and the cleared rows are read by the MMA through the async proxy
         tc_fence_before_sync();
         __syncwarp();
       }
