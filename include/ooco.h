@@ -7,7 +7,7 @@
  * the append of the new token's K/V into the cache, plus the Roofline byte /
  * FLOP count a bottleneck-aware scheduler feeds its latency predictor with.
  * Around that core: the same operations over an 8-bit cache (*_fp8) and for
- * several query tokens per sequence (*_mq), the movement of cache blocks that a
+ * several query tokens per sequence, up to a prefill chunk (*_mq), the movement of cache blocks that a
  * request migration needs (ooco_kv_*_blocks), and a variant with built-in
  * scratch memory (ooco_decode_attention_static).  The host-side latency model
  * and scheduling decisions are declared in ooco_sched.h.

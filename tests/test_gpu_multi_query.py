@@ -205,6 +205,39 @@ def test_fused_step_mq():
     assert_parity(out.reshape(-1, 32, 128), ref.out.reshape(-1, 32, 128), what="fused mq step")
 
 
+@pytest.mark.parametrize("Sq,tc", [(5, 1), (40, 1), (40, 0)], ids=["20-columns", "160-columns-tcgen05", "160-columns-mma-sync"])
+def test_fused_step_prefill_chunk(Sq, tc):
+    """ooco_decode_step_mq with a chunk long enough for the prefill-chunk kernels: the fused append of q_len
+    tokens (bit-exact over the whole pool) is seen by the attention of the same call."""
+    cfg = C("ck-step", 32, 8, 128, 16, (G(6, 40, 1500),), seed=120, pool_fill=0.85)
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    sh = binding.shape_of(batch)
+    g = torch.Generator(device="cuda").manual_seed(9)
+    q = torch.randn((cfg.batch, Sq, 32, 128), generator=g, device="cuda").to(torch.bfloat16)
+    k_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    v_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    lens = batch.context_lens                                              # contexts INCLUDING the new tokens
+    positions = (lens - Sq).contiguous()
+    k_ref, v_ref = inputs.as_u16(batch.k_cache).copy(), inputs.as_u16(batch.v_cache).copy()
+    table = batch.block_table.cpu().numpy()
+    for i in range(Sq):
+        oracle.kv_append(inputs.as_u16(k_new[:, i].contiguous()), inputs.as_u16(v_new[:, i].contiguous()), k_ref, v_ref,
+                         table, (positions + i).cpu().numpy(), block_size=16, strides=batch.strides)
+    binding.set_tuning(chunk_tcgen05=tc)
+    try:
+        ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+        out = torch.full_like(q, float("nan"))
+        binding.decode_step_mq(sh, q, k_new, v_new, batch.k_cache, batch.v_cache, batch.block_table, positions, lens,
+                               cfg.scale, out, ws)
+        assert binding.workspace_status(ws) == 0 and binding.last_launch_count() == 3
+    finally:
+        binding.set_tuning(chunk_tcgen05=1)
+    assert np.array_equal(inputs.as_u16(batch.k_cache), k_ref) and np.array_equal(inputs.as_u16(batch.v_cache), v_ref)
+    ref = oracle.decode_attention_mq(inputs.as_u16(q), k_ref, v_ref, table, lens.cpu().numpy(), cfg.scale,
+                                     num_kv_heads=8, block_size=16, strides=batch.strides)
+    assert_parity(out.reshape(-1, 32, 128), ref.out.reshape(-1, 32, 128), what=f"fused chunk step Sq={Sq}")
+
+
 @pytest.mark.parametrize("cfg,Sq", [
     (C("mq8-edges", 32, 8, 128, 16, fixed(0, 1, 2, 3, 4, 15, 16, 17, 18, 63, 64, 65, 66, 127, 129, 300), seed=94,
        pool_fill=0.7, shuffle_batch=False), 4),
