@@ -124,3 +124,39 @@ def test_very_long_context_next_to_very_short_ones():
     for b, h in pairs:
         err = np.abs(got[b, h] - ref.out[b, h])
         assert err.max() <= 1e-2 and err.mean() <= 1e-3, (b, h, err.max())
+
+
+@pytest.mark.parametrize("Sq", [4, 64], ids=["16-columns", "256-columns"])
+def test_prefill_chunk_full_size_sampled_sequences(Sq):
+    """Several query tokens per sequence at benchmark size and launch shape (cfg1 with the chunk added to every
+    context): the 16-column row-layout kernel and the tcgen05 chunk kernel; whole sampled sequences against
+    the oracle, which gets a compacted host copy of just their blocks."""
+    base = inputs.CONFIGS["cfg1"]
+    cfg = inputs.replace(base, groups=tuple(inputs.replace(g, lo=g.lo + Sq, hi=g.hi + Sq) for g in base.groups))
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    B, Hq, D, bs = cfg.batch, cfg.num_q_heads, cfg.head_dim, cfg.block_size
+    gen = torch.Generator(device="cuda").manual_seed(77)
+    q = torch.randn((B, Sq, Hq, D), generator=gen, device="cuda").to(torch.bfloat16)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_attention_mq(sh, q, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens, cfg.scale,
+                                out, ws)
+    assert binding.workspace_status(ws) == 0
+    assert torch.isfinite(out.float()).all()
+    seqs = sample_sequences(batch.context_lens, n_each=1)
+    lens, table = batch.context_lens.cpu(), batch.block_table.cpu()
+    ids, rows = [], []
+    for b in seqs:
+        n = (int(lens[b]) + bs - 1) // bs
+        row = torch.zeros(table.shape[1], dtype=torch.int32)
+        row[:n] = torch.arange(len(ids), len(ids) + n, dtype=torch.int32)
+        ids.extend(table[b, :n].tolist())
+        rows.append(row)
+    idx = torch.tensor(ids, dtype=torch.long, device="cuda")
+    ref = oracle.decode_attention_mq(inputs.as_u16(q[seqs].contiguous()), inputs.as_u16(batch.k_cache.index_select(0, idx)),
+                                     inputs.as_u16(batch.v_cache.index_select(0, idx)), torch.stack(rows).numpy(),
+                                     lens[seqs].numpy(), cfg.scale, num_kv_heads=cfg.num_kv_heads, block_size=bs,
+                                     strides=batch.strides)
+    mx, mean = assert_parity(out[seqs].reshape(-1, Hq, D), ref.out.reshape(-1, Hq, D), what=f"cfg1 + chunk of {Sq}")
+    print(f"cfg1 with {Sq} query tokens, {len(seqs)} sampled sequences: max abs {mx:.3e} mean abs {mean:.3e}")
