@@ -661,9 +661,10 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (di.sm_count <= 0) return OOCO_E_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
-  // Launch shape: 4 consumer warps x 2 CTAs per SM; the 8-bit path wants 16 consumer warps per SM (it is
-  // latency-bound): 8 x 2; groups of more than 8 query heads need two MMA column tiles and too many
-  // registers for two CTAs of any shape: 8 x 1.  A knob set by the caller wins.
+  // Launch shape of the decode kernel: 4 consumer warps x 2 CTAs per SM; the 8-bit path wants 16 consumer
+  // warps per SM (it is latency-bound): 8 x 2; more than 8 score columns need two MMA column tiles and too
+  // many registers for two CTAs of any shape: 8 x 1 (bf16 caches leave the decode kernel there, see below).
+  // A knob set by the caller wins.
   const int G_ = s->num_q_heads / s->num_kv_heads * q_len;
   int ncw = g_knobs[kKnobWarps].load(), cps = g_knobs[kKnobCtasPerSm].load();
   if (!g_overridden[kKnobWarps].load() && (kv8 || G_ > 8)) ncw = 8;
