@@ -530,7 +530,9 @@ def run_multi_query(args, local_rank):
     peak, peak_kind = measured_peak()
     achieved = nbytes / (attn * 1e-3) / 1e9
     columns = Sq * (cfg.num_q_heads // cfg.num_kv_heads)
-    kernel = "chunk_main_kernel" if columns > 16 else ("row16_main_kernel" if columns > 8 else "decode_main_kernel")
+    tcgen05 = columns > 64 and cfg.head_dim == 128 and not any(k.startswith("chunk_tcgen05=0") for k in args.knob)
+    kernel = ("chunk_tc_kernel" if tcgen05 else "chunk_main_kernel") if columns > 16 else (
+        "row16_main_kernel" if columns > 8 else "decode_main_kernel")
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "kernel": kernel, "algorithmic_bytes_per_launch": nbytes,
                 "traffic": None}
@@ -541,7 +543,7 @@ def run_multi_query(args, local_rank):
         roofline = {"bound": "tensor", "achieved": tflops, "peak": tf_peak, "unit": "TFLOP/s", "frac": tflops / tf_peak,
                     "peak_kind": f"of {tf_kind} (bf16 GEMM burst)", "kernel": kernel,
                     "algorithmic_flops_per_launch": cost["flops"], "traffic": None,
-                    "note": "flops as the operator table prints them (no causal discount); mma.sync path"}
+                    "note": "flops as the operator table prints them (no causal discount)"}
     print(json.dumps({
         "metric": METRIC + f" ({Sq} query tokens per sequence)", "value": nbytes / (ms * 1e-3) / 1e12, "unit": "TB/s",
         "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
