@@ -256,7 +256,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains: the row is one thread's work
 #pragma unroll
-        for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sr[j >> 5][j & 31]));
+        for (int j = 0; j < 64; j += 2)  // three-input maximum: two scores per instruction
+          mx4[(j >> 1) & 3] = fmax3(mx4[(j >> 1) & 3], __uint_as_float(sr[j >> 5][j & 31]),
+                                    __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]));
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;  // the scale is positive
         // reference maximum: raised only when the row maximum is more than kTcRescaleStep above it
         const bool raise = m_ref != -INFINITY && mx > m_ref + kTcRescaleStep;
@@ -286,17 +288,22 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
           l_run *= alpha;
         }
         const float neg_mu = m_ref == -INFINITY ? 0.f : -m_ref;
-        float add4[4] = {0.f, 0.f, 0.f, 0.f};
+        float2 add4[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+        const float2 scale2 = make_float2(p.scale_log2e, p.scale_log2e), neg_mu2 = make_float2(neg_mu, neg_mu);
         uint32_t pw[32];  // this row of P: 64 weights, two bf16 per word, in token order
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
+        for (int i = 0; i < 32; ++i) {  // the scaling and the sums work on packed pairs: one instruction for two weights
           const int j = 2 * i;
-          const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2e, neg_mu));
-          const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2e, neg_mu));
-          add4[i & 3] += p0 + p1;
-          pw[i] = pack_bf16x2(p0, p1);
+          const float2 x = ffma2(make_float2(__uint_as_float(sr[j >> 5][j & 31]), __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31])),
+                                 scale2, neg_mu2);
+          const float2 w = make_float2(ex2(x.x), ex2(x.y));
+          add4[i & 3] = fadd2(add4[i & 3], w);
+          pw[i] = pack_bf16x2(w.x, w.y);
         }
-        l_run += (add4[0] + add4[1]) + (add4[2] + add4[3]);
+        {
+          const float2 a01 = fadd2(add4[0], add4[1]), a23 = fadd2(add4[2], add4[3]);
+          l_run += (a01.x + a01.y) + (a23.x + a23.y);
+        }
         // over the first half of this row's scores (all of them are in registers by now)
         tmem_st32(trow + kTcColS, pw);
         tmem_st_wait();
