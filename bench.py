@@ -530,7 +530,7 @@ def run_multi_query(args, local_rank):
     peak, peak_kind = measured_peak()
     achieved = nbytes / (attn * 1e-3) / 1e9
     columns = Sq * (cfg.num_q_heads // cfg.num_kv_heads)
-    tcgen05 = columns > 64 and cfg.head_dim == 128 and not any(k.startswith("chunk_tcgen05=0") for k in args.knob)
+    tcgen05 = columns > 32 and cfg.head_dim == 128 and not any(k.startswith("chunk_tcgen05=0") for k in args.knob)
     kernel = ("chunk_tc_kernel" if tcgen05 else "chunk_main_kernel") if columns > 16 else (
         "row16_main_kernel" if columns > 8 else "decode_main_kernel")
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

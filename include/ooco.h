@@ -190,7 +190,7 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  * read once); more columns run a prefill-chunk kernel, which cuts the columns into row tiles of
  * up to 128, reads the cache once per row tile (the repeats hit L2) and never loads tokens a tile
  * cannot see; it becomes bound by the tensor pipe from about 64 columns on.  At head_dim 128 and
- * more than 64 columns that kernel runs on tcgen05 (scores and output in tensor memory), otherwise
+ * more than 32 columns that kernel runs on tcgen05 (scores and output in tensor memory), otherwise
  * on mma.sync.  The 8-bit cache
  * (ooco_decode_step_mq_fp8) has the decode kernel only.  The workspace grows with q_len: one fp32
  * partial row per (split item, score column).  q_len = 1 is ooco_decode_attention /
@@ -431,7 +431,7 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * page-locked inputs through their device mapping and lets the kernels write a page-locked result
  * directly (zero = always one copy per buffer); 11 non-zero = 9 to 16 score columns per
  * (sequence, kv head) run the kernel whose warps share 16 score rows and split the tokens of a
- * stage (zero = the decode kernel with two 8-column tiles); 12 non-zero = more than 64 score columns
+ * stage (zero = the decode kernel with two 8-column tiles); 12 non-zero = more than 32 score columns
  * at head_dim 128 run the tcgen05 kernel (zero = the mma.sync kernel of the prefill-chunk path).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.

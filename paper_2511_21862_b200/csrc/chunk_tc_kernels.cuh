@@ -1,5 +1,5 @@
 // Prefill-chunk attention over the paged cache on the 5th-generation tensor cores (tcgen05), head_dim 128,
-// for 65 or more score columns per (sequence, kv head).  Same units of work, producer warp, stage layout and
+// for 33 or more score columns per (sequence, kv head).  Same units of work, producer warp, stage layout and
 // meta words as chunk_main_kernel (chunk_kernels.cuh); row tiles are 128 score rows = the MMA's M.
 //
 //   warp 4      producer: TMA K / V stages of 64 tokens ([half][64 tok][64 dims], 128-byte swizzle)

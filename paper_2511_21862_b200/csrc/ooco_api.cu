@@ -312,7 +312,8 @@ static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the chunk attention kernel", (long)e);
 }
 
-// Prefill chunk on tcgen05 (head_dim 128, more than 64 score columns): 128-row tiles, two CTAs per SM.
+// Prefill chunk on tcgen05 (head_dim 128, more than 32 score columns: from there on it beats the mma.sync
+// kernel on every workload measured, a half-empty 128-row tile included): two CTAs per SM.
 static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                            int ctas_per_sm, cudaStream_t st, int dev) {
   auto kern = chunk_tc_kernel;
@@ -680,7 +681,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // 9 .. 16 columns: the row layout with the tokens of a stage split over 4 warps x 2 CTAs per SM (the
   // column layout of the decode kernel needs a second MMA tile and a transposition per tile there)
   const bool row16 = !chunk && !kv8 && G_ > 8 && g_knobs[kKnobRowLayout16].load() != 0;
-  const bool chunk_tc = chunk && G_ > 64 && s->head_dim == 128 && g_knobs[kKnobChunkTcgen05].load() != 0;
+  const bool chunk_tc = chunk && G_ > 32 && s->head_dim == 128 && g_knobs[kKnobChunkTcgen05].load() != 0;
   if (chunk) {
     ncw = chunk_warps(G_);
     cps = (ncw == 8 && !chunk_tc) ? 1 : 2;

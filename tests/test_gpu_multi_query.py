@@ -90,7 +90,7 @@ def test_prefill_chunk_matches_oracle(cfg, Sq):
                                     ("ck-g4-sq33", "ck-g4-sq128-fresh", "ck-g8-sq64-bs64", "ck-split")],
                          ids=lambda v: getattr(v, "name", str(v)))
 def test_prefill_chunk_on_the_mma_sync_kernel(cfg, Sq):
-    """head_dim 128 with more than 64 score columns runs the tcgen05 kernel by default; the mma.sync kernel
+    """head_dim 128 with more than 32 score columns runs the tcgen05 kernel by default; the mma.sync kernel
     of the same shape stays selectable and must agree with the oracle too."""
     binding.set_tuning(chunk_tcgen05=0)
     try:
