@@ -6,9 +6,11 @@ batch: ooco_decode_step, i.e. the append of the new token's K/V fused into the p
 split-KV attention kernel and the LSE merge kernel (three launches).  Successive steps use different pool replicas (as successive layers of a
 model do), so the KV working set of the timed region is far larger than L2.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl ours|reference]
 
-Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs an independent replica of the
+Prints ONE JSON line.  The default workload is the largest long-context configuration (cfg4: 512 sequences of
+1 K to 16 K tokens over a fragmented pool, with the append); at N = 1 the other full-size workloads are timed
+in the same run and reported under `per_config`.  With N > 1 (under torchrun) every rank runs an independent replica of the
 workload (its own seed); there is no collective on the data path.
 """
 from __future__ import annotations
@@ -33,9 +35,6 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 METRIC = "paged decode-attn achieved HBM TB/s"
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one attention-kernel launch, from the
-# ncu capture summarised in profiles/ (null for workloads without a capture).
-NCU_TRAFFIC_BYTES = {"cfg1": 579_344_768 + 7_974_016}   # mean of the two launches in profiles/decode_main_kernel_cfg1_ncu_full.md
 
 
 def measured_peak():
@@ -141,33 +140,41 @@ def replica_count(pool_bytes: int, free_bytes: int) -> int:
     return max(1, min(want, fit, 16))
 
 
+def sample_bytes_of(cfg, tokens: int, nseq: int) -> int:
+    """Model bytes (operator table, d = 2) of `nseq` whole sequences holding `tokens` cached tokens."""
+    return tokens * 2 * 2 * cfg.num_kv_heads * cfg.head_dim + 2 * 2 * nseq * cfg.num_q_heads * cfg.head_dim
+
+
 def run_reference(args, rank, world):
-    """The oracle as it stands, on the host cores, on a bounded sample of the workload per step."""
+    """The oracle as it stands, on the host cores, on a bounded sample of the workload per step.
+
+    Only the sampled sequences' blocks are synthesised on the host (lengths and block-table rows are the
+    full workload's own draws), so the largest workloads need no 20 GB host pool."""
     if rank != 0:
         return
     import numpy as np
     import oracle
     cfg = inputs.CONFIGS[args.workload]
-    batch = inputs.make_batch(cfg, "cpu", poison=False)
-    lens = batch.context_lens.numpy()
+    lens_all = inputs.draw_layout(cfg).lens.numpy()
     # sample: whole sequences, shortest first, up to ~budget tokens * heads per step
     budget = args.ref_token_heads
-    order = np.argsort(lens, kind="stable")
+    order = np.argsort(lens_all, kind="stable")
     chosen, acc = [], 0
     for b in order:
-        cost = int(lens[b]) * cfg.num_q_heads
+        cost = int(lens_all[b]) * cfg.num_q_heads
         if chosen and acc + cost > budget:
             break
         chosen.append(int(b)); acc += cost
-    pairs = np.array([(b, h) for b in chosen for h in range(cfg.num_q_heads)], dtype=np.int32)
-    tok = int(sum(int(lens[b]) for b in chosen))
-    sample_bytes = tok * 2 * 2 * cfg.num_kv_heads * cfg.head_dim + 2 * 2 * len(chosen) * cfg.num_q_heads * cfg.head_dim
+    batch = inputs.make_sample_batch(cfg, chosen, "cpu")
+    lens = batch.context_lens.numpy()
+    tok = int(lens.sum())
+    sample_bytes = sample_bytes_of(cfg, tok, len(chosen))
     q, k, v = inputs.as_u16(batch.q), inputs.as_u16(batch.k_cache), inputs.as_u16(batch.v_cache)
     table = batch.block_table.numpy()
 
     def step():
         oracle.decode_attention(q, k, v, table, lens, cfg.scale, num_kv_heads=cfg.num_kv_heads,
-                                block_size=cfg.block_size, strides=batch.strides, pairs=pairs)
+                                block_size=cfg.block_size, strides=batch.strides)
     for _ in range(args.warmup):
         step()
     t0 = time.perf_counter()
@@ -176,7 +183,8 @@ def run_reference(args, rank, world):
     dt = time.perf_counter() - t0
     ms = dt / args.steps * 1e3
     val = sample_bytes / (ms * 1e-3) / 1e12
-    sample = f"{len(chosen)} shortest sequences of {cfg.name} ({tok} tokens, all {cfg.num_q_heads} q heads) per step"
+    sample = (f"{len(chosen)} shortest of the {len(lens_all)} sequences of {cfg.name} ({tok} tokens, all "
+              f"{cfg.num_q_heads} q heads) per step")
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": "TB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
@@ -191,63 +199,98 @@ def run_reference(args, rank, world):
     print(json.dumps(line))
 
 
-def cpu_baseline(cfg, batch_host_fn, budget_s=15.0):
-    """Oracle timed on the host cores on a bounded sample of the same workload (rank 0, N = 1)."""
+def cpu_baseline(cfg, batch, budget_s=12.0, max_sample_bytes=4 << 30):
+    """Oracle timed on the host cores on a bounded sample of the same workload (rank 0, N = 1): whole
+    sequences, longest first, at most `max_sample_bytes` of K + V, repeated for about `budget_s`.  The
+    sample's blocks are compacted on the device and copied to the host; the oracle call is the stock one."""
     import numpy as np
     import oracle
-    hb = batch_host_fn()
-    lens = hb["lens"]
-    order = np.argsort(lens, kind="stable")
-    per_unit = None
-    # calibrate on the shortest sequence, then take whole sequences up to ~budget_s of CPU work
-    def run(seqs):
-        pairs = np.array([(b, h) for b in seqs for h in range(cfg.num_q_heads)], dtype=np.int32)
-        t0 = time.perf_counter()
-        oracle.decode_attention(hb["q"], hb["k"], hb["v"], hb["table"], lens, cfg.scale,
-                                num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size,
-                                strides=hb["strides"], pairs=pairs)
-        return time.perf_counter() - t0
-    first = [int(order[len(order) // 2])]
-    t_cal = run(first)
-    per_unit = t_cal / max(1, int(lens[first[0]]))
-    chosen, acc = [], 0.0
-    for b in order[::-1]:                                   # longest first: fewest partial sequences
-        est = per_unit * int(lens[b])
-        if chosen and acc + est > budget_s:
+    lens = batch.context_lens.cpu().numpy()
+    table = batch.block_table.cpu()
+    bs = cfg.block_size
+    per_token = 2 * 2 * cfg.num_kv_heads * cfg.head_dim
+    order = np.argsort(lens, kind="stable")[::-1]
+    chosen, acc = [], 0
+    for b in order:
+        need = int(lens[b]) * per_token
+        if chosen and acc + need > max_sample_bytes:
             continue
-        chosen.append(int(b)); acc += est
-        if acc > budget_s:
-            break
-    dt = run(chosen)
-    reps = 1
-    while dt * reps < 3.0 and reps < 64:                   # short workloads: repeat for a stable figure
-        reps *= 2
-    if reps > 1:
+        chosen.append(int(b)); acc += need
+    chosen.sort()
+    ids, rows = [], []
+    for b in chosen:
+        n = (int(lens[b]) + bs - 1) // bs
+        row = torch.zeros(table.shape[1], dtype=torch.int32)
+        row[:n] = torch.arange(len(ids), len(ids) + n, dtype=torch.int32)
+        ids.extend(table[b, :n].tolist())
+        rows.append(row)
+    idx = torch.tensor(ids if ids else [0], dtype=torch.long, device=batch.k_cache.device)
+    k = inputs.as_u16(batch.k_cache.index_select(0, idx))
+    v = inputs.as_u16(batch.v_cache.index_select(0, idx))
+    q = inputs.as_u16(batch.q[chosen].contiguous())
+    tab, ln = torch.stack(rows).numpy(), lens[chosen].astype(np.int32)
+
+    def run():
+        t0 = time.perf_counter()
+        oracle.decode_attention(q, k, v, tab, ln, cfg.scale, num_kv_heads=cfg.num_kv_heads, block_size=bs,
+                                strides=batch.strides)
+        return time.perf_counter() - t0
+    dt = run()
+    reps = int(max(1, min(256, round(budget_s / max(dt, 1e-4)) - 1)))
+    if reps > 1 or dt < 1.0:
         t0 = time.perf_counter()
         for _ in range(reps):
-            run(chosen)
+            run()
         dt = (time.perf_counter() - t0) / reps
-    tok = int(sum(int(lens[b]) for b in chosen))
-    nbytes = tok * 2 * 2 * cfg.num_kv_heads * cfg.head_dim + 2 * 2 * len(chosen) * cfg.num_q_heads * cfg.head_dim
-    return {"value": nbytes / dt / 1e12, "unit": "TB/s", "cores": oracle.num_threads(), "kind": "oracle",
+    tok = int(ln.sum())
+    return {"value": sample_bytes_of(cfg, tok, len(chosen)) / dt / 1e12, "unit": "TB/s", "cores": oracle.num_threads(),
+            "kind": "oracle",
             "sample": f"{len(chosen)} of {len(lens)} sequences of {cfg.name} ({tok} of {int(lens.sum())} tokens, "
                       f"all q heads), {dt:.2f} s per pass x {reps}",
             "decode_tokens_per_s": len(chosen) / dt}
 
 
-def run_ours(args, rank, local_rank, world):
-    from paper_2511_21862_b200 import binding, build
-    build.build()
-    binding.lib()
-    for kv in args.knob:
-        name, val = kv.split("=")
-        binding.set_tuning(**{name: int(val)})
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+def kernel_source_digest() -> str:
+    """Digest of the sources the attention kernel is compiled from (ncu counters taken on another
+    version of them are not reported)."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("decode_kernels.cuh", "ptx.cuh"):
+        with open(os.path.join(ROOT, "paper_2511_21862_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload: str, algorithmic_bytes: int):
+    """(DRAM bytes read + written per launch of the attention kernel, how it was obtained) from the ncu
+    figures recorded in profiles/decode_main_kernel_dram_traffic.txt, or (None, why).
+
+    A workload with a capture of its own reports it; the others are scaled from the capture the file
+    marks `scale_from`, by algorithmic bytes (traffic grows in proportion to the tokens read).  Lines:
+    `source <digest>`, `capture <name> <dram bytes> <algorithmic bytes>`, `scale_from <name>`."""
+    path = os.path.join(ROOT, "profiles", "decode_main_kernel_dram_traffic.txt")
+    try:
+        rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    except OSError:
+        return None, "no capture recorded"
+    digest = next((r[1] for r in rows if r[0] == "source"), None)
+    if digest != kernel_source_digest():
+        return None, "kernel sources changed since the capture"
+    caps = {r[1]: (int(r[2]), int(r[3])) for r in rows if r[0] == "capture"}
+    if workload in caps:
+        return caps[workload][0], f"ncu capture of {workload}"
+    base = next((r[1] for r in rows if r[0] == "scale_from"), None)
+    if base in caps:
+        return int(round(caps[base][0] / caps[base][1] * algorithmic_bytes)), f"scaled from the ncu capture of {base}"
+    return None, "no capture recorded"
+
+
+def measure_workload(args, cfg, dev, rank, world, *, e2e=True, baseline=False):
+    """Times one workload: K steps device-resident (value), the same K steps with events between the
+    kernels (kernel_ms), and the host-buffer step (e2e).  Returns a dict of local (this rank's) figures."""
+    from paper_2511_21862_b200 import binding
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    cfg = inputs.replace(inputs.CONFIGS[args.workload], seed=inputs.CONFIGS[args.workload].seed + 100 * rank)
     batch = inputs.make_batch(cfg, dev, poison=False)
     fp8 = args.kv == "fp8"
     K_SCALE, V_SCALE = 1.0 / 32, 1.0 / 32                                 # N(0, sigma) values sit well inside +-448
@@ -256,9 +299,10 @@ def run_ours(args, rank, local_rank, world):
     sh = binding.shape_of(batch)
     B = sh.batch
     lens_host = batch.context_lens.cpu().contiguous()
-    cost = binding.decode_bytes_model(sh, lens_host)
+    lens1_host = (lens_host + 1).contiguous()                             # the step attends T_b + 1 tokens
+    cost = binding.decode_bytes_model(sh, lens1_host)
     if fp8:                                                               # K / V stored with d = 1, q / out with d = 2
-        cost = dict(cost, bytes_kv=binding.decode_bytes_model(sh, lens_host, 1)["bytes_kv"])
+        cost = dict(cost, bytes_kv=binding.decode_bytes_model(sh, lens1_host, 1)["bytes_kv"])
         cost["bytes_paper"] = cost["bytes_q"] + cost["bytes_out"] + cost["bytes_kv"]
     kv_b = 1 if fp8 else 2
     append_bytes = 2 * B * cfg.num_kv_heads * cfg.head_dim * (2 + kv_b)   # K and V rows: bf16 read, cache written
@@ -266,7 +310,7 @@ def run_ours(args, rank, local_rank, world):
 
     pool_bytes = 2 * batch.k_cache.numel() * batch.k_cache.element_size()
     free, _ = torch.cuda.mem_get_info(dev)
-    R = replica_count(pool_bytes, free)
+    R = args.replicas if args.replicas > 0 else replica_count(pool_bytes, free)
     pools = [(batch.k_cache, batch.v_cache)] + [(batch.k_cache.clone(), batch.v_cache.clone()) for _ in range(R - 1)]
     ws = torch.empty(binding.workspace_bytes(sh), dtype=torch.uint8, device=dev)
     out = torch.empty_like(batch.q)
@@ -283,14 +327,13 @@ def run_ours(args, rank, local_rank, world):
             binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, k, v, batch.block_table, positions, lens1,
                                 cfg.scale, out, ws, stream)
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev.index)
     sampler.start()
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
     assert binding.workspace_status(ws) == 0
     if world > 1:
-        import torch.distributed as dist
         dist.barrier()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -316,73 +359,128 @@ def run_ours(args, rank, local_rank, world):
         step(i)
     recs = binding.profile_read(args.steps)
     binding.profile_enable(0)
+    res = {"cfg": cfg, "B": B, "cost": cost, "step_bytes": step_bytes, "ms": ms_local, "recs": recs, "clocks": clocks,
+           "R": R, "pool_bytes": pool_bytes, "launches_per_step": launches_per_step, "e2e_ms": None}
 
     # ---- end to end through the host-buffer entry point (pinned inputs in, result out, every step)
-    if fp8:
-        return finish_fp8(args, world, cfg, B, cost, step_bytes, ms_local, recs, clocks, R, pool_bytes, sampler)
-    pin = lambda t: t.cpu().contiguous().pin_memory()
-    hq, hk, hv, ht = pin(batch.q), pin(batch.k_new), pin(batch.v_new), pin(batch.block_table)
-    hp, hl = pin(positions), pin(lens1)
-    hout = torch.empty(batch.q.shape, dtype=torch.bfloat16).pin_memory()
-    stg = torch.empty(binding.step_staging_bytes(sh), dtype=torch.uint8, device=dev)
-    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, ht, hp, hl))
-    d2h = hout.numel() * hout.element_size()
-    e2e_steps = max(3, min(args.steps, 200))
+    if e2e and not fp8:
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        hq, hk, hv, ht = pin(batch.q), pin(batch.k_new), pin(batch.v_new), pin(batch.block_table)
+        hp, hl = pin(positions), pin(lens1)
+        hout = torch.empty(batch.q.shape, dtype=torch.bfloat16).pin_memory()
+        stg = torch.empty(binding.step_staging_bytes(sh), dtype=torch.uint8, device=dev)
+        res["h2d"] = sum(t.numel() * t.element_size() for t in (hq, hk, hv, ht, hp, hl))
+        res["d2h"] = hout.numel() * hout.element_size()
+        e2e_steps = max(3, min(args.steps, 200))
 
-    def e2e_step(i):
-        k, v = pools[i % R]
-        binding.decode_step_host(sh, hq, hk, hv, ht, hp, hl, k, v, cfg.scale, hout, stg, ws, stream)
-    for i in range(3):
-        e2e_step(i)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for i in range(e2e_steps):
-        e2e_step(i)
-    torch.cuda.synchronize()
-    e2e_ms_local = (time.perf_counter() - t0) / e2e_steps * 1e3
+        def e2e_step(i):
+            k, v = pools[i % R]
+            binding.decode_step_host(sh, hq, hk, hv, ht, hp, hl, k, v, cfg.scale, hout, stg, ws, stream)
+        for i in range(3):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        res["e2e_ms"] = (time.perf_counter() - t0) / e2e_steps * 1e3
+        res["e2e_steps"] = e2e_steps
     sampler.stop()
+    if baseline:
+        res["cpu_baseline"] = cpu_baseline(cfg, batch, args.cpu_seconds)
+    return res
 
-    ms, total_bytes = aggregate(world, ms_local, float(step_bytes))
-    e2e_ms, _ = aggregate(world, e2e_ms_local, 0.0)
-    _, total_seqs = aggregate(world, 0.0, float(B))
-    if rank != 0:
-        return
-    value = total_bytes / (ms * 1e-3) / 1e12
-    peak, peak_kind = measured_peak()
-    attn_ms = sorted(r[1] for r in recs)
+
+def roofline_of(res, peak, peak_kind):
+    cost = res["cost"]
+    attn_ms = sorted(r[1] for r in res["recs"])
     attn_avg = sum(attn_ms) / len(attn_ms)
     kernel_bytes = cost["bytes_kv"] + cost["bytes_q"] + cost["bytes_out"]
     achieved = kernel_bytes / (attn_avg * 1e-3) / 1e9
+    traffic, how = ncu_traffic(res["cfg"].name, kernel_bytes) if res["cfg"].name in inputs.CONFIGS else (None, "no capture recorded")
+    kernel_ms = {"plan": sum(r[0] for r in res["recs"]) / len(res["recs"]), "attention": attn_avg,
+                 "attention_median": attn_ms[len(attn_ms) // 2], "merge": sum(r[2] for r in res["recs"]) / len(res["recs"])}
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbps": achieved / NOMINAL_HBM_GBS,
+            "kernel": "decode_main_kernel", "algorithmic_bytes_per_launch": kernel_bytes,
+            "traffic": traffic, "traffic_source": how}
+    return kernel_ms, roof
+
+
+def run_ours(args, rank, local_rank, world):
+    from paper_2511_21862_b200 import binding, build
+    build.build()
+    binding.lib()
+    for kv in args.knob:
+        name, val = kv.split("=")
+        binding.set_tuning(**{name: int(val)})
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = inputs.replace(inputs.CONFIGS[args.workload], seed=inputs.CONFIGS[args.workload].seed + 100 * rank)
+    fp8 = args.kv == "fp8"
+    res = measure_workload(args, cfg, dev, rank, world, e2e=True,
+                           baseline=world == 1 and not args.no_cpu_baseline and not fp8)
+    if fp8:
+        return finish_fp8(args, world, cfg, res["B"], res["cost"], res["step_bytes"], res["ms"], res["recs"],
+                          res["clocks"], res["R"], res["pool_bytes"])
+    B, cost, step_bytes, R, pool_bytes = res["B"], res["cost"], res["step_bytes"], res["R"], res["pool_bytes"]
+    ms, total_bytes = aggregate(world, res["ms"], float(step_bytes))
+    e2e_ms, _ = aggregate(world, res["e2e_ms"], 0.0)
+    _, total_seqs = aggregate(world, 0.0, float(B))
+    # the other full-size workloads, timed the same way in the same run (N = 1 only)
+    per_config = {}
+    peak, peak_kind = measured_peak()
+    if world == 1 and not args.no_per_config:
+        torch.cuda.empty_cache()
+        for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+            if name == args.workload:
+                continue
+            torch.cuda.empty_cache()
+            sub = argparse.Namespace(**vars(args))
+            sub.steps = args.steps if name in ("cfg2", "cfg4") else 5 * args.steps   # short steps: a longer timed region
+            r = measure_workload(sub, inputs.CONFIGS[name], dev, rank, world, e2e=True, baseline=False)
+            km, roof = roofline_of(r, peak, peak_kind)
+            v = r["step_bytes"] / (r["ms"] * 1e-3) / 1e12
+            per_config[name] = {
+                "step_TBps": v, "ms_per_step": r["ms"], "steps": sub.steps, "pct_of_nominal_8tbps": 100.0 * v * 1e3 / NOMINAL_HBM_GBS,
+                "pct_of_measured_copy": 100.0 * v * 1e3 / peak, "kernel_ms": km,
+                "kernel_GBps": roof["achieved"], "kernel_frac_of_measured": roof["frac"],
+                "kernel_frac_of_nominal_8tbps": roof["frac_of_nominal_8tbps"], "traffic": roof["traffic"],
+                "traffic_source": roof["traffic_source"], "e2e_ms_per_step": r["e2e_ms"],
+                "total_tokens": r["cost"]["total_tokens"], "batch": r["B"], "pool_replicas": r["R"], "clocks": r["clocks"]}
+    if rank != 0:
+        return
+    value = total_bytes / (ms * 1e-3) / 1e12
+    kernel_ms, roof = roofline_of(res, peak, peak_kind)
     line = {
         "metric": METRIC, "value": value, "unit": "TB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "description": cfg.description, "batch": B,
                    "total_tokens": cost["total_tokens"], "step": "ooco_decode_step: fused kv append + plan, split-KV attention, LSE merge; one layer",
-                   "l2": f"inputs larger than L2: steps rotate over {R} pool replicas ({R * pool_bytes / 2**30:.2f} GiB)",
+                   "l2": f"inputs larger than L2: steps rotate over {R} pool replica(s) ({R * pool_bytes / 2**30:.2f} GiB), "
+                         f"{cost['bytes_kv'] / 2**30:.2f} GiB of K + V read per step",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "pct_of_nominal_8tbps": 100.0 * value * 1e3 / (NOMINAL_HBM_GBS * world),
         "pct_of_measured_copy": 100.0 * value * 1e3 / (peak * world),
         "decode_tokens_per_s": total_seqs / (ms * 1e-3),
         "step_bytes": step_bytes,
-        "kernel_ms": {"plan": sum(r[0] for r in recs) / len(recs), "attention": attn_avg,
-                      "attention_median": attn_ms[len(attn_ms) // 2], "merge": sum(r[2] for r in recs) / len(recs)},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbps": achieved / NOMINAL_HBM_GBS,
-                     "kernel": "decode_main_kernel", "algorithmic_bytes_per_launch": kernel_bytes,
-                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
-        "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e12, "unit": "TB/s", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
-        "gpu_launches": args.steps * launches_per_step,
-        "clocks": clocks,
+        "kernel_ms": kernel_ms,
+        "roofline": roof,
+        "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e12, "unit": "TB/s", "h2d_bytes_per_step": res["h2d"],
+                "d2h_bytes_per_step": res["d2h"], "ms_per_step": e2e_ms, "steps": res["e2e_steps"]},
+        "gpu_launches": args.steps * res["launches_per_step"],
+        "clocks": res["clocks"],
     }
-    if world == 1 and not args.no_cpu_baseline:
-        def host_batch():
-            return {"q": inputs.as_u16(batch.q), "k": inputs.as_u16(batch.k_cache), "v": inputs.as_u16(batch.v_cache),
-                    "table": batch.block_table.cpu().numpy(), "lens": lens_host.numpy(), "strides": batch.strides}
-        line["cpu_baseline"] = cpu_baseline(cfg, host_batch, args.cpu_seconds)
+    if per_config:
+        line["per_config"] = per_config
+    if "cpu_baseline" in res:
+        line["cpu_baseline"] = res["cpu_baseline"]
     print(json.dumps(line))
 
 
@@ -839,9 +937,8 @@ def run_model_fit(args, local_rank):
     print(json.dumps(line))
 
 
-def finish_fp8(args, world, cfg, B, cost, step_bytes, ms, recs, clocks, R, pool_bytes, sampler):
+def finish_fp8(args, world, cfg, B, cost, step_bytes, ms, recs, clocks, R, pool_bytes):
     """JSON line of the 8-bit-cache variant (single GPU; device-resident inputs only)."""
-    sampler.stop()
     peak, peak_kind = measured_peak()
     attn = sorted(r[1] for r in recs)
     attn_avg = sum(attn) / len(attn)
@@ -870,11 +967,13 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--workload", default="cfg4", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="time only --workload, not the other full-size workloads")
+    ap.add_argument("--replicas", type=int, default=0, help="pool replicas the steps rotate over (0: enough for 4 GiB)")
     ap.add_argument("--knob", action="append", default=[], help="launch-shape override name=value (sweeps)")
-    ap.add_argument("--cpu-seconds", type=float, default=15.0)
-    ap.add_argument("--ref-token-heads", type=int, default=400000,
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--ref-token-heads", type=int, default=4_000_000,
                     help="reference arm: (tokens x q heads) of oracle work per step")
     ap.add_argument("--op", default="decode_step", choices=["decode_step", "kv_migrate", "model_fit", "decode_mq", "serve_loop"],
                     help="decode_step: the decode hot path (default); kv_migrate: paged block gather + scatter; "

@@ -21,8 +21,14 @@
  *     stream).  All device work is enqueued on it; no entry point synchronises
  *     with the host unless its comment says so.
  *   - Return value: OOCO_OK (0) or a negative OOCO_E_* code.  Argument
- *     validation happens on the host before anything is launched; a call that
- *     returns an error has enqueued nothing.
+ *     validation (pointers, shape, sizes, alignment, the fit of the chosen
+ *     kernel's shared memory) happens on the host before anything is enqueued:
+ *     a call that returns OOCO_E_NULLPTR, _SHAPE, _UNSUPPORTED or _WORKSPACE
+ *     has enqueued nothing and touched no buffer.  OOCO_E_CUDA reports a
+ *     failing CUDA call or launch; launches of the same call that preceded it
+ *     (the plan, a fused append) may already be enqueued.
+ *   - `scale` (the softmax scale) must be positive and finite (OOCO_E_SHAPE
+ *     otherwise).
  */
 #ifndef OOCO_H_
 #define OOCO_H_
@@ -272,11 +278,16 @@ int ooco_decode_step_mq_fp8(const ooco_shape_t* shape, int32_t q_len, const void
  *   - A shape whose ooco_decode_workspace_bytes exceeds OOCO_STATIC_SCRATCH_BYTES is refused
  *     with OOCO_E_WORKSPACE before anything is launched, and ooco_last_error_detail names
  *     both sizes.  The exact test is ooco_decode_workspace_bytes(shape) <=
- *     OOCO_STATIC_SCRATCH_BYTES; with head_dim 128 and block tables of up to 8 K tokens that
- *     admits about 300 sequences of 32 q / 8 kv heads (64 sequences need 8.2 MiB) and about
- *     50 sequences of 64 q / 8 kv heads.
+ *     OOCO_STATIC_SCRATCH_BYTES; with the default tuning, head_dim 128 and block tables of up
+ *     to 8 K tokens that admits about 500 sequences of 32 q / 8 kv heads and about 50 of
+ *     64 q / 8 kv heads.  The bound moves with ooco_set_tuning knobs 4 and 5, which change
+ *     ooco_decode_workspace_bytes.
  *   - The first call on each device looks up the array's device address (that device must be
- *     current, as for every call); make that first call outside any stream capture.
+ *     current, as for every call); make that first call outside any stream capture.  With
+ *     CUDA's lazy module loading that first call is also when the device receives the
+ *     library's code and the array itself: "allocates nothing" holds from the second call on,
+ *     so make one warm-up call per device BEFORE handing the rest of the device's memory to a
+ *     pool; a first call on a device that is already full can fail with OOCO_E_CUDA.
  *   - All calls on a device share the one array: two calls that may overlap on the GPU (other
  *     streams, other host threads) race on it and corrupt each other's results.  Calls on one
  *     stream are ordered and safe.  The array keeps the previous call's contents; nothing in
@@ -439,8 +450,10 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
 int ooco_set_tuning(int knob, int value);
 
 /*
- * Text naming the CUDA call that made the last OOCO_E_CUDA on this thread fail, with its
- * error code ("" if none yet).  The pointer stays valid for the thread's lifetime.
+ * Text about the last OOCO_E_CUDA or OOCO_E_WORKSPACE on this thread ("" if none yet): the CUDA
+ * call that failed with its error code, or, from ooco_decode_attention_static, the scratch size
+ * the shape needs next to the size of the built-in array.  The pointer stays valid for the
+ * thread's lifetime.
  */
 const char* ooco_last_error_detail(void);
 

@@ -991,7 +991,6 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, co
   // the wait below; only the partial results need the attention grid to be complete.
   int first = 0, n = 0;
   grid_dep_launch();  // a programmatically launched successor may start its own prologue
-  if (p.hdr->status & kStatusPlanOverflow) return;  // no work list, no partials (status is reported)
   {
     const int u = blockIdx.x * units_per_block + (warp >> wpu_log2);
     if (u < n_units) {
@@ -999,7 +998,10 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, co
       n = p.seq_first[u / per_seq + 1] - first;
     }
   }
+  // (also on the overflow path: this grid's completion must imply the attention grid's, because the next
+  // call's first kernel waits on this grid only before it rewrites the workspace and the cache)
   grid_dep_wait();
+  if (p.hdr->status & kStatusPlanOverflow) return;  // no work list, no partials (status is reported)
   for (int ub = blockIdx.x * units_per_block; ub < n_units; ub += gridDim.x * units_per_block, first = -1) {
     const int u = ub + (warp >> wpu_log2);
     const bool live = u < n_units;

@@ -207,7 +207,7 @@ static cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size
 
 template <int D, int NCW, int NT, int TPW, bool KV8 = false>
 static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
-                       int ctas_per_sm, int want_stages, cudaStream_t st, int dev) {
+                       int ctas_per_sm, int want_stages, cudaStream_t st, int dev, bool dry) {
   using L = SmemLayout<D, NCW, NT, TPW, KV8>;
   auto kern = decode_main_kernel<D, NCW, NT, TPW, KV8>;
   // the opt-in limit covers static + dynamic shared memory of the kernel
@@ -233,6 +233,7 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
     if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
+  if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
   cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + 1) * 32), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
@@ -241,48 +242,48 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
 
 template <int D, int NCW, int TPW>
 static int launch_main_nt(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
-                          int cps, int stages, cudaStream_t st, int dev) {
-  if (p.GQ <= 8) return launch_main<D, NCW, 1, TPW>(tk, tv, p, di, cps, stages, st, dev);
-  return launch_main<D, NCW, 2, TPW>(tk, tv, p, di, cps, stages, st, dev);
+                          int cps, int stages, cudaStream_t st, int dev, bool dry) {
+  if (p.GQ <= 8) return launch_main<D, NCW, 1, TPW>(tk, tv, p, di, cps, stages, st, dev, dry);
+  return launch_main<D, NCW, 2, TPW>(tk, tv, p, di, cps, stages, st, dev, dry);
 }
 
 // 8-bit cache: head_dim 128, one tile per warp.
 static int launch_main_kv8(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
-                           const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev) {
+                           const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev, bool dry) {
   const bool wide = p.GQ > 8;
   switch (ncw) {
     case 2:
-      return wide ? launch_main<128, 2, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev)
-                  : launch_main<128, 2, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev);
+      return wide ? launch_main<128, 2, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry)
+                  : launch_main<128, 2, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry);
     case 8:
-      return wide ? launch_main<128, 8, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev)
-                  : launch_main<128, 8, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev);
+      return wide ? launch_main<128, 8, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry)
+                  : launch_main<128, 8, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry);
     default:
-      return wide ? launch_main<128, 4, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev)
-                  : launch_main<128, 4, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev);
+      return wide ? launch_main<128, 4, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry)
+                  : launch_main<128, 4, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry);
   }
 }
 
 template <int D>
 static int launch_main_ncw(int ncw, int tpw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
-                           const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev) {
+                           const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev, bool dry) {
   if (tpw == 2) {
     switch (ncw) {
-      case 2: return launch_main_nt<D, 2, 2>(tk, tv, p, di, cps, stages, st, dev);
-      default: return launch_main_nt<D, 4, 2>(tk, tv, p, di, cps, stages, st, dev);
+      case 2: return launch_main_nt<D, 2, 2>(tk, tv, p, di, cps, stages, st, dev, dry);
+      default: return launch_main_nt<D, 4, 2>(tk, tv, p, di, cps, stages, st, dev, dry);
     }
   }
   switch (ncw) {
-    case 2: return launch_main_nt<D, 2, 1>(tk, tv, p, di, cps, stages, st, dev);
-    case 8: return launch_main_nt<D, 8, 1>(tk, tv, p, di, cps, stages, st, dev);
-    default: return launch_main_nt<D, 4, 1>(tk, tv, p, di, cps, stages, st, dev);
+    case 2: return launch_main_nt<D, 2, 1>(tk, tv, p, di, cps, stages, st, dev, dry);
+    case 8: return launch_main_nt<D, 8, 1>(tk, tv, p, di, cps, stages, st, dev, dry);
+    default: return launch_main_nt<D, 4, 1>(tk, tv, p, di, cps, stages, st, dev, dry);
   }
 }
 
 // Prefill-chunk kernel: as many 64-token stages as the CTA's share of shared memory holds (at most 8).
 template <int D, int NCW>
 static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
-                        int ctas_per_sm, cudaStream_t st, int dev) {
+                        int ctas_per_sm, cudaStream_t st, int dev, bool dry) {
   using L = ChunkSmem<D>;
   auto kern = chunk_main_kernel<D, NCW>;
   static std::atomic<int> static_smem{-1};
@@ -306,6 +307,7 @@ static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
     if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
+  if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
   cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + 1) * 32), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
@@ -315,7 +317,7 @@ static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
 // Prefill chunk on tcgen05 (head_dim 128, more than 32 score columns: from there on it beats the mma.sync
 // kernel on every workload measured, a half-empty 128-row tile included): two CTAs per SM.
 static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
-                           int ctas_per_sm, cudaStream_t st, int dev) {
+                           int ctas_per_sm, cudaStream_t st, int dev, bool dry) {
   auto kern = chunk_tc_kernel;
   static std::atomic<int> static_smem{-1};
   if (static_smem.load() < 0) {
@@ -338,6 +340,7 @@ static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeP
     if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
+  if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
   cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(192), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
@@ -347,7 +350,7 @@ static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeP
 // 9 .. 16 score columns: the warps of a CTA share one 16-row tile and split the tokens of a stage.
 template <int D>
 static int launch_row16(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
-                        int ctas_per_sm, cudaStream_t st, int dev) {
+                        int ctas_per_sm, cudaStream_t st, int dev, bool dry) {
   constexpr int NCW = 4;
   using M = Row16Smem<NCW>;
   auto kern = row16_main_kernel<D, NCW>;
@@ -372,6 +375,7 @@ static int launch_row16(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
     if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
+  if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
   cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + 1) * 32), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
@@ -380,11 +384,11 @@ static int launch_row16(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
 
 template <int D>
 static int launch_chunk_ncw(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
-                            const DeviceInfo& di, int cps, cudaStream_t st, int dev) {
+                            const DeviceInfo& di, int cps, cudaStream_t st, int dev, bool dry) {
   switch (ncw) {
-    case 2: return launch_chunk<D, 2>(tk, tv, p, di, cps, st, dev);
-    case 4: return launch_chunk<D, 4>(tk, tv, p, di, cps, st, dev);
-    default: return launch_chunk<D, 8>(tk, tv, p, di, cps, st, dev);
+    case 2: return launch_chunk<D, 2>(tk, tv, p, di, cps, st, dev, dry);
+    case 4: return launch_chunk<D, 4>(tk, tv, p, di, cps, st, dev, dry);
+    default: return launch_chunk<D, 8>(tk, tv, p, di, cps, st, dev, dry);
   }
 }
 
@@ -652,6 +656,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   if (rc) return rc;
   if ((rc = validate_kv8(s, kv8))) return rc;
   if ((rc = validate_q_len(s, q_len, kv8 != nullptr))) return rc;
+  if (!(scale > 0.f) || !(scale <= 3.0e38f)) return OOCO_E_SHAPE;  // positive and finite (NaN fails both)
   if (!q || !k_cache || !v_cache || !block_table || !context_lens || !out || !workspace) return OOCO_E_NULLPTR;
   if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q | (uintptr_t)out) & 15) return OOCO_E_UNSUPPORTED;
   const WsLayout w = ws_layout(s, q_len);
@@ -740,6 +745,23 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   }
   p.split_halves = five_d ? 0 : 1;
 
+  // Everything of the attention launch that can refuse the call (shared-memory fit, function attributes) runs
+  // once without launching, before the first kernel of the call is enqueued.
+  const int stages = g_knobs[kKnobStages].load();
+  auto launch_attention = [&](bool dry) -> int {
+    if (chunk_tc) return launch_chunk_tc(tk, tv, p, di, cps, st, dev, dry);
+    if (chunk)
+      return s->head_dim == 128 ? launch_chunk_ncw<128>(ncw, tk, tv, p, di, cps, st, dev, dry)
+                                : launch_chunk_ncw<64>(ncw, tk, tv, p, di, cps, st, dev, dry);
+    if (row16)
+      return s->head_dim == 128 ? launch_row16<128>(tk, tv, p, di, cps, st, dev, dry)
+                                : launch_row16<64>(tk, tv, p, di, cps, st, dev, dry);
+    if (kv8) return launch_main_kv8(ncw, tk, tv, p, di, cps, stages, st, dev, dry);
+    return s->head_dim == 128 ? launch_main_ncw<128>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev, dry)
+                              : launch_main_ncw<64>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev, dry);
+  };
+  if ((rc = launch_attention(true))) return rc;
+
   cudaEvent_t* pe = nullptr;
   if (g_prof_on.load(std::memory_order_acquire)) {
     std::lock_guard<std::mutex> lk(g_prof.mu);
@@ -771,21 +793,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
                             hs);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("launch of the plan kernel", (long)e);
-  const int stages = g_knobs[kKnobStages].load();
   if (pe) cudaEventRecord(pe[1], st);
-  if (chunk_tc)
-    rc = launch_chunk_tc(tk, tv, p, di, cps, st, dev);
-  else if (chunk)
-    rc = s->head_dim == 128 ? launch_chunk_ncw<128>(ncw, tk, tv, p, di, cps, st, dev)
-                            : launch_chunk_ncw<64>(ncw, tk, tv, p, di, cps, st, dev);
-  else if (row16)
-    rc = s->head_dim == 128 ? launch_row16<128>(tk, tv, p, di, cps, st, dev) : launch_row16<64>(tk, tv, p, di, cps, st, dev);
-  else if (kv8)
-    rc = launch_main_kv8(ncw, tk, tv, p, di, cps, stages, st, dev);
-  else if (s->head_dim == 128)
-    rc = launch_main_ncw<128>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);
-  else
-    rc = launch_main_ncw<64>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev);
+  rc = launch_attention(false);
   if (rc) return rc;
   if (pe) cudaEventRecord(pe[2], st);
   {
@@ -1056,6 +1065,9 @@ int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void*
       !k_cache || !v_cache || !out_host || !staging || !workspace)
     return OOCO_E_NULLPTR;
   if (staging_bytes < ooco_step_staging_bytes(s) || ((uintptr_t)staging & 255)) return OOCO_E_WORKSPACE;
+  if (workspace_bytes < ws_layout(s).total || ((uintptr_t)workspace & 255)) return OOCO_E_WORKSPACE;
+  if (!(scale > 0.f) || !(scale <= 3.0e38f)) return OOCO_E_SHAPE;
+  if (((uintptr_t)k_cache | (uintptr_t)v_cache) & 15) return OOCO_E_UNSUPPORTED;
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const size_t qb = (size_t)s->batch * s->num_q_heads * s->head_dim * 2;

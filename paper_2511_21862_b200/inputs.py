@@ -143,20 +143,22 @@ def _randn_bf16(shape, sigma, gen, device, chunk_elems=1 << 28):
     return out
 
 
-def make_batch(cfg: DecodeConfig, device="cpu", *, poison: bool = True, table_pad: int = -1,
-               context_lens: torch.Tensor | None = None) -> DecodeBatch:
-    """Draw one decode batch.
+@dataclass
+class BatchLayout:
+    """Everything of a batch that is drawn on the CPU generator: lengths, block table, pool size."""
+    lens: torch.Tensor           # int32 [B]
+    table: torch.Tensor          # int32 [B, MB]
+    nblk: torch.Tensor           # int64 [B] blocks owned by each sequence (room for the append included)
+    num_blocks: int              # NB
+    used_blocks: int
+    valid_slots: torch.Tensor    # int32 [NB] tokens < T_b held by each block
 
-    Every sequence owns ceil((T_b + 1) / bs) distinct physical blocks (room for the one-token
-    append at position T_b), taken from a random permutation of the pool, so tables are shuffled
-    and non-contiguous; with pool_fill < 1 the unused blocks are holes spread over the pool.
-    With `poison`, every slot at or beyond T_b (and every unused block) is NaN and every table
-    entry beyond a sequence's blocks is `table_pad`, so any out-of-range read shows up.
-    """
-    device = torch.device(device)
+
+def draw_layout(cfg: DecodeConfig, *, table_pad: int = -1, context_lens: torch.Tensor | None = None) -> BatchLayout:
+    """Lengths and block table of `cfg` (identical on every machine: CPU generator, seed of the config)."""
     cgen = torch.Generator(device="cpu").manual_seed(cfg.seed)
     lens = draw_context_lens(cfg, cgen) if context_lens is None else context_lens.to(torch.int32).cpu()
-    B, bs, Hkv, Hq, D = lens.numel(), cfg.block_size, cfg.num_kv_heads, cfg.num_q_heads, cfg.head_dim
+    B, bs = lens.numel(), cfg.block_size
     nblk = (lens.to(torch.int64) + 1 + bs - 1) // bs           # blocks owned, incl. room for the append
     used = int(nblk.sum())
     if cfg.pool_blocks:
@@ -177,6 +179,23 @@ def make_batch(cfg: DecodeConfig, device="cpu", *, poison: bool = True, table_pa
         cnt = torch.clamp(T - torch.arange(n, dtype=torch.int64) * bs, 0, bs).to(torch.int32)
         valid_slots[ids.long()] = cnt
         off += n
+    return BatchLayout(lens, table, nblk, NB, used, valid_slots)
+
+
+def make_batch(cfg: DecodeConfig, device="cpu", *, poison: bool = True, table_pad: int = -1,
+               context_lens: torch.Tensor | None = None) -> DecodeBatch:
+    """Draw one decode batch.
+
+    Every sequence owns ceil((T_b + 1) / bs) distinct physical blocks (room for the one-token
+    append at position T_b), taken from a random permutation of the pool, so tables are shuffled
+    and non-contiguous; with pool_fill < 1 the unused blocks are holes spread over the pool.
+    With `poison`, every slot at or beyond T_b (and every unused block) is NaN and every table
+    entry beyond a sequence's blocks is `table_pad`, so any out-of-range read shows up.
+    """
+    device = torch.device(device)
+    lay = draw_layout(cfg, table_pad=table_pad, context_lens=context_lens)
+    lens, table, NB, used, valid_slots = lay.lens, lay.table, lay.num_blocks, lay.used_blocks, lay.valid_slots
+    B, bs, Hkv, Hq, D = lens.numel(), cfg.block_size, cfg.num_kv_heads, cfg.num_q_heads, cfg.head_dim
 
     dgen = torch.Generator(device=device).manual_seed(cfg.seed + 1000)
     if cfg.layout == "head_major":
@@ -205,6 +224,41 @@ def make_batch(cfg: DecodeConfig, device="cpu", *, poison: bool = True, table_pa
             v_cache[s:e].masked_fill_(dead, float("nan"))
     return DecodeBatch(cfg, q, k_cache, v_cache, table.to(device), lens.to(device), k_new, v_new,
                        NB, strides, extras={"used_blocks": used, "valid_slots": valid_slots})
+
+
+def make_sample_batch(cfg: DecodeConfig, seqs, device="cpu") -> DecodeBatch:
+    """The sequences `seqs` of `cfg`'s batch alone, over a pool that holds just their blocks.
+
+    Lengths and block-table rows are those of the full batch (same CPU draws); the sampled sequences'
+    blocks are renumbered in the shuffled order of their original ids, so the compact pool is as
+    non-contiguous as the original one.  Values are drawn for the sampled blocks only (same
+    distribution as `make_batch`, other draws), which keeps the host footprint to the sample's size.
+    The batch index of sequence seqs[i] is i."""
+    device = torch.device(device)
+    lay = draw_layout(cfg)
+    seqs = [int(b) for b in seqs]
+    bs, Hkv, Hq, D = cfg.block_size, cfg.num_kv_heads, cfg.num_q_heads, cfg.head_dim
+    ids = torch.cat([lay.table[b, : int(lay.nblk[b])] for b in seqs]).to(torch.int64)
+    order = torch.argsort(ids)                                   # rank of each original id = its new id
+    new_id = torch.empty_like(order)
+    new_id[order] = torch.arange(ids.numel())
+    NB, MB = ids.numel(), int(max(int(lay.nblk[b]) for b in seqs))
+    table = torch.full((len(seqs), MB), -1, dtype=torch.int32)
+    off = 0
+    for i, b in enumerate(seqs):
+        n = int(lay.nblk[b])
+        table[i, :n] = new_id[off:off + n].to(torch.int32)
+        off += n
+    lens = lay.lens[seqs].contiguous()
+    dgen = torch.Generator(device=device).manual_seed(cfg.seed + 2000)
+    assert cfg.layout == "head_major"
+    k_cache = _randn_bf16((NB, Hkv, bs, D), cfg.sigma, dgen, device)
+    v_cache = _randn_bf16((NB, Hkv, bs, D), cfg.sigma, dgen, device)
+    q = _randn_bf16((len(seqs), Hq, D), cfg.sigma, dgen, device)
+    k_new = _randn_bf16((len(seqs), Hkv, D), cfg.sigma, dgen, device)
+    v_new = _randn_bf16((len(seqs), Hkv, D), cfg.sigma, dgen, device)
+    return DecodeBatch(cfg, q, k_cache, v_cache, table.to(device), lens.to(device), k_new, v_new, NB,
+                       (Hkv * bs * D, bs * D, D), extras={"used_blocks": NB, "sampled_from": seqs})
 
 
 def as_u16(t: torch.Tensor):

@@ -113,6 +113,15 @@ def test_argument_validation_without_a_device():
     assert attn(dataclasses.replace(good, num_q_heads=64, num_kv_heads=2)) == -3        # group of 32
     assert attn(dataclasses.replace(good, kv_token_stride=68)) == -3                    # not 16-byte multiple
     assert attn(good, ws_bytes=1024) == -4                                              # WORKSPACE
+    # the softmax scale must be positive and finite (every kernel may then take the maximum before scaling)
+    for bad_scale in (0.0, -0.125, float("inf"), float("nan")):
+        assert L.ooco_decode_attention(ctypes.byref(good.c()), one, one, one, one, one, bad_scale, one, one, 1 << 40,
+                                       None) == -2
+        assert L.ooco_decode_step_host(ctypes.byref(good.c()), one, one, one, one, one, one, one, one, bad_scale, one,
+                                       one, 1 << 40, one, 1 << 40, None) == -2
+    # the host-buffer step checks both scratch buffers before it enqueues its first copy
+    assert L.ooco_decode_step_host(ctypes.byref(good.c()), one, one, one, one, one, one, one, one, 1.0, one,
+                                   one, 1 << 40, one, 1024, None) == -4
     assert L.ooco_kv_append(ctypes.byref(good.c()), None, one, one, one, one, one, None) == -1
     assert L.ooco_decode_bytes_model(ctypes.byref(good.c()), None, 2, None) == -1
     assert L.ooco_set_tuning(99, 1) == -2 and L.ooco_set_tuning(0, 3) == -2

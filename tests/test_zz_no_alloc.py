@@ -5,8 +5,10 @@ engine gave the whole device to its KV pool at start-up, or the decode loop cann
 device-wide synchronisation an allocation implies, or the host framework forbids allocations outside
 its own pool.  For them the library carries a 16 MiB scratch array in its device image and an entry
 point that uses it instead of a caller-provided workspace.  These tests call that entry point through
-the C ABI and compare it with the ordinary entry point (same tolerance as the parity tests), twice in
-a row on different batches, because the shared array still holds the previous call's contents.
+the C ABI, several times in a row on different batches (the shared array still holds the previous
+call's contents), and require its output to be bit for bit the ordinary entry point's (both run the same
+launches on the same plan), to match the fp64 oracle within the parity tolerance, and the call to
+leave the device's free memory and torch's allocation counter untouched.
 
 This file is collected last on purpose: a failure here cannot hide another test's result in a run
 that stops at the first failure.
@@ -17,6 +19,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2511_21862_b200 import binding, build, inputs
 
 MAX_ABS_TOL, MEAN_ABS_TOL = 1e-2, 1e-3          # the tolerance of the parity tests
@@ -42,7 +45,7 @@ def both_entry_points(cfg):
     binding.decode_attention_static(sh, batch.q, batch.k_cache, batch.v_cache, batch.block_table,
                                     batch.context_lens, cfg.scale, got)
     torch.cuda.synchronize()
-    return got, want
+    return batch, got, want
 
 
 @pytest.mark.gpu
@@ -50,11 +53,36 @@ def test_static_scratch_entry_point_matches_the_workspace_one_twice_in_a_row():
     first = C("noalloc-a", 32, 8, 128, 16, (G(20, 1, 2500), G(2, 5000, 7000)), seed=60, pool_fill=0.8)   # split + unsplit
     second = C("noalloc-b", 8, 2, 64, 32, (G(7, 0, 300),), seed=61)                                        # other shape, stale scratch
     for cfg in (first, second, first):
-        got, want = both_entry_points(cfg)
-        g, w = got.double().cpu().numpy(), want.double().cpu().numpy()
-        assert not np.isnan(g).any() and not np.isnan(w).any()
-        err = np.abs(g - w)
+        batch, got, want = both_entry_points(cfg)
+        assert not torch.isnan(got.float()).any()
+        assert torch.equal(got.view(torch.int16), want.view(torch.int16)), cfg.name       # same launches, same plan
+        ref = oracle.decode_attention(inputs.as_u16(batch.q), inputs.as_u16(batch.k_cache), inputs.as_u16(batch.v_cache),
+                                      batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                      num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size, strides=batch.strides)
+        err = np.abs(got.double().cpu().numpy() - ref.out)
         assert err.max() <= MAX_ABS_TOL and err.mean() <= MEAN_ABS_TOL, (cfg.name, err.max(), err.mean())
+
+
+@pytest.mark.gpu
+def test_static_scratch_entry_point_allocates_nothing_after_its_first_call():
+    """After one warm-up call on the device (module loading and the symbol look-up happen there) a call
+    changes neither the device's free memory nor the bytes torch has handed out."""
+    cfg = C("noalloc-c", 32, 8, 128, 16, (G(12, 1, 3000),), seed=62)
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    sh = binding.shape_of(batch)
+    out = torch.empty_like(batch.q)
+    call = lambda: binding.decode_attention_static(sh, batch.q, batch.k_cache, batch.v_cache, batch.block_table,
+                                                   batch.context_lens, cfg.scale, out)
+    call()
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (held0, reserved0)
 
 
 def test_static_scratch_entry_point_rejects_shapes_beyond_its_array():

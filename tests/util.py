@@ -27,9 +27,10 @@ def gpu_attention(batch, context_lens=None, scale=None, check_status=True):
     return out
 
 
-def oracle_attention(batch, context_lens=None, scale=None, seqs=None):
+def oracle_attention(batch, context_lens=None, scale=None, seqs=None, kv8=None):
     """fp64 oracle on a host copy; with `seqs`, only those sequences (other rows NaN), using a
-    compacted copy of just their blocks (plain torch indexing) so huge pools need not be copied."""
+    compacted copy of just their blocks (plain torch indexing) so huge pools need not be copied.
+    `kv8` = (k_scale, v_scale): the pools hold E4M3 codes (the 8-bit oracle)."""
     cfg = batch.cfg
     lens = (batch.context_lens if context_lens is None else context_lens).cpu()
     table = batch.block_table.cpu()
@@ -47,10 +48,46 @@ def oracle_attention(batch, context_lens=None, scale=None, seqs=None):
         idx = torch.tensor(ids if ids else [0], dtype=torch.long, device=k.device)
         k, v, table = k.index_select(0, idx), v.index_select(0, idx), new_table
         pairs = np.array([(b, h) for b in seqs for h in range(cfg.num_q_heads)], dtype=np.int32)
+    if kv8 is not None:
+        return oracle.decode_attention_fp8(
+            inputs.as_u16(batch.q), inputs.as_u8(k), inputs.as_u8(v), table.numpy(), lens.numpy(),
+            cfg.scale if scale is None else scale, kv8[0], kv8[1], num_kv_heads=cfg.num_kv_heads,
+            block_size=cfg.block_size, strides=batch.strides, pairs=pairs)
     return oracle.decode_attention(
         inputs.as_u16(batch.q), inputs.as_u16(k), inputs.as_u16(v), table.numpy(), lens.numpy(),
         cfg.scale if scale is None else scale, num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size,
         strides=batch.strides, pairs=pairs)
+
+
+def sequence_slices(lens, block_size, block_bytes, slice_bytes):
+    """Consecutive runs of sequences whose cache blocks add up to at most `slice_bytes` each
+    (a single sequence larger than that is a run of its own)."""
+    runs, cur, acc = [], [], 0
+    for b, T in enumerate(int(x) for x in lens):
+        need = -(-T // block_size) * block_bytes
+        if cur and acc + need > slice_bytes:
+            runs.append(cur)
+            cur, acc = [], 0
+        cur.append(b)
+        acc += need
+    if cur:
+        runs.append(cur)
+    return runs
+
+
+def oracle_attention_every_sequence(batch, context_lens=None, scale=None, kv8=None, slice_bytes=3 << 30):
+    """The oracle's output for EVERY sequence of a batch whose pool is too large to copy to the host in
+    one piece: the sequences are taken in consecutive runs, each run gets a compacted host copy of just
+    its blocks, and the rows are put together.  fp64 [B, Hq, D]."""
+    cfg = batch.cfg
+    lens = (batch.context_lens if context_lens is None else context_lens).cpu()
+    block_bytes = 2 * cfg.num_kv_heads * cfg.block_size * cfg.head_dim * batch.k_cache.element_size()
+    out = np.full(tuple(batch.q.shape), np.nan, dtype=np.float64)
+    for run in sequence_slices(lens.tolist(), cfg.block_size, block_bytes, slice_bytes):
+        r = oracle_attention(batch, context_lens=lens, scale=scale, seqs=run, kv8=kv8)
+        out[run] = r.out[run]
+    assert not np.isnan(out).any()
+    return out
 
 
 def assert_parity(out_gpu: torch.Tensor, ref: np.ndarray, rows=None, what=""):
