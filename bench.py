@@ -381,12 +381,17 @@ def measure_workload(args, cfg, dev, rank, world, *, e2e=True, baseline=False):
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
+        enq = wait = 0
         t0 = time.perf_counter()
         for i in range(e2e_steps):
             e2e_step(i)
+            a, b = binding.last_host_step_ns()
+            enq, wait = enq + a, wait + b
         torch.cuda.synchronize()
         res["e2e_ms"] = (time.perf_counter() - t0) / e2e_steps * 1e3
         res["e2e_steps"] = e2e_steps
+        # host time inside the call: until everything was enqueued / waiting for the stream (microseconds)
+        res["e2e_host_us"] = {"enqueue": enq / e2e_steps / 1e3, "wait": wait / e2e_steps / 1e3}
     sampler.stop()
     if baseline:
         res["cpu_baseline"] = cpu_baseline(cfg, batch, args.cpu_seconds)
@@ -451,7 +456,7 @@ def run_ours(args, rank, local_rank, world):
                 "pct_of_measured_copy": 100.0 * v * 1e3 / peak, "kernel_ms": km,
                 "kernel_GBps": roof["achieved"], "kernel_frac_of_measured": roof["frac"],
                 "kernel_frac_of_nominal_8tbps": roof["frac_of_nominal_8tbps"], "traffic": roof["traffic"],
-                "traffic_source": roof["traffic_source"], "e2e_ms_per_step": r["e2e_ms"],
+                "traffic_source": roof["traffic_source"], "e2e_ms_per_step": r["e2e_ms"], "e2e_host_us_per_call": r["e2e_host_us"],
                 "total_tokens": r["cost"]["total_tokens"], "batch": r["B"], "pool_replicas": r["R"], "clocks": r["clocks"]}
     if rank != 0:
         return
@@ -473,7 +478,8 @@ def run_ours(args, rank, local_rank, world):
         "kernel_ms": kernel_ms,
         "roofline": roof,
         "e2e": {"value": total_bytes / (e2e_ms * 1e-3) / 1e12, "unit": "TB/s", "h2d_bytes_per_step": res["h2d"],
-                "d2h_bytes_per_step": res["d2h"], "ms_per_step": e2e_ms, "steps": res["e2e_steps"]},
+                "d2h_bytes_per_step": res["d2h"], "ms_per_step": e2e_ms, "steps": res["e2e_steps"],
+                "host_us_per_call": res["e2e_host_us"]},
         "gpu_launches": args.steps * res["launches_per_step"],
         "clocks": res["clocks"],
     }

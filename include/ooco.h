@@ -412,6 +412,13 @@ int ooco_decode_step_host(const ooco_shape_t* shape, const void* q_host,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Where the host time of the last successful ooco_decode_step_host call on this thread went:
+ * *enqueue_ns = from entry until everything was enqueued (validation, pointer queries, tensor-map
+ * encoding, launches), *wait_ns = the wait for the stream after that.  Host clocks; for benchmarks.
+ */
+int ooco_last_host_step_ns(int64_t* enqueue_ns, int64_t* wait_ns);
+
+/*
  * Number of kernels the last successful ooco_decode_attention call on this
  * thread enqueued (for launch accounting in benchmarks); 0 before any call.
  */
@@ -444,10 +451,37 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * (sequence, kv head) run the kernel whose warps share 16 score rows and split the tokens of a
  * stage (zero = the decode kernel with two 8-column tiles); 12 non-zero = more than 32 score columns
  * at head_dim 128 run the tcgen05 kernel (zero = the mma.sync kernel of the prefill-chunk path).
+ * 13 non-zero = diagnostic fp32 output: `out` of the attention entry points is then fp32 (same
+ * shape, 4 bytes per value) and holds the values the kernels would otherwise round to bf16 (every
+ * row goes through the partial-result and merge path; an unsplit row passes it unchanged), so a
+ * test can separate the arithmetic's error from the output format's rounding; not for the host-buffer
+ * step (OOCO_E_UNSUPPORTED).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
- * unknown knob or a value outside its range.
+ * unknown knob or a value outside its range.  ooco_get_tuning returns a knob's current value
+ * (OOCO_E_SHAPE, which is negative, for an unknown knob).
  */
 int ooco_set_tuning(int knob, int value);
+int ooco_get_tuning(int knob);
+
+/*
+ * The checked build.  Compiling the library with -DOOCO_CHECKS (build.py writes it to
+ * libooco_checked.so) makes the kernels range-check every index they derive from device data: each
+ * block-table entry they read, the fields of each work item, each partial-result slot and output
+ * row, and the shared-memory destination of each asynchronous copy.  A violation is OR-ed into the
+ * status word ooco_workspace_status reads (8: table entry outside [0, num_blocks), 16: work-item
+ * field out of range, 32: partial-slot / work-list / output index out of range, 64: shared-memory
+ * destination outside its region) and the access is skipped (a bad table entry reads as zeros); the
+ * kernels never trap.  It stands in for a memory checker on machines where none can be run; the
+ * release build compiles the checks to nothing.
+ *   ooco_checked_build     1 in the checked build, 0 otherwise.
+ *   ooco_check_predicate   evaluates one of the range predicates on the HOST (for unit tests of the
+ *                          predicates themselves): which = 0 table entry {id, num_blocks};
+ *                          1 index {i, n}; 2 work item {sequence, slot, first token, end token, B,
+ *                          max items, table capacity in tokens}; 3 span {offset, bytes, lo, hi}.
+ *                          Returns 1 / 0, or a negative OOCO_E_* for a NULL pointer or unknown `which`.
+ */
+int ooco_checked_build(void);
+int ooco_check_predicate(int which, const int64_t* args_host);
 
 /*
  * Text about the last OOCO_E_CUDA or OOCO_E_WORKSPACE on this thread ("" if none yet): the CUDA

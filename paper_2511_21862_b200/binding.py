@@ -23,7 +23,8 @@ EXPORTS = (
     "ooco_kv_gather_blocks", "ooco_kv_scatter_blocks", "ooco_kv_copy_blocks",
     "ooco_kv_append_fp8", "ooco_decode_attention_fp8", "ooco_decode_step_fp8",
     "ooco_decode_workspace_bytes_mq", "ooco_decode_attention_mq", "ooco_kv_append_mq", "ooco_attention_bytes_model",
-    "ooco_decode_step_mq", "ooco_decode_step_mq_fp8",
+    "ooco_decode_step_mq", "ooco_decode_step_mq_fp8", "ooco_get_tuning", "ooco_checked_build", "ooco_check_predicate",
+    "ooco_last_host_step_ns",
 )
 
 
@@ -47,6 +48,17 @@ class ooco_cost_t(ctypes.Structure):
 
 
 _lib = None
+
+
+def use_library(path: str | None):
+    """Makes `path` (e.g. the checked build, `build.LIB_CHECKED`) the library every call below goes to;
+    None returns to the default library.  Returns the path that was in use."""
+    global _lib, LIB_PATH
+    old = LIB_PATH
+    LIB_PATH = path or os.path.join(_HERE, "libooco.so")
+    _lib = None
+    lib()
+    return old
 
 
 def lib() -> ctypes.CDLL:
@@ -113,6 +125,13 @@ def lib() -> ctypes.CDLL:
         L.ooco_last_error_detail.restype = ctypes.c_char_p
         L.ooco_set_tuning.restype = ctypes.c_int
         L.ooco_set_tuning.argtypes = [ctypes.c_int, ctypes.c_int]
+        L.ooco_get_tuning.restype = ctypes.c_int
+        L.ooco_get_tuning.argtypes = [ctypes.c_int]
+        L.ooco_last_host_step_ns.restype = ctypes.c_int
+        L.ooco_last_host_step_ns.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]
+        L.ooco_checked_build.restype = ctypes.c_int
+        L.ooco_check_predicate.restype = ctypes.c_int
+        L.ooco_check_predicate.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int64)]
         L.ooco_status_string.restype = ctypes.c_char_p
         L.ooco_status_string.argtypes = [ctypes.c_int]
         L.ooco_version.restype = ctypes.c_int
@@ -153,12 +172,41 @@ class Shape:
 
 
 KNOBS = {"warps": 0, "stages": 1, "ctas_per_sm": 2, "chunk_min": 3, "chunk_max": 4, "items_per_cta": 5,
-         "split_halves": 6, "tiles_per_warp": 7, "pdl": 8, "copy_ctas_per_sm": 9, "host_stage_kernel": 10, "row_layout_16": 11, "chunk_tcgen05": 12}
+         "split_halves": 6, "tiles_per_warp": 7, "pdl": 8, "copy_ctas_per_sm": 9, "host_stage_kernel": 10, "row_layout_16": 11, "chunk_tcgen05": 12,
+         "out_f32": 13}
 
 
 def set_tuning(**kw):
     for k, v in kw.items():
         _check(lib().ooco_set_tuning(KNOBS[k], int(v)), f"ooco_set_tuning({k}={v})")
+
+
+def get_tuning(knob: str) -> int:
+    v = lib().ooco_get_tuning(KNOBS[knob])
+    if v < 0:
+        raise OocoError(v, f"ooco_get_tuning({knob})")
+    return int(v)
+
+
+def last_host_step_ns():
+    """(ns until everything of the last decode_step_host call was enqueued, ns it then waited for the stream)."""
+    a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(lib().ooco_last_host_step_ns(ctypes.byref(a), ctypes.byref(b)), "ooco_last_host_step_ns")
+    return int(a.value), int(b.value)
+
+
+def checked_build() -> bool:
+    """True when the loaded library is the variant whose kernels range-check device-derived indices."""
+    return bool(lib().ooco_checked_build())
+
+
+def check_predicate(which: int, *args) -> bool:
+    """Host evaluation of one of the checked build's range predicates (see ooco_check_predicate)."""
+    a = (ctypes.c_int64 * max(1, len(args)))(*[int(x) for x in args])
+    r = lib().ooco_check_predicate(int(which), a)
+    if r < 0:
+        raise OocoError(r, "ooco_check_predicate")
+    return bool(r)
 
 
 def _stream_ptr(stream) -> int:
@@ -172,6 +220,12 @@ def _dev(t: torch.Tensor, dtype=None) -> int:
     if dtype is not None:
         assert t.dtype == dtype, (t.dtype, dtype)
     return t.data_ptr()
+
+
+def _out(t: torch.Tensor) -> int:
+    """`out` is bf16, or fp32 while the diagnostic fp32-output knob is set."""
+    want = torch.float32 if get_tuning("out_f32") else torch.bfloat16
+    return _dev(t, want)
 
 
 def workspace_bytes(shape: Shape) -> int:
@@ -200,7 +254,7 @@ def decode_attention(shape: Shape, q, k_cache, v_cache, block_table, context_len
     _check(lib().ooco_decode_attention(
         ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_cache, torch.bfloat16),
         _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
-        float(scale), _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        float(scale), _out(out), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_attention")
 
 
@@ -210,7 +264,7 @@ def decode_step(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table, po
     _check(lib().ooco_decode_step(
         ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_new, torch.bfloat16), _dev(v_new, torch.bfloat16),
         _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32),
-        _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), _dev(out, torch.bfloat16),
+        _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), _out(out),
         _dev(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step")
 
 
@@ -229,7 +283,7 @@ def decode_attention_fp8(shape: Shape, q, k_cache, v_cache, block_table, context
     _check(lib().ooco_decode_attention_fp8(
         ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_cache, torch.uint8), _dev(v_cache, torch.uint8),
         _dev(block_table, torch.int32), _dev(context_lens, torch.int32), float(scale), float(k_scale),
-        float(v_scale), _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        float(v_scale), _out(out), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_attention_fp8")
 
 
@@ -240,7 +294,7 @@ def decode_step_fp8(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table
         ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_new, torch.bfloat16), _dev(v_new, torch.bfloat16),
         _dev(k_cache, torch.uint8), _dev(v_cache, torch.uint8), _dev(block_table, torch.int32),
         _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale), float(k_scale), float(v_scale),
-        _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        _out(out), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_step_fp8")
 
 
@@ -258,7 +312,7 @@ def decode_attention_mq(shape: Shape, q, k_cache, v_cache, block_table, context_
     _check(lib().ooco_decode_attention_mq(
         ctypes.byref(shape.c()), int(q.shape[1]), _dev(q, torch.bfloat16), _dev(k_cache, torch.bfloat16),
         _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
-        float(scale), _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        float(scale), _out(out), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_attention_mq")
 
 
@@ -270,7 +324,7 @@ def decode_step_mq(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_table,
         ctypes.byref(shape.c()), int(q.shape[1]), _dev(q, torch.bfloat16), _dev(k_new, torch.bfloat16),
         _dev(v_new, torch.bfloat16), _dev(k_cache, torch.bfloat16), _dev(v_cache, torch.bfloat16),
         _dev(block_table, torch.int32), _dev(positions, torch.int32), _dev(context_lens, torch.int32), float(scale),
-        _dev(out, torch.bfloat16), _dev(workspace), workspace.numel() * workspace.element_size(),
+        _out(out), _dev(workspace), workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)), "ooco_decode_step_mq")
 
 
@@ -282,7 +336,7 @@ def decode_step_mq_fp8(shape: Shape, q, k_new, v_new, k_cache, v_cache, block_ta
         ctypes.byref(shape.c()), int(q.shape[1]), _dev(q, torch.bfloat16), _opt_dev(k_new, torch.bfloat16),
         _opt_dev(v_new, torch.bfloat16), _dev(k_cache, torch.uint8), _dev(v_cache, torch.uint8),
         _dev(block_table, torch.int32), _opt_dev(positions, torch.int32), _dev(context_lens, torch.int32),
-        float(scale), float(k_scale), float(v_scale), _dev(out, torch.bfloat16), _dev(workspace),
+        float(scale), float(k_scale), float(v_scale), _out(out), _dev(workspace),
         workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "ooco_decode_step_mq_fp8")
 
 
@@ -307,7 +361,7 @@ def decode_attention_static(shape: Shape, q, k_cache, v_cache, block_table, cont
     _check(lib().ooco_decode_attention_static(
         ctypes.byref(shape.c()), _dev(q, torch.bfloat16), _dev(k_cache, torch.bfloat16),
         _dev(v_cache, torch.bfloat16), _dev(block_table, torch.int32), _dev(context_lens, torch.int32),
-        float(scale), _dev(out, torch.bfloat16), _stream_ptr(stream)), "ooco_decode_attention_static")
+        float(scale), _out(out), _stream_ptr(stream)), "ooco_decode_attention_static")
 
 
 def _opt_dev(t, dtype=None):

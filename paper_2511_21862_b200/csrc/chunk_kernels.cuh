@@ -168,6 +168,12 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
     slot = it % nst;
     return warp_wait(s_empty + 8 * slot, (((uint32_t)(it / nst)) & 1u) ^ 1u, s_abort);
   };
+  // checked build: see the producer of decode_main_kernel
+  auto table_entry = [&](const int32_t* e) {
+    const int v = *e;
+    return checked(chk_table_entry(v, p.NB), &p.hdr->status, kStatusBadTableEntry) ? v : p.NB;
+  };
+  bool violated = false;
   while (unit < n_units && ok) {
     int nxt = 0;
     if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
@@ -175,6 +181,12 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
     // the last row tile of an item sees the most tokens: it goes first (longest work first)
     const int item = (int)(unit / nrt), rt = nrt - 1 - (int)(unit - (long long)item * nrt);
     const int4 d = p.items[item];
+    if (!checked(chk_item(d.x, d.y, d.z, d.w, p.B, p.max_items, cap_tokens), &p.hdr->status, kStatusBadItem)) {
+      *s_abort = 1;  // stop the CTA: the other warps leave through the abort flag
+      violated = true;
+      ok = false;
+      break;
+    }
     const int b = d.x, h = d.y % p.Hkv, t0 = d.z, t1 = d.w;
     long long T = p.context_lens[b];
     T = T < 0 ? 0 : (T > cap_tokens ? cap_tokens : T);
@@ -186,7 +198,7 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
     int blk_cur = 0;
     {
       const int tb = t0 + lane * p.tile_rows;
-      if (lane < boxes_per_stage && tb < t1e) blk_cur = row[tb / p.bs];
+      if (lane < boxes_per_stage && tb < t1e) blk_cur = table_entry(row + tb / p.bs);
     }
     if (nstage == 0) {  // the tile sees nothing of this chunk: one empty stage carries the bookkeeping
       int slot;
@@ -208,7 +220,7 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
       int blk_n = 0;  // table entries of the following stage, one stage ahead of their use
       {
         const int tb = tok0 + kChunkStageTok + lane * p.tile_rows;
-        if (s + 1 < nstage && lane < boxes_per_stage && tb < t1e) blk_n = row[tb / p.bs];
+        if (s + 1 < nstage && lane < boxes_per_stage && tb < t1e) blk_n = table_entry(row + tb / p.bs);
       }
       int slot;
       if (!acquire(slot)) {
@@ -223,16 +235,30 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
         mbar_arrive_expect_tx(full, 2u * (uint32_t)nbox * box_rows_bytes * (D / 64));
       }
       __syncwarp();
+      bool span_ok = true;
       if (lane < nbox) {
         const int tb = tok0 + lane * p.tile_rows;
         const int c_tok = tb % p.bs;
         const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + (uint32_t)lane * box_rows_bytes;
         const uint32_t dv = dk + L::kTileBytes;
+        // checked build: the box lands inside the first 64-dim half of the stage's K tile (the others follow it)
+        span_ok = checked(chk_span(dk, box_rows_bytes, s_stage + (long long)slot * L::kStageBytes,
+                                   s_stage + (long long)slot * L::kStageBytes + L::kHalfBytes) &&
+                              chk_span(slot, 1, 0, nst),
+                          &p.hdr->status, kStatusBadSmem);
+        if (span_ok) {
 #pragma unroll
-        for (int j = 0; j < D / 64; ++j) {
-          tma_load_4d(dk + j * L::kHalfBytes, &tm_k, full, 64 * j, c_tok, h, blk_cur);
-          tma_load_4d(dv + j * L::kHalfBytes, &tm_v, full, 64 * j, c_tok, h, blk_cur);
+          for (int j = 0; j < D / 64; ++j) {
+            tma_load_4d(dk + j * L::kHalfBytes, &tm_k, full, 64 * j, c_tok, h, blk_cur);
+            tma_load_4d(dv + j * L::kHalfBytes, &tm_v, full, 64 * j, c_tok, h, blk_cur);
+          }
         }
+      }
+      if (kChecked && !__all_sync(0xffffffffu, span_ok)) {  // a skipped copy leaves the stage incomplete: stop
+        *s_abort = 1;
+        violated = true;
+        ok = false;
+        break;
       }
       blk_cur = blk_n;
     }
@@ -252,7 +278,7 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
   }
   if (!ok) {
     // stop path: record it, then wait (bounded) until every copy already issued has landed
-    if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+    if (lane == 0 && !violated) atomicOr(&p.hdr->status, kStatusWaitTimeout);
     int dummy_abort = 0;
     const int pending = it < nst ? it : nst;
     for (int k = 0; k < pending; ++k) {
@@ -385,7 +411,9 @@ chunk_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (last && live) {
       // ---- the warp's 16 rows are complete for this item: normalise and write them
       const int slot_id = meta.x;
-      const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
+      const bool dst_ok = checked(chk_index(slot_id, p.max_items) && chk_index(b, p.B) && chk_index(h, p.Hkv),
+                                  &p.hdr->status, kStatusBadIndex);
+      const int n_chunks = dst_ok ? p.seq_first[b + 1] - p.seq_first[b] : 1;
       float l0 = l_run[0], l1 = l_run[1];
 #pragma unroll
       for (int o = 1; o < 4; o <<= 1) {
@@ -395,10 +423,10 @@ chunk_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
         const int col = colw + g + 8 * r;
-        if (col >= p.GQ) continue;
+        if (col >= p.GQ || (kChecked && !dst_ok)) continue;
         const float l = r ? l1 : l0, m = r ? m_run[1] : m_run[0];
         const float inv = l > 0.f ? 1.f / l : 0.f;  // l = 0: the row saw no token of this chunk
-        if (n_chunks == 1) {
+        if (n_chunks == 1 && !p.out_f32) {
           const int qi = col / p.G, head = col - qi * p.G;
           __nv_bfloat16* dst = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D + 2 * t;
 #pragma unroll
@@ -560,7 +588,9 @@ row16_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // ---- the item is complete: combine the NCW warps' running states through this stage's memory
     {
       const int slot_id = meta.x;
-      const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
+      const bool dst_ok = checked(chk_index(slot_id, p.max_items) && chk_index(b, p.B) && chk_index(h, p.Hkv),
+                                  &p.hdr->status, kStatusBadIndex);
+      const int n_chunks = dst_ok ? p.seq_first[b + 1] - p.seq_first[b] : 1;
       float l0 = l_run[0], l1 = l_run[1];
 #pragma unroll
       for (int o = 1; o < 4; o <<= 1) {
@@ -617,7 +647,8 @@ row16_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
           num.w += sw * o.w;
         }
         const float inv = den > 0.f ? 1.f / den : 0.f;
-        if (n_chunks == 1) {
+        if (kChecked && !dst_ok) continue;
+        if (n_chunks == 1 && !p.out_f32) {
           const int qi = col / p.G, head = col - qi * p.G;
           __nv_bfloat16* dst = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D + 4 * c;
           const __nv_bfloat162 lo = __floats2bfloat162_rn(num.x * inv, num.y * inv);

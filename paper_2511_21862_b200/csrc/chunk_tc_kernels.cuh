@@ -324,7 +324,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
       if (last) {
         // ---- the unit is complete: normalise this row of O and write it
         const int slot_id = meta.x;
-        const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
+        const bool dst_ok = checked(chk_index(slot_id, p.max_items) && chk_index(b, p.B) && chk_index(h, p.Hkv),
+                                    &p.hdr->status, kStatusBadIndex);
+        const int n_chunks = dst_ok ? p.seq_first[b + 1] - p.seq_first[b] : 1;
+        const bool write_row = real_row && (!kChecked || dst_ok);
         if (ntok > 0) {
           if (!wait_pv(n_pv - 1)) {
             ok = false;
@@ -345,7 +348,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
 #pragma unroll
             for (int j = 0; j < 32; ++j) o[j] = 0u;
           }
-          if (real_row && n_chunks == 1) {
+          if (write_row && n_chunks == 1 && !p.out_f32) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
               uint32_t w[4];
@@ -354,7 +357,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
                 w[i] = pack_bf16x2(__uint_as_float(o[8 * v + 2 * i]) * inv, __uint_as_float(o[8 * v + 2 * i + 1]) * inv);
               *reinterpret_cast<uint4*>(orow + 32 * c4 + 8 * v) = make_uint4(w[0], w[1], w[2], w[3]);
             }
-          } else if (real_row) {
+          } else if (write_row) {
 #pragma unroll
             for (int v = 0; v < 8; ++v)
               *reinterpret_cast<float4*>(prow_o + 32 * c4 + 4 * v) =
@@ -363,7 +366,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
           }
           __syncwarp();  // the tensor-memory loads are warp-wide: reconverge before the next one
         }
-        if (real_row && n_chunks > 1)
+        if (write_row && (n_chunks > 1 || p.out_f32))
           p.part_lse[(size_t)slot_id * p.GQ + col] = l_run > 0.f ? m_ref + lg2(l_run) : -INFINITY;
         tc_fence_before_sync();  // the next unit's first P.V overwrites O: ordered behind these reads by q-ready
       }

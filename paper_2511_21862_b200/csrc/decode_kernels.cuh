@@ -22,6 +22,41 @@ namespace ooco {
 
 constexpr int kStatusPlanOverflow = 1;
 constexpr int kStatusWaitTimeout = 2;
+// Reported by the checked build only (compiled with -DOOCO_CHECKS):
+constexpr int kStatusBadTableEntry = 8;   // a block-table entry that is read lies outside [0, num_blocks)
+constexpr int kStatusBadItem = 16;        // a work-item field outside its range
+constexpr int kStatusBadIndex = 32;       // a partial-result slot, work-list or output index outside its buffer
+constexpr int kStatusBadSmem = 64;        // a shared-memory destination outside the region it belongs to
+
+// ------------------------------------------------------------------------------------ checked build
+// With -DOOCO_CHECKS every index the kernels derive from device data (table entries, work items,
+// partial-result slots) and every shared-memory destination of a copy is range-checked; a violation
+// sets a bit of the workspace's status word and the access is skipped (or, for a table entry, replaced
+// by an id the tensor-map bounds check turns into zeros).  Nothing traps.  Without the macro the
+// checks compile to nothing.
+#ifdef OOCO_CHECKS
+constexpr bool kChecked = true;
+#else
+constexpr bool kChecked = false;
+#endif
+__host__ __device__ inline bool chk_table_entry(long long blk, long long num_blocks) { return blk >= 0 && blk < num_blocks; }
+__host__ __device__ inline bool chk_index(long long i, long long n) { return i >= 0 && i < n; }
+// item = {sequence, partial slot, first token, end token}
+__host__ __device__ inline bool chk_item(long long b, long long slot, long long t0, long long t1, long long B,
+                                         long long max_items, long long cap_tokens) {
+  return b >= 0 && b < B && slot >= 0 && slot < max_items && t0 >= 0 && t0 <= t1 && t1 <= cap_tokens;
+}
+__host__ __device__ inline bool chk_span(long long off, long long bytes, long long lo, long long hi) {
+  return off >= lo && bytes >= 0 && off + bytes <= hi;
+}
+// true = proceed.  In the checked build a failed predicate is recorded and answers false.
+__device__ __forceinline__ bool checked(bool ok, int32_t* status, int bit) {
+  if (kChecked && !ok) {
+    atomicOr(status, bit);
+    return false;
+  }
+  return true;
+}
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every in-kernel wait gives up after 2 s
 
 struct WsHeader {  // first 256 bytes of the workspace
@@ -44,6 +79,8 @@ struct DecodeParams {
   float* part_o;          // [max_items, GQ, D] normalised partial outputs
   float* part_lse;        // [max_items, GQ] log2-domain log-sum-exp of each partial
   int32_t B, Hq, Hkv, G, D, bs, MB;
+  int32_t NB;             // physical blocks in the pool (read by the checked build only)
+  int32_t out_f32;        // diagnostic: `out` holds fp32 and every row goes through the partial + merge path
   int32_t Sq;             // query tokens per sequence (the last Sq tokens of its context); 1 = decode
   int32_t GQ;             // G * Sq: score columns of one (sequence, kv head), column = query * G + head
   int32_t max_items;
@@ -311,13 +348,19 @@ __global__ void __launch_bounds__(kThreads) plan_kernel(DecodeParams p, int stag
     int b, t0, t1;
     const int r = chunk_of(ci, b, t0, t1);
     const long long pos = atomicAdd(&s_cursor[r], 1);
-    for (int h = 0; h < p.Hkv; ++h) p.items[pos * p.Hkv + h] = make_int4(b, ci * p.Hkv + h, t0, t1);
+    for (int h = 0; h < p.Hkv; ++h)
+      if (checked(chk_index(pos * p.Hkv + h, p.max_items), &p.hdr->status, kStatusBadIndex))
+        p.items[pos * p.Hkv + h] = make_int4(b, ci * p.Hkv + h, t0, t1);
   }
   // sequences without context produce zeros
   const int row = p.Sq * p.Hq * p.D;
   for (int b = wid; b < p.B; b += kThreads / 32) {
     if (len_of(b) > 0) continue;
-    for (int i = lane; i < row; i += 32) p.out[(size_t)b * row + i] = __float2bfloat16(0.f);
+    if (p.out_f32) {
+      for (int i = lane; i < row; i += 32) reinterpret_cast<float*>(p.out)[(size_t)b * row + i] = 0.f;
+    } else {
+      for (int i = lane; i < row; i += 32) p.out[(size_t)b * row + i] = __float2bfloat16(0.f);
+    }
   }
 }
 
@@ -662,14 +705,32 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       const long long T = p.context_lens[b];
       return (int)(T < 0 ? 0 : (T > cap_tokens ? cap_tokens : T));
     };
+    // checked build: an item whose fields are out of range is never dereferenced; a table entry outside
+    // the pool is recorded and replaced by an id beyond the tensor map (the copy then delivers zeros)
+    auto item_ok = [&](const int4& x) {
+      return checked(chk_item(x.x, x.y, x.z, x.w, p.B, p.max_items, cap_tokens), &p.hdr->status, kStatusBadItem);
+    };
+    auto table_entry = [&](const int32_t* e) {
+      const int v = *e;
+      return checked(chk_table_entry(v, p.NB), &p.hdr->status, kStatusBadTableEntry) ? v : p.NB;
+    };
+    bool violated = false;
     if (item < n_items) {
       d = p.items[item];
-      const int tb = d.z + lane * p.tile_rows;
-      if (lane < boxes_per_stage && tb < d.w) blk_cur = p.block_table[(size_t)d.x * p.MB + tb / p.bs];
-      if (p.Sq > 1) T_cur = seq_len(d.x);
+      if (item_ok(d)) {
+        const int tb = d.z + lane * p.tile_rows;
+        if (lane < boxes_per_stage && tb < d.w) blk_cur = table_entry(p.block_table + (size_t)d.x * p.MB + tb / p.bs);
+        if (p.Sq > 1) T_cur = seq_len(d.x);
+      }
     }
     bool ok = true;
     while (item < n_items && ok) {
+      if (kChecked && !item_ok(d)) {  // stop the CTA: the consumers leave through the abort flag
+        *s_abort = 1;
+        violated = true;
+        ok = false;
+        break;
+      }
       int nxt = 0;
       if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
       int4 nd = make_int4(0, 0, 0, 0);
@@ -685,7 +746,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         int blk_n = 0;
         {
           const int tb = tok0 + kStageTok + lane * p.tile_rows;
-          if (s + 1 < nstage_item && lane < boxes_per_stage && tb < t1) blk_n = row[tb / p.bs];
+          if (s + 1 < nstage_item && lane < boxes_per_stage && tb < t1) blk_n = table_entry(row + tb / p.bs);
         }
         const int slot = it % nst;
         const uint32_t ph = (uint32_t)(it / nst) & 1u;
@@ -709,12 +770,19 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           mbar_arrive_expect_tx(full, bytes);
         }
         __syncwarp();
+        bool span_ok = true;  // checked build: every copy lands inside its stage (and the q rows inside their slot)
         if (lane < nbox) {
           const int tb = tok0 + lane * p.tile_rows;
           const int c_tok = tb % p.bs;
           const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + lane * box_bytes;
           const uint32_t dv = dk + L::kTileBytes;
-          if (KV8) {  // a token row is one 128-byte swizzle row: one 4-d copy per box
+          span_ok = checked(chk_span(dk, box_bytes, s_stage + (long long)slot * L::kStageBytes,
+                                     s_stage + (long long)slot * L::kStageBytes + L::kTileBytes) &&
+                                chk_span(slot, 1, 0, nst),
+                            &p.hdr->status, kStatusBadSmem);
+          if (!span_ok) {
+            // skipped
+          } else if (KV8) {  // a token row is one 128-byte swizzle row: one 4-d copy per box
             tma_load_4d(dk, &tm_k, full, 0, c_tok, h, blk_cur);
             tma_load_4d(dv, &tm_v, full, 0, c_tok, h, blk_cur);
           } else if (D == 128 && !p.split_halves) {
@@ -728,17 +796,28 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             }
           }
         }
-        if (s == 0 && lane < p.Sq)  // one run of G heads per query token, side by side: [query][head][D]
-          bulk_g2s(s_q + (uint32_t)slot * qslot + (uint32_t)lane * p.G * D * 2,
-                   p.q + (((size_t)b * p.Sq + lane) * p.Hq + (size_t)h * p.G) * D, (uint32_t)p.G * D * 2, full);
+        if (s == 0 && lane < p.Sq) {  // one run of G heads per query token, side by side: [query][head][D]
+          const uint32_t dq = s_q + (uint32_t)slot * qslot + (uint32_t)lane * p.G * D * 2;
+          if (checked(chk_span(dq, (long long)p.G * D * 2, s_q + (long long)slot * qslot, s_q + (long long)(slot + 1) * qslot),
+                      &p.hdr->status, kStatusBadSmem))
+            bulk_g2s(dq, p.q + (((size_t)b * p.Sq + lane) * p.Hq + (size_t)h * p.G) * D, (uint32_t)p.G * D * 2, full);
+          else
+            span_ok = false;
+        }
+        if (kChecked && !__all_sync(0xffffffffu, span_ok)) {  // a skipped copy leaves the stage incomplete: stop
+          *s_abort = 1;
+          violated = true;
+          ok = false;
+          break;
+        }
         // look ahead to the next item: its descriptor, then its first table entries
         if (s == 0) {
           nxt = __shfl_sync(0xffffffffu, nxt, 0);
           if (nxt < n_items) nd = p.items[nxt];
         }
-        if (s == (nstage_item > 1 ? 1 : 0) && nxt < n_items) {
+        if (s == (nstage_item > 1 ? 1 : 0) && nxt < n_items && (!kChecked || item_ok(nd))) {
           const int tb = nd.z + lane * p.tile_rows;
-          if (lane < boxes_per_stage && tb < nd.w) blk_nxt_item = p.block_table[(size_t)nd.x * p.MB + tb / p.bs];
+          if (lane < boxes_per_stage && tb < nd.w) blk_nxt_item = table_entry(p.block_table + (size_t)nd.x * p.MB + tb / p.bs);
           if (p.Sq > 1) T_nxt = seq_len(nd.x);
         }
         blk_cur = blk_n;
@@ -765,7 +844,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
     if (!ok) {
       // stop path: record it, then wait (bounded) until every copy already issued has landed
-      if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+      if (lane == 0 && !violated) atomicOr(&p.hdr->status, kStatusWaitTimeout);
       int dummy_abort = 0;
       const int pending = it < nst ? it : nst;
       for (int k = 0; k < pending; ++k) {
@@ -889,7 +968,10 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (last) {
       // ---- combine the NCW warps' running states (64 dims per pass), then write the item's result
       const int item = meta.x, b = meta.y, h = meta.z;
-      const int n_chunks = p.seq_first[b + 1] - p.seq_first[b];
+      // checked build: the partial slot and the sequence index address the workspace and `out`
+      const bool dst_ok = checked(chk_index(item, p.max_items) && chk_index(b, p.B) && chk_index(h, p.Hkv),
+                                  &p.hdr->status, kStatusBadIndex);
+      const int n_chunks = dst_ok ? p.seq_first[b + 1] - p.seq_first[b] : 1;
       float* mo = g_merge + (size_t)warp * L::kHeads * L::kOStride;
       float* all_m = g_merge + L::kMergeOBytes / 4;
       float lsum[NT][2];
@@ -955,7 +1037,8 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           }
           float o = den > 0.f ? num / den : 0.f;
           if (KV8) o *= p.v_scale;
-          if (n_chunks == 1) {
+          if (kChecked && !dst_ok) continue;
+          if (n_chunks == 1 && !p.out_f32) {
             const int qi = p.Sq > 1 ? col / p.G : 0, head = col - qi * p.G;
             p.out[(((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D + dim] = __float2bfloat16_rn(o);
           } else {
@@ -1012,7 +1095,12 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, co
       first = p.seq_first[b];
       n = p.seq_first[b + 1] - first;
     }
-    const bool work = live && n > 1;  // unsplit (or empty) sequence: the attention kernel wrote the row itself
+    // unsplit (or empty) sequence: the attention kernel wrote the row itself -- except with fp32 output, where
+    // every row is a partial (an unsplit row passes through unchanged: one chunk of weight 1)
+    bool work = live && (n > 1 || (p.out_f32 && n == 1));
+    if (work && !checked(chk_index((long long)(first + n) * p.Hkv - 1, p.max_items) && first >= 0, &p.hdr->status,
+                         kStatusBadIndex))
+      work = false;
     float M = -INFINITY, den = 0.f, acc[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) acc[i] = 0.f;
@@ -1076,11 +1164,16 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const DecodeParams p, co
       __syncthreads();  // the shares are consumed before the next round overwrites them
     }
     if (work && sub == 0) {
-      __nv_bfloat16* dst = p.out + (((size_t)b * p.Sq + qi) * p.Hq + hq) * D + lane * V;
+      const size_t at = (((size_t)b * p.Sq + qi) * p.Hq + hq) * D + lane * V;
       const float inv = den > 0.f ? 1.f / den : 0.f;  // den = 0: the query saw no token at all
+      if (p.out_f32) {
 #pragma unroll
-      for (int i = 0; i < V; i += 2)
-        *reinterpret_cast<__nv_bfloat162*>(dst + i) = __floats2bfloat162_rn(acc[i] * inv, acc[i + 1] * inv);
+        for (int i = 0; i < V; ++i) reinterpret_cast<float*>(p.out)[at + i] = acc[i] * inv;
+      } else {
+#pragma unroll
+        for (int i = 0; i < V; i += 2)
+          *reinterpret_cast<__nv_bfloat162*>(p.out + at + i) = __floats2bfloat162_rn(acc[i] * inv, acc[i + 1] * inv);
+      }
     }
   }
 }

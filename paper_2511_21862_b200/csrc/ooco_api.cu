@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <chrono>
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
@@ -21,14 +22,15 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobOutF32, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}, {0}};
 static std::atomic<int> g_overridden[kKnobCount];  // knob set through ooco_set_tuning
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
 static thread_local int tl_last_launches = 0;
 static thread_local bool tl_events_between_kernels = false;  // profiling: no programmatic overlap
 static thread_local char tl_detail[160] = "";
+static thread_local int64_t tl_host_ns[2] = {0, 0};  // last host-buffer step: host work before the wait, the wait
 
 // Remembers where a CUDA-side failure happened (read back through ooco_last_error_detail).
 static int fail_cuda(const char* where, long code) {
@@ -597,9 +599,28 @@ int ooco_set_tuning(int knob, int value) {
   if (knob == kKnobItemsPerCta && (value < 1 || value > 64)) return OOCO_E_SHAPE;
   if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
   if (knob == kKnobCopyCtasPerSm && (value < 1 || value > 3)) return OOCO_E_SHAPE;
+  if (knob == kKnobOutF32 && value != 0 && value != 1) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
   g_overridden[knob].store(1);
   return OOCO_OK;
+}
+
+int ooco_get_tuning(int knob) {
+  if (knob < 0 || knob >= kKnobCount) return OOCO_E_SHAPE;
+  return g_knobs[knob].load();
+}
+
+int ooco_checked_build(void) { return kChecked ? 1 : 0; }
+
+int ooco_check_predicate(int which, const int64_t* a) {
+  if (!a) return OOCO_E_NULLPTR;
+  switch (which) {
+    case 0: return chk_table_entry(a[0], a[1]) ? 1 : 0;
+    case 1: return chk_index(a[0], a[1]) ? 1 : 0;
+    case 2: return chk_item(a[0], a[1], a[2], a[3], a[4], a[5], a[6]) ? 1 : 0;
+    case 3: return chk_span(a[0], a[1], a[2], a[3]) ? 1 : 0;
+    default: return OOCO_E_SHAPE;
+  }
 }
 
 int ooco_kv_append(const ooco_shape_t* s, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
@@ -717,6 +738,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.D = s->head_dim;
   p.bs = s->block_size;
   p.MB = s->max_blocks_per_seq;
+  p.NB = s->num_blocks;
+  p.out_f32 = g_knobs[kKnobOutF32].load() != 0;
   p.max_items = w.max_items;
   p.tile_rows = s->block_size < stage_tok ? s->block_size : stage_tok;
   p.grid_main = di.sm_count * cps;
@@ -1068,6 +1091,8 @@ int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void*
   if (workspace_bytes < ws_layout(s).total || ((uintptr_t)workspace & 255)) return OOCO_E_WORKSPACE;
   if (!(scale > 0.f) || !(scale <= 3.0e38f)) return OOCO_E_SHAPE;
   if (((uintptr_t)k_cache | (uintptr_t)v_cache) & 15) return OOCO_E_UNSUPPORTED;
+  if (g_knobs[kKnobOutF32].load()) return OOCO_E_UNSUPPORTED;  // the staging and the host result are sized for bf16
+  const auto t_enter = std::chrono::steady_clock::now();
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const size_t qb = (size_t)s->batch * s->num_q_heads * s->head_dim * 2;
@@ -1124,7 +1149,18 @@ int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void*
   }
   if (!out_mapped && cudaMemcpyAsync(out_host, d_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return fail_cuda("cudaMemcpyAsync(device to host)", -1);
+  const auto t_enqueued = std::chrono::steady_clock::now();
   if (cudaStreamSynchronize(st) != cudaSuccess) return fail_cuda("cudaStreamSynchronize", -1);
+  const auto t_done = std::chrono::steady_clock::now();
+  tl_host_ns[0] = std::chrono::duration_cast<std::chrono::nanoseconds>(t_enqueued - t_enter).count();
+  tl_host_ns[1] = std::chrono::duration_cast<std::chrono::nanoseconds>(t_done - t_enqueued).count();
+  return OOCO_OK;
+}
+
+int ooco_last_host_step_ns(int64_t* enqueue_ns, int64_t* wait_ns) {
+  if (!enqueue_ns || !wait_ns) return OOCO_E_NULLPTR;
+  *enqueue_ns = tl_host_ns[0];
+  *wait_ns = tl_host_ns[1];
   return OOCO_OK;
 }
 

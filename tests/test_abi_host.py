@@ -149,7 +149,7 @@ def test_query_length_limits_and_workspace_growth_without_a_device():
     assert attn(8193) == -3 and attn(0) == -2
     assert attn(64, q=odd) == -3 and attn(64, out=odd) == -3
     assert attn(64, ws_bytes=binding.workspace_bytes_mq(sh, 4)) == -4
-    assert L.ooco_set_tuning(11, 0) == 0 and L.ooco_set_tuning(11, 1) == 0 and L.ooco_set_tuning(12, 1) == 0 and L.ooco_set_tuning(13, 1) == -2
+    assert L.ooco_set_tuning(11, 0) == 0 and L.ooco_set_tuning(11, 1) == 0 and L.ooco_set_tuning(12, 1) == 0 and L.ooco_set_tuning(14, 1) == -2
 
 
 def test_missing_library_fails_loudly(monkeypatch):
@@ -196,3 +196,43 @@ def test_attention_bytes_model_with_several_query_tokens():
         assert got["bytes_q"] == got["bytes_out"] == d * Sq * Hq * D * len(lens)
         if Sq == 1:
             assert got == binding.decode_bytes_model(sh, torch.from_numpy(lens), d)
+
+
+def test_range_predicates_of_the_checked_build():
+    """The predicates the checked build guards its accesses with, evaluated on the host: each accepts the
+    whole legal range and refuses the first value on either side of it."""
+    P = binding.check_predicate
+    NB = 1000
+    assert P(0, 0, NB) and P(0, NB - 1, NB)
+    assert not P(0, -1, NB) and not P(0, NB, NB) and not P(0, 2**31 - 1, NB) and not P(0, -7, NB)
+    assert P(1, 0, 5) and P(1, 4, 5) and not P(1, 5, 5) and not P(1, -1, 5) and not P(1, 0, 0)
+    # work item {sequence, slot, t0, t1, B, max_items, capacity in tokens}
+    ok = (3, 17, 64, 128, 4, 18, 128)
+    assert P(2, *ok)
+    assert P(2, 0, 0, 0, 0, 4, 18, 128)                                            # an empty chunk at the start is in range
+    for i, bad in ((0, -1), (0, 4), (1, -1), (1, 18), (2, -64), (2, 192), (3, 63), (3, 129)):
+        args = list(ok)
+        args[i] = bad
+        assert not P(2, *args), (i, bad)
+    # span {offset, bytes, lo, hi}: [offset, offset + bytes) inside [lo, hi)
+    assert P(3, 1024, 4096, 1024, 5120) and P(3, 1024, 0, 1024, 1024)
+    assert not P(3, 1023, 16, 1024, 5120) and not P(3, 5105, 16, 1024, 5120) and not P(3, 2048, -16, 1024, 5120)
+    with pytest.raises(binding.OocoError):
+        P(9, 0, 0)
+    assert binding.checked_build() is False
+
+
+def test_fp32_output_knob_is_a_switch():
+    assert binding.get_tuning("out_f32") == 0
+    L = binding.lib()
+    assert L.ooco_set_tuning(13, 2) == -2 and L.ooco_set_tuning(14, 1) == -2 and L.ooco_get_tuning(99) == -2
+    binding.set_tuning(out_f32=1)
+    try:
+        assert binding.get_tuning("out_f32") == 1
+        good = binding.Shape(2, 8, 2, 64, 16, 8, 4, 2 * 16 * 64, 16 * 64, 64)
+        one = ctypes.c_void_p(256)
+        # the host-buffer step has no fp32 result buffer: refused before anything is enqueued
+        assert L.ooco_decode_step_host(ctypes.byref(good.c()), one, one, one, one, one, one, one, one, 1.0, one,
+                                       one, 1 << 40, one, 1 << 40, None) == -3
+    finally:
+        binding.set_tuning(out_f32=0)

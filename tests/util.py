@@ -9,6 +9,28 @@ MAX_ABS_TOL = 1e-2    # bf16 in / fp32 accumulate / bf16 out vs the fp64 oracle:
 MEAN_ABS_TOL = 1e-3   # and mean |err|, over all B * Hq * D outputs
 
 
+import contextlib
+
+
+@contextlib.contextmanager
+def fp32_output():
+    """The library's diagnostic output mode: `out` tensors are fp32 and hold the values before the bf16 rounding."""
+    binding.set_tuning(out_f32=1)
+    try:
+        yield
+    finally:
+        binding.set_tuning(out_f32=0)
+
+
+def assert_parity_and_rounding(out_bf16: torch.Tensor, out_f32: torch.Tensor, ref: np.ndarray, what=""):
+    """The stated tolerance on the fp32 output (no allowance for the output format), and the bf16 output must be
+    exactly the fp32 output rounded to nearest even: together they hold the bf16 path to the same arithmetic."""
+    mx, mean = assert_parity(out_f32, ref, what=what + " (fp32 out)")
+    want = out_f32.to(torch.bfloat16)
+    assert torch.equal(out_bf16.view(torch.int16), want.view(torch.int16)), f"{what}: bf16 out is not round(fp32 out)"
+    return mx, mean
+
+
 def bf16_to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().to(torch.float64).numpy()
 
