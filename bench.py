@@ -588,6 +588,10 @@ def run_multi_query(args, local_rank):
     cfg = inputs.replace(base, groups=tuple(inputs.replace(g, lo=g.lo + Sq, hi=g.hi + Sq) if g.dist != "fixed" else g
                                             for g in base.groups))
     batch = inputs.make_batch(cfg, dev, poison=False)
+    fp8 = args.kv == "fp8"
+    KS = VS = 1.0 / 32
+    if fp8:
+        batch = inputs.to_e4m3_pool(batch, KS, VS, poison=False)
     sh = binding.shape_of(batch)
     B = sh.batch
     gen = torch.Generator(device=dev).manual_seed(cfg.seed + 7)
@@ -597,8 +601,11 @@ def run_multi_query(args, local_rank):
     positions = (batch.context_lens - Sq).contiguous()                   # the new tokens are the last q_len of each context
     lens_host = batch.context_lens.cpu().contiguous()
     cost = binding.attention_bytes_model(sh, Sq, lens_host)                     # table row with S_q = q_len
+    if fp8:                                                                     # K / V stored with d = 1
+        cost = dict(cost, bytes_kv=cost["bytes_kv"] // 2)
+        cost["bytes_paper"] = cost["bytes_q"] + cost["bytes_out"] + cost["bytes_kv"]
     nbytes = cost["bytes_paper"]
-    pool_bytes = 2 * batch.k_cache.numel() * 2
+    pool_bytes = 2 * batch.k_cache.numel() * batch.k_cache.element_size()
     free, _ = torch.cuda.mem_get_info(dev)
     R = replica_count(pool_bytes, free)
     pools = [(batch.k_cache, batch.v_cache)] + [(batch.k_cache.clone(), batch.v_cache.clone()) for _ in range(R - 1)]
@@ -607,8 +614,12 @@ def run_multi_query(args, local_rank):
 
     def step(i):
         k, v = pools[i % R]
-        binding.decode_step_mq(sh, q, k_new, v_new, k, v, batch.block_table, positions, batch.context_lens, cfg.scale,
-                               out, ws, stream)
+        if fp8:
+            binding.decode_step_mq_fp8(sh, q, k_new, v_new, k, v, batch.block_table, positions, batch.context_lens,
+                                       cfg.scale, KS, VS, out, ws, stream)
+        else:
+            binding.decode_step_mq(sh, q, k_new, v_new, k, v, batch.block_table, positions, batch.context_lens,
+                                   cfg.scale, out, ws, stream)
     sampler = ClockSampler(local_rank)
     sampler.start()
     for i in range(args.warmup):
@@ -634,7 +645,8 @@ def run_multi_query(args, local_rank):
     peak, peak_kind = measured_peak()
     achieved = nbytes / (attn * 1e-3) / 1e9
     columns = Sq * (cfg.num_q_heads // cfg.num_kv_heads)
-    tcgen05 = columns > 32 and cfg.head_dim == 128 and not any(k.startswith("chunk_tcgen05=0") for k in args.knob)
+    tcgen05 = (columns > 32 and cfg.head_dim == 128 and not any(k.startswith("chunk_tcgen05=0") for k in args.knob)) or \
+              (fp8 and columns > 16)
     kernel = ("chunk_tc_kernel" if tcgen05 else "chunk_main_kernel") if columns > 16 else (
         "row16_main_kernel" if columns > 8 else "decode_main_kernel")
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -649,10 +661,10 @@ def run_multi_query(args, local_rank):
                     "algorithmic_flops_per_launch": cost["flops"], "traffic": None,
                     "note": "flops as the operator table prints them (no causal discount)"}
     print(json.dumps({
-        "metric": METRIC + f" ({Sq} query tokens per sequence)", "value": nbytes / (ms * 1e-3) / 1e12, "unit": "TB/s",
+        "metric": METRIC + f" ({Sq} query tokens per sequence" + (", 8-bit E4M3 KV cache)" if fp8 else ")"), "value": nbytes / (ms * 1e-3) / 1e12, "unit": "TB/s",
         "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}, {Sq} query tokens per sequence", "batch": B,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16 (e4m3 codes widened)" if fp8 else "bf16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}, {Sq} query tokens per sequence" + (", 8-bit cache" if fp8 else ""), "batch": B,
                    "total_tokens": cost["total_tokens"], "step": "ooco_decode_step_mq, one layer",
                    "l2": f"inputs larger than L2: steps rotate over {R} pool replicas"},
         "query_tokens_per_s": B * Sq / (ms * 1e-3),

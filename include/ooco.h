@@ -197,8 +197,9 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  * up to 128, reads the cache once per row tile (the repeats hit L2) and never loads tokens a tile
  * cannot see; it becomes bound by the tensor pipe from about 64 columns on.  At head_dim 128 and
  * more than 32 columns that kernel runs on tcgen05 (scores and output in tensor memory), otherwise
- * on mma.sync.  The 8-bit cache
- * (ooco_decode_step_mq_fp8) has the decode kernel only.  The workspace grows with q_len: one fp32
+ * on mma.sync.  Over the 8-bit cache
+ * (ooco_decode_step_mq_fp8) every chunk of more than 16 columns runs the tcgen05 kernel, whose extra
+ * warps widen each 8-bit stage to f16 in shared memory first.  The workspace grows with q_len: one fp32
  * partial row per (split item, score column).  q_len = 1 is ooco_decode_attention /
  * ooco_kv_append exactly.  Everything else as for those two.
  */
@@ -251,7 +252,9 @@ int ooco_decode_step_fp8(const ooco_shape_t* shape, const void* q, const void* k
  * Both variants at once: q_len query tokens per sequence over an 8-bit cache.  With k_new and v_new
  * (bf16 [B, q_len, Hkv, head_dim]) the quantising append of the q_len new tokens at positions[b] + i
  * is fused into the first launch, as in ooco_decode_step_mq; with both NULL (positions may be NULL
- * too) only the attention runs.  Restrictions: those of the two variants together.
+ * too) only the attention runs.  Restrictions: those of the two variants together (head_dim 128,
+ * 1 <= q_len <= 8192); codes are widened exactly to f16, q and the softmax weights are rounded to
+ * f16, accumulation is fp32 -- for every q_len.
  */
 int ooco_decode_step_mq_fp8(const ooco_shape_t* shape, int32_t q_len, const void* q, const void* k_new,
                             const void* v_new, void* k_cache, void* v_cache, const int32_t* block_table,

@@ -144,12 +144,18 @@ __device__ __forceinline__ void chunk_consume(uint32_t kst, uint32_t vst, const 
 // The producer warp of both kernels below: walks its units of work (item, row tile of RT score columns),
 // streams the K / V stages of each through TMA and describes every stage in two int4 of `g_meta`:
 //   {partial slot, sequence, kv head, tokens | first << 16 | last << 17}  {first token, T - S_q + 1, chunk end, row tile}
-template <int D>
+// KV8: the caches hold 8-bit codes; a stage is [64 tok][D bytes] of K, then of V (one 128-byte row per token at
+// head_dim 128, one copy per box), for a consumer that widens it before use.
+template <int D, bool KV8 = false>
 __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const DecodeParams& p,
                                               const int RT, const int nst, const uint32_t s_stage,
                                               const uint32_t s_full, const uint32_t s_empty, int4* g_meta,
                                               volatile int* s_abort, const int lane) {
   using L = ChunkSmem<D>;
+  static_assert(!KV8 || D == 128, "the 8-bit stage layout is one 128-byte row per token");
+  constexpr uint32_t kStageBytesP = KV8 ? 2u * kChunkStageTok * D : (uint32_t)L::kStageBytes;
+  constexpr uint32_t kTileBytesP = KV8 ? (uint32_t)kChunkStageTok * D : (uint32_t)L::kTileBytes;
+  constexpr uint32_t kCopiesPerBox = KV8 ? 1u : (uint32_t)(D / 64);
   const int nrt = (p.GQ + RT - 1) / RT;
   const long long n_units = (long long)p.hdr->n_items * nrt;
   // ================================================================= producer warp
@@ -232,21 +238,24 @@ __device__ __forceinline__ void chunk_produce(const CUtensorMap& tm_k, const CUt
         const int flags = (s == 0 ? 1 : 0) | (s == nstage - 1 ? 2 : 0);
         g_meta[2 * slot] = make_int4(d.y, b, h, ntok | (flags << 16));
         g_meta[2 * slot + 1] = make_int4(tok0, lim_base, t1, rt);
-        mbar_arrive_expect_tx(full, 2u * (uint32_t)nbox * box_rows_bytes * (D / 64));
+        mbar_arrive_expect_tx(full, 2u * (uint32_t)nbox * box_rows_bytes * kCopiesPerBox);
       }
       __syncwarp();
       bool span_ok = true;
       if (lane < nbox) {
         const int tb = tok0 + lane * p.tile_rows;
         const int c_tok = tb % p.bs;
-        const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + (uint32_t)lane * box_rows_bytes;
-        const uint32_t dv = dk + L::kTileBytes;
+        const uint32_t dk = s_stage + (uint32_t)slot * kStageBytesP + (uint32_t)lane * box_rows_bytes;
+        const uint32_t dv = dk + kTileBytesP;
         // checked build: the box lands inside the first 64-dim half of the stage's K tile (the others follow it)
-        span_ok = checked(chk_span(dk, box_rows_bytes, s_stage + (long long)slot * L::kStageBytes,
-                                   s_stage + (long long)slot * L::kStageBytes + L::kHalfBytes) &&
+        span_ok = checked(chk_span(dk, box_rows_bytes, s_stage + (long long)slot * kStageBytesP,
+                                   s_stage + (long long)slot * kStageBytesP + L::kHalfBytes) &&
                               chk_span(slot, 1, 0, nst),
                           &p.hdr->status, kStatusBadSmem);
-        if (span_ok) {
+        if (span_ok && KV8) {
+          tma_load_4d(dk, &tm_k, full, 0, c_tok, h, blk_cur);
+          tma_load_4d(dv, &tm_v, full, 0, c_tok, h, blk_cur);
+        } else if (span_ok) {
 #pragma unroll
           for (int j = 0; j < D / 64; ++j) {
             tma_load_4d(dk + j * L::kHalfBytes, &tm_k, full, 64 * j, c_tok, h, blk_cur);

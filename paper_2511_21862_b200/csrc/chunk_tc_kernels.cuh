@@ -15,6 +15,13 @@
 //               happens a few times per unit instead of once per stage), stores the bf16 weights as its P
 //               row, and at the end of the unit normalises its O row and writes it.
 // Every wait is bounded; on a wait that gives up the CTA stops issuing, drains and releases the tensor memory.
+//
+// KV8 (the caches hold E4M3 codes): the producer's TMA copies land the 8-bit stages ([64 tok][128 B] of K, then of
+// V) in a ring of their own, and two more warps (6, 7) widen every stage into the 16-bit stage layout above --
+// exactly, to f16 holding value / 256 (e4m3x2_to_f16x2; the factor goes into the softmax scale and the output
+// scale) -- so both contractions run unchanged as kind::f16 MMAs with f16 operands (Q and P are rounded to f16, as
+// in the 8-bit decode kernel).  The widening costs integer work on warps that do nothing else; the tensor pipe,
+// not HBM, bounds this kernel, so the halved cache bytes buy capacity, not time.
 #pragma once
 #include "chunk_kernels.cuh"
 
@@ -25,30 +32,38 @@ constexpr int kTcTmemCols = 256;    // allocated columns (a power of two)
 constexpr int kTcColS = 0, kTcColO = 64, kTcColQ = 192;
 constexpr float kTcRescaleStep = 8.f;
 
+constexpr int kTcRawStageBytes = 2 * kChunkStageTok * 128;  // 8-bit cache: K, then V, one 128-byte row per token
 struct ChunkTcSmem {
-  __host__ __device__ static size_t total(int nstages) {
-    return 1024 + (size_t)nstages * (ChunkSmem<128>::kStageBytes + 32 + 16) + 128;
+  __host__ __device__ static size_t total(int nstages, int nraw = 0) {
+    return 1024 + (size_t)nstages * (ChunkSmem<128>::kStageBytes + 32 + 16) + (size_t)nraw * (kTcRawStageBytes + 32 + 16) +
+           128;
   }
 };
 
 // Barrier bookkeeping.  Barriers that come in pairs ([2]) are used alternately by consecutive stages, and use
 // number n of a pair takes barrier n & 1 with phase parity (n >> 1) & 1: a waiter can then never be overtaken
 // by two completions of the barrier it waits on (the completion after next needs the waiter's own progress).
-__global__ void __launch_bounds__(192, 2)
+template <bool KV8>
+__global__ void __launch_bounds__(KV8 ? 256 : 192, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                 const DecodeParams p) {
   constexpr int D = 128;
+  constexpr int kConvThreads = 64;  // KV8: warps 6 and 7
   using L = ChunkSmem<D>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
-  const int nst = p.nstages;
+  const int nst = p.nstages, nraw = KV8 ? p.nstages_raw : 0;
   const uint32_t s_stage = base;
-  const uint32_t s_meta = s_stage + (uint32_t)nst * L::kStageBytes;
-  const uint32_t s_full = s_meta + (uint32_t)nst * 32;
+  const uint32_t s_rstage = s_stage + (uint32_t)nst * L::kStageBytes;  // KV8: ring of 8-bit stages (1024-byte aligned)
+  const uint32_t s_meta = s_rstage + (uint32_t)nraw * kTcRawStageBytes;
+  const uint32_t s_rmeta = s_meta + (uint32_t)nst * 32;
+  const uint32_t s_full = s_rmeta + (uint32_t)nraw * 32;
   const uint32_t s_empty = s_full + (uint32_t)nst * 8;
-  const uint32_t s_sready = s_empty + (uint32_t)nst * 8;  // [2] S buffer holds the stage's scores       (MMA commit)
+  const uint32_t s_rfull = s_empty + (uint32_t)nst * 8;   // KV8: the 8-bit stage has landed                (TMA)
+  const uint32_t s_rempty = s_rfull + (uint32_t)nraw * 8;  // KV8: the 8-bit stage has been widened         (64 threads)
+  const uint32_t s_sready = s_rempty + (uint32_t)nraw * 8;  // [2] S buffer holds the stage's scores       (MMA commit)
   const uint32_t s_sfree = s_sready + 16;                 // [2] S buffer has been read into registers  (128 softmax threads)
   const uint32_t s_pready = s_sfree + 16;                 // [2] meta words consumed, P written         (128 softmax threads)
   const uint32_t s_pvdone = s_pready + 16;                // [2] the stage's P.V is complete            (MMA commit)
@@ -56,6 +71,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   const uint32_t s_drain = s_qready + 8;
   const uint32_t s_slot = s_drain + 8;
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
+  int4* g_rmeta = reinterpret_cast<int4*>(gen + (s_rmeta - base));
   volatile uint32_t* g_slot = reinterpret_cast<volatile uint32_t*>(gen + (s_slot - base));
   volatile int* s_abort = reinterpret_cast<volatile int*>(gen + (s_slot + 4 - base));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -63,8 +79,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   if (threadIdx.x == 0) {
     *s_abort = 0;
     for (int i = 0; i < nst; ++i) {
-      mbar_init(s_full + 8 * i, 1);
+      mbar_init(s_full + 8 * i, KV8 ? kConvThreads : 1);  // KV8: filled by the widening threads, not by TMA
       mbar_init(s_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < nraw; ++i) {
+      mbar_init(s_rfull + 8 * i, 1);
+      mbar_init(s_rempty + 8 * i, kConvThreads);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(s_sready + 8 * i, 1);
@@ -85,11 +105,59 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   grid_dep_launch();  // the merge kernel may queue up behind this grid
 
   if (warp == 4) {
-    chunk_produce<D>(tm_k, tm_v, p, kTcRows, nst, s_stage, s_full, s_empty, g_meta, s_abort, lane);
+    if (KV8)
+      chunk_produce<D, true>(tm_k, tm_v, p, kTcRows, nraw, s_rstage, s_rfull, s_rempty, g_rmeta, s_abort, lane);
+    else
+      chunk_produce<D>(tm_k, tm_v, p, kTcRows, nst, s_stage, s_full, s_empty, g_meta, s_abort, lane);
+  } else if (KV8 && warp >= 6) {
+    // ================================================================= widening warps (8-bit cache only)
+    // Stage number `it` of the 8-bit ring becomes stage number `it` of the 16-bit ring (bookkeeping stages and
+    // the end marker included).  A unit of work is (tile K / V, token row r, 16-byte chunk c of the row's 128
+    // codes): one 16-byte load, sixteen codes widened, two 16-byte stores into the row's 64-dim half c / 4.
+    const int ctid = threadIdx.x - 192;
+    bool ok = true;
+    for (int it = 0;; ++it) {
+      const int rs = it % nraw, slot = it % nst;
+      if (!warp_wait(s_rfull + 8 * rs, (uint32_t)(it / nraw) & 1u, s_abort) ||
+          !warp_wait(s_empty + 8 * slot, ((uint32_t)(it / nst) & 1u) ^ 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      const int4 meta = g_rmeta[2 * rs], meta2 = g_rmeta[2 * rs + 1];
+      const int ntok = meta.x < 0 ? 0 : (meta.w & 0xffff);
+      if (ntok > 0) {
+        const uint8_t* rsrc = gen + (s_rstage - base) + (size_t)rs * kTcRawStageBytes;
+        uint8_t* sdst = gen + (size_t)slot * L::kStageBytes;
+#pragma unroll 4
+        for (int i = 0; i < 2 * kChunkStageTok * 8 / kConvThreads; ++i) {
+          const int u = i * kConvThreads + ctid;
+          const int tile = u >> 9, r = (u >> 3) & 63, c = u & 7;
+          if (r >= ntok) continue;  // rows beyond the stage's tokens are never used (masked scores, cleared V rows)
+          const uint4 w = *reinterpret_cast<const uint4*>(rsrc + (size_t)tile * (kTcRawStageBytes / 2) + (size_t)r * 128 +
+                                                          ((c ^ (r & 7)) << 4));
+          uint8_t* drow = sdst + (size_t)tile * L::kTileBytes + (size_t)(c >> 2) * L::kHalfBytes + (size_t)r * 128;
+          *reinterpret_cast<uint4*>(drow + (((2 * (c & 3)) ^ (r & 7)) << 4)) =
+              make_uint4(e4m3x2_to_f16x2<kSelB0B1>(w.x), e4m3x2_to_f16x2<kSelB2B3>(w.x), e4m3x2_to_f16x2<kSelB0B1>(w.y),
+                         e4m3x2_to_f16x2<kSelB2B3>(w.y));
+          *reinterpret_cast<uint4*>(drow + (((2 * (c & 3) + 1) ^ (r & 7)) << 4)) =
+              make_uint4(e4m3x2_to_f16x2<kSelB0B1>(w.z), e4m3x2_to_f16x2<kSelB2B3>(w.z), e4m3x2_to_f16x2<kSelB0B1>(w.w),
+                         e4m3x2_to_f16x2<kSelB2B3>(w.w));
+        }
+      }
+      if (ctid == 0) {
+        g_meta[2 * slot] = meta;
+        g_meta[2 * slot + 1] = meta2;
+      }
+      fence_proxy_async_smem();  // the widened stage is read by the MMAs through the async proxy
+      mbar_arrive(s_full + 8 * slot);
+      mbar_arrive(s_rempty + 8 * rs);
+      if (meta.x < 0) break;
+    }
+    if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
   } else if (warp == 5) {
     // ================================================================= MMA warp
-    const uint32_t idesc_s = umma_idesc_bf16(kTcRows, kChunkStageTok, 0);
-    const uint32_t idesc_o = umma_idesc_bf16(kTcRows, D, 1);
+    const uint32_t idesc_s = umma_idesc_16bit(kTcRows, kChunkStageTok, 0, !KV8);
+    const uint32_t idesc_o = umma_idesc_16bit(kTcRows, D, 1, !KV8);
     uint32_t ph_q = 0, full_phase = 1u;
     uint32_t n_s = 0, n_p = 0, n_pv = 0;  // score MMAs issued, stages handed over by the softmax threads, P.V issued
     int slot = -1;
@@ -220,10 +288,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
               const uint4 v = real_row ? src[8 * half + c] : make_uint4(0u, 0u, 0u, 0u);
-              qw[4 * c] = v.x;
-              qw[4 * c + 1] = v.y;
-              qw[4 * c + 2] = v.z;
-              qw[4 * c + 3] = v.w;
+              qw[4 * c] = KV8 ? bf16x2_to_f16x2(v.x) : v.x;  // the widened codes are f16: so is the query
+              qw[4 * c + 1] = KV8 ? bf16x2_to_f16x2(v.y) : v.y;
+              qw[4 * c + 2] = KV8 ? bf16x2_to_f16x2(v.z) : v.z;
+              qw[4 * c + 3] = KV8 ? bf16x2_to_f16x2(v.w) : v.w;
             }
             tmem_st32(trow + kTcColQ + 32 * half, qw);
           }
@@ -298,7 +366,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
                                  scale2, neg_mu2);
           const float2 w = make_float2(ex2(x.x), ex2(x.y));
           add4[i & 3] = fadd2(add4[i & 3], w);
-          pw[i] = pack_bf16x2(w.x, w.y);
+          pw[i] = KV8 ? pack_f16x2(w.x, w.y) : pack_bf16x2(w.x, w.y);
         }
         {
           const float2 a01 = fadd2(add4[0], add4[1]), a23 = fadd2(add4[2], add4[3]);
@@ -335,7 +403,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
           }
           tc_fence_after_sync();
         }
-        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // l = 0: the row saw no token of this chunk
+        // l = 0: the row saw no token of this chunk; the 8-bit cache's V scale (and widening factor) comes in here
+        const float inv = (l_run > 0.f ? 1.f / l_run : 0.f) * (KV8 ? p.v_scale : 1.f);
         __nv_bfloat16* orow = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D;
         float* prow_o = p.part_o + ((size_t)slot_id * p.GQ + col) * D;
 #pragma unroll 1

@@ -87,6 +87,7 @@ struct DecodeParams {
   int32_t tile_rows;      // token rows per TMA box = min(bs, stage tokens)
   int32_t split_halves;   // 1: one 4-d TMA per 64-dim half; 0: one 5-d TMA per box
   int32_t nstages;
+  int32_t nstages_raw;    // 8-bit prefill-chunk kernel: stages of its ring of 8-bit copies
   int32_t grid_main;      // CTAs the plan sizes the chunks for
   int32_t next_item_init; // start of the dynamic work counter = CTAs of the attention grid (they take the first units statically)
   int32_t chunk_min, chunk_max, items_per_cta;

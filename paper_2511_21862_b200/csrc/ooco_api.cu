@@ -318,9 +318,10 @@ static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
 
 // Prefill chunk on tcgen05 (head_dim 128, more than 32 score columns: from there on it beats the mma.sync
 // kernel on every workload measured, a half-empty 128-row tile included): two CTAs per SM.
+template <bool KV8>
 static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                            int ctas_per_sm, cudaStream_t st, int dev, bool dry) {
-  auto kern = chunk_tc_kernel;
+  auto kern = chunk_tc_kernel<KV8>;
   static std::atomic<int> static_smem{-1};
   if (static_smem.load() < 0) {
     cudaFuncAttributes fa;
@@ -331,11 +332,14 @@ static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeP
   const size_t dyn_max = (size_t)di.smem_optin - (size_t)static_smem.load();
   const size_t budget = ctas_per_sm > 1 ? ((size_t)di.smem_optin + 1024) / ctas_per_sm - 1024 - static_smem.load()
                                         : dyn_max;
-  int nst = 6;
-  while (nst > 2 && ChunkTcSmem::total(nst) > budget) --nst;
-  if (ChunkTcSmem::total(nst) > dyn_max) return OOCO_E_UNSUPPORTED;
+  // 8-bit cache: two 16-bit stages (the MMAs' double buffer) and as many 8-bit stages as fit beside them
+  int nst = KV8 ? 2 : 6, nraw = KV8 ? 4 : 0;
+  while (!KV8 && nst > 2 && ChunkTcSmem::total(nst) > budget) --nst;
+  while (KV8 && nraw > 2 && ChunkTcSmem::total(nst, nraw) > budget) --nraw;
+  if (ChunkTcSmem::total(nst, nraw) > dyn_max) return OOCO_E_UNSUPPORTED;
   p.nstages = nst;
-  const size_t smem = ChunkTcSmem::total(nst);
+  p.nstages_raw = nraw;
+  const size_t smem = ChunkTcSmem::total(nst, nraw);
   static std::atomic<size_t> configured[64];
   if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max);
@@ -343,7 +347,7 @@ static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeP
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
   if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
-  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(192), smem, st,
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(KV8 ? 256 : 192), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the tcgen05 chunk attention kernel", (long)e);
@@ -648,8 +652,8 @@ static int validate_q_len(const ooco_shape_t* s, int q_len, bool kv8 = false) {
   if (q_len < 1) return OOCO_E_SHAPE;
   if (q_len == 1) return OOCO_OK;
   if (q_len > kMaxQLen) return OOCO_E_UNSUPPORTED;
-  // the 8-bit cache has the decode kernel only
-  if (kv8 && (long long)(s->num_q_heads / s->num_kv_heads) * q_len > kDecodeMaxColumns) return OOCO_E_UNSUPPORTED;
+  (void)s;
+  (void)kv8;  // the 8-bit cache runs the decode kernel up to 16 score columns and the tcgen05 chunk kernel beyond
   return OOCO_OK;
 }
 
@@ -707,7 +711,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // 9 .. 16 columns: the row layout with the tokens of a stage split over 4 warps x 2 CTAs per SM (the
   // column layout of the decode kernel needs a second MMA tile and a transposition per tile there)
   const bool row16 = !chunk && !kv8 && G_ > 8 && g_knobs[kKnobRowLayout16].load() != 0;
-  const bool chunk_tc = chunk && G_ > 32 && s->head_dim == 128 && g_knobs[kKnobChunkTcgen05].load() != 0;
+  // (the 8-bit cache has no mma.sync chunk kernel: every chunk over it runs the tcgen05 kernel)
+  const bool chunk_tc = chunk && s->head_dim == 128 && (kv8 || (G_ > 32 && g_knobs[kKnobChunkTcgen05].load() != 0));
   if (chunk) {
     ncw = chunk_warps(G_);
     cps = (ncw == 8 && !chunk_tc) ? 1 : 2;
@@ -772,7 +777,9 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // once without launching, before the first kernel of the call is enqueued.
   const int stages = g_knobs[kKnobStages].load();
   auto launch_attention = [&](bool dry) -> int {
-    if (chunk_tc) return launch_chunk_tc(tk, tv, p, di, cps, st, dev, dry);
+    if (chunk_tc)
+      return kv8 ? launch_chunk_tc<true>(tk, tv, p, di, cps, st, dev, dry)
+                 : launch_chunk_tc<false>(tk, tv, p, di, cps, st, dev, dry);
     if (chunk)
       return s->head_dim == 128 ? launch_chunk_ncw<128>(ncw, tk, tv, p, di, cps, st, dev, dry)
                                 : launch_chunk_ncw<64>(ncw, tk, tv, p, di, cps, st, dev, dry);

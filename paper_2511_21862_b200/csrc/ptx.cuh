@@ -178,6 +178,12 @@ __device__ __forceinline__ float lg2(float x) {
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Packed bf16x2 -> packed f16x2 (round to nearest even; exact for magnitudes the f16 range holds).
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(w & 0xffff0000u)), "f"(__uint_as_float(w << 16)));
+  return d;
+}
 // Two fp32 -> packed bf16x2 (round to nearest even); `lo` lands in the low half.
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t d;
@@ -201,11 +207,15 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr, uint32_t lbo_
   d |= (uint64_t)2 << 61;  // 128-byte swizzle
   return d;
 }
-// Instruction descriptor of kind::f16 with bf16 A and B (the same type, as the instruction requires), fp32 D,
-// A K-major, B K-major or MN-major, D = M x N.
-__device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N, int b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
+// Instruction descriptor of kind::f16 with A and B both f16 or both bf16 (the same type, as the instruction
+// requires), fp32 D, A K-major, B K-major or MN-major, D = M x N.
+__device__ __forceinline__ uint32_t umma_idesc_16bit(int M, int N, int b_mn_major, bool bf16) {
+  const uint32_t fmt = bf16 ? 1u : 0u;  // A and B format: 0 = f16, 1 = bf16
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
          ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N, int b_mn_major) {
+  return umma_idesc_16bit(M, N, b_mn_major, true);
 }
 // D[tmem] (+)= A[smem] x B[smem]; issued by ONE thread; completion is observed through umma_commit.
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {

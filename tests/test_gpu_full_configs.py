@@ -127,3 +127,26 @@ def test_prefill_chunk_full_size_every_output(Sq):
     assert ref.out.shape == (B, Sq, Hq, D)
     mx, mean = assert_parity(out.reshape(-1, Hq, D), ref.out.reshape(-1, Hq, D), what=f"cfg1 + chunk of {Sq}")
     print(f"cfg1 with {Sq} query tokens, all {ref.out.size} outputs: max abs {mx:.3e} mean abs {mean:.3e}")
+
+
+def test_prefill_chunk_over_8bit_cache_full_size_every_output():
+    """cfg1 with a 64-token chunk per sequence over E4M3 caches (256 score columns: two row tiles of the tcgen05
+    kernel, stages widened in shared memory), every output against the 8-bit oracle."""
+    Sq, ks, vs = 64, 1.0 / 32, 1.0 / 32
+    base = inputs.CONFIGS["cfg1"]
+    cfg = inputs.replace(base, groups=tuple(inputs.replace(g, lo=g.lo + Sq, hi=g.hi + Sq) for g in base.groups))
+    batch = inputs.to_e4m3_pool(inputs.make_batch(cfg, "cuda", poison=True), ks, vs)
+    B, Hq, D, bs = cfg.batch, cfg.num_q_heads, cfg.head_dim, cfg.block_size
+    gen = torch.Generator(device="cuda").manual_seed(78)
+    q = torch.randn((B, Sq, Hq, D), generator=gen, device="cuda").to(torch.bfloat16)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_step_mq_fp8(sh, q, None, None, batch.k_cache, batch.v_cache, batch.block_table, None,
+                               batch.context_lens, cfg.scale, ks, vs, out, ws)
+    assert binding.workspace_status(ws) == 0
+    ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), inputs.as_u8(batch.k_cache), inputs.as_u8(batch.v_cache),
+                                         batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                         ks, vs, num_kv_heads=cfg.num_kv_heads, block_size=bs, strides=batch.strides)
+    mx, mean = assert_parity(out.reshape(-1, Hq, D), ref.out.reshape(-1, Hq, D), what="cfg1 + chunk of 64, 8-bit cache")
+    print(f"cfg1 with 64 query tokens over an 8-bit cache, all {ref.out.size} outputs: max abs {mx:.3e} mean abs {mean:.3e}")

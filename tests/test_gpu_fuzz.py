@@ -142,10 +142,11 @@ def draw_chunk_case(seed):
 @pytest.mark.parametrize("seed", range(32))
 def test_random_chunk_case(seed):
     cfg, Sq = draw_chunk_case(seed)
-    batch, q, out = run_case(cfg, "mq", Sq, seed, torch.bfloat16)
+    mode = "mq8" if cfg.head_dim == 128 and seed % 3 == 1 else "mq"          # a third of the head_dim-128 chunks over E4M3 caches
+    batch, q, out = run_case(cfg, mode, Sq, seed, torch.bfloat16)
     with fp32_output():
-        _, _, out32 = run_case(cfg, "mq", Sq, seed, torch.float32)
-    ref = oracle_case(cfg, "mq", batch, q)
+        _, _, out32 = run_case(cfg, mode, Sq, seed, torch.float32)
+    ref = oracle_case(cfg, mode, batch, q)
     assert_parity_and_rounding(out, out32, ref,
-                               what=f"{cfg.name} Sq={Sq} G={cfg.num_q_heads // cfg.num_kv_heads} D={cfg.head_dim} "
+                               what=f"{cfg.name} {mode} Sq={Sq} G={cfg.num_q_heads // cfg.num_kv_heads} D={cfg.head_dim} "
                                     f"bs={cfg.block_size} {cfg.layout} lens={batch.context_lens.cpu().tolist()}")

@@ -160,13 +160,12 @@ def test_unsupported_shapes_are_refused():
     sh = binding.shape_of(batch)
     with pytest.raises(binding.OocoError):
         binding.workspace_bytes_mq(sh, 8193)                               # beyond the largest chunk
-    # the 8-bit cache has no prefill-chunk kernel: 8 heads x 3 tokens > 16 columns
-    ws = torch.empty(binding.workspace_bytes_mq(sh, 3), dtype=torch.uint8, device="cuda")
-    q = torch.zeros((1, 3, 64, 128), dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(binding.OocoError) as e:
-        binding.decode_step_mq_fp8(sh, q, None, None, batch.k_cache, batch.v_cache, batch.block_table, None,
-                                   batch.context_lens, 1.0, 1.0, 1.0, torch.empty_like(q), ws)
-    assert e.value.status == -3
+    # the 8-bit cache is built for head_dim 128 only (refused on the host, before anything is launched)
+    import ctypes
+    sh64 = binding.Shape(1, 8, 2, 64, 16, 8, 4, 2 * 16 * 64, 16 * 64, 64)
+    one = ctypes.c_void_p(256)
+    assert binding.lib().ooco_decode_step_mq_fp8(ctypes.byref(sh64.c()), 3, one, None, None, one, one, one, None, one,
+                                                 1.0, 1.0, 1.0, one, one, 1 << 40, None) == -3
     # a workspace sized for fewer query tokens is refused
     b16 = inputs.make_batch(cfg, "cuda", poison=False)
     sh16 = binding.shape_of(b16)
@@ -289,3 +288,67 @@ def test_fused_step_mq_over_8bit_cache():
     ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), k_ref, v_ref, table, lens.cpu().numpy(), cfg.scale, ks, vs,
                                          num_kv_heads=8, block_size=16, strides=batch.strides)
     assert_parity(out.reshape(-1, 32, 128), ref.out.reshape(-1, 32, 128), what="fused mq step, 8-bit cache")
+
+
+def run_case_8bit(cfg, Sq, seed, ks=1.0 / 32, vs=0.04):
+    b16 = inputs.make_batch(cfg, "cuda", poison=True, table_pad=2**31 - 1)
+    batch = inputs.to_e4m3_pool(b16, ks, vs)
+    B, Hq, D = cfg.batch, cfg.num_q_heads, cfg.head_dim
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    q = (torch.randn((B, Sq, Hq, D), generator=g, device="cuda") * cfg.sigma).to(torch.bfloat16)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_step_mq_fp8(sh, q, None, None, batch.k_cache, batch.v_cache, batch.block_table, None,
+                               batch.context_lens, cfg.scale, ks, vs, out, ws)
+    assert binding.workspace_status(ws) == 0
+    ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), inputs.as_u8(batch.k_cache), inputs.as_u8(batch.v_cache),
+                                         batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                         ks, vs, num_kv_heads=cfg.num_kv_heads, block_size=cfg.block_size,
+                                         strides=batch.strides)
+    assert_parity(out.reshape(B * Sq, Hq, D), ref.out.reshape(B * Sq, Hq, D), what=f"{cfg.name} Sq={Sq} (8-bit cache)")
+    return batch, q, out
+
+
+@pytest.mark.parametrize("cfg,Sq", [c for c in CHUNK_CASES if c[0].head_dim == 128],
+                         ids=lambda v: getattr(v, "name", str(v)))
+def test_prefill_chunk_over_8bit_cache(cfg, Sq):
+    """More than 16 score columns over E4M3 caches: the tcgen05 chunk kernel with the stages widened to f16 in
+    shared memory (17 columns up to several row tiles, every block size, split sequences)."""
+    batch, q, out = run_case_8bit(cfg, Sq, seed=cfg.seed)
+    out2 = torch.full_like(out, float("nan"))
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    binding.decode_step_mq_fp8(sh, q, None, None, batch.k_cache, batch.v_cache, batch.block_table, None,
+                               batch.context_lens, cfg.scale, 1.0 / 32, 0.04, out2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))                    # run-to-run bitwise
+
+
+def test_fused_step_prefill_chunk_over_8bit_cache():
+    """The quantising append of a 40-token chunk (bit-exact over the whole pool) fused into the first launch, seen by
+    the attention of the same call."""
+    cfg = C("ck8-step", 32, 8, 128, 16, (G(6, 40, 1500),), seed=121, pool_fill=0.85)
+    Sq, ks, vs = 40, 1.0 / 32, 1.0 / 32
+    batch = inputs.to_e4m3_pool(inputs.make_batch(cfg, "cuda", poison=True), ks, vs)
+    sh = binding.shape_of(batch)
+    g = torch.Generator(device="cuda").manual_seed(10)
+    q = torch.randn((cfg.batch, Sq, 32, 128), generator=g, device="cuda").to(torch.bfloat16)
+    k_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    v_new = torch.randn((cfg.batch, Sq, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    lens = batch.context_lens
+    positions = (lens - Sq).contiguous()
+    k_ref, v_ref = inputs.as_u8(batch.k_cache).copy(), inputs.as_u8(batch.v_cache).copy()
+    table = batch.block_table.cpu().numpy()
+    for i in range(Sq):
+        oracle.kv_append_fp8(inputs.as_u16(k_new[:, i].contiguous()), inputs.as_u16(v_new[:, i].contiguous()), k_ref,
+                             v_ref, table, (positions + i).cpu().numpy(), ks, vs, block_size=16, strides=batch.strides)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    binding.decode_step_mq_fp8(sh, q, k_new, v_new, batch.k_cache, batch.v_cache, batch.block_table, positions, lens,
+                               cfg.scale, ks, vs, out, ws)
+    assert binding.workspace_status(ws) == 0 and binding.last_launch_count() == 3
+    assert np.array_equal(inputs.as_u8(batch.k_cache), k_ref) and np.array_equal(inputs.as_u8(batch.v_cache), v_ref)
+    ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), k_ref, v_ref, table, lens.cpu().numpy(), cfg.scale, ks, vs,
+                                         num_kv_heads=8, block_size=16, strides=batch.strides)
+    assert_parity(out.reshape(-1, 32, 128), ref.out.reshape(-1, 32, 128), what="fused chunk step, 8-bit cache")
