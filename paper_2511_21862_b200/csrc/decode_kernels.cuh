@@ -373,18 +373,25 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
 // ------------------------------------------------------------------------------------ main
 // Shared-memory carve-up, shared by host (sizing) and device.  TPW = 16-token tiles each
 // consumer warp owns per stage.
-template <int D, int NCW, int NT, int TPW, bool KV8 = false>
+// KVM: 0 = bf16 cache; 1 = 8-bit cache, scores on mma.sync from codes widened in registers; 2 = 8-bit cache,
+// scores on tcgen05 (kind::f8f6f4) straight from the stage, read back from tensor memory.
+template <int D, int NCW, int NT, int TPW, int KVM = 0>
 struct SmemLayout {
   static constexpr int kStageTok = 16 * NCW * TPW;
-  static constexpr int kTileBytes = kStageTok * D * (KV8 ? 1 : 2);  // K (or V) bytes of one stage
+  static constexpr int kTileBytes = kStageTok * D * (KVM ? 1 : 2);  // K (or V) bytes of one stage
   static constexpr int kStageBytes = 2 * kTileBytes;
   static constexpr int kHeads = NT * 8;
   static constexpr int kOStride = 64 + 4;                    // floats per head row of one 64-dim pass
   static constexpr int kMergeOBytes = NCW * kHeads * kOStride * 4;
   static constexpr int kMergeBytes = kMergeOBytes + NCW * kHeads * 2 * 4;
+  // KVM 2: the query of a work item as two E4M3 terms ([2 * kHeads rows][128 bytes], 1024-byte aligned) and one
+  // inverse row scale per head, two of each (consecutive items alternate); per stage one "scores ready" barrier
+  static constexpr int kQSplitBytes = KVM == 2 ? 2 * kHeads * 128 : 0;
+  static constexpr int kTcSColumns = 2 * kHeads;             // tensor-memory columns of one stage's scores
   __host__ __device__ static int q_slot_bytes(int G) { return ((G * D * 2 + 127) / 128) * 128; }
   __host__ __device__ static size_t total(int nstages, int G) {
-    return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16) + kMergeBytes + 64;
+    return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16 + (KVM == 2 ? 8 : 0)) + kMergeBytes + 64 +
+           (KVM == 2 ? 2 * kQSplitBytes + 2 * kHeads * 4 + 32 : 0);
   }
 };
 
@@ -541,6 +548,14 @@ constexpr float kE4m3WidenFactor = 256.f;                  // what the widened v
 __device__ __forceinline__ float f16_lo(uint32_t x) { return __half2float(__ushort_as_half((unsigned short)(x & 0xffffu))); }
 __device__ __forceinline__ float f16_hi(uint32_t x) { return __half2float(__ushort_as_half((unsigned short)(x >> 16))); }
 
+// Softmax and value part of a 16-token tile over the 8-bit cache; `sv[nt]` holds the tile's scaled scores (log2
+// domain) in the MMA accumulator layout: (token g, head 2t) (token g, head 2t+1) (token g+8, 2t) (token g+8, 2t+1).
+template <int D, int NT, bool kTail>
+__device__ __forceinline__ void kv8_softmax_values(uint32_t vst, uint32_t tile_off, const uint32_t (&pat)[D / 16],
+                                                   float (&sv)[NT][4], float (&m_run)[NT][2], float (&l_run)[NT][2],
+                                                   float (&o_acc)[NT][D / 16][4], int valid, int g, int t, int lim_w,
+                                                   const int (*qi_col)[2]);
+
 template <int D, int NT, bool kTail>
 __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uint32_t tile_off,
                                                  const uint32_t (&pat)[D / 16], const uint32_t (&qf)[NT][D / 16][2],
@@ -570,12 +585,24 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
       mma_f16(sc[nt][1], c0, c1, c2, c3, qf[nt][2 * j + 1][0], qf[nt][2 * j + 1][1]);
     }
   }
+  float sv[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sv[nt][e] = (sc[nt][0][e] + sc[nt][1][e]) * scale_log2e;
+  kv8_softmax_values<D, NT, kTail>(vst, tile_off, pat, sv, m_run, l_run, o_acc, valid, g, t, lim_w, qi_col);
+}
+
+template <int D, int NT, bool kTail>
+__device__ __forceinline__ void kv8_softmax_values(uint32_t vst, uint32_t tile_off, const uint32_t (&pat)[D / 16],
+                                                   float (&sv)[NT][4], float (&m_run)[NT][2], float (&l_run)[NT][2],
+                                                   float (&o_acc)[NT][D / 16][4], int valid, int g, int t, int lim_w,
+                                                   const int (*qi_col)[2]) {
+  constexpr int KS = D / 16;
   uint32_t pb[NT][2];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
-    float s[4];  // (token g, head 2t) (token g, head 2t+1) (token g+8, 2t) (token g+8, 2t+1)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) s[e] = (sc[nt][0][e] + sc[nt][1][e]) * scale_log2e;
+    float (&s)[4] = sv[nt];
     if (kTail) {
       const int l0 = min(valid, lim_w + qi_col[nt][0]), l1 = min(valid, lim_w + qi_col[nt][1]);
       if (g >= l0) s[0] = -INFINITY;
@@ -643,17 +670,56 @@ __device__ __forceinline__ void consume_tile_kv8(uint32_t kst, uint32_t vst, uin
   }
 }
 
+// D[tmem] (+)= A[smem] x B[smem] with 8-bit floating-point operands (the formats are in the instruction descriptor).
+__device__ __forceinline__ void umma_f8_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 16 lanes x (8 * N) fp32 columns of tensor memory in the accumulator layout of mma.sync m16n8: for column
+// block i, registers 4i .. 4i + 3 of lane (g = lane / 4, t = lane % 4) hold (row g, columns 2t, 2t + 1) and
+// (row g + 8, columns 2t, 2t + 1).  The lane field of the address may be the warp's lane quarter base or 16 more.
+__device__ __forceinline__ void tmem_ld_frag(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_frag(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+// Two fp32 -> two E4M3 codes (round to nearest even, saturating); `lo` lands in the low byte.
+__device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
+  uint16_t d;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
 // The 8-bit path is bound by the consumer warps' instruction latency, not by HBM, so its 8-warp shape
-// is compiled for two CTAs per SM (16 consumer warps), which caps it at 112 registers per thread.
-template <int D, int NCW, int NT, int TPW, bool KV8 = false>
-__global__ void __launch_bounds__((NCW + 1) * 32, (KV8 && NCW == 8 && NT == 1) ? 2 : 1)
-decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                   const DecodeParams p) {
-  using L = SmemLayout<D, NCW, NT, TPW, KV8>;
+// is compiled for two CTAs per SM (16 consumer warps), which caps it at 112 registers per thread (102 with the
+// extra MMA warp of KVM 2).
+//
+// KVM 2 -- scores of the 8-bit cache on the 5th-generation tensor cores.  A stage is 128 tokens = the M of one
+// tcgen05.mma: one more warp (NCW + 1) waits for each stage, splits the stage's query rows into two E4M3 terms
+// (q * a = hi + lo / 16 with a power-of-two row scale a: as precise as the bf16 query) in a swizzled [16 x 128 B]
+// tile and issues S[128 tok x 16] = K_stage . Qsplit^T (4 MMAs of K 32, kind::f8f6f4, both operands straight from
+// shared memory, K as the TMA wrote it) into the stage's own tensor-memory columns.  The consumer warps load their
+// 16-token tile of S in the mma.sync accumulator layout and go on with the softmax and the value MMAs as in KVM 1;
+// the codes of K are never widened.
+template <int D, int NCW, int NT, int TPW, int KVM>
+__device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                                     const DecodeParams& p, uint8_t* smem_raw) {
+  constexpr bool KV8 = KVM != 0, KVTC = KVM == 2;
+  using L = SmemLayout<D, NCW, NT, TPW, KVM>;
   static_assert(!KV8 || (D == 128 && TPW == 1), "the 8-bit path is built for head_dim 128, one tile per warp");
+  static_assert(!KVTC || NCW == 8, "a stage must hold the 128 tokens of one tcgen05 MMA");
   constexpr int kStageTok = L::kStageTok;
   constexpr int KS = D / 16;  // k-steps of the score MMA = m-tiles of the value MMA
-  extern __shared__ uint8_t smem_raw[];
 
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -661,12 +727,18 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   const int nst = p.nstages;
   const int qslot = L::q_slot_bytes(p.GQ);
   const uint32_t s_stage = base;
-  const uint32_t s_q = s_stage + (uint32_t)nst * L::kStageBytes;
+  const uint32_t s_qs = s_stage + (uint32_t)nst * L::kStageBytes;  // KVM 2: two split query tiles (1024-byte aligned)
+  const uint32_t s_q = s_qs + 2u * L::kQSplitBytes;
   const uint32_t s_merge = s_q + (uint32_t)nst * qslot;
   const uint32_t s_meta = s_merge + L::kMergeBytes;
   const uint32_t s_full = s_meta + (uint32_t)nst * 16;
   const uint32_t s_empty = s_full + (uint32_t)nst * 8;
   const uint32_t s_mbar = s_empty + (uint32_t)nst * 8;
+  const uint32_t s_inva = s_mbar + 16;                     // KVM 2: [2][heads] inverse row scales of the split
+  const uint32_t s_sready = s_inva + 2u * L::kHeads * 4;    // KVM 2: [nst] the stage's scores are in tensor memory
+  const uint32_t s_drain = s_sready + (uint32_t)nst * 8;
+  const uint32_t s_tslot = s_drain + 8;
+  const uint32_t s_qfree = s_tslot + 8;                     // KVM 2: [2] the MMAs that read split tile i are complete
   float* g_merge = reinterpret_cast<float*>(gen + (s_merge - base));
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
   uint8_t* g_q = gen + (s_q - base);
@@ -679,14 +751,117 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     for (int i = 0; i < nst; ++i) {
       mbar_init(s_full + 8 * i, 1);
       mbar_init(s_empty + 8 * i, NCW);
+      if (KVTC) mbar_init(s_sready + 8 * i, 1);
     }
     mbar_init(s_mbar, NCW * 32);
+    if (KVTC) {
+      mbar_init(s_drain, 1);
+      mbar_init(s_qfree, 1);
+      mbar_init(s_qfree + 8, 1);
+    }
     fence_mbar_init();
   }
+  uint32_t tmem = 0;
+  if (KVTC) {
+    if (warp == NCW + 1) {
+      uint32_t cols = 32;
+      while (cols < (uint32_t)nst * L::kTcSColumns) cols <<= 1;
+      tmem_alloc(s_tslot, cols);
+    }
+    tc_fence_before_sync();
+  }
   __syncthreads();
+  if (KVTC) {
+    tc_fence_after_sync();
+    tmem = *reinterpret_cast<volatile uint32_t*>(gen + (s_tslot - base));
+  }
   grid_dep_wait();    // the plan (and a fused append) must have completed
   grid_dep_launch();  // the merge kernel may queue up behind this grid
   const int n_items = p.hdr->n_items;
+
+  if (KVTC && warp == NCW + 1) {
+    // ================================================================= score MMA warp (KVM 2)
+    // kind::f8f6f4: E4M3 x E4M3 -> fp32, both operands K-major, M = 128 tokens, N = 2 * heads (high and low term)
+    const uint32_t idesc = (1u << 4) | ((uint32_t)(L::kTcSColumns >> 3) << 17) | ((uint32_t)(kStageTok >> 4) << 24);
+    int slot = -1;
+    uint32_t full_phase = 1u;
+    bool issued = false;
+    // items seen so far; item n (counted from 1) uses split tile (n - 1) & 1, as that tile's use number (n - 1) >> 1.
+    // A tile is rewritten only once the MMAs of its previous use are complete: the item's last stage commits to
+    // the tile's own barrier.
+    uint32_t n_item = 0;
+    for (;;) {
+      if (++slot == nst) slot = 0;
+      if (slot == 0) full_phase ^= 1u;
+      if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
+        if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+        break;
+      }
+      const int4 meta = g_meta[slot];
+      if (meta.x < 0) break;
+      const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+      if (first) ++n_item;
+      const uint32_t qb = (n_item - 1) & 1, q_use = (n_item - 1) >> 1;
+      if (first && !warp_wait(s_qfree + 8 * qb, (q_use & 1u) ^ 1u, s_abort)) {  // passes at once for a tile's first use
+        if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+        break;
+      }
+      // ---- at the item's first stage: its query rows, row r as hi + lo / 16, scaled by a power of two that
+      // brings the row's largest magnitude into [128, 256) (E4M3 goes up to 448); lane l owns dims 4l .. 4l + 3
+      const uint8_t* qs = g_q + (size_t)slot * qslot;
+      uint8_t* qd = gen + (s_qs - base) + (size_t)qb * L::kQSplitBytes;
+      float* inva = reinterpret_cast<float*>(gen + (s_inva - base)) + qb * L::kHeads;
+#pragma unroll 2
+      for (int hr = 0; first && hr < L::kHeads; ++hr) {
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        if (hr < p.GQ) {
+          const uint2 w = *reinterpret_cast<const uint2*>(qs + ((size_t)hr * D + 4 * lane) * 2);
+          x[0] = __uint_as_float(w.x << 16);
+          x[1] = __uint_as_float(w.x & 0xffff0000u);
+          x[2] = __uint_as_float(w.y << 16);
+          x[3] = __uint_as_float(w.y & 0xffff0000u);
+        }
+        float mx = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+#pragma unroll
+        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (!(mx <= 3.0e38f)) mx = 0.f;  // a row holding NaN or infinity is outside the contract: keep the scale finite
+        // a = 2^(7 - exponent of mx), its biased exponent clamped to the normal range; 1 for an all-zero row
+        int ae = 127 + 7 + 127 - (int)((__float_as_uint(mx) >> 23) & 0xffu);
+        ae = mx > 0.f ? (ae > 254 ? 254 : ae) : 127;
+        const float a = __uint_as_float((uint32_t)ae << 23), inv_a = __uint_as_float((uint32_t)(254 - ae) << 23);
+        const uint32_t h01 = pack_e4m3x2(x[0] * a, x[1] * a), h23 = pack_e4m3x2(x[2] * a, x[3] * a);
+        const uint32_t f01 = e4m3x2_to_f16x2<kSelB0B1>(h01), f23 = e4m3x2_to_f16x2<kSelB0B1>(h23);  // values / 256
+        const uint32_t l01 = pack_e4m3x2((x[0] * a - f16_lo(f01) * kE4m3WidenFactor) * 16.f,
+                                         (x[1] * a - f16_hi(f01) * kE4m3WidenFactor) * 16.f);
+        const uint32_t l23 = pack_e4m3x2((x[2] * a - f16_lo(f23) * kE4m3WidenFactor) * 16.f,
+                                         (x[3] * a - f16_hi(f23) * kE4m3WidenFactor) * 16.f);
+        const uint32_t off = (uint32_t)hr * 128 + ((((uint32_t)lane >> 2) ^ ((uint32_t)hr & 7)) << 4) + ((uint32_t)lane & 3) * 4;
+        *reinterpret_cast<uint32_t*>(qd + off) = h01 | (h23 << 16);
+        *reinterpret_cast<uint32_t*>(qd + L::kHeads * 128 + off) = l01 | (l23 << 16);
+        if (lane == 0) inva[hr] = inv_a;
+      }
+      if (first) fence_proxy_async_smem();  // the tile is read by the MMAs through the async proxy
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes, qst = s_qs + qb * L::kQSplitBytes;
+#pragma unroll
+        for (int k = 0; k < D / 32; ++k)  // 32 contraction bytes per MMA
+          umma_f8_ss(tmem + (uint32_t)slot * L::kTcSColumns, umma_smem_desc(kst + k * 32, 0, 1024),
+                     umma_smem_desc(qst + k * 32, 0, 1024), idesc, k ? 1u : 0u);
+        umma_commit(s_sready + 8 * slot);
+        if (last) umma_commit(s_qfree + 8 * qb);
+      }
+      __syncwarp();
+      issued = true;
+    }
+    if (issued) {  // the tensor memory must not be released under MMAs in flight
+      if (lane == 0) umma_commit(s_drain);
+      __syncwarp();
+      int dummy = 0;
+      mbar_wait_bounded(s_drain, 0u, &dummy, kWaitLimitNs / 8);
+    }
+    return tmem;
+  }
 
   if (warp == NCW) {
     // ================================================================= producer warp
@@ -853,7 +1028,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         mbar_wait_bounded(s_full + 8 * (j % nst), (uint32_t)(j / nst) & 1u, &dummy_abort, kWaitLimitNs / 8);
       }
     }
-    return;
+    return tmem;
   }
 
   // =================================================================== consumer warps
@@ -873,7 +1048,8 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   }
   // Per-lane byte offsets of the ldmatrix rows inside a stage's K / V tile.  A box holds
   // [D/64 halves][tile_rows][64 dims] with the 128-byte swizzle (16-byte chunk ^= row & 7).
-  const int r0 = 16 * TPW * warp;  // first token row of this warp inside a stage
+  // first token row of this warp inside a stage (KVM 2: a warp reads tensor memory in its own lane quarter only)
+  const int r0 = KVTC ? 32 * (warp & 3) + 16 * (warp >> 2) : 16 * TPW * warp;
   const uint32_t box_bytes = (uint32_t)p.tile_rows * D * (KV8 ? 1 : 2);
   const uint32_t half_bytes = (uint32_t)p.tile_rows * 128;
   const int lr_k = (lane & 7) + ((lane >> 3) & 1) * 8, cs_k = lane >> 4;
@@ -899,6 +1075,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     qi_col[nt][0] = p.Sq > 1 ? (8 * nt + 2 * t) / p.G : 0;
     qi_col[nt][1] = p.Sq > 1 ? (8 * nt + 2 * t + 1) / p.G : 0;
   }
+  uint32_t n_item_c = 0;  // items seen so far (KVM 2: item n reads the row scales of split tile n & 1)
   uint32_t mphase = 0;  // parity of the next merge-barrier phase to wait for
   bool merge_pending_read = false;
 
@@ -909,12 +1086,13 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (slot == 0) full_phase ^= 1u;
     if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
       if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
-      return;
+      return tmem;
     }
     const int4 meta = g_meta[slot];
     if (meta.x < 0) break;
     const int ntok = meta.w & 0xffff;
     const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+    if (first) ++n_item_c;
     if (first) {
       const uint8_t* qs = g_q + (size_t)slot * qslot;
 #pragma unroll
@@ -926,7 +1104,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         for (int k = 0; k < KS; ++k) {
           o_acc[nt][k][0] = o_acc[nt][k][1] = o_acc[nt][k][2] = o_acc[nt][k][3] = 0.f;
           uint32_t v0 = 0u, v1 = 0u;
-          if (head < p.GQ) {
+          if (!KVTC && head < p.GQ) {
             if (KV8) {  // dims 16k + 4t .. + 3 as two f16 pairs (the k order of the 8-bit score MMA)
               const uint2 w = *reinterpret_cast<const uint2*>(qs + ((size_t)head * D + 16 * k + 4 * t) * 2);
               v0 = pack_f16x2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u));
@@ -948,7 +1126,31 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       const uint32_t vst = kst + L::kTileBytes;
       // rows of this warp the first query token may see; with one query token that is all of them
       const int lim_w = ((meta.w >> 18) & 1023) - 16 - r0;
-      if (KV8) {
+      if (KVTC) {
+        // this warp's 16 x (2 * heads) tile of the stage's scores, in the accumulator layout of mma.sync
+        if (!warp_wait(s_sready + 8 * slot, full_phase, s_abort)) {
+          if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+          return tmem;
+        }
+        tc_fence_after_sync();
+        uint32_t f[8 * NT];
+        tmem_ld_frag(tmem + ((uint32_t)r0 << 16) + (uint32_t)slot * L::kTcSColumns, f);
+        tmem_ld_wait();
+        const float* inva = reinterpret_cast<const float*>(gen + (s_inva - base)) + ((n_item_c - 1) & 1) * L::kHeads;
+        float sv[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const float2 ia = *reinterpret_cast<const float2*>(inva + 8 * nt + 2 * t);
+          const float m0 = ia.x * p.scale_log2e, m1 = ia.y * p.scale_log2e;
+#pragma unroll
+          for (int e = 0; e < 4; ++e)  // high term + low term / 16
+            sv[nt][e] = fmaf(__uint_as_float(f[4 * (NT + nt) + e]), 0.0625f, __uint_as_float(f[4 * nt + e])) * ((e & 1) ? m1 : m0);
+        }
+        if (valid >= 16 && lim_w >= 16)
+          kv8_softmax_values<D, NT, false>(vst, tile_k[0], kpat, sv, m_run, l_run, o_acc, valid, g, t, 0, nullptr);
+        else
+          kv8_softmax_values<D, NT, true>(vst, tile_k[0], kpat, sv, m_run, l_run, o_acc, valid, g, t, lim_w, qi_col);
+      } else if (KV8) {
         if (valid >= 16 && lim_w >= 16)
           consume_tile_kv8<D, NT, false>(kst, vst, tile_k[0], kpat, qf, m_run, l_run, o_acc, p.scale_log2e, valid, g, t);
         else
@@ -992,7 +1194,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         if (merge_pending_read) {  // earlier readers must be done with the buffer
           if (!warp_wait(s_mbar, mphase, s_abort)) {
             if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
-            return;
+            return tmem;
           }
           mphase ^= 1u;
         }
@@ -1020,7 +1222,7 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         mbar_arrive(s_mbar);
         if (!warp_wait(s_mbar, mphase, s_abort)) {
           if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
-          return;
+          return tmem;
         }
         mphase ^= 1u;
         for (int idx = threadIdx.x; idx < p.GQ * 64; idx += NCW * 32) {
@@ -1050,6 +1252,24 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         mbar_arrive(s_mbar);
         merge_pending_read = true;
       }
+    }
+  }
+  return tmem;
+}
+
+template <int D, int NCW, int NT, int TPW, int KVM = 0>
+__global__ void __launch_bounds__((NCW + (KVM == 2 ? 2 : 1)) * 32, (KVM && NCW == 8 && NT == 1) ? 2 : 1)
+decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                   const DecodeParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t tmem = decode_main_body<D, NCW, NT, TPW, KVM>(tm_k, tm_v, p, smem_raw);
+  if (KVM == 2) {  // common exit: release the tensor memory once every warp is done with it
+    tc_fence_before_sync();
+    __syncthreads();
+    if ((threadIdx.x >> 5) == NCW + 1) {
+      uint32_t cols = 32;
+      while (cols < (uint32_t)p.nstages * SmemLayout<D, NCW, NT, TPW, KVM>::kTcSColumns) cols <<= 1;
+      tmem_dealloc(tmem, cols);
     }
   }
 }

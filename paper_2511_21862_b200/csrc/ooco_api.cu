@@ -22,8 +22,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobOutF32, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}, {0}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobOutF32, kKnobKv8Tcgen05, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}, {0}, {1}};
 static std::atomic<int> g_overridden[kKnobCount];  // knob set through ooco_set_tuning
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
@@ -207,11 +207,11 @@ static cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size
   return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
-template <int D, int NCW, int NT, int TPW, bool KV8 = false>
+template <int D, int NCW, int NT, int TPW, int KVM = 0>
 static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                        int ctas_per_sm, int want_stages, cudaStream_t st, int dev, bool dry) {
-  using L = SmemLayout<D, NCW, NT, TPW, KV8>;
-  auto kern = decode_main_kernel<D, NCW, NT, TPW, KV8>;
+  using L = SmemLayout<D, NCW, NT, TPW, KVM>;
+  auto kern = decode_main_kernel<D, NCW, NT, TPW, KVM>;
   // the opt-in limit covers static + dynamic shared memory of the kernel
   static std::atomic<int> static_smem{-1};
   if (static_smem.load() < 0) {
@@ -225,6 +225,7 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
   const size_t budget = ctas_per_sm > 1 ? ((size_t)di.smem_optin + 1024) / ctas_per_sm - 1024 - static_smem.load()
                                         : dyn_max;
   int nst = want_stages > 0 ? want_stages : 32;
+  if (KVM == 2 && nst > 8) nst = 8;  // every stage owns tensor-memory columns for its scores
   while (nst > 2 && L::total(nst, p.GQ) > budget) --nst;
   if (L::total(nst, p.GQ) > dyn_max) return OOCO_E_UNSUPPORTED;
   p.nstages = nst;
@@ -236,7 +237,7 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
   if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
-  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + 1) * 32), smem, st,
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + (KVM == 2 ? 2 : 1)) * 32), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the attention kernel", (long)e);
@@ -249,20 +250,23 @@ static int launch_main_nt(const CUtensorMap& tk, const CUtensorMap& tv, DecodePa
   return launch_main<D, NCW, 2, TPW>(tk, tv, p, di, cps, stages, st, dev, dry);
 }
 
-// 8-bit cache: head_dim 128, one tile per warp.
-static int launch_main_kv8(int ncw, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
+// 8-bit cache: head_dim 128, one tile per warp.  `tc`: the 8-warp shape with the scores on tcgen05.
+static int launch_main_kv8(int ncw, bool tc, const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p,
                            const DeviceInfo& di, int cps, int stages, cudaStream_t st, int dev, bool dry) {
   const bool wide = p.GQ > 8;
+  if (tc && ncw == 8)
+    return wide ? launch_main<128, 8, 2, 1, 2>(tk, tv, p, di, cps, stages, st, dev, dry)
+                : launch_main<128, 8, 1, 1, 2>(tk, tv, p, di, cps, stages, st, dev, dry);
   switch (ncw) {
     case 2:
-      return wide ? launch_main<128, 2, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry)
-                  : launch_main<128, 2, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry);
+      return wide ? launch_main<128, 2, 2, 1, 1>(tk, tv, p, di, cps, stages, st, dev, dry)
+                  : launch_main<128, 2, 1, 1, 1>(tk, tv, p, di, cps, stages, st, dev, dry);
     case 8:
-      return wide ? launch_main<128, 8, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry)
-                  : launch_main<128, 8, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry);
+      return wide ? launch_main<128, 8, 2, 1, 1>(tk, tv, p, di, cps, stages, st, dev, dry)
+                  : launch_main<128, 8, 1, 1, 1>(tk, tv, p, di, cps, stages, st, dev, dry);
     default:
-      return wide ? launch_main<128, 4, 2, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry)
-                  : launch_main<128, 4, 1, 1, true>(tk, tv, p, di, cps, stages, st, dev, dry);
+      return wide ? launch_main<128, 4, 2, 1, 1>(tk, tv, p, di, cps, stages, st, dev, dry)
+                  : launch_main<128, 4, 1, 1, 1>(tk, tv, p, di, cps, stages, st, dev, dry);
   }
 }
 
@@ -603,7 +607,7 @@ int ooco_set_tuning(int knob, int value) {
   if (knob == kKnobItemsPerCta && (value < 1 || value > 64)) return OOCO_E_SHAPE;
   if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
   if (knob == kKnobCopyCtasPerSm && (value < 1 || value > 3)) return OOCO_E_SHAPE;
-  if (knob == kKnobOutF32 && value != 0 && value != 1) return OOCO_E_SHAPE;
+  if ((knob == kKnobOutF32 || knob == kKnobKv8Tcgen05) && value != 0 && value != 1) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
   g_overridden[knob].store(1);
   return OOCO_OK;
@@ -755,8 +759,10 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.chunk_max = g_knobs[kKnobChunkMax].load();
   if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
   p.items_per_cta = plan_items_per_cta(G_);
-  // the 8-bit path widens codes to value / 256 (kE4m3WidenFactor): both scales carry the factor back
-  p.scale_log2e = scale * 1.4426950408889634f * (kv8 ? kv8->k_scale * kE4m3WidenFactor : 1.f);
+  // the 8-bit path widens codes to value / 256 (kE4m3WidenFactor): both scales carry the factor back (K's only
+  // where K is widened: the tcgen05 score path multiplies the codes' own values)
+  const bool kv8_tc = kv8 && !chunk && ncw == 8 && g_knobs[kKnobKv8Tcgen05].load() != 0;
+  p.scale_log2e = scale * 1.4426950408889634f * (kv8 ? kv8->k_scale * (kv8_tc ? 1.f : kE4m3WidenFactor) : 1.f);
   p.v_scale = kv8 ? kv8->v_scale * kE4m3WidenFactor : 1.f;
 
   CUtensorMap tk, tv;
@@ -786,7 +792,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
     if (row16)
       return s->head_dim == 128 ? launch_row16<128>(tk, tv, p, di, cps, st, dev, dry)
                                 : launch_row16<64>(tk, tv, p, di, cps, st, dev, dry);
-    if (kv8) return launch_main_kv8(ncw, tk, tv, p, di, cps, stages, st, dev, dry);
+    if (kv8) return launch_main_kv8(ncw, kv8_tc, tk, tv, p, di, cps, stages, st, dev, dry);
     return s->head_dim == 128 ? launch_main_ncw<128>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev, dry)
                               : launch_main_ncw<64>(ncw, tpw, tk, tv, p, di, cps, stages, st, dev, dry);
   };

@@ -149,7 +149,7 @@ def test_query_length_limits_and_workspace_growth_without_a_device():
     assert attn(8193) == -3 and attn(0) == -2
     assert attn(64, q=odd) == -3 and attn(64, out=odd) == -3
     assert attn(64, ws_bytes=binding.workspace_bytes_mq(sh, 4)) == -4
-    assert L.ooco_set_tuning(11, 0) == 0 and L.ooco_set_tuning(11, 1) == 0 and L.ooco_set_tuning(12, 1) == 0 and L.ooco_set_tuning(14, 1) == -2
+    assert L.ooco_set_tuning(11, 0) == 0 and L.ooco_set_tuning(11, 1) == 0 and L.ooco_set_tuning(12, 1) == 0 and L.ooco_set_tuning(15, 1) == -2
 
 
 def test_missing_library_fails_loudly(monkeypatch):
@@ -225,7 +225,7 @@ def test_range_predicates_of_the_checked_build():
 def test_fp32_output_knob_is_a_switch():
     assert binding.get_tuning("out_f32") == 0
     L = binding.lib()
-    assert L.ooco_set_tuning(13, 2) == -2 and L.ooco_set_tuning(14, 1) == -2 and L.ooco_get_tuning(99) == -2
+    assert L.ooco_set_tuning(13, 2) == -2 and L.ooco_set_tuning(15, 1) == -2 and L.ooco_get_tuning(99) == -2
     binding.set_tuning(out_f32=1)
     try:
         assert binding.get_tuning("out_f32") == 1
