@@ -384,14 +384,20 @@ struct SmemLayout {
   static constexpr int kOStride = 64 + 4;                    // floats per head row of one 64-dim pass
   static constexpr int kMergeOBytes = NCW * kHeads * kOStride * 4;
   static constexpr int kMergeBytes = kMergeOBytes + NCW * kHeads * 2 * 4;
-  // KVM 2: the query of a work item as two E4M3 terms ([2 * kHeads rows][128 bytes], 1024-byte aligned) and one
-  // inverse row scale per head, two of each (consecutive items alternate); per stage one "scores ready" barrier
+  // KVM 2: K and V have rings of their own.  The K tile of a stage is dead as soon as its score MMAs are complete
+  // (the scores wait in tensor memory, kTcSBuffers stages of them), so kTcKSlots slots keep the K stream going and
+  // the rest of the shared memory gives the V ring (`nstages` slots) the depth the consumers' latency needs.
+  // Besides: the query of a work item as two E4M3 terms ([2 * kHeads rows][128 bytes], 1024-byte aligned) and one
+  // inverse row scale per head, two of each (consecutive items alternate).
+  static constexpr int kTcKSlots = 2, kTcSBuffers = 8;
   static constexpr int kQSplitBytes = KVM == 2 ? 2 * kHeads * 128 : 0;
   static constexpr int kTcSColumns = 2 * kHeads;             // tensor-memory columns of one stage's scores
   __host__ __device__ static int q_slot_bytes(int G) { return ((G * D * 2 + 127) / 128) * 128; }
   __host__ __device__ static size_t total(int nstages, int G) {
-    return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16 + (KVM == 2 ? 8 : 0)) + kMergeBytes + 64 +
-           (KVM == 2 ? 2 * kQSplitBytes + 2 * kHeads * 4 + 32 : 0);
+    if (KVM == 2)
+      return 1024 + (size_t)kTcKSlots * (kTileBytes + q_slot_bytes(G) + 16 + 16) + (size_t)nstages * (kTileBytes + 16 + 16) +
+             kMergeBytes + 64 + 2 * kQSplitBytes + 2 * kHeads * 4 + kTcSBuffers * 8 + 32;
+    return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16) + kMergeBytes + 64;
   }
 };
 
@@ -726,19 +732,28 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
   uint8_t* gen = smem_raw + (base - raw);
   const int nst = p.nstages;
   const int qslot = L::q_slot_bytes(p.GQ);
+  constexpr int kNK = L::kTcKSlots, kNS = L::kTcSBuffers;
+  // stages: [nst][K tile, V tile]; KVM 2: K ring [kNK][K tile], then V ring [nst][V tile] (full / empty / meta below
+  // are the V ring's, i.e. what the consumer warps see, in every mode)
   const uint32_t s_stage = base;
-  const uint32_t s_qs = s_stage + (uint32_t)nst * L::kStageBytes;  // KVM 2: two split query tiles (1024-byte aligned)
+  const uint32_t s_vring = s_stage + (uint32_t)kNK * L::kTileBytes;
+  const uint32_t s_qs = KVTC ? s_vring + (uint32_t)nst * L::kTileBytes
+                             : s_stage + (uint32_t)nst * L::kStageBytes;  // KVM 2: two split query tiles (1024-byte aligned)
   const uint32_t s_q = s_qs + 2u * L::kQSplitBytes;
-  const uint32_t s_merge = s_q + (uint32_t)nst * qslot;
+  const uint32_t s_merge = s_q + (uint32_t)(KVTC ? kNK : nst) * qslot;  // (KVM 2: the query rows travel with the K tile)
   const uint32_t s_meta = s_merge + L::kMergeBytes;
-  const uint32_t s_full = s_meta + (uint32_t)nst * 16;
+  const uint32_t s_kmeta = s_meta + (uint32_t)nst * 16;
+  const uint32_t s_full = s_kmeta + (KVTC ? kNK * 16u : 0u);
   const uint32_t s_empty = s_full + (uint32_t)nst * 8;
   const uint32_t s_mbar = s_empty + (uint32_t)nst * 8;
   const uint32_t s_inva = s_mbar + 16;                     // KVM 2: [2][heads] inverse row scales of the split
-  const uint32_t s_sready = s_inva + 2u * L::kHeads * 4;    // KVM 2: [nst] the stage's scores are in tensor memory
-  const uint32_t s_drain = s_sready + (uint32_t)nst * 8;
+  const uint32_t s_sready = s_inva + 2u * L::kHeads * 4;    // KVM 2: [kNS] the stage's scores are in tensor memory
+  const uint32_t s_drain = s_sready + (uint32_t)kNS * 8;
   const uint32_t s_tslot = s_drain + 8;
   const uint32_t s_qfree = s_tslot + 8;                     // KVM 2: [2] the MMAs that read split tile i are complete
+  const uint32_t s_kfull = s_qfree + 16;                    // KVM 2: [kNK] the K tile (and the item's query rows) has landed
+  const uint32_t s_kempty = s_kfull + (uint32_t)kNK * 8;    // KVM 2: [kNK] the MMAs that read the K tile are complete
+  int4* g_kmeta = reinterpret_cast<int4*>(gen + (s_kmeta - base));
   float* g_merge = reinterpret_cast<float*>(gen + (s_merge - base));
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
   uint8_t* g_q = gen + (s_q - base);
@@ -751,10 +766,14 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     for (int i = 0; i < nst; ++i) {
       mbar_init(s_full + 8 * i, 1);
       mbar_init(s_empty + 8 * i, NCW);
-      if (KVTC) mbar_init(s_sready + 8 * i, 1);
     }
     mbar_init(s_mbar, NCW * 32);
     if (KVTC) {
+      for (int i = 0; i < kNS; ++i) mbar_init(s_sready + 8 * i, 1);
+      for (int i = 0; i < kNK; ++i) {
+        mbar_init(s_kfull + 8 * i, 1);
+        mbar_init(s_kempty + 8 * i, 1);
+      }
       mbar_init(s_drain, 1);
       mbar_init(s_qfree, 1);
       mbar_init(s_qfree + 8, 1);
@@ -764,9 +783,7 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
   uint32_t tmem = 0;
   if (KVTC) {
     if (warp == NCW + 1) {
-      uint32_t cols = 32;
-      while (cols < (uint32_t)nst * L::kTcSColumns) cols <<= 1;
-      tmem_alloc(s_tslot, cols);
+      tmem_alloc(s_tslot, kNS * L::kTcSColumns);  // 128 or 256 columns
     }
     tc_fence_before_sync();
   }
@@ -783,21 +800,18 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     // ================================================================= score MMA warp (KVM 2)
     // kind::f8f6f4: E4M3 x E4M3 -> fp32, both operands K-major, M = 128 tokens, N = 2 * heads (high and low term)
     const uint32_t idesc = (1u << 4) | ((uint32_t)(L::kTcSColumns >> 3) << 17) | ((uint32_t)(kStageTok >> 4) << 24);
-    int slot = -1;
-    uint32_t full_phase = 1u;
     bool issued = false;
     // items seen so far; item n (counted from 1) uses split tile (n - 1) & 1, as that tile's use number (n - 1) >> 1.
     // A tile is rewritten only once the MMAs of its previous use are complete: the item's last stage commits to
     // the tile's own barrier.
     uint32_t n_item = 0;
-    for (;;) {
-      if (++slot == nst) slot = 0;
-      if (slot == 0) full_phase ^= 1u;
-      if (!warp_wait(s_full + 8 * slot, full_phase, s_abort)) {
+    for (uint32_t it = 0;; ++it) {
+      const uint32_t slot = it % kNK, sbuf = it % kNS;  // K ring slot (the query rows share it), score buffer
+      if (!warp_wait(s_kfull + 8 * slot, (it / kNK) & 1u, s_abort)) {
         if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
         break;
       }
-      const int4 meta = g_meta[slot];
+      const int4 meta = g_kmeta[slot];
       if (meta.x < 0) break;
       const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
       if (first) ++n_item;
@@ -843,12 +857,13 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
       if (first) fence_proxy_async_smem();  // the tile is read by the MMAs through the async proxy
       __syncwarp();
       if (lane == 0) {
-        const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes, qst = s_qs + qb * L::kQSplitBytes;
+        const uint32_t kst = s_stage + slot * L::kTileBytes, qst = s_qs + qb * L::kQSplitBytes;
 #pragma unroll
         for (int k = 0; k < D / 32; ++k)  // 32 contraction bytes per MMA
-          umma_f8_ss(tmem + (uint32_t)slot * L::kTcSColumns, umma_smem_desc(kst + k * 32, 0, 1024),
+          umma_f8_ss(tmem + sbuf * L::kTcSColumns, umma_smem_desc(kst + k * 32, 0, 1024),
                      umma_smem_desc(qst + k * 32, 0, 1024), idesc, k ? 1u : 0u);
-        umma_commit(s_sready + 8 * slot);
+        umma_commit(s_sready + 8 * sbuf);
+        umma_commit(s_kempty + 8 * slot);  // the K tile (and the query rows beside it) may be refilled
         if (last) umma_commit(s_qfree + 8 * qb);
       }
       __syncwarp();
@@ -926,11 +941,14 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
         }
         const int slot = it % nst;
         const uint32_t ph = (uint32_t)(it / nst) & 1u;
-        if (!warp_wait(s_empty + 8 * slot, ph ^ 1u, s_abort)) {
+        const int kslot = KVTC ? it % kNK : slot;  // KVM 2: the K tile and the query rows go to the K ring
+        if (!warp_wait(s_empty + 8 * slot, ph ^ 1u, s_abort) ||
+            (KVTC && !warp_wait(s_kempty + 8 * kslot, (((uint32_t)it / kNK) & 1u) ^ 1u, s_abort))) {
           ok = false;
           break;
         }
         const uint32_t full = s_full + 8 * slot;
+        const uint32_t kfull = KVTC ? s_kfull + 8 * kslot : full;
         if (lane == 0) {
           const int flags = (s == 0 ? 1 : 0) | (s == nstage_item - 1 ? 2 : 0);
           // rows of this stage the first query token may see, biased by 16 and clipped to 10 bits
@@ -940,26 +958,33 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
             const long long lim0 = (long long)T_cur - p.Sq + 1 - tok0 + 16;
             cm = lim0 < 0 ? 0 : (lim0 > 1023 ? 1023 : (int)lim0);
           }
-          g_meta[slot] = make_int4(slot_id, b, h, ntok | (flags << 16) | (cm << 18));
-          uint32_t bytes = 2u * nbox * box_bytes;
-          if (s == 0) bytes += (uint32_t)p.GQ * D * 2;
-          mbar_arrive_expect_tx(full, bytes);
+          const int4 meta = make_int4(slot_id, b, h, ntok | (flags << 16) | (cm << 18));
+          g_meta[slot] = meta;
+          const uint32_t qbytes = s == 0 ? (uint32_t)p.GQ * D * 2 : 0u;
+          if (KVTC) {
+            g_kmeta[kslot] = meta;
+            mbar_arrive_expect_tx(kfull, nbox * box_bytes + qbytes);
+            mbar_arrive_expect_tx(full, nbox * box_bytes);
+          } else {
+            mbar_arrive_expect_tx(full, 2u * nbox * box_bytes + qbytes);
+          }
         }
         __syncwarp();
         bool span_ok = true;  // checked build: every copy lands inside its stage (and the q rows inside their slot)
         if (lane < nbox) {
           const int tb = tok0 + lane * p.tile_rows;
           const int c_tok = tb % p.bs;
-          const uint32_t dk = s_stage + (uint32_t)slot * L::kStageBytes + lane * box_bytes;
-          const uint32_t dv = dk + L::kTileBytes;
-          span_ok = checked(chk_span(dk, box_bytes, s_stage + (long long)slot * L::kStageBytes,
-                                     s_stage + (long long)slot * L::kStageBytes + L::kTileBytes) &&
-                                chk_span(slot, 1, 0, nst),
+          const uint32_t k0 = KVTC ? s_stage + (uint32_t)kslot * L::kTileBytes : s_stage + (uint32_t)slot * L::kStageBytes;
+          const uint32_t v0 = KVTC ? s_vring + (uint32_t)slot * L::kTileBytes : k0 + L::kTileBytes;
+          const uint32_t dk = k0 + lane * box_bytes, dv = v0 + lane * box_bytes;
+          span_ok = checked(chk_span(dk, box_bytes, k0, (long long)k0 + L::kTileBytes) &&
+                                chk_span(dv, box_bytes, v0, (long long)v0 + L::kTileBytes) && chk_span(slot, 1, 0, nst) &&
+                                chk_span(kslot, 1, 0, KVTC ? kNK : nst),
                             &p.hdr->status, kStatusBadSmem);
           if (!span_ok) {
             // skipped
           } else if (KV8) {  // a token row is one 128-byte swizzle row: one 4-d copy per box
-            tma_load_4d(dk, &tm_k, full, 0, c_tok, h, blk_cur);
+            tma_load_4d(dk, &tm_k, kfull, 0, c_tok, h, blk_cur);
             tma_load_4d(dv, &tm_v, full, 0, c_tok, h, blk_cur);
           } else if (D == 128 && !p.split_halves) {
             tma_load_5d(dk, &tm_k, full, 0, c_tok, 0, h, blk_cur);
@@ -973,10 +998,10 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
           }
         }
         if (s == 0 && lane < p.Sq) {  // one run of G heads per query token, side by side: [query][head][D]
-          const uint32_t dq = s_q + (uint32_t)slot * qslot + (uint32_t)lane * p.G * D * 2;
-          if (checked(chk_span(dq, (long long)p.G * D * 2, s_q + (long long)slot * qslot, s_q + (long long)(slot + 1) * qslot),
+          const uint32_t dq = s_q + (uint32_t)kslot * qslot + (uint32_t)lane * p.G * D * 2;
+          if (checked(chk_span(dq, (long long)p.G * D * 2, s_q + (long long)kslot * qslot, s_q + (long long)(kslot + 1) * qslot),
                       &p.hdr->status, kStatusBadSmem))
-            bulk_g2s(dq, p.q + (((size_t)b * p.Sq + lane) * p.Hq + (size_t)h * p.G) * D, (uint32_t)p.G * D * 2, full);
+            bulk_g2s(dq, p.q + (((size_t)b * p.Sq + lane) * p.Hq + (size_t)h * p.G) * D, (uint32_t)p.G * D * 2, kfull);
           else
             span_ok = false;
         }
@@ -1006,12 +1031,17 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     }
     // end marker (one stage, seen by every consumer warp)
     if (ok) {
-      const int slot = it % nst;
+      const int slot = it % nst, kslot = it % kNK;
       const uint32_t ph = (uint32_t)(it / nst) & 1u;
-      if (warp_wait(s_empty + 8 * slot, ph ^ 1u, s_abort)) {
+      if (warp_wait(s_empty + 8 * slot, ph ^ 1u, s_abort) &&
+          (!KVTC || warp_wait(s_kempty + 8 * kslot, (((uint32_t)it / kNK) & 1u) ^ 1u, s_abort))) {
         if (lane == 0) {
           g_meta[slot] = make_int4(-1, 0, 0, 0);
           mbar_arrive(s_full + 8 * slot);
+          if (KVTC) {
+            g_kmeta[kslot] = make_int4(-1, 0, 0, 0);
+            mbar_arrive(s_kfull + 8 * kslot);
+          }
         }
         ++it;
       } else {
@@ -1026,6 +1056,10 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
       for (int k = 0; k < pending; ++k) {
         const int j = it - 1 - k;
         mbar_wait_bounded(s_full + 8 * (j % nst), (uint32_t)(j / nst) & 1u, &dummy_abort, kWaitLimitNs / 8);
+      }
+      for (int k = 0; KVTC && k < (it < kNK ? it : kNK); ++k) {
+        const int j = it - 1 - k;
+        mbar_wait_bounded(s_kfull + 8 * (j % kNK), (uint32_t)(j / kNK) & 1u, &dummy_abort, kWaitLimitNs / 8);
       }
     }
     return tmem;
@@ -1122,19 +1156,20 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     }
     const int valid = ntok - r0;  // this warp's rows [0, valid) of 16 * TPW hold tokens of the chunk
     if (valid > 0) {
-      const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;
-      const uint32_t vst = kst + L::kTileBytes;
+      const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes;  // (not read with KVM 2)
+      const uint32_t vst = KVTC ? s_vring + (uint32_t)slot * L::kTileBytes : kst + L::kTileBytes;
       // rows of this warp the first query token may see; with one query token that is all of them
       const int lim_w = ((meta.w >> 18) & 1023) - 16 - r0;
       if (KVTC) {
         // this warp's 16 x (2 * heads) tile of the stage's scores, in the accumulator layout of mma.sync
-        if (!warp_wait(s_sready + 8 * slot, full_phase, s_abort)) {
+        const uint32_t sbuf = (uint32_t)it % kNS;
+        if (!warp_wait(s_sready + 8 * sbuf, ((uint32_t)it / kNS) & 1u, s_abort)) {
           if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
           return tmem;
         }
         tc_fence_after_sync();
         uint32_t f[8 * NT];
-        tmem_ld_frag(tmem + ((uint32_t)r0 << 16) + (uint32_t)slot * L::kTcSColumns, f);
+        tmem_ld_frag(tmem + ((uint32_t)r0 << 16) + sbuf * L::kTcSColumns, f);
         tmem_ld_wait();
         const float* inva = reinterpret_cast<const float*>(gen + (s_inva - base)) + ((n_item_c - 1) & 1) * L::kHeads;
         float sv[NT][4];
@@ -1267,9 +1302,8 @@ decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     tc_fence_before_sync();
     __syncthreads();
     if ((threadIdx.x >> 5) == NCW + 1) {
-      uint32_t cols = 32;
-      while (cols < (uint32_t)p.nstages * SmemLayout<D, NCW, NT, TPW, KVM>::kTcSColumns) cols <<= 1;
-      tmem_dealloc(tmem, cols);
+      using L = SmemLayout<D, NCW, NT, TPW, KVM>;
+      tmem_dealloc(tmem, L::kTcSBuffers * L::kTcSColumns);
     }
   }
 }
