@@ -387,8 +387,8 @@ struct SmemLayout {
   // KVM 2: K and V have rings of their own.  The K tile of a stage is dead as soon as its score MMAs are complete
   // (the scores wait in tensor memory, kTcSBuffers stages of them), so kTcKSlots slots keep the K stream going and
   // the rest of the shared memory gives the V ring (`nstages` slots) the depth the consumers' latency needs.
-  // Besides: the query of a work item as two E4M3 terms ([2 * kHeads rows][128 bytes], 1024-byte aligned) and one
-  // inverse row scale per head, two of each (consecutive items alternate).
+  // Besides: the query of a work item as two E4M3 terms ([2 * kHeads rows][128 bytes], 1024-byte aligned), two
+  // such tiles (consecutive items alternate), and beside every score buffer the inverse row scales of its item.
   static constexpr int kTcKSlots = 2, kTcSBuffers = 8;
   static constexpr int kQSplitBytes = KVM == 2 ? 2 * kHeads * 128 : 0;
   static constexpr int kTcSColumns = 2 * kHeads;             // tensor-memory columns of one stage's scores
@@ -396,7 +396,7 @@ struct SmemLayout {
   __host__ __device__ static size_t total(int nstages, int G) {
     if (KVM == 2)
       return 1024 + (size_t)kTcKSlots * (kTileBytes + q_slot_bytes(G) + 16 + 16) + (size_t)nstages * (kTileBytes + 16 + 16) +
-             kMergeBytes + 64 + 2 * kQSplitBytes + 2 * kHeads * 4 + kTcSBuffers * 8 + 32;
+             kMergeBytes + 64 + 2 * kQSplitBytes + kTcSBuffers * (kHeads * 4 + 8) + 32;
     return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16) + kMergeBytes + 64;
   }
 };
@@ -746,8 +746,8 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
   const uint32_t s_full = s_kmeta + (KVTC ? kNK * 16u : 0u);
   const uint32_t s_empty = s_full + (uint32_t)nst * 8;
   const uint32_t s_mbar = s_empty + (uint32_t)nst * 8;
-  const uint32_t s_inva = s_mbar + 16;                     // KVM 2: [2][heads] inverse row scales of the split
-  const uint32_t s_sready = s_inva + 2u * L::kHeads * 4;    // KVM 2: [kNS] the stage's scores are in tensor memory
+  const uint32_t s_inva = s_mbar + 16;                     // KVM 2: [kNS][heads] inverse row scales, one set per score buffer
+  const uint32_t s_sready = s_inva + (uint32_t)kNS * L::kHeads * 4;  // KVM 2: [kNS] the stage's scores are in tensor memory
   const uint32_t s_drain = s_sready + (uint32_t)kNS * 8;
   const uint32_t s_tslot = s_drain + 8;
   const uint32_t s_qfree = s_tslot + 8;                     // KVM 2: [2] the MMAs that read split tile i are complete
@@ -805,6 +805,7 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     // A tile is rewritten only once the MMAs of its previous use are complete: the item's last stage commits to
     // the tile's own barrier.
     uint32_t n_item = 0;
+    float my_inva = 0.f;  // lane r: the inverse scale of row r of the current item
     for (uint32_t it = 0;; ++it) {
       const uint32_t slot = it % kNK, sbuf = it % kNS;  // K ring slot (the query rows share it), score buffer
       if (!warp_wait(s_kfull + 8 * slot, (it / kNK) & 1u, s_abort)) {
@@ -824,7 +825,6 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
       // brings the row's largest magnitude into [128, 256) (E4M3 goes up to 448); lane l owns dims 4l .. 4l + 3
       const uint8_t* qs = g_q + (size_t)slot * qslot;
       uint8_t* qd = gen + (s_qs - base) + (size_t)qb * L::kQSplitBytes;
-      float* inva = reinterpret_cast<float*>(gen + (s_inva - base)) + qb * L::kHeads;
 #pragma unroll 2
       for (int hr = 0; first && hr < L::kHeads; ++hr) {
         float x[4] = {0.f, 0.f, 0.f, 0.f};
@@ -852,9 +852,13 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
         const uint32_t off = (uint32_t)hr * 128 + ((((uint32_t)lane >> 2) ^ ((uint32_t)hr & 7)) << 4) + ((uint32_t)lane & 3) * 4;
         *reinterpret_cast<uint32_t*>(qd + off) = h01 | (h23 << 16);
         *reinterpret_cast<uint32_t*>(qd + L::kHeads * 128 + off) = l01 | (l23 << 16);
-        if (lane == 0) inva[hr] = inv_a;
+        if (lane == hr) my_inva = inv_a;
       }
       if (first) fence_proxy_async_smem();  // the tile is read by the MMAs through the async proxy
+      // the row scales travel with the stage's score buffer (the consumer warps may be several stages, and items,
+      // behind this warp): written and fenced before the MMAs whose completion the consumers wait for are issued
+      if (lane < L::kHeads) reinterpret_cast<float*>(gen + (s_inva - base))[sbuf * L::kHeads + lane] = my_inva;
+      __threadfence_block();
       __syncwarp();
       if (lane == 0) {
         const uint32_t kst = s_stage + slot * L::kTileBytes, qst = s_qs + qb * L::kQSplitBytes;
@@ -1109,7 +1113,6 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     qi_col[nt][0] = p.Sq > 1 ? (8 * nt + 2 * t) / p.G : 0;
     qi_col[nt][1] = p.Sq > 1 ? (8 * nt + 2 * t + 1) / p.G : 0;
   }
-  uint32_t n_item_c = 0;  // items seen so far (KVM 2: item n reads the row scales of split tile n & 1)
   uint32_t mphase = 0;  // parity of the next merge-barrier phase to wait for
   bool merge_pending_read = false;
 
@@ -1126,7 +1129,6 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     if (meta.x < 0) break;
     const int ntok = meta.w & 0xffff;
     const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
-    if (first) ++n_item_c;
     if (first) {
       const uint8_t* qs = g_q + (size_t)slot * qslot;
 #pragma unroll
@@ -1171,7 +1173,7 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
         uint32_t f[8 * NT];
         tmem_ld_frag(tmem + ((uint32_t)r0 << 16) + sbuf * L::kTcSColumns, f);
         tmem_ld_wait();
-        const float* inva = reinterpret_cast<const float*>(gen + (s_inva - base)) + ((n_item_c - 1) & 1) * L::kHeads;
+        const float* inva = reinterpret_cast<const float*>(gen + (s_inva - base)) + sbuf * L::kHeads;
         float sv[NT][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
