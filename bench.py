@@ -427,6 +427,12 @@ def run_ours(args, rank, local_rank, world):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     cfg = inputs.replace(inputs.CONFIGS[args.workload], seed=inputs.CONFIGS[args.workload].seed + 100 * rank)
+    if args.batch_div > 1 or args.len_div > 1:                            # a smaller sibling (profiler captures)
+        cfg = inputs.scaled_config(cfg, batch_div=args.batch_div, len_div=args.len_div)
+        cfg = inputs.replace(cfg, description=cfg.description + f" [batch / {args.batch_div}, lengths / {args.len_div}]")
+    if args.block_size:                                                   # the same sequences over a pool of other blocks
+        cfg = inputs.replace(cfg, block_size=args.block_size, name=f"{cfg.name}-bs{args.block_size}",
+                             description=cfg.description + f" [block size overridden: {args.block_size}]")
     fp8 = args.kv == "fp8"
     res = measure_workload(args, cfg, dev, rank, world, e2e=True,
                            baseline=world == 1 and not args.no_cpu_baseline and not fp8)
@@ -440,7 +446,7 @@ def run_ours(args, rank, local_rank, world):
     # the other full-size workloads, timed the same way in the same run (N = 1 only)
     per_config = {}
     peak, peak_kind = measured_peak()
-    if world == 1 and not args.no_per_config:
+    if world == 1 and not args.no_per_config and not args.block_size and args.batch_div == 1 and args.len_div == 1:
         torch.cuda.empty_cache()
         for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
             if name == args.workload:
@@ -988,6 +994,10 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="time only --workload, not the other full-size workloads")
+    ap.add_argument("--block-size", type=int, default=0, choices=[0, 16, 32, 64, 128, 256],
+                    help="decode_step: KV block size instead of the workload's own (a sensitivity measurement; 0: keep)")
+    ap.add_argument("--batch-div", type=int, default=1, help="decode_step: divide the workload's sequence counts (a smaller sibling)")
+    ap.add_argument("--len-div", type=int, default=1, help="decode_step: divide the workload's context lengths")
     ap.add_argument("--replicas", type=int, default=0, help="pool replicas the steps rotate over (0: enough for 4 GiB)")
     ap.add_argument("--knob", action="append", default=[], help="launch-shape override name=value (sweeps)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
