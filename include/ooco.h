@@ -393,10 +393,12 @@ size_t ooco_step_staging_bytes(const ooco_shape_t* shape);
  *
  * When all six input buffers are page-locked and 16-byte aligned (cudaHostAlloc / cudaHostRegister,
  * e.g. torch pinned memory) the step's first launch reads them through their device mapping (the
- * planning and append CTAs directly, extra CTAs staging q and the block table for the attention
- * kernel), and a page-locked out_host is written by the attention kernels directly: three launches,
- * no copy-engine transfer.  Pageable buffers are detected and go through one cudaMemcpyAsync each.
- * The results are the same.
+ * planning and append CTAs directly, extra CTAs staging the block table and the lengths for the
+ * attention kernel), the attention kernel fetches each work item's q rows from the host mapping
+ * itself (with up to 8 query heads per kv head; otherwise q is staged too), and a page-locked
+ * out_host is written by the attention kernels directly: three launches, no copy-engine transfer,
+ * and q and out cross the host link while the attention runs.  Pageable buffers are detected and
+ * go through one cudaMemcpyAsync each.  The results are the same.
  *
  *   q_host, k_new_host, v_new_host   HOST (pinned for full copy speed), bf16
  *                                    [B,Hq,D], [B,Hkv,D], [B,Hkv,D]
@@ -450,7 +452,8 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * merge kernels with programmatic dependent launch (their prologues overlap the predecessor);
  * 9 CTAs per SM of the block-movement kernel {1..3}; 10 non-zero = ooco_decode_step_host reads
  * page-locked inputs through their device mapping and lets the kernels write a page-locked result
- * directly (zero = always one copy per buffer); 11 non-zero = 9 to 16 score columns per
+ * directly (zero = always one copy per buffer; 2 = as 1, but q is staged on the device by the first launch
+ * instead of being fetched from the host mapping by the attention kernel); 11 non-zero = 9 to 16 score columns per
  * (sequence, kv head) run the kernel whose warps share 16 score rows and split the tokens of a
  * stage (zero = the decode kernel with two 8-column tiles); 12 non-zero = more than 32 score columns
  * at head_dim 128 run the tcgen05 kernel (zero = the mma.sync kernel of the prefill-chunk path).

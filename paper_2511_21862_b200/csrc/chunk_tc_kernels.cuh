@@ -115,10 +115,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     // the end marker included).  A unit of work is (tile K / V, token row r, 16-byte chunk c of the row's 128
     // codes): one 16-byte load, sixteen codes widened, two 16-byte stores into the row's 64-dim half c / 4.
     const int ctid = threadIdx.x - 192;
+    const int nrw = KV8 ? nraw : 1;  // (this branch only exists for the 8-bit cache)
     bool ok = true;
     for (int it = 0;; ++it) {
-      const int rs = it % nraw, slot = it % nst;
-      if (!warp_wait(s_rfull + 8 * rs, (uint32_t)(it / nraw) & 1u, s_abort) ||
+      const int rs = it % nrw, slot = it % nst;
+      if (!warp_wait(s_rfull + 8 * rs, (uint32_t)(it / nrw) & 1u, s_abort) ||
           !warp_wait(s_empty + 8 * slot, ((uint32_t)(it / nst) & 1u) ^ 1u, s_abort)) {
         ok = false;
         break;

@@ -1,8 +1,9 @@
 // Paged decode attention for sm_100a: plan -> split-KV partial attention -> LSE merge.
 //
 // Work item = (sequence b, kv head h, token chunk [t0, t1)).  One CTA processes an item with
-// one producer warp that streams K / V tiles global -> shared through TMA (128-byte swizzle)
-// into a ring of stages, and NCW consumer warps that each own 16 tokens of every stage:
+// a producer warp that streams K / V tiles global -> shared through TMA (128-byte swizzle)
+// into a ring of stages (at head_dim 128 a second warp issues the V copies, from a descriptor
+// the first posts per stage), and NCW consumer warps that each own 16 tokens of every stage:
 //   S[16 tok x 8 heads]  = K_tile (A, ldmatrix) x Q^T (B, registers)          mma.sync bf16
 //   online softmax over tokens (warp shuffles), P packed to bf16, transposed by movmatrix
 //   O^T[D x 8 heads]    += V_tile^T (A, ldmatrix.trans) x P (B)               mma.sync bf16
@@ -390,14 +391,22 @@ struct SmemLayout {
   // Besides: the query of a work item as two E4M3 terms ([2 * kHeads rows][128 bytes], 1024-byte aligned), two
   // such tiles (consecutive items alternate), and beside every score buffer the inverse row scales of its item.
   static constexpr int kTcKSlots = 2, kTcSBuffers = 8;
+  // A second producer warp issues the V copies of every stage (the first hands it a descriptor per stage): one
+  // warp issuing all copies of a stage is the limit with small boxes.  Present for the 8-bit tcgen05 mode and for
+  // the bf16 cache at head_dim 128 (at head_dim 64 the extra warp would cost the fourth CTA per SM).
+  static constexpr bool kVProducer = KVM == 2 || (KVM == 0 && D == 128);
+  static constexpr int kWarps = NCW + 1 + (KVM == 2 ? 1 : 0) + (kVProducer ? 1 : 0);  // consumers, producer, [MMA], [V producer]
+  static constexpr int kVDescBytes = 96;  // what the V producer warp needs for one stage (see VStageDesc)
   static constexpr int kQSplitBytes = KVM == 2 ? 2 * kHeads * 128 : 0;
   static constexpr int kTcSColumns = 2 * kHeads;             // tensor-memory columns of one stage's scores
   __host__ __device__ static int q_slot_bytes(int G) { return ((G * D * 2 + 127) / 128) * 128; }
   __host__ __device__ static size_t total(int nstages, int G) {
     if (KVM == 2)
-      return 1024 + (size_t)kTcKSlots * (kTileBytes + q_slot_bytes(G) + 16 + 16) + (size_t)nstages * (kTileBytes + 16 + 16) +
-             kMergeBytes + 64 + 2 * kQSplitBytes + kTcSBuffers * (kHeads * 4 + 8) + 32;
-    return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16) + kMergeBytes + 64;
+      return 1024 + (size_t)kTcKSlots * (kTileBytes + q_slot_bytes(G) + 16 + 16) +
+             (size_t)nstages * (kTileBytes + 16 + 16 + kVDescBytes + 8) + kMergeBytes + 64 + 2 * kQSplitBytes +
+             kTcSBuffers * (kHeads * 4 + 8) + 32;
+    return 1024 + (size_t)nstages * (kStageBytes + q_slot_bytes(G) + 16 + 16 + (kVProducer ? kVDescBytes + 8 : 0)) +
+           kMergeBytes + 64;
   }
 };
 
@@ -706,6 +715,17 @@ __device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
   return d;
 }
 
+// KVM 2: one stage's V copies as the K producer hands them to the V producer warp (one slot per V ring slot).
+struct VStageDesc {
+  int32_t nbox;      // boxes (TMA copies) of the stage; -1 = end marker: arrive on the stage's barrier and stop
+  int32_t h;         // kv head
+  int32_t pad[2];
+  int32_t blk[8];    // physical block of box i (8 boxes of 16 rows fill a 128-token stage)
+  int32_t c_tok[8];  // first token row of box i inside its block
+  int32_t pad2[4];
+};
+static_assert(sizeof(VStageDesc) == 96, "descriptor slot is 96 bytes");
+
 // The 8-bit path is bound by the consumer warps' instruction latency, not by HBM, so its 8-warp shape
 // is compiled for two CTAs per SM (16 consumer warps), which caps it at 112 registers per thread (102 with the
 // extra MMA warp of KVM 2).
@@ -721,6 +741,8 @@ template <int D, int NCW, int NT, int TPW, int KVM>
 __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                                      const DecodeParams& p, uint8_t* smem_raw) {
   constexpr bool KV8 = KVM != 0, KVTC = KVM == 2;
+  constexpr bool VP = SmemLayout<D, NCW, NT, TPW, KVM>::kVProducer;  // the V copies are issued by a warp of their own
+  constexpr int kVProducerWarp = NCW + (KVTC ? 2 : 1);
   using L = SmemLayout<D, NCW, NT, TPW, KVM>;
   static_assert(!KV8 || (D == 128 && TPW == 1), "the 8-bit path is built for head_dim 128, one tile per warp");
   static_assert(!KVTC || NCW == 8, "a stage must hold the 128 tokens of one tcgen05 MMA");
@@ -753,6 +775,9 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
   const uint32_t s_qfree = s_tslot + 8;                     // KVM 2: [2] the MMAs that read split tile i are complete
   const uint32_t s_kfull = s_qfree + 16;                    // KVM 2: [kNK] the K tile (and the item's query rows) has landed
   const uint32_t s_kempty = s_kfull + (uint32_t)kNK * 8;    // KVM 2: [kNK] the MMAs that read the K tile are complete
+  const uint32_t s_vdfull = KVTC ? s_kempty + (uint32_t)kNK * 8 : s_mbar + 16;  // [nst] the stage's V descriptor is posted
+  const uint32_t s_vdesc = s_vdfull + (uint32_t)nst * 8;    // [nst] VStageDesc
+  VStageDesc* g_vdesc = reinterpret_cast<VStageDesc*>(gen + (s_vdesc - base));
   int4* g_kmeta = reinterpret_cast<int4*>(gen + (s_kmeta - base));
   float* g_merge = reinterpret_cast<float*>(gen + (s_merge - base));
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
@@ -768,6 +793,8 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
       mbar_init(s_empty + 8 * i, NCW);
     }
     mbar_init(s_mbar, NCW * 32);
+    if (VP)
+      for (int i = 0; i < nst; ++i) mbar_init(s_vdfull + 8 * i, 1);
     if (KVTC) {
       for (int i = 0; i < kNS; ++i) mbar_init(s_sready + 8 * i, 1);
       for (int i = 0; i < kNK; ++i) {
@@ -882,11 +909,60 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
     return tmem;
   }
 
+  if (VP && warp == kVProducerWarp) {
+    // ================================================================= V producer warp
+    // With blocks of 16 tokens a stage is 4 to 8 K boxes and as many V boxes of 2 to 4 KiB; one warp issuing every
+    // copy of every stage does not keep up with HBM, so the producer below posts each stage's V boxes here.
+    if (lane == 0) prefetch_tmap(&tm_v);
+    const uint32_t vbox_bytes = (uint32_t)p.tile_rows * D * (KV8 ? 1 : 2);
+    int it = 0;
+    bool ok = true;
+    for (;; ++it) {
+      const int slot = it % nst;
+      if (!warp_wait(s_vdfull + 8 * slot, (uint32_t)(it / nst) & 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      const VStageDesc& vd = g_vdesc[slot];
+      const int nbox = vd.nbox;
+      const uint32_t full = s_full + 8 * slot;
+      if (nbox < 0) {  // end marker (KVM 2: the consumer warps see it through the V ring's barrier, arrived on here)
+        if (KVTC && lane == 0) mbar_arrive(full);
+        break;
+      }
+      // (bf16: the producer has armed the stage's barrier for the K, V and q bytes together)
+      if (KVTC && lane == 0) mbar_arrive_expect_tx(full, (uint32_t)nbox * vbox_bytes);
+      __syncwarp();
+      if (lane < nbox && lane < 8) {
+        const uint32_t dv = (KVTC ? s_vring + (uint32_t)slot * L::kTileBytes
+                                  : s_stage + (uint32_t)slot * L::kStageBytes + L::kTileBytes) + lane * vbox_bytes;
+        const int c_tok = vd.c_tok[lane], h = vd.h, blk = vd.blk[lane];
+        if (KV8) {
+          tma_load_4d(dv, &tm_v, full, 0, c_tok, h, blk);
+        } else if (D == 128 && !p.split_halves) {
+          tma_load_5d(dv, &tm_v, full, 0, c_tok, 0, h, blk);
+        } else {
+#pragma unroll
+          for (int j = 0; j < D / 64; ++j) tma_load_4d(dv + j * (vbox_bytes / (D / 64)), &tm_v, full, 64 * j, c_tok, h, blk);
+        }
+      }
+    }
+    if (!ok) {  // stop path: wait (bounded) until every V copy already issued has landed
+      if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+      int dummy_abort = 0;
+      for (int k = 0; k < (it < nst ? it : nst); ++k) {
+        const int j = it - 1 - k;
+        mbar_wait_bounded(s_full + 8 * (j % nst), (uint32_t)(j / nst) & 1u, &dummy_abort, kWaitLimitNs / 8);
+      }
+    }
+    return tmem;
+  }
+
   if (warp == NCW) {
     // ================================================================= producer warp
     if (lane == 0) {
       prefetch_tmap(&tm_k);
-      prefetch_tmap(&tm_v);
+      if (!VP) prefetch_tmap(&tm_v);
     }
     const int boxes_per_stage = kStageTok / p.tile_rows;
     const uint32_t box_bytes = (uint32_t)p.tile_rows * D * (KV8 ? 1 : 2);
@@ -965,12 +1041,17 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
           const int4 meta = make_int4(slot_id, b, h, ntok | (flags << 16) | (cm << 18));
           g_meta[slot] = meta;
           const uint32_t qbytes = s == 0 ? (uint32_t)p.GQ * D * 2 : 0u;
-          if (KVTC) {
+          if (KVTC) {  // (the V producer warp arms the stage's own barrier)
             g_kmeta[kslot] = meta;
             mbar_arrive_expect_tx(kfull, nbox * box_bytes + qbytes);
-            mbar_arrive_expect_tx(full, nbox * box_bytes);
+            g_vdesc[slot].nbox = nbox;
+            g_vdesc[slot].h = h;
           } else {
             mbar_arrive_expect_tx(full, 2u * nbox * box_bytes + qbytes);
+            if (VP) {
+              g_vdesc[slot].nbox = nbox;
+              g_vdesc[slot].h = h;
+            }
           }
         }
         __syncwarp();
@@ -987,18 +1068,26 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
                             &p.hdr->status, kStatusBadSmem);
           if (!span_ok) {
             // skipped
+          } else if (KVTC) {  // the K box here, the V box through the V producer warp
+            tma_load_4d(dk, &tm_k, kfull, 0, c_tok, h, blk_cur);
+            g_vdesc[slot].blk[lane & 7] = blk_cur;
+            g_vdesc[slot].c_tok[lane & 7] = c_tok;
           } else if (KV8) {  // a token row is one 128-byte swizzle row: one 4-d copy per box
             tma_load_4d(dk, &tm_k, kfull, 0, c_tok, h, blk_cur);
             tma_load_4d(dv, &tm_v, full, 0, c_tok, h, blk_cur);
           } else if (D == 128 && !p.split_halves) {
             tma_load_5d(dk, &tm_k, full, 0, c_tok, 0, h, blk_cur);
-            tma_load_5d(dv, &tm_v, full, 0, c_tok, 0, h, blk_cur);
+            if (!VP) tma_load_5d(dv, &tm_v, full, 0, c_tok, 0, h, blk_cur);
           } else {
 #pragma unroll
             for (int j = 0; j < D / 64; ++j) {
               tma_load_4d(dk + j * (box_bytes / (D / 64)), &tm_k, full, 64 * j, c_tok, h, blk_cur);
-              tma_load_4d(dv + j * (box_bytes / (D / 64)), &tm_v, full, 64 * j, c_tok, h, blk_cur);
+              if (!VP) tma_load_4d(dv + j * (box_bytes / (D / 64)), &tm_v, full, 64 * j, c_tok, h, blk_cur);
             }
+          }
+          if (VP && !KVTC && span_ok) {  // the V box goes through the V producer warp
+            g_vdesc[slot].blk[lane & 7] = blk_cur;
+            g_vdesc[slot].c_tok[lane & 7] = c_tok;
           }
         }
         if (s == 0 && lane < p.Sq) {  // one run of G heads per query token, side by side: [query][head][D]
@@ -1014,6 +1103,10 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
           violated = true;
           ok = false;
           break;
+        }
+        if (VP) {  // hand the stage's V boxes to the V producer warp
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s_vdfull + 8 * slot);
         }
         // look ahead to the next item: its descriptor, then its first table entries
         if (s == 0) {
@@ -1041,10 +1134,17 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
           (!KVTC || warp_wait(s_kempty + 8 * kslot, (((uint32_t)it / kNK) & 1u) ^ 1u, s_abort))) {
         if (lane == 0) {
           g_meta[slot] = make_int4(-1, 0, 0, 0);
-          mbar_arrive(s_full + 8 * slot);
-          if (KVTC) {
+          if (KVTC) {  // the consumers' marker travels through the V producer warp, which stops on it too
+            g_vdesc[slot].nbox = -1;
+            mbar_arrive(s_vdfull + 8 * slot);
             g_kmeta[kslot] = make_int4(-1, 0, 0, 0);
             mbar_arrive(s_kfull + 8 * kslot);
+          } else {
+            mbar_arrive(s_full + 8 * slot);
+            if (VP) {  // the V producer warp stops on the marker too
+              g_vdesc[slot].nbox = -1;
+              mbar_arrive(s_vdfull + 8 * slot);
+            }
           }
         }
         ++it;
@@ -1056,7 +1156,7 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
       // stop path: record it, then wait (bounded) until every copy already issued has landed
       if (lane == 0 && !violated) atomicOr(&p.hdr->status, kStatusWaitTimeout);
       int dummy_abort = 0;
-      const int pending = it < nst ? it : nst;
+      const int pending = KVTC ? 0 : (it < nst ? it : nst);  // (KVM 2: the V producer warp drains the V ring)
       for (int k = 0; k < pending; ++k) {
         const int j = it - 1 - k;
         mbar_wait_bounded(s_full + 8 * (j % nst), (uint32_t)(j / nst) & 1u, &dummy_abort, kWaitLimitNs / 8);
@@ -1295,7 +1395,7 @@ __device__ __forceinline__ uint32_t decode_main_body(const CUtensorMap& tm_k, co
 }
 
 template <int D, int NCW, int NT, int TPW, int KVM = 0>
-__global__ void __launch_bounds__((NCW + (KVM == 2 ? 2 : 1)) * 32, (KVM && NCW == 8 && NT == 1) ? 2 : 1)
+__global__ void __launch_bounds__(SmemLayout<D, NCW, NT, TPW, KVM>::kWarps * 32, (KVM && NCW == 8 && NT == 1) ? 2 : 1)
 decode_main_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const DecodeParams p) {
   extern __shared__ uint8_t smem_raw[];

@@ -237,7 +237,7 @@ static int launch_main(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParam
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
   if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
-  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3((NCW + (KVM == 2 ? 2 : 1)) * 32), smem, st,
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(L::kWarps * 32), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the attention kernel", (long)e);
@@ -1146,9 +1146,15 @@ int ooco_decode_step_host(const ooco_shape_t* s, const void* q_host, const void*
       hs.dst[k] = ddst[pick[k]];
       hs.bytes[k] = (uint32_t)nbytes[pick[k]];
     }
+    // The decode kernel (up to 8 query heads per kv head) fetches the q rows of a work item with one bulk copy
+    // beside the item's first K / V stage: it takes them from the host mapping itself, so q crosses the host link
+    // while the attention runs instead of in front of it.  (The 16-row kernel loads q with plain loads at the
+    // start of an item and keeps the staged copy.)
+    const bool q_direct = s->num_q_heads / s->num_kv_heads <= 8 && g_knobs[kKnobHostStageKernel].load() != 2;
+    if (q_direct) hs.bytes[0] = 0;
     const AppendParams ap = make_append_params(s, msrc[1], msrc[2], k_cache, v_cache, (const int32_t*)msrc[3],
                                                (const int32_t*)msrc[4]);
-    if ((rc = decode_core(s, d_q, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_len, scale, out_dev,
+    if ((rc = decode_core(s, q_direct ? msrc[0] : (const void*)d_q, k_cache, v_cache, (const int32_t*)d_tab, (const int32_t*)d_len, scale, out_dev,
                           workspace, workspace_bytes, st, &ap, nullptr, 1, &hs, (const int32_t*)msrc[5])))
       return rc;
   } else {

@@ -164,12 +164,23 @@ def test_kv_append_skips_bad_positions():
     assert np.array_equal(inputs.as_u16(batch.k_cache), k_ref) and np.array_equal(inputs.as_u16(batch.v_cache), v_ref)
 
 
-@pytest.mark.parametrize("pinned,launches", [(True, 3), (False, 3)], ids=["page-locked", "pageable"])
-def test_serving_step_from_host_buffers(pinned, launches):
+@pytest.mark.parametrize("pinned,stage_knob,hq", [(True, 1, 32), (True, 2, 32), (True, 1, 128), (False, 1, 32)],
+                         ids=["page-locked", "page-locked-q-staged", "page-locked-16-heads-per-kv-head", "pageable"])
+def test_serving_step_from_host_buffers(pinned, stage_knob, hq):
     """append at T then attend T + 1 through the host-buffer entry point: page-locked buffers are read
-    through their device mapping inside the first launch and the result is written to the host
-    directly; pageable ones are copied."""
-    cfg = C("step", 32, 8, 128, 16, (G(9, 1, 2500),), seed=50, pool_fill=0.8)
+    through their device mapping (q by the attention kernel itself, or staged by the first launch: behind
+    the knob and for the 16-row kernel) and the result is written to the host directly; pageable ones are
+    copied."""
+    launches = 3
+    cfg = C("step", hq, 8, 128, 16, (G(9, 1, 2500),), seed=50, pool_fill=0.8)
+    binding.set_tuning(host_stage_kernel=stage_knob)
+    try:
+        _serving_step_from_host_buffers(cfg, pinned, launches)
+    finally:
+        binding.set_tuning(host_stage_kernel=1)
+
+
+def _serving_step_from_host_buffers(cfg, pinned, launches):
     batch = inputs.make_batch(cfg, "cuda", poison=True)
     sh = binding.shape_of(batch)
     pin = (lambda t: t.cpu().contiguous().pin_memory()) if pinned else (lambda t: t.cpu().contiguous().clone())
@@ -190,6 +201,31 @@ def test_serving_step_from_host_buffers(pinned, launches):
                                   lens1.numpy(), cfg.scale, num_kv_heads=8, block_size=16, strides=batch.strides)
     assert_parity(out_h, ref.out, what="host step")
     assert binding.last_launch_count() == launches
+
+
+def test_refused_fused_step_enqueues_nothing():
+    """A call that returns an argument error has touched no buffer: the fused step with a workspace that is too
+    small (or misaligned) leaves the pool, `out` and the workspace as they were."""
+    cfg = C("refused", 32, 8, 128, 16, (G(6, 100, 900),), seed=53)
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    sh = binding.shape_of(batch)
+    ws = torch.zeros(binding.workspace_bytes(sh) + 256, dtype=torch.uint8, device="cuda")
+    out = torch.full_like(batch.q, float("nan"))
+    lens1 = (batch.context_lens + 1).contiguous()
+    k0, v0 = batch.k_cache.clone(), batch.v_cache.clone()
+    for bad_ws in (ws[:1024], ws[16:]):                                        # too small; not 256-byte aligned
+        with pytest.raises(binding.OocoError) as err:
+            binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, batch.k_cache, batch.v_cache, batch.block_table,
+                                batch.context_lens, lens1, cfg.scale, out, bad_ws)
+        assert err.value.status == -4
+    with pytest.raises(binding.OocoError) as err:                              # softmax scale must be positive
+        binding.decode_step(sh, batch.q, batch.k_new, batch.v_new, batch.k_cache, batch.v_cache, batch.block_table,
+                            batch.context_lens, lens1, 0.0, out, ws[:binding.workspace_bytes(sh)])
+    assert err.value.status == -2
+    torch.cuda.synchronize()
+    assert torch.equal(batch.k_cache.view(torch.int16), k0.view(torch.int16))
+    assert torch.equal(batch.v_cache.view(torch.int16), v0.view(torch.int16))
+    assert torch.isnan(out.float()).all() and int(ws.count_nonzero()) == 0
 
 
 def test_fused_step_on_device_buffers():
