@@ -463,6 +463,8 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * test can separate the arithmetic's error from the output format's rounding; not for the host-buffer
  * step (OOCO_E_UNSUPPORTED).  14 non-zero = the decode kernel over the 8-bit cache (8 consumer warps)
  * computes its scores on tcgen05 from the stored codes (zero = mma.sync on codes widened in registers).
+ * 15 non-zero = prefill chunks of more than 128 score columns over a bf16 cache (head_dim 128) run the tcgen05
+ * kernel that keeps two 128-row tiles per CTA (zero = one tile per CTA, two CTAs per SM).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.  ooco_get_tuning returns a knob's current value
  * (OOCO_E_SHAPE, which is negative, for an unknown knob).

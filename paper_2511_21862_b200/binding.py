@@ -173,7 +173,7 @@ class Shape:
 
 KNOBS = {"warps": 0, "stages": 1, "ctas_per_sm": 2, "chunk_min": 3, "chunk_max": 4, "items_per_cta": 5,
          "split_halves": 6, "tiles_per_warp": 7, "pdl": 8, "copy_ctas_per_sm": 9, "host_stage_kernel": 10, "row_layout_16": 11, "chunk_tcgen05": 12,
-         "out_f32": 13, "kv8_tcgen05": 14}
+         "out_f32": 13, "kv8_tcgen05": 14, "chunk_two_tiles": 15}
 
 
 def set_tuning(**kw):

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libooco.so")
 LIB_CHECKED = os.path.join(HERE, "libooco_checked.so")   # the same sources with -DOOCO_CHECKS
 SOURCES = ["ooco_api.cu", "ooco_sched.cpp"]
-HEADERS = ["decode_kernels.cuh", "chunk_kernels.cuh", "chunk_tc_kernels.cuh", "block_copy_kernels.cuh", "ptx.cuh", os.path.join("..", "..", "include", "ooco.h"),
+HEADERS = ["decode_kernels.cuh", "chunk_kernels.cuh", "chunk_tc_kernels.cuh", "chunk_tc2_kernels.cuh", "block_copy_kernels.cuh", "ptx.cuh", os.path.join("..", "..", "include", "ooco.h"),
            os.path.join("..", "..", "include", "ooco_sched.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",

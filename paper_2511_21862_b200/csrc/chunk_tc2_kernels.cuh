@@ -1,0 +1,614 @@
+// Prefill-chunk attention over the paged cache on tcgen05, two row tiles per CTA (head_dim 128, bf16 cache, more than
+// 128 score columns per (sequence, kv head)).  Same plan, merge and work items as chunk_tc_kernel
+// (chunk_tc_kernels.cuh); a unit of work is (item, PAIR of 128-row tiles), one persistent CTA per SM:
+//
+//   warps 0..3   softmax of tile 0: thread r owns score row r of the tile (tensor-memory lane r)
+//   warps 4..7   softmax of tile 1
+//   warp 8       K producer: walks the units, TMA copies of the K slots (128 tokens: [half][128 tok][64 dims],
+//                128-byte swizzle), posts each stage's meta words and a descriptor of its V boxes
+//   warp 9       V producer: TMA copies of the V slots from those descriptors
+//   warp 10      owns the tensor memory (512 columns); one lane issues the MMAs of both tiles:
+//                  S_t[128 x 128]   = Q_t[128 x 128] . K_slot^T    8 x tcgen05.mma M128 N128 K16, both operands shared memory
+//                  O_t[128 x 128] (+)= P_t[128 x 128] . V_slot      8 x tcgen05.mma M128 N128 K16, P from tensor memory,
+//                                                                   V MN-major from the slot
+//                columns of tile t: S_t at 256 t (P_t, two bf16 per column, over its first 64 once the softmax
+//                threads have read S_t), O_t at 256 t + 128.  Q_t lives in shared memory (32 KiB per tile).
+//
+// The two tiles share every K / V slot (half the shared-memory fills of one tile per CTA) and take turns on the tensor
+// pipe: the MMAs are issued in the order  S_0(j) S_1(j) | P.V_0(j) S_0(j+1) P.V_1(j) S_1(j+1) | P.V_0(j+1) ...  so that
+// while the softmax threads of one tile work on their scores the pipe runs the other tile's MMAs.  The pipe executes
+// one thread's MMAs in order, which makes it safe for S_t(j+1) to overwrite P_t(j), and means P.V_t(j-1) is complete
+// whenever S_t(j) is: a softmax thread may rescale its row of O_t as soon as it holds the scores.  With 128-token
+// slots the fetch of the shared-memory A operand (Q) is amortised over twice the columns: the score MMAs are no longer
+// bound by it.  Every wait is bounded; on a wait that gives up the CTA stops issuing, drains and releases the tensor
+// memory.
+#pragma once
+#include "chunk_tc_kernels.cuh"
+
+namespace ooco {
+
+constexpr int kTc2StageTok = 128;                    // tokens of K (or V) per slot
+constexpr int kTc2HalfBytes = kTc2StageTok * 128;    // [128 tok][64 dims] bf16
+constexpr int kTc2SlotBytes = 2 * kTc2HalfBytes;     // K (or V) of one stage: 32 KiB
+constexpr int kTc2QBytes = 2 * kTcRows * 128;        // one tile's queries: [half][128 rows][64 dims] bf16, 32 KiB
+constexpr int kTc2Rows = 2 * kTcRows;                // score rows of a unit
+constexpr int kTc2TmemCols = 512;
+constexpr int kTc2KSlots = 2, kTc2VSlots = 3, kTc2MetaRing = 8;
+
+struct ChunkTc2Smem {
+  __host__ __device__ static size_t total() {
+    return 1024 + 2 * (size_t)kTc2QBytes + (size_t)(kTc2KSlots + kTc2VSlots) * kTc2SlotBytes + kTc2MetaRing * 32 +
+           kTc2VSlots * sizeof(VStageDesc) + 256;
+  }
+};
+
+// Barrier bookkeeping.  Stage number n (counted over the whole kernel, bookkeeping stages and the end marker
+// included) uses K slot n % 2, V slot n % 3, meta entry n % 8 and, for each tile, barrier n & 1 of the pairs
+// [2] below with phase parity (n >> 1) & 1 -- every tile takes a turn of its barriers on every stage, with or
+// without work, so nobody can be overtaken by two completions of a barrier it waits on.
+__global__ void __launch_bounds__(352, 1)
+chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                 const DecodeParams p) {
+  constexpr int D = 128;
+  constexpr int NK = kTc2KSlots, NV = kTc2VSlots, NM = kTc2MetaRing;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const uint32_t s_q = base;                                       // [2] Q tiles
+  const uint32_t s_k = s_q + 2u * kTc2QBytes;                      // [NK] K slots
+  const uint32_t s_v = s_k + (uint32_t)NK * kTc2SlotBytes;         // [NV] V slots
+  const uint32_t s_meta = s_v + (uint32_t)NV * kTc2SlotBytes;      // [NM] two int4 per stage
+  const uint32_t s_vdesc = s_meta + (uint32_t)NM * 32;             // [NV] VStageDesc
+  const uint32_t s_bar = s_vdesc + (uint32_t)NV * sizeof(VStageDesc);
+  const uint32_t s_kfull = s_bar;                  // [NK] the K slot has landed                          (TMA)
+  const uint32_t s_kempty = s_kfull + NK * 8;      // [NK] the score MMAs that read it are complete       (MMA commit)
+  const uint32_t s_vfull = s_kempty + NK * 8;      // [NV] the V slot has landed                          (TMA)
+  const uint32_t s_vempty = s_vfull + NV * 8;      // [NV] the P.V MMAs that read it are complete         (MMA commit)
+  const uint32_t s_vdfull = s_vempty + NV * 8;     // [NV] the stage's V descriptor is posted             (K producer)
+  const uint32_t s_mfull = s_vdfull + NV * 8;      // [NM] the stage's meta words are posted              (K producer)
+  const uint32_t s_sready = s_mfull + NM * 8;      // [2 tiles][2] S_t holds the stage's scores            (MMA commit)
+  const uint32_t s_pready = s_sready + 32;         // [2 tiles][2] P_t written, O_t rescaled, V rows clean (128 threads)
+  const uint32_t s_pvdone = s_pready + 32;         // [2 tiles] the unit's last P.V_t is complete          (MMA commit)
+  const uint32_t s_qready = s_pvdone + 16;         // [2 tiles] Q_t of the unit is in shared memory        (128 threads)
+  const uint32_t s_drain = s_qready + 16;
+  const uint32_t s_slot = s_drain + 8;
+  int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
+  VStageDesc* g_vdesc = reinterpret_cast<VStageDesc*>(gen + (s_vdesc - base));
+  volatile uint32_t* g_slot = reinterpret_cast<volatile uint32_t*>(gen + (s_slot - base));
+  volatile int* s_abort = reinterpret_cast<volatile int*>(gen + (s_slot + 4 - base));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    *s_abort = 0;
+    for (int i = 0; i < NK; ++i) {
+      mbar_init(s_kfull + 8 * i, 1);
+      mbar_init(s_kempty + 8 * i, 1);
+    }
+    for (int i = 0; i < NV; ++i) {
+      mbar_init(s_vfull + 8 * i, 1);
+      mbar_init(s_vempty + 8 * i, 1);
+      mbar_init(s_vdfull + 8 * i, 1);
+    }
+    for (int i = 0; i < NM; ++i) mbar_init(s_mfull + 8 * i, 1);
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(s_sready + 8 * i, 1);
+      mbar_init(s_pready + 8 * i, 128);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(s_pvdone + 8 * i, 1);
+      mbar_init(s_qready + 8 * i, 128);
+    }
+    mbar_init(s_drain, 1);
+    fence_mbar_init();
+  }
+  if (warp == 10) tmem_alloc(s_slot, kTc2TmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = *g_slot;
+  grid_dep_wait();    // the plan (and a fused append) must have completed
+  grid_dep_launch();  // the merge kernel may queue up behind this grid
+
+  const int nrt = (p.GQ + kTc2Rows - 1) / kTc2Rows;  // tile pairs per work item
+  const long long cap_tokens = (long long)p.MB * p.bs;
+
+  if (warp == 8) {
+    // ================================================================= K producer (and the walk over the units)
+    if (lane == 0) prefetch_tmap(&tm_k);
+    const long long n_units = (long long)p.hdr->n_items * nrt;
+    const int boxes_per_stage = kTc2StageTok / p.tile_rows;   // at most 8 (blocks of 16 tokens)
+    const uint32_t box_rows_bytes = (uint32_t)p.tile_rows * 128;
+    int it = 0;
+    bool ok = true, violated = false;
+    long long unit = blockIdx.x;
+    auto table_entry = [&](const int32_t* e) {
+      const int v = *e;
+      return checked(chk_table_entry(v, p.NB), &p.hdr->status, kStatusBadTableEntry) ? v : p.NB;
+    };
+    // waits until K slot, V slot (and with it the V descriptor) of stage `it` are free; false when a wait gave up
+    auto acquire = [&]() {
+      return warp_wait(s_kempty + 8 * (it % NK), (((uint32_t)(it / NK)) & 1u) ^ 1u, s_abort) &&
+             warp_wait(s_vempty + 8 * (it % NV), (((uint32_t)(it / NV)) & 1u) ^ 1u, s_abort);
+    };
+    while (unit < n_units && ok) {
+      int nxt = 0;
+      if (lane == 0) nxt = atomicAdd(&p.hdr->next_item, 1);
+      nxt = __shfl_sync(0xffffffffu, nxt, 0);
+      // the last tile pair of an item sees the most tokens: it goes first (longest work first)
+      const int item = (int)(unit / nrt), rt = nrt - 1 - (int)(unit - (long long)item * nrt);
+      const int4 d = p.items[item];
+      if (!checked(chk_item(d.x, d.y, d.z, d.w, p.B, p.max_items, cap_tokens), &p.hdr->status, kStatusBadItem)) {
+        *s_abort = 1;
+        violated = true;
+        ok = false;
+        break;
+      }
+      const int b = d.x, h = d.y % p.Hkv, t0 = d.z, t1 = d.w;
+      long long T = p.context_lens[b];
+      T = T < 0 ? 0 : (T > cap_tokens ? cap_tokens : T);
+      const int lim_base = (int)T - p.Sq + 1;                      // tokens the first query token sees
+      const int col_hi = min(p.GQ, (rt + 1) * kTc2Rows) - 1;
+      const int t1e = min(t1, lim_base + col_hi / p.G);             // nothing beyond is visible to this tile pair
+      const int nstage = t1e > t0 ? (t1e - t0 + kTc2StageTok - 1) / kTc2StageTok : 0;
+      const int32_t* row = p.block_table + (size_t)b * p.MB;
+      int blk_cur = 0;
+      {
+        const int tb = t0 + lane * p.tile_rows;
+        if (lane < boxes_per_stage && tb < t1e) blk_cur = table_entry(row + tb / p.bs);
+      }
+      // a pair that sees nothing of this chunk passes one stage without tokens, which carries the bookkeeping
+      for (int s = 0; s < (nstage > 0 ? nstage : 1); ++s, ++it) {
+        const int tok0 = t0 + s * kTc2StageTok;
+        const int ntok = nstage > 0 ? min(kTc2StageTok, t1e - tok0) : 0;
+        const int nbox = (ntok + p.tile_rows - 1) / p.tile_rows;
+        int blk_n = 0;  // table entries of the following stage, one stage ahead of their use
+        {
+          const int tb = tok0 + kTc2StageTok + lane * p.tile_rows;
+          if (s + 1 < nstage && lane < boxes_per_stage && tb < t1e) blk_n = table_entry(row + tb / p.bs);
+        }
+        if (!acquire()) {
+          ok = false;
+          break;
+        }
+        const int ks = it % NK, vs = it % NV, ms = it % NM;
+        const uint32_t kfull = s_kfull + 8 * ks;
+        if (lane == 0) {
+          const int flags = (s == 0 ? 1 : 0) | (s == (nstage > 0 ? nstage : 1) - 1 ? 2 : 0);
+          g_meta[2 * ms] = make_int4(d.y, b, h, ntok | (flags << 16));
+          g_meta[2 * ms + 1] = make_int4(tok0, lim_base, t1, rt);
+          g_vdesc[vs].nbox = nbox;
+          g_vdesc[vs].h = h;
+          if (nbox > 0)
+            mbar_arrive_expect_tx(kfull, 2u * (uint32_t)nbox * box_rows_bytes);
+          else
+            mbar_arrive(kfull);
+        }
+        __syncwarp();
+        bool span_ok = true;
+        if (lane < nbox) {
+          const int tb = tok0 + lane * p.tile_rows;
+          const int c_tok = tb % p.bs;
+          const uint32_t k0 = s_k + (uint32_t)ks * kTc2SlotBytes;
+          const uint32_t dk = k0 + (uint32_t)lane * box_rows_bytes;
+          span_ok = checked(chk_span(dk, box_rows_bytes, k0, (long long)k0 + kTc2HalfBytes) && chk_span(lane, 1, 0, 8),
+                            &p.hdr->status, kStatusBadSmem);
+          if (span_ok) {
+            tma_load_4d(dk, &tm_k, kfull, 0, c_tok, h, blk_cur);
+            tma_load_4d(dk + kTc2HalfBytes, &tm_k, kfull, 64, c_tok, h, blk_cur);
+            g_vdesc[vs].blk[lane & 7] = blk_cur;
+            g_vdesc[vs].c_tok[lane & 7] = c_tok;
+          }
+        }
+        if (kChecked && !__all_sync(0xffffffffu, span_ok)) {  // a skipped copy leaves the stage incomplete: stop
+          *s_abort = 1;
+          violated = true;
+          ok = false;
+          break;
+        }
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(s_vdfull + 8 * vs);  // the V producer takes over the stage's V boxes
+          mbar_arrive(s_mfull + 8 * ms);   // the softmax threads may read the meta words
+        }
+        blk_cur = blk_n;
+      }
+      unit = nxt;
+    }
+    if (ok) {  // end marker: one more stage, seen by every other warp
+      if (acquire()) {
+        if (lane == 0) {
+          g_meta[2 * (it % NM)] = make_int4(-1, 0, 0, 0);
+          g_vdesc[it % NV].nbox = -1;
+          mbar_arrive(s_kfull + 8 * (it % NK));
+          mbar_arrive(s_vdfull + 8 * (it % NV));
+          mbar_arrive(s_mfull + 8 * (it % NM));
+        }
+        ++it;
+      } else {
+        ok = false;
+      }
+    }
+    if (!ok) {  // stop path: record it, then wait (bounded) until every K copy already issued has landed
+      if (lane == 0 && !violated) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+      int dummy_abort = 0;
+      for (int k = 0; k < (it < NK ? it : NK); ++k) {
+        const int j = it - 1 - k;
+        mbar_wait_bounded(s_kfull + 8 * (j % NK), (uint32_t)(j / NK) & 1u, &dummy_abort, kWaitLimitNs / 8);
+      }
+    }
+  } else if (warp == 9) {
+    // ================================================================= V producer
+    if (lane == 0) prefetch_tmap(&tm_v);
+    const uint32_t box_rows_bytes = (uint32_t)p.tile_rows * 128;
+    int it = 0;
+    bool ok = true;
+    for (;; ++it) {
+      const int vs = it % NV;
+      if (!warp_wait(s_vdfull + 8 * vs, (uint32_t)(it / NV) & 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      const VStageDesc& vd = g_vdesc[vs];
+      const int nbox = vd.nbox;
+      const uint32_t vfull = s_vfull + 8 * vs;
+      if (nbox <= 0) {  // a stage without tokens, or the end marker
+        if (lane == 0) mbar_arrive(vfull);
+        if (nbox < 0) break;
+        continue;
+      }
+      if (lane == 0) mbar_arrive_expect_tx(vfull, 2u * (uint32_t)nbox * box_rows_bytes);
+      __syncwarp();
+      if (lane < nbox && lane < 8) {
+        const uint32_t dv = s_v + (uint32_t)vs * kTc2SlotBytes + (uint32_t)lane * box_rows_bytes;
+        tma_load_4d(dv, &tm_v, vfull, 0, vd.c_tok[lane], vd.h, vd.blk[lane]);
+        tma_load_4d(dv + kTc2HalfBytes, &tm_v, vfull, 64, vd.c_tok[lane], vd.h, vd.blk[lane]);
+      }
+    }
+    if (!ok) {
+      if (lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+      int dummy_abort = 0;
+      for (int k = 0; k < (it < NV ? it : NV); ++k) {
+        const int j = it - 1 - k;
+        mbar_wait_bounded(s_vfull + 8 * (j % NV), (uint32_t)(j / NV) & 1u, &dummy_abort, kWaitLimitNs / 8);
+      }
+    }
+  } else if (warp == 10) {
+    // ================================================================= MMA warp
+    const uint32_t idesc_s = umma_idesc_16bit(kTcRows, kTc2StageTok, 0, true);
+    const uint32_t idesc_o = umma_idesc_16bit(kTcRows, D, 1, true);
+    uint32_t n_q[2] = {0u, 0u};  // units in which tile t had rows and tokens (uses of its q-ready barrier)
+    bool issued = false, ok = true;
+    // what is known about the stage whose P.V MMAs are still to be issued
+    struct Pending {
+      bool valid, act[2], first, last;
+      int ntok, vs;
+      uint32_t n;
+    } pend = {false, {false, false}, false, false, 0, 0, 0u};
+    // P.V of tile t for the pending stage: waits for the tile's softmax threads, then issues (or just takes the turn)
+    auto issue_pv = [&](int t) {
+      const uint32_t n = pend.n;
+      if (!warp_wait(s_pready + 8 * (2 * t + (n & 1)), (n >> 1) & 1u, s_abort)) return false;
+      if (pend.act[t] && pend.ntok > 0) {
+        if (!warp_wait(s_vfull + 8 * pend.vs, ((uint32_t)(n / NV)) & 1u, s_abort)) return false;
+        tc_fence_after_sync();
+        if (lane == 0) {
+          const uint32_t vst = s_v + (uint32_t)pend.vs * kTc2SlotBytes, ts = tmem + 256u * t;
+#pragma unroll
+          for (int k = 0; k < kTc2StageTok / 16; ++k)  // 16 tokens: 8 columns of P, 16 rows of 128 bytes of V in either half
+            umma_ts(ts + 128, ts + 8 * k, umma_smem_desc(vst + k * 2048, kTc2HalfBytes, 1024), idesc_o,
+                    (pend.first && k == 0) ? 0u : 1u);
+          if (pend.last) umma_commit(s_pvdone + 8 * t);
+        }
+        __syncwarp();
+        issued = true;
+      } else if (pend.act[t] && pend.last) {
+        if (lane == 0) mbar_arrive(s_pvdone + 8 * t);  // a unit without tokens: nothing to wait for
+        __syncwarp();
+      }
+      return true;
+    };
+    // the V slot of the pending stage is free once both tiles' P.V are complete
+    auto release_v = [&]() {
+      if (lane == 0) {
+        if (pend.ntok > 0 && (pend.act[0] || pend.act[1]))
+          umma_commit(s_vempty + 8 * pend.vs);
+        else
+          mbar_arrive(s_vempty + 8 * pend.vs);
+      }
+      __syncwarp();
+    };
+    for (uint32_t n = 0;; ++n) {
+      const int ks = n % NK, ms = n % NM;
+      if (!warp_wait(s_kfull + 8 * ks, (n / NK) & 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      const int4 meta = g_meta[2 * ms], meta2 = g_meta[2 * ms + 1];
+      const bool end = meta.x < 0;
+      const int ntok = end ? 0 : (meta.w & 0xffff);
+      const bool first = !end && ((meta.w >> 16) & 1), last = !end && ((meta.w >> 17) & 1);
+      const int rt = end ? 0 : meta2.w;
+      bool act[2];
+      act[0] = !end;                                            // a unit always has rows in its first tile
+      act[1] = !end && rt * kTc2Rows + kTcRows < p.GQ;
+      // ---- tile 0: S_0 of this stage goes behind P.V_0 of the pending one
+      if (pend.valid && !issue_pv(0)) {
+        ok = false;
+        break;
+      }
+#pragma unroll 1
+      for (int t = 0; t < 2; ++t) {
+        if (t == 1 && pend.valid) {  // ---- tile 1: the same, and the pending stage's V slot is then done with
+          if (!issue_pv(1)) {
+            ok = false;
+            break;
+          }
+          release_v();
+        }
+        if (act[t] && ntok > 0) {
+          if (first) {
+            if (!warp_wait(s_qready + 8 * t, n_q[t] & 1u, s_abort)) {
+              ok = false;
+              break;
+            }
+            ++n_q[t];
+          }
+          tc_fence_after_sync();
+          if (lane == 0) {
+            const uint32_t kst = s_k + (uint32_t)ks * kTc2SlotBytes, qst = s_q + (uint32_t)t * kTc2QBytes;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                umma_ss(tmem + 256u * t, umma_smem_desc(qst + hh * kTc2HalfBytes + k * 32, 0, 1024),
+                        umma_smem_desc(kst + hh * kTc2HalfBytes + k * 32, 0, 1024), idesc_s, (hh | k) ? 1u : 0u);
+            umma_commit(s_sready + 8 * (2 * t + (n & 1)));
+          }
+          __syncwarp();
+          issued = true;
+        } else {
+          // no scores for this tile: the turn of its barriers is taken all the same (also wakes the softmax
+          // threads for the end marker)
+          if (lane == 0) mbar_arrive(s_sready + 8 * (2 * t + (n & 1)));
+          __syncwarp();
+        }
+      }
+      if (!ok) break;
+      // the K slot is free once the score MMAs of both tiles are complete
+      if (lane == 0) {
+        if (ntok > 0)
+          umma_commit(s_kempty + 8 * ks);
+        else
+          mbar_arrive(s_kempty + 8 * ks);
+      }
+      __syncwarp();
+      if (end) break;
+      pend.valid = true;
+      pend.act[0] = act[0];
+      pend.act[1] = act[1];
+      pend.first = first;
+      pend.last = last;
+      pend.ntok = ntok;
+      pend.vs = n % NV;
+      pend.n = n;
+    }
+    if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+    if (!ok && issued) {  // the tensor memory must not be released under MMAs in flight
+      if (lane == 0) umma_commit(s_drain);
+      __syncwarp();
+      int dummy = 0;
+      mbar_wait_bounded(s_drain, 0u, &dummy, kWaitLimitNs / 8);
+    }
+  } else {
+    // ================================================================= softmax warps: thread = score row of tile t
+    const int t = warp >> 2, row = threadIdx.x & 127;
+    const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256u * t;  // this thread's lane, the tile's columns
+    uint8_t* q_gen = gen + (size_t)t * kTc2QBytes;
+    float m_ref = -INFINITY, l_run = 0.f;  // reference maximum (scaled, log2 domain), sum of the weights
+    int lim_row = 0;
+    uint32_t n_unit = 0;  // units in which this tile had rows
+    bool ok = true;
+    bool q_ahead = false;  // the Q rows of the unit that starts with the next stage are in shared memory already
+    // this thread's Q row of tile pair `rt_` of (sequence b_, kv head h_) into the swizzled K-major tile
+    // ([half][row][64 dims], 16-byte chunk ^= row & 7), then its arrival on the tile's q-ready barrier
+    auto load_q = [&](int b_, int h_, int rt_) {
+      const int col_ = rt_ * kTc2Rows + t * kTcRows + row;
+      const int qi_ = col_ / p.G, head_ = col_ - qi_ * p.G;
+      const bool real_ = col_ < p.GQ;
+      const uint4* src = reinterpret_cast<const uint4*>(
+          p.q + (((size_t)b_ * p.Sq + (real_ ? qi_ : 0)) * p.Hq + (size_t)h_ * p.G + (real_ ? head_ : 0)) * D);
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 v = real_ ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(q_gen + (size_t)(c >> 3) * kTc2HalfBytes + (size_t)row * 128 + (((c & 7) ^ (row & 7)) << 4)) = v;
+      }
+      fence_proxy_async_smem();  // the tile is read by the MMAs through the async proxy
+      mbar_arrive(s_qready + 8 * t);
+    };
+    for (uint32_t n = 0;; ++n) {
+      const int ms = n % NM;
+      if (!warp_wait(s_mfull + 8 * ms, (n / NM) & 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      const int4 meta = g_meta[2 * ms], meta2 = g_meta[2 * ms + 1];
+      const bool end = meta.x < 0;
+      const int ntok = end ? 0 : (meta.w & 0xffff);
+      const bool first = !end && ((meta.w >> 16) & 1), last = !end && ((meta.w >> 17) & 1);
+      const int b = meta.y, h = meta.z, rt = end ? 0 : meta2.w, lim_base = meta2.y;
+      const bool act = !end && (t == 0 || rt * kTc2Rows + kTcRows < p.GQ);
+      const int col = rt * kTc2Rows + t * kTcRows + row;
+      const int qi = col / p.G, head = col - qi * p.G;
+      const bool real_row = act && col < p.GQ;
+      if (first && act) {
+        m_ref = -INFINITY;
+        l_run = 0.f;
+        lim_row = lim_base + qi;
+        if (ntok > 0 && !q_ahead) load_q(b, h, rt);
+        q_ahead = false;
+        ++n_unit;
+      }
+      if (!warp_wait(s_sready + 8 * (2 * t + (n & 1)), (n >> 1) & 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      if (end) break;
+      if (act && ntok > 0) {
+        tc_fence_after_sync();
+        uint32_t sr[4][32];
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) tmem_ld32(trow + 32 * c4, sr[c4]);
+        tmem_ld_wait();
+        // tokens [0, e) of the stage are visible to this row
+        const int e = min(min(meta2.z, lim_row) - meta2.x, ntok);
+        if (e < kTc2StageTok) {
+#pragma unroll
+          for (int j = 0; j < kTc2StageTok; ++j)
+            if (j >= e) sr[j >> 5][j & 31] = 0xff800000u;  // -inf
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int j = 0; j < kTc2StageTok; j += 2)
+          mx4[(j >> 1) & 3] = fmax3(mx4[(j >> 1) & 3], __uint_as_float(sr[j >> 5][j & 31]),
+                                    __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]));
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;  // the scale is positive
+        // reference maximum: raised only when the row maximum is more than kTcRescaleStep above it
+        const bool raise = m_ref != -INFINITY && mx > m_ref + kTcRescaleStep;
+        float alpha = 1.f;
+        if (m_ref == -INFINITY) {
+          m_ref = mx;  // nothing accumulated for this row so far
+        } else if (raise) {
+          alpha = ex2(m_ref - mx);
+          m_ref = mx;
+        }
+        if (__any_sync(0xffffffffu, raise)) {
+          // P.V of the previous stage was issued before this stage's score MMAs, so it is complete: O may be rescaled
+#pragma unroll 1
+          for (int c4 = 0; c4 < D / 32; ++c4) {
+            uint32_t o[32];
+            tmem_ld32(trow + 128 + 32 * c4, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+            tmem_st32(trow + 128 + 32 * c4, o);
+          }
+          tmem_st_wait();
+          l_run *= alpha;
+        }
+        const float neg_mu = m_ref == -INFINITY ? 0.f : -m_ref;
+        const float2 scale2 = make_float2(p.scale_log2e, p.scale_log2e), neg_mu2 = make_float2(neg_mu, neg_mu);
+        float2 add4[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {  // 64 tokens at a time: 32 packed words of P
+          uint32_t pw[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int j = 64 * hf + 2 * i;
+            const float2 x = ffma2(make_float2(__uint_as_float(sr[j >> 5][j & 31]), __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31])),
+                                   scale2, neg_mu2);
+            const float2 w = make_float2(ex2(x.x), ex2(x.y));
+            add4[i & 3] = fadd2(add4[i & 3], w);
+            pw[i] = pack_bf16x2(w.x, w.y);
+          }
+          tmem_st32(trow + 32 * hf, pw);  // over this row's scores (all of them are in registers by now)
+        }
+        {
+          const float2 a01 = fadd2(add4[0], add4[1]), a23 = fadd2(add4[2], add4[3]);
+          l_run += (a01.x + a01.y) + (a23.x + a23.y);
+        }
+        tmem_st_wait();
+        if (ntok < kTc2StageTok) {
+          // V rows beyond the stage's tokens may hold anything (NaN included): clear them once the slot has landed
+          const int vs = n % NV;
+          if (!warp_wait(s_vfull + 8 * vs, (n / NV) & 1u, s_abort)) {
+            ok = false;
+            break;
+          }
+          uint8_t* vgen = gen + (s_v - base) + (size_t)vs * kTc2SlotBytes;
+          for (int idx = row; idx < (kTc2StageTok - ntok) * 16; idx += 128) {
+            const int r = ntok + (idx >> 4), c = idx & 15;
+            *reinterpret_cast<uint4*>(vgen + (size_t)(c >> 3) * kTc2HalfBytes + (size_t)r * 128 + ((c & 7) << 4)) =
+                make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_proxy_async_smem();  // the cleared rows are read by the MMA through the async proxy
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+      }
+      mbar_arrive(s_pready + 8 * (2 * t + (n & 1)));
+
+      if (last && act) {
+        // The unit's last score MMAs are complete, so the tile's Q rows are free: when the next stage opens a unit
+        // with rows in this tile, its Q goes to shared memory now and the score MMAs of that stage need not wait
+        // for the epilogue below.
+        {
+          const int ms1 = (n + 1) % NM;
+          if (!warp_wait(s_mfull + 8 * ms1, ((n + 1) / NM) & 1u, s_abort)) {
+            ok = false;
+            break;
+          }
+          const int4 nm = g_meta[2 * ms1], nm2 = g_meta[2 * ms1 + 1];
+          if (nm.x >= 0 && (nm.w & 0xffff) > 0 && (t == 0 || nm2.w * kTc2Rows + kTcRows < p.GQ)) {
+            load_q(nm.y, nm.z, nm2.w);
+            q_ahead = true;
+          }
+        }
+        // ---- the unit is complete: normalise this row of O and write it
+        const int slot_id = meta.x;
+        const bool dst_ok = checked(chk_index(slot_id, p.max_items) && chk_index(b, p.B) && chk_index(h, p.Hkv),
+                                    &p.hdr->status, kStatusBadIndex);
+        const int n_chunks = dst_ok ? p.seq_first[b + 1] - p.seq_first[b] : 1;
+        const bool write_row = real_row && (!kChecked || dst_ok);
+        // use number n_unit - 1 of the tile's pv-done barrier
+        if (!warp_wait(s_pvdone + 8 * t, (n_unit - 1) & 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after_sync();
+        const bool unit_has_tokens = ntok > 0;                // (a unit without tokens is one stage: nothing is in O)
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;    // l = 0: the row saw no token of this chunk
+        __nv_bfloat16* orow = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D;
+        float* prow_o = p.part_o + ((size_t)slot_id * p.GQ + col) * D;
+#pragma unroll 1
+        for (int c4 = 0; c4 < D / 32; ++c4) {
+          uint32_t o[32];
+          if (unit_has_tokens) {
+            tmem_ld32(trow + 128 + 32 * c4, o);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = 0u;
+          }
+          if (write_row && n_chunks == 1 && !p.out_f32) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                w[i] = pack_bf16x2(__uint_as_float(o[8 * v + 2 * i]) * inv, __uint_as_float(o[8 * v + 2 * i + 1]) * inv);
+              *reinterpret_cast<uint4*>(orow + 32 * c4 + 8 * v) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          } else if (write_row) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+              *reinterpret_cast<float4*>(prow_o + 32 * c4 + 4 * v) =
+                  make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
+                              __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
+          }
+          __syncwarp();  // the tensor-memory loads are warp-wide: reconverge before the next one
+        }
+        if (write_row && (n_chunks > 1 || p.out_f32))
+          p.part_lse[(size_t)slot_id * p.GQ + col] = l_run > 0.f ? m_ref + lg2(l_run) : -INFINITY;
+        tc_fence_before_sync();  // the next unit's first P.V overwrites O: ordered behind these reads by q-ready / p-ready
+      }
+    }
+    if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+  }
+  // ---- common exit: release the tensor memory once every warp is done with it
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 10) tmem_dealloc(tmem, kTc2TmemCols);
+}
+
+}  // namespace ooco

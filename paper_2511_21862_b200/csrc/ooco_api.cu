@@ -15,6 +15,7 @@
 #include "block_copy_kernels.cuh"
 #include "chunk_kernels.cuh"
 #include "chunk_tc_kernels.cuh"
+#include "chunk_tc2_kernels.cuh"
 #include "decode_kernels.cuh"
 
 namespace ooco {
@@ -22,8 +23,8 @@ namespace ooco {
 // ------------------------------------------------------------------------------------ tuning
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
-            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobOutF32, kKnobKv8Tcgen05, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}, {0}, {1}};
+            kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobOutF32, kKnobKv8Tcgen05, kKnobChunkTwoTiles, kKnobCount };
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}, {0}, {1}, {1}};
 static std::atomic<int> g_overridden[kKnobCount];  // knob set through ooco_set_tuning
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
@@ -357,6 +358,34 @@ static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeP
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the tcgen05 chunk attention kernel", (long)e);
 }
 
+// Prefill chunk on tcgen05 with two 128-row tiles per CTA (head_dim 128, bf16 cache, more than 128 score columns):
+// one persistent CTA per SM, 512 tensor-memory columns, 128-token K / V slots.
+static int launch_chunk_tc2(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
+                            cudaStream_t st, int dev, bool dry) {
+  auto kern = chunk_tc2_kernel;
+  static std::atomic<int> static_smem{-1};
+  if (static_smem.load() < 0) {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncGetAttributes", (long)e);
+    static_smem.store((int)fa.sharedSizeBytes);
+  }
+  const size_t dyn_max = (size_t)di.smem_optin - (size_t)static_smem.load();
+  const size_t smem = ChunkTc2Smem::total();
+  if (smem > dyn_max) return OOCO_E_UNSUPPORTED;
+  static std::atomic<size_t> configured[64];
+  if (dev < 0 || dev >= 64 || configured[dev].load() < smem) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max);
+    if (e != cudaSuccess) return fail_cuda("cudaFuncSetAttribute(max dynamic smem)", (long)e);
+    if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
+  }
+  if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(352), smem, st,
+                            g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the two-tile tcgen05 chunk attention kernel", (long)e);
+}
+
 // 9 .. 16 score columns: the warps of a CTA share one 16-row tile and split the tokens of a stage.
 template <int D>
 static int launch_row16(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
@@ -607,7 +636,7 @@ int ooco_set_tuning(int knob, int value) {
   if (knob == kKnobItemsPerCta && (value < 1 || value > 64)) return OOCO_E_SHAPE;
   if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
   if (knob == kKnobCopyCtasPerSm && (value < 1 || value > 3)) return OOCO_E_SHAPE;
-  if ((knob == kKnobOutF32 || knob == kKnobKv8Tcgen05) && value != 0 && value != 1) return OOCO_E_SHAPE;
+  if ((knob == kKnobOutF32 || knob == kKnobKv8Tcgen05 || knob == kKnobChunkTwoTiles) && value != 0 && value != 1) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
   g_overridden[knob].store(1);
   return OOCO_OK;
@@ -717,15 +746,18 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   const bool row16 = !chunk && !kv8 && G_ > 8 && g_knobs[kKnobRowLayout16].load() != 0;
   // (the 8-bit cache has no mma.sync chunk kernel: every chunk over it runs the tcgen05 kernel)
   const bool chunk_tc = chunk && s->head_dim == 128 && (kv8 || (G_ > 32 && g_knobs[kKnobChunkTcgen05].load() != 0));
+  // (more than one 128-row tile per item, bf16: the kernel that keeps two tiles per CTA on the tensor pipe in turns)
+  const bool chunk_tc2 = chunk_tc && !kv8 && G_ > kTcRows && g_knobs[kKnobChunkTwoTiles].load() != 0;
   if (chunk) {
     ncw = chunk_warps(G_);
     cps = (ncw == 8 && !chunk_tc) ? 1 : 2;
     if (chunk_tc && g_overridden[kKnobCtasPerSm].load()) cps = g_knobs[kKnobCtasPerSm].load() > 1 ? 2 : 1;
+    if (chunk_tc2) cps = 1;
   } else if (row16) {
     ncw = 4;
     cps = 2;
   }
-  const int stage_tok = (chunk || row16) ? kChunkStageTok : 16 * ncw * tpw;
+  const int stage_tok = chunk_tc2 ? kTc2StageTok : ((chunk || row16) ? kChunkStageTok : 16 * ncw * tpw);
   DecodeParams p;
   memset(&p, 0, sizeof p);
   uint8_t* ws = (uint8_t*)workspace;
@@ -754,7 +786,10 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   p.grid_main = di.sm_count * cps;
   if (p.grid_main > kGridCap) p.grid_main = kGridCap;
   p.next_item_init = p.grid_main;
-  if (chunk) p.grid_main = (p.grid_main + chunk_row_tiles(G_) - 1) / chunk_row_tiles(G_);
+  if (chunk_tc2)
+    p.grid_main = (p.grid_main + (G_ + kTc2Rows - 1) / kTc2Rows - 1) / ((G_ + kTc2Rows - 1) / kTc2Rows);
+  else if (chunk)
+    p.grid_main = (p.grid_main + chunk_row_tiles(G_) - 1) / chunk_row_tiles(G_);
   p.chunk_min = g_knobs[kKnobChunkMin].load();
   p.chunk_max = g_knobs[kKnobChunkMax].load();
   if (p.chunk_max < p.chunk_min) p.chunk_max = p.chunk_min;
@@ -783,6 +818,7 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // once without launching, before the first kernel of the call is enqueued.
   const int stages = g_knobs[kKnobStages].load();
   auto launch_attention = [&](bool dry) -> int {
+    if (chunk_tc2) return launch_chunk_tc2(tk, tv, p, di, st, dev, dry);
     if (chunk_tc)
       return kv8 ? launch_chunk_tc<true>(tk, tv, p, di, cps, st, dev, dry)
                  : launch_chunk_tc<false>(tk, tv, p, di, cps, st, dev, dry);
