@@ -34,11 +34,12 @@ constexpr int kTc2QBytes = 2 * kTcRows * 128;        // one tile's queries: [hal
 constexpr int kTc2Rows = 2 * kTcRows;                // score rows of a unit
 constexpr int kTc2TmemCols = 512;
 constexpr int kTc2KSlots = 2, kTc2VSlots = 3, kTc2MetaRing = 8;
+constexpr int kTc2Threads = 20 * 32;               // 16 softmax warps, K producer, V producer, one MMA warp per tile
 
 struct ChunkTc2Smem {
   __host__ __device__ static size_t total() {
     return 1024 + 2 * (size_t)kTc2QBytes + (size_t)(kTc2KSlots + kTc2VSlots) * kTc2SlotBytes + kTc2MetaRing * 32 +
-           kTc2VSlots * sizeof(VStageDesc) + 256;
+           kTc2VSlots * sizeof(VStageDesc) + 512;
   }
 };
 
@@ -46,11 +47,12 @@ struct ChunkTc2Smem {
 // included) uses K slot n % 2, V slot n % 3, meta entry n % 8 and, for each tile, barrier n & 1 of the pairs
 // [2] below with phase parity (n >> 1) & 1 -- every tile takes a turn of its barriers on every stage, with or
 // without work, so nobody can be overtaken by two completions of a barrier it waits on.
-__global__ void __launch_bounds__(352, 1)
+__global__ void __launch_bounds__(kTc2Threads, 1)
 chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const DecodeParams p) {
   constexpr int D = 128;
   constexpr int NK = kTc2KSlots, NV = kTc2VSlots, NM = kTc2MetaRing;
+  constexpr int kWarpK = 16, kWarpV = 17, kWarpM = 18;  // warps 0 .. 15: softmax; 18, 19: MMA of tile 0, 1
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -72,7 +74,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const uint32_t s_pvdone = s_pready + 32;         // [2 tiles] the unit's last P.V_t is complete          (MMA commit)
   const uint32_t s_qready = s_pvdone + 16;         // [2 tiles] Q_t of the unit is in shared memory        (128 threads)
   const uint32_t s_drain = s_qready + 16;
-  const uint32_t s_slot = s_drain + 8;
+  const uint32_t s_slot = s_drain + 16;
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
   VStageDesc* g_vdesc = reinterpret_cast<VStageDesc*>(gen + (s_vdesc - base));
   volatile uint32_t* g_slot = reinterpret_cast<volatile uint32_t*>(gen + (s_slot - base));
@@ -83,26 +85,27 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     *s_abort = 0;
     for (int i = 0; i < NK; ++i) {
       mbar_init(s_kfull + 8 * i, 1);
-      mbar_init(s_kempty + 8 * i, 1);
+      mbar_init(s_kempty + 8 * i, 2);  // one arrival per MMA warp
     }
     for (int i = 0; i < NV; ++i) {
       mbar_init(s_vfull + 8 * i, 1);
-      mbar_init(s_vempty + 8 * i, 1);
+      mbar_init(s_vempty + 8 * i, 2);
       mbar_init(s_vdfull + 8 * i, 1);
     }
     for (int i = 0; i < NM; ++i) mbar_init(s_mfull + 8 * i, 1);
     for (int i = 0; i < 4; ++i) {
       mbar_init(s_sready + 8 * i, 1);
-      mbar_init(s_pready + 8 * i, 128);
+      mbar_init(s_pready + 8 * i, 256);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(s_pvdone + 8 * i, 1);
-      mbar_init(s_qready + 8 * i, 128);
+      mbar_init(s_qready + 8 * i, 256);
     }
     mbar_init(s_drain, 1);
+    mbar_init(s_drain + 8, 1);
     fence_mbar_init();
   }
-  if (warp == 10) tmem_alloc(s_slot, kTc2TmemCols);
+  if (warp == kWarpM) tmem_alloc(s_slot, kTc2TmemCols);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -113,7 +116,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const int nrt = (p.GQ + kTc2Rows - 1) / kTc2Rows;  // tile pairs per work item
   const long long cap_tokens = (long long)p.MB * p.bs;
 
-  if (warp == 8) {
+  if (warp == kWarpK) {
     // ================================================================= K producer (and the walk over the units)
     if (lane == 0) prefetch_tmap(&tm_k);
     const long long n_units = (long long)p.hdr->n_items * nrt;
@@ -237,7 +240,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         mbar_wait_bounded(s_kfull + 8 * (j % NK), (uint32_t)(j / NK) & 1u, &dummy_abort, kWaitLimitNs / 8);
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == kWarpV) {
     // ================================================================= V producer
     if (lane == 0) prefetch_tmap(&tm_v);
     const uint32_t box_rows_bytes = (uint32_t)p.tile_rows * 128;
@@ -273,51 +276,23 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         mbar_wait_bounded(s_vfull + 8 * (j % NV), (uint32_t)(j / NV) & 1u, &dummy_abort, kWaitLimitNs / 8);
       }
     }
-  } else if (warp == 10) {
-    // ================================================================= MMA warp
+  } else if (warp >= kWarpM) {
+    // ================================================================= MMA warps: warp kWarpM + t issues tile t's MMAs
+    // One thread issues an MMA about every 110 to 130 cycles whatever its size (measured: M128 N64 or N128 K16, either
+    // operand source), twice what the pipe needs for N = 128, and the pipe overlaps the MMAs of two threads (two
+    // issuers: one N = 128 MMA per 70 cycles).  So each tile has an issuing warp of its own; the order inside a tile,
+    // P.V_t(n - 1) before S_t(n), is the program order of its thread, and the tiles need no order between them.
+    const int t = warp - kWarpM;
     const uint32_t idesc_s = umma_idesc_16bit(kTcRows, kTc2StageTok, 0, true);
     const uint32_t idesc_o = umma_idesc_16bit(kTcRows, D, 1, true);
-    uint32_t n_q[2] = {0u, 0u};  // units in which tile t had rows and tokens (uses of its q-ready barrier)
+    const uint32_t ts = tmem + 256u * t;
+    const uint64_t dq = umma_smem_desc(s_q + (uint32_t)t * kTc2QBytes, 0, 1024);
+    uint32_t n_q = 0;  // units in which the tile had rows and tokens (uses of its q-ready barrier)
     bool issued = false, ok = true;
     // what is known about the stage whose P.V MMAs are still to be issued
-    struct Pending {
-      bool valid, act[2], first, last;
-      int ntok, vs;
-      uint32_t n;
-    } pend = {false, {false, false}, false, false, 0, 0, 0u};
-    // P.V of tile t for the pending stage: waits for the tile's softmax threads, then issues (or just takes the turn)
-    auto issue_pv = [&](int t) {
-      const uint32_t n = pend.n;
-      if (!warp_wait(s_pready + 8 * (2 * t + (n & 1)), (n >> 1) & 1u, s_abort)) return false;
-      if (pend.act[t] && pend.ntok > 0) {
-        if (!warp_wait(s_vfull + 8 * pend.vs, ((uint32_t)(n / NV)) & 1u, s_abort)) return false;
-        tc_fence_after_sync();
-        if (lane == 0) {
-          const uint32_t vst = s_v + (uint32_t)pend.vs * kTc2SlotBytes, ts = tmem + 256u * t;
-#pragma unroll
-          for (int k = 0; k < kTc2StageTok / 16; ++k)  // 16 tokens: 8 columns of P, 16 rows of 128 bytes of V in either half
-            umma_ts(ts + 128, ts + 8 * k, umma_smem_desc(vst + k * 2048, kTc2HalfBytes, 1024), idesc_o,
-                    (pend.first && k == 0) ? 0u : 1u);
-          if (pend.last) umma_commit(s_pvdone + 8 * t);
-        }
-        __syncwarp();
-        issued = true;
-      } else if (pend.act[t] && pend.last) {
-        if (lane == 0) mbar_arrive(s_pvdone + 8 * t);  // a unit without tokens: nothing to wait for
-        __syncwarp();
-      }
-      return true;
-    };
-    // the V slot of the pending stage is free once both tiles' P.V are complete
-    auto release_v = [&]() {
-      if (lane == 0) {
-        if (pend.ntok > 0 && (pend.act[0] || pend.act[1]))
-          umma_commit(s_vempty + 8 * pend.vs);
-        else
-          mbar_arrive(s_vempty + 8 * pend.vs);
-      }
-      __syncwarp();
-    };
+    bool p_valid = false, p_act = false, p_first = false, p_last = false;
+    int p_ntok = 0;
+    uint32_t p_n = 0;
     for (uint32_t n = 0;; ++n) {
       const int ks = n % NK, ms = n % NM;
       if (!warp_wait(s_kfull + 8 * ks, (n / NK) & 1u, s_abort)) {
@@ -329,99 +304,127 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const int ntok = end ? 0 : (meta.w & 0xffff);
       const bool first = !end && ((meta.w >> 16) & 1), last = !end && ((meta.w >> 17) & 1);
       const int rt = end ? 0 : meta2.w;
-      bool act[2];
-      act[0] = !end;                                            // a unit always has rows in its first tile
-      act[1] = !end && rt * kTc2Rows + kTcRows < p.GQ;
-      // ---- tile 0: S_0 of this stage goes behind P.V_0 of the pending one
-      if (pend.valid && !issue_pv(0)) {
-        ok = false;
-        break;
-      }
-#pragma unroll 1
-      for (int t = 0; t < 2; ++t) {
-        if (t == 1 && pend.valid) {  // ---- tile 1: the same, and the pending stage's V slot is then done with
-          if (!issue_pv(1)) {
+      const bool act = !end && (t == 0 || rt * kTc2Rows + kTcRows < p.GQ);  // a unit always has rows in its first tile
+      // ---- P.V of the pending stage: waits for the tile's softmax threads, then issues (or just takes the turn)
+      if (p_valid) {
+        const int vs = p_n % NV;
+        if (!warp_wait(s_pready + 8 * (2 * t + (p_n & 1)), (p_n >> 1) & 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        if (p_act && p_ntok > 0) {
+          if (!warp_wait(s_vfull + 8 * vs, (p_n / NV) & 1u, s_abort)) {
             ok = false;
             break;
           }
-          release_v();
-        }
-        if (act[t] && ntok > 0) {
-          if (first) {
-            if (!warp_wait(s_qready + 8 * t, n_q[t] & 1u, s_abort)) {
-              ok = false;
-              break;
-            }
-            ++n_q[t];
-          }
           tc_fence_after_sync();
           if (lane == 0) {
-            const uint32_t kst = s_k + (uint32_t)ks * kTc2SlotBytes, qst = s_q + (uint32_t)t * kTc2QBytes;
+            const uint64_t dv = umma_smem_desc(s_v + (uint32_t)vs * kTc2SlotBytes, kTc2HalfBytes, 1024);
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-              for (int k = 0; k < 4; ++k)
-                umma_ss(tmem + 256u * t, umma_smem_desc(qst + hh * kTc2HalfBytes + k * 32, 0, 1024),
-                        umma_smem_desc(kst + hh * kTc2HalfBytes + k * 32, 0, 1024), idesc_s, (hh | k) ? 1u : 0u);
-            umma_commit(s_sready + 8 * (2 * t + (n & 1)));
+            for (int k = 0; k < kTc2StageTok / 16; ++k)  // 16 tokens: 8 columns of P, 16 rows of 128 bytes of V in either half
+              umma_ts(ts + 128, ts + 8 * k, dv + (uint64_t)(k * (2048 >> 4)), idesc_o, (p_first && k == 0) ? 0u : 1u);
+            if (p_last) umma_commit(s_pvdone + 8 * t);
+            umma_commit(s_vempty + 8 * vs);  // (one of the two arrivals that free the V slot)
           }
           __syncwarp();
           issued = true;
         } else {
-          // no scores for this tile: the turn of its barriers is taken all the same (also wakes the softmax
-          // threads for the end marker)
-          if (lane == 0) mbar_arrive(s_sready + 8 * (2 * t + (n & 1)));
+          if (lane == 0) {
+            if (p_act && p_last) mbar_arrive(s_pvdone + 8 * t);  // a unit without tokens: nothing to wait for
+            mbar_arrive(s_vempty + 8 * vs);
+          }
           __syncwarp();
         }
       }
-      if (!ok) break;
-      // the K slot is free once the score MMAs of both tiles are complete
-      if (lane == 0) {
-        if (ntok > 0)
-          umma_commit(s_kempty + 8 * ks);
-        else
-          mbar_arrive(s_kempty + 8 * ks);
+      // ---- scores of this stage
+      // The tiles take turns, half a stage apart: S_0(n), S_1(n), S_0(n + 1), ... in this order, so that one tile's
+      // softmax runs beside the other tile's MMAs (P.V of the stage before, then these scores) instead of both tiles
+      // doing the same thing at once.  Tile 1 waits for tile 0's scores of this stage, tile 0 for tile 1's of the
+      // stage before -- on every stage, with or without work, so that neither warp can get two turns ahead of the
+      // other on a barrier pair.
+      if (t == 1 ? !warp_wait(s_sready + 8 * (n & 1), (n >> 1) & 1u, s_abort)
+                 : (n > 0 && !warp_wait(s_sready + 8 * (2 + ((n - 1) & 1)), ((n - 1) >> 1) & 1u, s_abort))) {
+        ok = false;
+        break;
       }
-      __syncwarp();
+      if (act && ntok > 0) {
+        if (first) {
+          if (!warp_wait(s_qready + 8 * t, n_q & 1u, s_abort)) {
+            ok = false;
+            break;
+          }
+          ++n_q;
+        }
+        tc_fence_after_sync();
+        if (lane == 0) {
+          const uint64_t dk = umma_smem_desc(s_k + (uint32_t)ks * kTc2SlotBytes, 0, 1024);
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {  // 16 dims = 32 bytes further along the rows; the second 64 dims = the next half
+              const uint64_t off = (uint64_t)((hh * kTc2HalfBytes + k * 32) >> 4);
+              umma_ss(ts, dq + off, dk + off, idesc_s, (hh | k) ? 1u : 0u);
+            }
+          umma_commit(s_sready + 8 * (2 * t + (n & 1)));
+          umma_commit(s_kempty + 8 * ks);  // (one of the two arrivals that free the K slot)
+        }
+        __syncwarp();
+        issued = true;
+      } else {
+        // no scores for this tile: the turn of its barriers is taken all the same (also wakes the softmax threads
+        // for the end marker)
+        if (lane == 0) {
+          mbar_arrive(s_sready + 8 * (2 * t + (n & 1)));
+          mbar_arrive(s_kempty + 8 * ks);
+        }
+        __syncwarp();
+      }
       if (end) break;
-      pend.valid = true;
-      pend.act[0] = act[0];
-      pend.act[1] = act[1];
-      pend.first = first;
-      pend.last = last;
-      pend.ntok = ntok;
-      pend.vs = n % NV;
-      pend.n = n;
+      p_valid = true;
+      p_act = act;
+      p_first = first;
+      p_last = last;
+      p_ntok = ntok;
+      p_n = n;
     }
     if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
     if (!ok && issued) {  // the tensor memory must not be released under MMAs in flight
-      if (lane == 0) umma_commit(s_drain);
+      if (lane == 0) umma_commit(s_drain + 8 * t);
       __syncwarp();
       int dummy = 0;
-      mbar_wait_bounded(s_drain, 0u, &dummy, kWaitLimitNs / 8);
+      mbar_wait_bounded(s_drain + 8 * t, 0u, &dummy, kWaitLimitNs / 8);
     }
   } else {
-    // ================================================================= softmax warps: thread = score row of tile t
-    const int t = warp >> 2, row = threadIdx.x & 127;
-    const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256u * t;  // this thread's lane, the tile's columns
+    // ================================================================= softmax warps
+    // Tile t = warps 8 t .. 8 t + 7.  Warp (q = warp & 3, hf = (warp >> 2) & 1) owns the 16 score rows
+    // 32 q + 16 hf .. + 15 of the tile (a warp reaches the 32 tensor-memory lanes of its quarter q only) and reads
+    // them in the 16-lane shape: lane (g, tq) holds rows g and g + 8, columns 8 i + 2 tq, + 1 -- two threads would be
+    // too few per row to hide the latency of the row's chain, four share it here and combine with quad shuffles.
+    const int t = warp >> 3, q4 = warp & 3, hf = (warp >> 2) & 1;
+    const int g = lane >> 2, tq = lane & 3;
+    const int row0 = 32 * q4 + 16 * hf + g;  // this thread's rows of the tile: row0 and row0 + 8
+    const uint32_t trow = tmem + ((uint32_t)(32 * q4 + 16 * hf) << 16) + 256u * t;  // the warp's lanes, the tile's columns
+    const int tid_t = threadIdx.x & 255;     // index among the tile's 256 threads
     uint8_t* q_gen = gen + (size_t)t * kTc2QBytes;
-    float m_ref = -INFINITY, l_run = 0.f;  // reference maximum (scaled, log2 domain), sum of the weights
-    int lim_row = 0;
+    float m_ref[2] = {-INFINITY, -INFINITY};  // reference maximum per row (scaled, log2 domain)
+    float l_part[2] = {0.f, 0.f};             // this thread's share of the row's sum of weights
+    int lim_row[2] = {0, 0};
     uint32_t n_unit = 0;  // units in which this tile had rows
     bool ok = true;
     bool q_ahead = false;  // the Q rows of the unit that starts with the next stage are in shared memory already
-    // this thread's Q row of tile pair `rt_` of (sequence b_, kv head h_) into the swizzled K-major tile
-    // ([half][row][64 dims], 16-byte chunk ^= row & 7), then its arrival on the tile's q-ready barrier
+    // Q of tile pair `rt_` of (sequence b_, kv head h_) into the swizzled K-major tile ([half][row][64 dims], 16-byte
+    // chunk ^= row & 7): thread i of the tile writes 64 dims (half i & 1) of row i >> 1; then the q-ready arrival
     auto load_q = [&](int b_, int h_, int rt_) {
-      const int col_ = rt_ * kTc2Rows + t * kTcRows + row;
+      const int r_ = tid_t >> 1, half_ = tid_t & 1;
+      const int col_ = rt_ * kTc2Rows + t * kTcRows + r_;
       const int qi_ = col_ / p.G, head_ = col_ - qi_ * p.G;
       const bool real_ = col_ < p.GQ;
       const uint4* src = reinterpret_cast<const uint4*>(
-          p.q + (((size_t)b_ * p.Sq + (real_ ? qi_ : 0)) * p.Hq + (size_t)h_ * p.G + (real_ ? head_ : 0)) * D);
+          p.q + (((size_t)b_ * p.Sq + (real_ ? qi_ : 0)) * p.Hq + (size_t)h_ * p.G + (real_ ? head_ : 0)) * D + 64 * half_);
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
+      for (int c = 0; c < 8; ++c) {
         const uint4 v = real_ ? src[c] : make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4*>(q_gen + (size_t)(c >> 3) * kTc2HalfBytes + (size_t)row * 128 + (((c & 7) ^ (row & 7)) << 4)) = v;
+        *reinterpret_cast<uint4*>(q_gen + (size_t)half_ * kTc2HalfBytes + (size_t)r_ * 128 + ((c ^ (r_ & 7)) << 4)) = v;
       }
       fence_proxy_async_smem();  // the tile is read by the MMAs through the async proxy
       mbar_arrive(s_qready + 8 * t);
@@ -438,13 +441,14 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const bool first = !end && ((meta.w >> 16) & 1), last = !end && ((meta.w >> 17) & 1);
       const int b = meta.y, h = meta.z, rt = end ? 0 : meta2.w, lim_base = meta2.y;
       const bool act = !end && (t == 0 || rt * kTc2Rows + kTcRows < p.GQ);
-      const int col = rt * kTc2Rows + t * kTcRows + row;
-      const int qi = col / p.G, head = col - qi * p.G;
-      const bool real_row = act && col < p.GQ;
+      const int col0 = rt * kTc2Rows + t * kTcRows + row0;  // score column (query token x head) of row0; row0 + 8: col0 + 8
       if (first && act) {
-        m_ref = -INFINITY;
-        l_run = 0.f;
-        lim_row = lim_base + qi;
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          m_ref[rr] = -INFINITY;
+          l_part[rr] = 0.f;
+          lim_row[rr] = lim_base + (col0 + 8 * rr) / p.G;
+        }
         if (ntok > 0 && !q_ahead) load_q(b, h, rt);
         q_ahead = false;
         ++n_unit;
@@ -456,67 +460,82 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       if (end) break;
       if (act && ntok > 0) {
         tc_fence_after_sync();
-        uint32_t sr[4][32];
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) tmem_ld32(trow + 32 * c4, sr[c4]);
+        uint32_t sr[64];  // sr[4 i + 2 rr + c] = score of row (row0 + 8 rr), token 8 i + 2 tq + c of the stage
+        tmem_ld_16x256b_x16(trow, sr);
         tmem_ld_wait();
-        // tokens [0, e) of the stage are visible to this row
-        const int e = min(min(meta2.z, lim_row) - meta2.x, ntok);
-        if (e < kTc2StageTok) {
+        // tokens [0, e) of the stage are visible to the row
+        const int e0 = min(min(meta2.z, lim_row[0]) - meta2.x, ntok), e1 = min(min(meta2.z, lim_row[1]) - meta2.x, ntok);
+        if (__any_sync(0xffffffffu, min(e0, e1) < kTc2StageTok)) {
 #pragma unroll
-          for (int j = 0; j < kTc2StageTok; ++j)
-            if (j >= e) sr[j >> 5][j & 31] = 0xff800000u;  // -inf
-        }
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          for (int i = 0; i < 16; ++i)
 #pragma unroll
-        for (int j = 0; j < kTc2StageTok; j += 2)
-          mx4[(j >> 1) & 3] = fmax3(mx4[(j >> 1) & 3], __uint_as_float(sr[j >> 5][j & 31]),
-                                    __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]));
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;  // the scale is positive
-        // reference maximum: raised only when the row maximum is more than kTcRescaleStep above it
-        const bool raise = m_ref != -INFINITY && mx > m_ref + kTcRescaleStep;
-        float alpha = 1.f;
-        if (m_ref == -INFINITY) {
-          m_ref = mx;  // nothing accumulated for this row so far
-        } else if (raise) {
-          alpha = ex2(m_ref - mx);
-          m_ref = mx;
+            for (int c = 0; c < 2; ++c) {
+              const int j = 8 * i + 2 * tq + c;
+              if (j >= e0) sr[4 * i + c] = 0xff800000u;  // -inf
+              if (j >= e1) sr[4 * i + 2 + c] = 0xff800000u;
+            }
         }
-        if (__any_sync(0xffffffffu, raise)) {
+        float alpha[2] = {1.f, 1.f}, neg_mu[2];
+        bool raise_any = false;
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          float ma = -INFINITY, mb = -INFINITY;
+#pragma unroll
+          for (int i = 0; i < 16; i += 2) {  // three-input maximum: two scores per instruction, two chains
+            ma = fmax3(ma, __uint_as_float(sr[4 * i + 2 * rr]), __uint_as_float(sr[4 * i + 2 * rr + 1]));
+            mb = fmax3(mb, __uint_as_float(sr[4 * i + 4 + 2 * rr]), __uint_as_float(sr[4 * i + 4 + 2 * rr + 1]));
+          }
+          float mx = fmaxf(ma, mb);
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+          mx *= p.scale_log2e;  // the scale is positive
+          // reference maximum: raised only when the row maximum is more than kTcRescaleStep above it
+          const bool raise = m_ref[rr] != -INFINITY && mx > m_ref[rr] + kTcRescaleStep;
+          if (m_ref[rr] == -INFINITY) {
+            m_ref[rr] = mx;  // nothing accumulated for this row so far
+          } else if (raise) {
+            alpha[rr] = ex2(m_ref[rr] - mx);
+            m_ref[rr] = mx;
+          }
+          raise_any |= raise;
+          neg_mu[rr] = m_ref[rr] == -INFINITY ? 0.f : -m_ref[rr];
+        }
+        if (__any_sync(0xffffffffu, raise_any)) {
           // P.V of the previous stage was issued before this stage's score MMAs, so it is complete: O may be rescaled
 #pragma unroll 1
-          for (int c4 = 0; c4 < D / 32; ++c4) {
+          for (int c2 = 0; c2 < 2; ++c2) {
             uint32_t o[32];
-            tmem_ld32(trow + 128 + 32 * c4, o);
+            tmem_ld_16x256b_x8(trow + 128 + 64 * c2, o);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-            tmem_st32(trow + 128 + 32 * c4, o);
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha[(j >> 1) & 1]);
+            tmem_st_16x256b_x8(trow + 128 + 64 * c2, o);
           }
           tmem_st_wait();
-          l_run *= alpha;
+          l_part[0] *= alpha[0];
+          l_part[1] *= alpha[1];
         }
-        const float neg_mu = m_ref == -INFINITY ? 0.f : -m_ref;
-        const float2 scale2 = make_float2(p.scale_log2e, p.scale_log2e), neg_mu2 = make_float2(neg_mu, neg_mu);
-        float2 add4[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+        const float2 scale2 = make_float2(p.scale_log2e, p.scale_log2e);
+        const float2 nm0 = make_float2(neg_mu[0], neg_mu[0]), nm1 = make_float2(neg_mu[1], neg_mu[1]);
+        float2 add0 = {0.f, 0.f}, add1 = {0.f, 0.f};
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {  // 64 tokens at a time: 32 packed words of P
-          uint32_t pw[32];
+        for (int h2 = 0; h2 < 2; ++h2) {  // 64 tokens at a time: 16 packed words of P per thread
+          uint32_t pw[16];  // pw[2 i + rr]: row (row0 + 8 rr), tokens 64 h2 + 8 i + 2 tq, + 1 = P column 32 h2 + 4 i + tq
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int j = 64 * hf + 2 * i;
-            const float2 x = ffma2(make_float2(__uint_as_float(sr[j >> 5][j & 31]), __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31])),
-                                   scale2, neg_mu2);
-            const float2 w = make_float2(ex2(x.x), ex2(x.y));
-            add4[i & 3] = fadd2(add4[i & 3], w);
-            pw[i] = pack_bf16x2(w.x, w.y);
+          for (int i = 0; i < 8; ++i) {
+            const int r = 4 * (8 * h2 + i);
+            const float2 x0 = ffma2(make_float2(__uint_as_float(sr[r]), __uint_as_float(sr[r + 1])), scale2, nm0);
+            const float2 x1 = ffma2(make_float2(__uint_as_float(sr[r + 2]), __uint_as_float(sr[r + 3])), scale2, nm1);
+            const float2 w0 = make_float2(ex2(x0.x), ex2(x0.y)), w1 = make_float2(ex2(x1.x), ex2(x1.y));
+            add0 = fadd2(add0, w0);
+            add1 = fadd2(add1, w1);
+            pw[2 * i] = pack_bf16x2(w0.x, w0.y);
+            pw[2 * i + 1] = pack_bf16x2(w1.x, w1.y);
           }
-          tmem_st32(trow + 32 * hf, pw);  // over this row's scores (all of them are in registers by now)
+          tmem_st_16x128b_x8(trow + 32 * h2, pw);  // over the rows' scores (all of them are in registers by now)
         }
-        {
-          const float2 a01 = fadd2(add4[0], add4[1]), a23 = fadd2(add4[2], add4[3]);
-          l_run += (a01.x + a01.y) + (a23.x + a23.y);
-        }
+        l_part[0] += add0.x + add0.y;
+        l_part[1] += add1.x + add1.y;
         tmem_st_wait();
         if (ntok < kTc2StageTok) {
           // V rows beyond the stage's tokens may hold anything (NaN included): clear them once the slot has landed
@@ -526,7 +545,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             break;
           }
           uint8_t* vgen = gen + (s_v - base) + (size_t)vs * kTc2SlotBytes;
-          for (int idx = row; idx < (kTc2StageTok - ntok) * 16; idx += 128) {
+          for (int idx = tid_t; idx < (kTc2StageTok - ntok) * 16; idx += 256) {
             const int r = ntok + (idx >> 4), c = idx & 15;
             *reinterpret_cast<uint4*>(vgen + (size_t)(c >> 3) * kTc2HalfBytes + (size_t)r * 128 + ((c & 7) << 4)) =
                 make_uint4(0u, 0u, 0u, 0u);
@@ -554,53 +573,62 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             q_ahead = true;
           }
         }
-        // ---- the unit is complete: normalise this row of O and write it
+        // ---- the unit is complete: normalise the rows of O and write them
         const int slot_id = meta.x;
         const bool dst_ok = checked(chk_index(slot_id, p.max_items) && chk_index(b, p.B) && chk_index(h, p.Hkv),
                                     &p.hdr->status, kStatusBadIndex);
         const int n_chunks = dst_ok ? p.seq_first[b + 1] - p.seq_first[b] : 1;
-        const bool write_row = real_row && (!kChecked || dst_ok);
         // use number n_unit - 1 of the tile's pv-done barrier
         if (!warp_wait(s_pvdone + 8 * t, (n_unit - 1) & 1u, s_abort)) {
           ok = false;
           break;
         }
         tc_fence_after_sync();
-        const bool unit_has_tokens = ntok > 0;                // (a unit without tokens is one stage: nothing is in O)
-        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;    // l = 0: the row saw no token of this chunk
-        __nv_bfloat16* orow = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D;
-        float* prow_o = p.part_o + ((size_t)slot_id * p.GQ + col) * D;
+        const bool unit_has_tokens = ntok > 0;  // (a unit without tokens is one stage: nothing is in O)
+        float inv[2], lse[2];
+        __nv_bfloat16* orow[2];
+        float* prow[2];
+        bool write_row[2];
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          float l = l_part[rr];
+          l += __shfl_xor_sync(0xffffffffu, l, 1);
+          l += __shfl_xor_sync(0xffffffffu, l, 2);
+          inv[rr] = l > 0.f ? 1.f / l : 0.f;  // l = 0: the row saw no token of this chunk
+          lse[rr] = l > 0.f ? m_ref[rr] + lg2(l) : -INFINITY;
+          const int col = col0 + 8 * rr;
+          const int qi = col / p.G, head = col - qi * p.G;
+          write_row[rr] = col < p.GQ && (!kChecked || dst_ok);
+          orow[rr] = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D;
+          prow[rr] = p.part_o + ((size_t)slot_id * p.GQ + col) * D;
+          if (write_row[rr] && tq == 0 && (n_chunks > 1 || p.out_f32)) p.part_lse[(size_t)slot_id * p.GQ + col] = lse[rr];
+        }
 #pragma unroll 1
-        for (int c4 = 0; c4 < D / 32; ++c4) {
-          uint32_t o[32];
+        for (int c2 = 0; c2 < 2; ++c2) {
+          uint32_t o[32];  // o[4 i + 2 rr + c] = row (row0 + 8 rr), dim 64 c2 + 8 i + 2 tq + c
           if (unit_has_tokens) {
-            tmem_ld32(trow + 128 + 32 * c4, o);
+            tmem_ld_16x256b_x8(trow + 128 + 64 * c2, o);
             tmem_ld_wait();
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j) o[j] = 0u;
           }
-          if (write_row && n_chunks == 1 && !p.out_f32) {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint32_t w[4];
+          for (int rr = 0; rr < 2; ++rr) {
+            if (!write_row[rr]) continue;
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                w[i] = pack_bf16x2(__uint_as_float(o[8 * v + 2 * i]) * inv, __uint_as_float(o[8 * v + 2 * i + 1]) * inv);
-              *reinterpret_cast<uint4*>(orow + 32 * c4 + 8 * v) = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int i = 0; i < 8; ++i) {
+              const float a = __uint_as_float(o[4 * i + 2 * rr]) * inv[rr], c = __uint_as_float(o[4 * i + 2 * rr + 1]) * inv[rr];
+              const int dim = 64 * c2 + 8 * i + 2 * tq;
+              if (n_chunks == 1 && !p.out_f32)
+                *reinterpret_cast<uint32_t*>(orow[rr] + dim) = pack_bf16x2(a, c);
+              else
+                *reinterpret_cast<float2*>(prow[rr] + dim) = make_float2(a, c);
             }
-          } else if (write_row) {
-#pragma unroll
-            for (int v = 0; v < 8; ++v)
-              *reinterpret_cast<float4*>(prow_o + 32 * c4 + 4 * v) =
-                  make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
-                              __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
           }
           __syncwarp();  // the tensor-memory loads are warp-wide: reconverge before the next one
         }
-        if (write_row && (n_chunks > 1 || p.out_f32))
-          p.part_lse[(size_t)slot_id * p.GQ + col] = l_run > 0.f ? m_ref + lg2(l_run) : -INFINITY;
-        tc_fence_before_sync();  // the next unit's first P.V overwrites O: ordered behind these reads by q-ready / p-ready
+        tc_fence_before_sync();  // the next unit's first P.V overwrites O: ordered behind these reads by p-ready
       }
     }
     if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
@@ -608,7 +636,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   // ---- common exit: release the tensor memory once every warp is done with it
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 10) tmem_dealloc(tmem, kTc2TmemCols);
+  if (warp == kWarpM) tmem_dealloc(tmem, kTc2TmemCols);
 }
 
 }  // namespace ooco

@@ -169,13 +169,15 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
       if (!warp_wait(s_sfree + 8 * (n_s & 1), ((n_s >> 1) & 1u) ^ 1u, s_abort)) return false;
       tc_fence_after_sync();
       if (lane == 0) {
-        const uint32_t kst = s_stage + (uint32_t)sl * L::kStageBytes;
+        // (one descriptor per stage, advanced by adding to its address field: building one per MMA costs the issuing
+        // thread more time than the MMA takes)
+        const uint64_t dk = umma_smem_desc(s_stage + (uint32_t)sl * L::kStageBytes, 0, 1024);
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
           for (int k = 0; k < 4; ++k)  // 16 dims of Q are 8 tensor-memory columns
-            umma_ts(tmem + kTcColS, tmem + kTcColQ + 8 * (4 * h + k),
-                    umma_smem_desc(kst + h * L::kHalfBytes + k * 32, 0, 1024), idesc_s, (h | k) ? 1u : 0u);
+            umma_ts(tmem + kTcColS, tmem + kTcColQ + 8 * (4 * h + k), dk + (uint64_t)((h * L::kHalfBytes + k * 32) >> 4), idesc_s,
+                    (h | k) ? 1u : 0u);
         umma_commit(s_sready + 8 * (n_s & 1));
       }
       __syncwarp();
@@ -227,10 +229,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
       if (ntok > 0) {
         tc_fence_after_sync();
         if (lane == 0) {
-          const uint32_t kst = s_stage + (uint32_t)slot * L::kStageBytes, vst = kst + L::kTileBytes;
+          const uint64_t dv = umma_smem_desc(s_stage + (uint32_t)slot * L::kStageBytes + L::kTileBytes, L::kHalfBytes, 1024);
 #pragma unroll
           for (int k = 0; k < 4; ++k)  // 16 tokens: 8 columns of P, 16 rows of 128 bytes of V in either half
-            umma_ts(tmem + kTcColO, tmem + kTcColS + 8 * k, umma_smem_desc(vst + k * 2048, L::kHalfBytes, 1024), idesc_o,
+            umma_ts(tmem + kTcColO, tmem + kTcColS + 8 * k, dv + (uint64_t)(k * (2048 >> 4)), idesc_o,
                     (first && k == 0) ? 0u : 1u);
           umma_commit(s_empty + 8 * slot);
           umma_commit(s_pvdone + 8 * (n_pv & 1));

@@ -380,7 +380,7 @@ static int launch_chunk_tc2(const CUtensorMap& tk, const CUtensorMap& tv, Decode
     if (dev >= 0 && dev < 64) configured[dev].store(dyn_max);
   }
   if (dry) return OOCO_OK;  // sizing and attributes only: the caller launches nothing before these have passed
-  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(352), smem, st,
+  cudaError_t e = launch_ex(kern, dim3(p.next_item_init), dim3(kTc2Threads), smem, st,
                             g_knobs[kKnobPdl].load() != 0 && !tl_events_between_kernels, tk, tv, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the two-tile tcgen05 chunk attention kernel", (long)e);
