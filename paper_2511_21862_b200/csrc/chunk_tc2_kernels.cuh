@@ -305,6 +305,22 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const bool first = !end && ((meta.w >> 16) & 1), last = !end && ((meta.w >> 17) & 1);
       const int rt = end ? 0 : meta2.w;
       const bool act = !end && (t == 0 || rt * kTc2Rows + kTcRows < p.GQ);  // a unit always has rows in its first tile
+      // Everything that is normally there already is waited for first (the pending stage's V slot, the other tile's
+      // turn: see below), so that nothing but the MMAs themselves follows the softmax threads' hand-over.
+      if (p_valid && p_act && p_ntok > 0 && !warp_wait(s_vfull + 8 * (p_n % NV), (p_n / NV) & 1u, s_abort)) {
+        ok = false;
+        break;
+      }
+      // The tiles take turns, half a stage apart: S_0(n), S_1(n), S_0(n + 1), ... in this order, so that one tile's
+      // softmax runs beside the other tile's MMAs (P.V of the stage before, then these scores) instead of both tiles
+      // doing the same thing at once.  Tile 1 waits for tile 0's scores of this stage, tile 0 for tile 1's of the
+      // stage before -- on every stage, with or without work, so that neither warp can get two turns ahead of the
+      // other on a barrier pair.
+      if (t == 1 ? !warp_wait(s_sready + 8 * (n & 1), (n >> 1) & 1u, s_abort)
+                 : (n > 0 && !warp_wait(s_sready + 8 * (2 + ((n - 1) & 1)), ((n - 1) >> 1) & 1u, s_abort))) {
+        ok = false;
+        break;
+      }
       // ---- P.V of the pending stage: waits for the tile's softmax threads, then issues (or just takes the turn)
       if (p_valid) {
         const int vs = p_n % NV;
@@ -313,10 +329,6 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           break;
         }
         if (p_act && p_ntok > 0) {
-          if (!warp_wait(s_vfull + 8 * vs, (p_n / NV) & 1u, s_abort)) {
-            ok = false;
-            break;
-          }
           tc_fence_after_sync();
           if (lane == 0) {
             const uint64_t dv = umma_smem_desc(s_v + (uint32_t)vs * kTc2SlotBytes, kTc2HalfBytes, 1024);
@@ -337,16 +349,6 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
       }
       // ---- scores of this stage
-      // The tiles take turns, half a stage apart: S_0(n), S_1(n), S_0(n + 1), ... in this order, so that one tile's
-      // softmax runs beside the other tile's MMAs (P.V of the stage before, then these scores) instead of both tiles
-      // doing the same thing at once.  Tile 1 waits for tile 0's scores of this stage, tile 0 for tile 1's of the
-      // stage before -- on every stage, with or without work, so that neither warp can get two turns ahead of the
-      // other on a barrier pair.
-      if (t == 1 ? !warp_wait(s_sready + 8 * (n & 1), (n >> 1) & 1u, s_abort)
-                 : (n > 0 && !warp_wait(s_sready + 8 * (2 + ((n - 1) & 1)), ((n - 1) >> 1) & 1u, s_abort))) {
-        ok = false;
-        break;
-      }
       if (act && ntok > 0) {
         if (first) {
           if (!warp_wait(s_qready + 8 * t, n_q & 1u, s_abort)) {
