@@ -462,32 +462,47 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       if (end) break;
       if (act && ntok > 0) {
         tc_fence_after_sync();
-        uint32_t sr[64];  // sr[4 i + 2 rr + c] = score of row (row0 + 8 rr), token 8 i + 2 tq + c of the stage
-        tmem_ld_16x256b_x16(trow, sr);
-        tmem_ld_wait();
+        // Two passes over the stage's scores, 64 tokens at a time (32 registers): the row maxima first, then, with the
+        // reference maxima known, the weights.  Reading the scores twice costs little (tensor memory is close) and
+        // keeps the threads clear of spills.  sh[4 i + 2 rr + c] = score of row (row0 + 8 rr), token 64 h2 + 8 i + 2 tq + c.
         // tokens [0, e) of the stage are visible to the row
         const int e0 = min(min(meta2.z, lim_row[0]) - meta2.x, ntok), e1 = min(min(meta2.z, lim_row[1]) - meta2.x, ntok);
-        if (__any_sync(0xffffffffu, min(e0, e1) < kTc2StageTok)) {
+        const bool masked = __any_sync(0xffffffffu, min(e0, e1) < kTc2StageTok);
+        auto load_half = [&](int h2, uint32_t (&sh)[32]) {
+          tmem_ld_16x256b_x8(trow + 64 * h2, sh);
+          tmem_ld_wait();
+          if (masked) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i)
+            for (int i = 0; i < 8; ++i)
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              const int j = 8 * i + 2 * tq + c;
-              if (j >= e0) sr[4 * i + c] = 0xff800000u;  // -inf
-              if (j >= e1) sr[4 * i + 2 + c] = 0xff800000u;
+              for (int c = 0; c < 2; ++c) {
+                const int j = 64 * h2 + 8 * i + 2 * tq + c;
+                if (j >= e0) sh[4 * i + c] = 0xff800000u;  // -inf
+                if (j >= e1) sh[4 * i + 2 + c] = 0xff800000u;
+              }
+          }
+        };
+        float mxr[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+          uint32_t sh[32];
+          load_half(h2, sh);
+#pragma unroll
+          for (int rr = 0; rr < 2; ++rr) {
+            float ma = mxr[rr], mb = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) {  // three-input maximum: two scores per instruction, two chains
+              ma = fmax3(ma, __uint_as_float(sh[4 * i + 2 * rr]), __uint_as_float(sh[4 * i + 2 * rr + 1]));
+              mb = fmax3(mb, __uint_as_float(sh[4 * i + 4 + 2 * rr]), __uint_as_float(sh[4 * i + 4 + 2 * rr + 1]));
             }
+            mxr[rr] = fmaxf(ma, mb);
+          }
         }
         float alpha[2] = {1.f, 1.f}, neg_mu[2];
         bool raise_any = false;
 #pragma unroll
         for (int rr = 0; rr < 2; ++rr) {
-          float ma = -INFINITY, mb = -INFINITY;
-#pragma unroll
-          for (int i = 0; i < 16; i += 2) {  // three-input maximum: two scores per instruction, two chains
-            ma = fmax3(ma, __uint_as_float(sr[4 * i + 2 * rr]), __uint_as_float(sr[4 * i + 2 * rr + 1]));
-            mb = fmax3(mb, __uint_as_float(sr[4 * i + 4 + 2 * rr]), __uint_as_float(sr[4 * i + 4 + 2 * rr + 1]));
-          }
-          float mx = fmaxf(ma, mb);
+          float mx = mxr[rr];
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
           mx *= p.scale_log2e;  // the scale is positive
@@ -522,19 +537,23 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         float2 add0 = {0.f, 0.f}, add1 = {0.f, 0.f};
 #pragma unroll
         for (int h2 = 0; h2 < 2; ++h2) {  // 64 tokens at a time: 16 packed words of P per thread
+          uint32_t sh[32];
+          load_half(h2, sh);
+          // (P of the first 64 tokens lands on score columns 0 .. 31, read by now; the second 64 tokens' scores, still
+          // to be read, are columns 64 .. 127)
           uint32_t pw[16];  // pw[2 i + rr]: row (row0 + 8 rr), tokens 64 h2 + 8 i + 2 tq, + 1 = P column 32 h2 + 4 i + tq
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const int r = 4 * (8 * h2 + i);
-            const float2 x0 = ffma2(make_float2(__uint_as_float(sr[r]), __uint_as_float(sr[r + 1])), scale2, nm0);
-            const float2 x1 = ffma2(make_float2(__uint_as_float(sr[r + 2]), __uint_as_float(sr[r + 3])), scale2, nm1);
+            const int r = 4 * i;
+            const float2 x0 = ffma2(make_float2(__uint_as_float(sh[r]), __uint_as_float(sh[r + 1])), scale2, nm0);
+            const float2 x1 = ffma2(make_float2(__uint_as_float(sh[r + 2]), __uint_as_float(sh[r + 3])), scale2, nm1);
             const float2 w0 = make_float2(ex2(x0.x), ex2(x0.y)), w1 = make_float2(ex2(x1.x), ex2(x1.y));
             add0 = fadd2(add0, w0);
             add1 = fadd2(add1, w1);
             pw[2 * i] = pack_bf16x2(w0.x, w0.y);
             pw[2 * i + 1] = pack_bf16x2(w1.x, w1.y);
           }
-          tmem_st_16x128b_x8(trow + 32 * h2, pw);  // over the rows' scores (all of them are in registers by now)
+          tmem_st_16x128b_x8(trow + 32 * h2, pw);
         }
         l_part[0] += add0.x + add0.y;
         l_part[1] += add1.x + add1.y;
