@@ -1,27 +1,28 @@
 // Prefill-chunk attention over the paged cache on tcgen05, two row tiles per CTA (head_dim 128, bf16 cache, more than
 // 128 score columns per (sequence, kv head)).  Same plan, merge and work items as chunk_tc_kernel
-// (chunk_tc_kernels.cuh); a unit of work is (item, PAIR of 128-row tiles), one persistent CTA per SM:
+// (chunk_tc_kernels.cuh); a unit of work is (item, PAIR of 128-row tiles), one persistent CTA of 20 warps per SM:
 //
-//   warps 0..3   softmax of tile 0: thread r owns score row r of the tile (tensor-memory lane r)
-//   warps 4..7   softmax of tile 1
-//   warp 8       K producer: walks the units, TMA copies of the K slots (128 tokens: [half][128 tok][64 dims],
-//                128-byte swizzle), posts each stage's meta words and a descriptor of its V boxes
-//   warp 9       V producer: TMA copies of the V slots from those descriptors
-//   warp 10      owns the tensor memory (512 columns); one lane issues the MMAs of both tiles:
-//                  S_t[128 x 128]   = Q_t[128 x 128] . K_slot^T    8 x tcgen05.mma M128 N128 K16, both operands shared memory
-//                  O_t[128 x 128] (+)= P_t[128 x 128] . V_slot      8 x tcgen05.mma M128 N128 K16, P from tensor memory,
-//                                                                   V MN-major from the slot
-//                columns of tile t: S_t at 256 t (P_t, two bf16 per column, over its first 64 once the softmax
-//                threads have read S_t), O_t at 256 t + 128.  Q_t lives in shared memory (32 KiB per tile).
+//   warps 0..7    softmax of tile 0, warps 8..15 of tile 1: a warp owns 16 score rows (tensor-memory lanes), four
+//                 threads share a row (16-lane tensor-memory shapes, quad shuffles)
+//   warp 16       K producer: walks the units, TMA copies of the K slots (128 tokens: [half][128 tok][64 dims],
+//                 128-byte swizzle), posts each stage's meta words and a descriptor of its V boxes
+//   warp 17       V producer: TMA copies of the V slots from those descriptors
+//   warps 18, 19  one lane of warp 18 + t issues the MMAs of tile t into the 512 tensor-memory columns:
+//                   S_t[128 x 128]   = Q_t[128 x 128] . K_slot^T    8 x tcgen05.mma M128 N128 K16, both operands shared memory
+//                   O_t[128 x 128] (+)= P_t[128 x 128] . V_slot      8 x tcgen05.mma M128 N128 K16, P from tensor memory,
+//                                                                    V MN-major from the slot
+//                 columns of tile t: S_t at 256 t (P_t, two bf16 per column, over its first 64 once the softmax
+//                 threads have read S_t), O_t at 256 t + 128.  Q_t lives in shared memory (32 KiB per tile).
 //
-// The two tiles share every K / V slot (half the shared-memory fills of one tile per CTA) and take turns on the tensor
-// pipe: the MMAs are issued in the order  S_0(j) S_1(j) | P.V_0(j) S_0(j+1) P.V_1(j) S_1(j+1) | P.V_0(j+1) ...  so that
-// while the softmax threads of one tile work on their scores the pipe runs the other tile's MMAs.  The pipe executes
-// one thread's MMAs in order, which makes it safe for S_t(j+1) to overwrite P_t(j), and means P.V_t(j-1) is complete
-// whenever S_t(j) is: a softmax thread may rescale its row of O_t as soon as it holds the scores.  With 128-token
-// slots the fetch of the shared-memory A operand (Q) is amortised over twice the columns: the score MMAs are no longer
-// bound by it.  Every wait is bounded; on a wait that gives up the CTA stops issuing, drains and releases the tensor
-// memory.
+// Why this shape.  One thread gets an MMA issued about every 110 cycles whatever its size (measured: N 64 or 128, either
+// operand source; N 256: 165), so MMAs should be as large as tensor memory allows (128-token slots: N = 128 for the
+// scores) and each tile needs an issuing thread of its own (two issuers run side by side: one N = 128 MMA per 70
+// cycles).  A tile's chain per stage is  scores -> softmax -> P.V -> next scores  (S_t(n+1) overwrites P_t(n), and the
+// pipe executes one thread's MMAs in order, so P.V_t(n) is issued first; it also means P.V_t(n-1) is complete whenever
+// S_t(n) is: a softmax thread may rescale its rows of O_t as soon as it holds the scores).  The chain is latency-bound,
+// so the two tiles run half a stage apart -- the issuing warps keep the order S_0(n), S_1(n), S_0(n+1), ... -- and one
+// tile's softmax runs beside the other tile's MMAs.  The tiles share every K / V slot.  Every wait is bounded; on a
+// wait that gives up the CTA stops issuing, drains and releases the tensor memory.
 #pragma once
 #include "chunk_tc_kernels.cuh"
 
