@@ -196,7 +196,8 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  * read once); more columns run a prefill-chunk kernel, which cuts the columns into row tiles of
  * up to 128, reads the cache once per row tile (the repeats hit L2) and never loads tokens a tile
  * cannot see; it becomes bound by the tensor pipe from about 64 columns on.  At head_dim 128 and
- * more than 32 columns that kernel runs on tcgen05 (scores and output in tensor memory), otherwise
+ * more than 32 columns that kernel runs on tcgen05 (scores and output in tensor memory; beyond 128
+ * columns over a bf16 cache with two 128-row tiles per CTA taking turns on the tensor pipe), otherwise
  * on mma.sync.  Over the 8-bit cache
  * (ooco_decode_step_mq_fp8) every chunk of more than 16 columns runs the tcgen05 kernel, whose extra
  * warps widen each 8-bit stage to f16 in shared memory first.  The workspace grows with q_len: one fp32
