@@ -226,7 +226,7 @@ def test_range_predicates_of_the_checked_build():
 def test_fp32_output_knob_is_a_switch():
     assert binding.get_tuning("out_f32") == 0
     L = binding.lib()
-    assert L.ooco_set_tuning(13, 2) == -2 and L.ooco_set_tuning(15, 1) == -2 and L.ooco_get_tuning(99) == -2
+    assert L.ooco_set_tuning(13, 2) == -2 and L.ooco_set_tuning(16, 1) == -2 and L.ooco_get_tuning(99) == -2
     binding.set_tuning(out_f32=1)
     try:
         assert binding.get_tuning("out_f32") == 1
