@@ -653,7 +653,8 @@ def run_multi_query(args, local_rank):
     columns = Sq * (cfg.num_q_heads // cfg.num_kv_heads)
     tcgen05 = (columns > 32 and cfg.head_dim == 128 and not any(k.startswith("chunk_tcgen05=0") for k in args.knob)) or \
               (fp8 and columns > 16)
-    kernel = ("chunk_tc_kernel" if tcgen05 else "chunk_main_kernel") if columns > 16 else (
+    two_tiles = tcgen05 and not fp8 and columns > 128 and not any(k.startswith("chunk_two_tiles=0") for k in args.knob)
+    kernel = (("chunk_tc2_kernel" if two_tiles else "chunk_tc_kernel") if tcgen05 else "chunk_main_kernel") if columns > 16 else (
         "row16_main_kernel" if columns > 8 and not fp8 else "decode_main_kernel")   # (the 8-bit cache has no row16 kernel)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "kernel": kernel, "algorithmic_bytes_per_launch": nbytes,

@@ -78,6 +78,11 @@ CHUNK_CASES = [
     # split into several chunks (few long sequences)
     (C("ck-split", 32, 8, 128, 16, fixed(9000, 2049, 70), seed=110, pool_fill=0.9, shuffle_batch=False), 48),
     (C("ck-split-g2", 16, 8, 128, 16, fixed(20000, 4100), seed=111, shuffle_batch=False), 9),
+    # 320 columns: a pair of 128-row tiles, then a pair whose second tile has no rows; contexts around the slot size
+    # (sigma 0.5: the first queries of a fresh prompt return single V entries, whose bf16 rounding alone would pass
+    # 1e-2 beyond |v| = 2.56)
+    (C("ck-g4-sq80", 32, 8, 128, 16, fixed(80, 81, 127, 128, 129, 208, 2600, 9100), seed=112, pool_fill=0.8,
+       shuffle_batch=False, sigma=0.5), 80),
 ]
 
 
@@ -97,6 +102,19 @@ def test_prefill_chunk_on_the_mma_sync_kernel(cfg, Sq):
         run_case(cfg, Sq, seed=cfg.seed)
     finally:
         binding.set_tuning(chunk_tcgen05=1)
+
+
+@pytest.mark.parametrize("cfg,Sq", [c for c in CHUNK_CASES if c[0].name in
+                                    ("ck-g4-sq33", "ck-g4-sq128-fresh", "ck-g8-sq64-bs64", "ck-split", "ck-g4-sq80")],
+                         ids=lambda v: getattr(v, "name", str(v)))
+def test_prefill_chunk_on_the_one_tile_tcgen05_kernel(cfg, Sq):
+    """More than 128 score columns over a bf16 cache run the kernel with two 128-row tiles per CTA by default;
+    the one-tile tcgen05 kernel stays selectable and must agree with the oracle too."""
+    binding.set_tuning(chunk_two_tiles=0)
+    try:
+        run_case(cfg, Sq, seed=cfg.seed)
+    finally:
+        binding.set_tuning(chunk_two_tiles=1)
 
 
 def test_chunk_rows_agree_with_decode_rows():
