@@ -1,5 +1,5 @@
-// Thin wrappers over the sm_100a PTX the kernels use: mbarrier, bulk / tensor async copies (TMA, never
-// multicast), ldmatrix, movmatrix, bf16 mma.sync, ex2, and tcgen05 (MMA from shared memory into tensor memory).
+// Thin wrappers over the sm_100a PTX the kernels use: mbarrier, bulk / tensor async copies (TMA, one
+// destination CTA each), ldmatrix, movmatrix, bf16 mma.sync, ex2, and tcgen05 (MMA from shared memory into tensor memory).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
