@@ -71,9 +71,9 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const uint32_t s_vdfull = s_vempty + NV * 8;     // [NV] the stage's V descriptor is posted             (K producer)
   const uint32_t s_mfull = s_vdfull + NV * 8;      // [NM] the stage's meta words are posted              (K producer)
   const uint32_t s_sready = s_mfull + NM * 8;      // [2 tiles][2] S_t holds the stage's scores            (MMA commit)
-  const uint32_t s_pready = s_sready + 32;         // [2 tiles][2] P_t written, O_t rescaled, V rows clean (128 threads)
+  const uint32_t s_pready = s_sready + 32;         // [2 tiles][2] P_t written, O_t rescaled, V rows clean (256 threads)
   const uint32_t s_pvdone = s_pready + 32;         // [2 tiles] the unit's last P.V_t is complete          (MMA commit)
-  const uint32_t s_qready = s_pvdone + 16;         // [2 tiles] Q_t of the unit is in shared memory        (128 threads)
+  const uint32_t s_qready = s_pvdone + 16;         // [2 tiles] Q_t of the unit is in shared memory        (256 threads)
   const uint32_t s_drain = s_qready + 16;
   const uint32_t s_slot = s_drain + 16;
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
