@@ -651,9 +651,11 @@ def run_multi_query(args, local_rank):
     peak, peak_kind = measured_peak()
     achieved = nbytes / (attn * 1e-3) / 1e9
     columns = Sq * (cfg.num_q_heads // cfg.num_kv_heads)
-    tcgen05 = (columns > 32 and cfg.head_dim == 128 and not any(k.startswith("chunk_tcgen05=0") for k in args.knob)) or \
-              (fp8 and columns > 16)
-    two_tiles = tcgen05 and not fp8 and columns > 128 and not any(k.startswith("chunk_two_tiles=0") for k in args.knob)
+    knobs = dict(k.split("=", 1) for k in args.knob)
+    tc_knob, tt_knob = int(knobs.get("chunk_tcgen05", 1)), int(knobs.get("chunk_two_tiles", 2))
+    tc_from = 17 if tc_knob == 1 else tc_knob                              # first column count on the tcgen05 kernels
+    tcgen05 = columns > 16 and cfg.head_dim == 128 and (fp8 or (tc_knob != 0 and columns >= tc_from))
+    two_tiles = tcgen05 and not fp8 and tt_knob != 0 and (columns > 128 or tt_knob == 2)
     kernel = (("chunk_tc2_kernel" if two_tiles else "chunk_tc_kernel") if tcgen05 else "chunk_main_kernel") if columns > 16 else (
         "row16_main_kernel" if columns > 8 and not fp8 else "decode_main_kernel")   # (the 8-bit cache has no row16 kernel)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -195,10 +195,10 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  * (sequence, kv head), (Hq / Hkv) * q_len <= 16, run the decode kernels (HBM-bound: the cache is
  * read once); more columns run a prefill-chunk kernel, which cuts the columns into row tiles of
  * up to 128, reads the cache once per row tile (the repeats hit L2) and never loads tokens a tile
- * cannot see; it becomes bound by the tensor pipe from about 64 columns on.  At head_dim 128 and
- * more than 32 columns that kernel runs on tcgen05 (scores and output in tensor memory; beyond 128
- * columns over a bf16 cache with two 128-row tiles per CTA taking turns on the tensor pipe), otherwise
- * on mma.sync.  Over the 8-bit cache
+ * cannot see; it becomes bound by the tensor pipe beyond 128 columns.  At head_dim 128 that kernel
+ * runs on tcgen05 (scores and output in tensor memory; over a bf16 cache one CTA per SM with two
+ * 128-row tiles taking turns on the tensor pipe, or, up to 128 columns, one tile whose scores run a
+ * stage ahead of its softmax), otherwise on mma.sync.  Over the 8-bit cache
  * (ooco_decode_step_mq_fp8) every chunk of more than 16 columns runs the tcgen05 kernel, whose extra
  * warps widen each 8-bit stage to f16 in shared memory first.  The workspace grows with q_len: one fp32
  * partial row per (split item, score column).  q_len = 1 is ooco_decode_attention /
@@ -456,16 +456,19 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * directly (zero = always one copy per buffer; 2 = as 1, but q is staged on the device by the first launch
  * instead of being fetched from the host mapping by the attention kernel); 11 non-zero = 9 to 16 score columns per
  * (sequence, kv head) run the kernel whose warps share 16 score rows and split the tokens of a
- * stage (zero = the decode kernel with two 8-column tiles); 12 non-zero = more than 32 score columns
- * at head_dim 128 run the tcgen05 kernel (zero = the mma.sync kernel of the prefill-chunk path).
+ * stage (zero = the decode kernel with two 8-column tiles); 12 = which prefill chunks (more than 16 score
+ * columns) run the tcgen05 kernels at head_dim 128 over a bf16 cache: 1 = all of them (default), n in
+ * [17, 65536] = those with n or more score columns, 0 = none (the mma.sync kernel of the prefill-chunk path).
  * 13 non-zero = diagnostic fp32 output: `out` of the attention entry points is then fp32 (same
  * shape, 4 bytes per value) and holds the values the kernels would otherwise round to bf16 (every
  * row goes through the partial-result and merge path; an unsplit row passes it unchanged), so a
  * test can separate the arithmetic's error from the output format's rounding; not for the host-buffer
  * step (OOCO_E_UNSUPPORTED).  14 non-zero = the decode kernel over the 8-bit cache (8 consumer warps)
  * computes its scores on tcgen05 from the stored codes (zero = mma.sync on codes widened in registers).
- * 15 non-zero = prefill chunks of more than 128 score columns over a bf16 cache (head_dim 128) run the tcgen05
- * kernel that keeps two 128-row tiles per CTA (zero = one tile per CTA, two CTAs per SM).
+ * 15 = the tcgen05 kernel with one CTA per SM and two 128-row tiles per CTA (bf16 cache, head_dim 128): 2 (default) =
+ * every chunk that knob 12 sends to tcgen05 (with 128 score columns or fewer the kernel runs one tile and gives the
+ * second tile's score buffer and issuing warp to it), 1 = only chunks of more than 128 score columns, 0 = never (one
+ * tile per CTA, two CTAs per SM).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.  ooco_get_tuning returns a knob's current value
  * (OOCO_E_SHAPE, which is negative, for an unknown knob).

@@ -52,21 +52,26 @@ __global__ void __launch_bounds__(kTc2Threads, 1)
 chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const DecodeParams p) {
   constexpr int D = 128;
-  constexpr int NK = kTc2KSlots, NV = kTc2VSlots, NM = kTc2MetaRing;
+  constexpr int NV = kTc2VSlots, NM = kTc2MetaRing;
+  // One-tile mode: no work item has rows for tile 1 (at most 128 score columns).  The kernel is then bound by HBM,
+  // not by the tensor pipe, and what would idle serves the one tile: tile 1's Q region is a third K slot, tile 1's
+  // score columns a second S buffer, and tile 1's issuing warp issues the P.V MMAs (see the MMA warps).
+  const bool solo = p.GQ <= kTcRows;
+  const int NK = solo ? kTc2KSlots + 1 : kTc2KSlots;
   constexpr int kWarpK = 16, kWarpV = 17, kWarpM = 18;  // warps 0 .. 15: softmax; 18, 19: MMA of tile 0, 1
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const uint32_t s_q = base;                                       // [2] Q tiles
-  const uint32_t s_k = s_q + 2u * kTc2QBytes;                      // [NK] K slots
-  const uint32_t s_v = s_k + (uint32_t)NK * kTc2SlotBytes;         // [NV] V slots
+  const uint32_t s_k = s_q + (solo ? 1u : 2u) * kTc2QBytes;        // [NK] K slots
+  const uint32_t s_v = s_q + 2u * kTc2QBytes + (uint32_t)kTc2KSlots * kTc2SlotBytes;  // [NV] V slots
   const uint32_t s_meta = s_v + (uint32_t)NV * kTc2SlotBytes;      // [NM] two int4 per stage
   const uint32_t s_vdesc = s_meta + (uint32_t)NM * 32;             // [NV] VStageDesc
   const uint32_t s_bar = s_vdesc + (uint32_t)NV * sizeof(VStageDesc);
   const uint32_t s_kfull = s_bar;                  // [NK] the K slot has landed                          (TMA)
-  const uint32_t s_kempty = s_kfull + NK * 8;      // [NK] the score MMAs that read it are complete       (MMA commit)
-  const uint32_t s_vfull = s_kempty + NK * 8;      // [NV] the V slot has landed                          (TMA)
+  const uint32_t s_kempty = s_kfull + (kTc2KSlots + 1) * 8;      // [NK] the score MMAs that read it are complete       (MMA commit)
+  const uint32_t s_vfull = s_kempty + (kTc2KSlots + 1) * 8;      // [NV] the V slot has landed                          (TMA)
   const uint32_t s_vempty = s_vfull + NV * 8;      // [NV] the P.V MMAs that read it are complete         (MMA commit)
   const uint32_t s_vdfull = s_vempty + NV * 8;     // [NV] the stage's V descriptor is posted             (K producer)
   const uint32_t s_mfull = s_vdfull + NV * 8;      // [NM] the stage's meta words are posted              (K producer)
@@ -74,7 +79,8 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const uint32_t s_pready = s_sready + 32;         // [2 tiles][2] P_t written, O_t rescaled, V rows clean (256 threads)
   const uint32_t s_pvdone = s_pready + 32;         // [2 tiles] the unit's last P.V_t is complete          (MMA commit)
   const uint32_t s_qready = s_pvdone + 16;         // [2 tiles] Q_t of the unit is in shared memory        (256 threads)
-  const uint32_t s_drain = s_qready + 16;
+  const uint32_t s_pvstage = s_qready + 16;       // [2] one-tile mode: the stage's P.V is complete              (MMA commit)
+  const uint32_t s_drain = s_pvstage + 16;
   const uint32_t s_slot = s_drain + 16;
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
   VStageDesc* g_vdesc = reinterpret_cast<VStageDesc*>(gen + (s_vdesc - base));
@@ -86,11 +92,11 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     *s_abort = 0;
     for (int i = 0; i < NK; ++i) {
       mbar_init(s_kfull + 8 * i, 1);
-      mbar_init(s_kempty + 8 * i, 2);  // one arrival per MMA warp
+      mbar_init(s_kempty + 8 * i, solo ? 1 : 2);  // one arrival per MMA warp that reads K
     }
     for (int i = 0; i < NV; ++i) {
       mbar_init(s_vfull + 8 * i, 1);
-      mbar_init(s_vempty + 8 * i, 2);
+      mbar_init(s_vempty + 8 * i, solo ? 1 : 2);
       mbar_init(s_vdfull + 8 * i, 1);
     }
     for (int i = 0; i < NM; ++i) mbar_init(s_mfull + 8 * i, 1);
@@ -101,6 +107,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (int i = 0; i < 2; ++i) {
       mbar_init(s_pvdone + 8 * i, 1);
       mbar_init(s_qready + 8 * i, 256);
+      mbar_init(s_pvstage + 8 * i, 1);
     }
     mbar_init(s_drain, 1);
     mbar_init(s_drain + 8, 1);
@@ -277,6 +284,121 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         mbar_wait_bounded(s_vfull + 8 * (j % NV), (uint32_t)(j / NV) & 1u, &dummy_abort, kWaitLimitNs / 8);
       }
     }
+  } else if (warp >= kWarpM && solo) {
+    // ================================================================= MMA warps, one-tile mode
+    // One thread issues an MMA about every 100 cycles, so a single issuing thread needs longer for the 16 MMAs of a
+    // stage than HBM needs for the stage's bytes.  With one tile the two issuing warps split the stage instead: warp
+    // kWarpM issues the scores S(n) = Q . K_slot^T into S buffer n & 1 (columns 256 (n & 1); buffer 1 is what tile 1's
+    // scores would occupy), warp kWarpM + 1 the values O += P(n) . V_slot.  The pipe keeps no order between two
+    // threads' MMAs, so each hand-over has a barrier: S(n) overwrites P(n - 2), hence waits for P.V(n - 2) to be
+    // complete (s_pvstage, one completion per stage, with or without tokens); P.V(n) waits for the softmax threads'
+    // P(n).  The scores of a stage are thus computed while the softmax threads still work on the one before.
+    const int t = warp - kWarpM;
+    bool issued = false, ok = true;
+    if (t == 0) {
+      const uint32_t idesc_s = umma_idesc_16bit(kTcRows, kTc2StageTok, 0, true);
+      const uint64_t dq = umma_smem_desc(s_q, 0, 1024);
+      uint32_t n_q = 0;  // units with tokens (uses of the q-ready barrier)
+      for (uint32_t n = 0;; ++n) {
+        const int ks = n % NK, ms = n % NM;
+        if (!warp_wait(s_kfull + 8 * ks, (n / NK) & 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        const int4 meta = g_meta[2 * ms];
+        const bool end = meta.x < 0;
+        const int ntok = end ? 0 : (meta.w & 0xffff);
+        const bool first = !end && ((meta.w >> 16) & 1);
+        // The buffer's previous contents, P(n - 2), have been consumed.  Waited for on every stage, with or without
+        // tokens (the end marker included): it also means that the softmax threads are past their wait for S(n - 2),
+        // so this stage's completion of the score barrier n & 1 cannot overtake them.
+        if (n >= 2 && !warp_wait(s_pvstage + 8 * (n & 1), ((n - 2) >> 1) & 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        if (ntok > 0) {
+          if (first) {
+            if (!warp_wait(s_qready, n_q & 1u, s_abort)) {
+              ok = false;
+              break;
+            }
+            ++n_q;
+          }
+          tc_fence_after_sync();
+          if (lane == 0) {
+            const uint64_t dk = umma_smem_desc(s_k + (uint32_t)ks * kTc2SlotBytes, 0, 1024);
+            const uint32_t ts = tmem + 256u * (n & 1);
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {  // 16 dims = 32 bytes further along the rows; the second 64 dims = the next half
+                const uint64_t off = (uint64_t)((hh * kTc2HalfBytes + k * 32) >> 4);
+                umma_ss(ts, dq + off, dk + off, idesc_s, (hh | k) ? 1u : 0u);
+              }
+            umma_commit(s_sready + 8 * (n & 1));
+            umma_commit(s_kempty + 8 * ks);
+          }
+          __syncwarp();
+          issued = true;
+        } else {
+          // no scores: the turn of the barriers is taken all the same (also wakes the softmax threads for the end marker)
+          if (lane == 0) {
+            mbar_arrive(s_sready + 8 * (n & 1));
+            mbar_arrive(s_kempty + 8 * ks);
+          }
+          __syncwarp();
+        }
+        if (end) break;
+      }
+    } else {
+      const uint32_t idesc_o = umma_idesc_16bit(kTcRows, D, 1, true);
+      for (uint32_t n = 0;; ++n) {
+        const int vs = n % NV, ms = n % NM;
+        if (!warp_wait(s_mfull + 8 * ms, (n / NM) & 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        const int4 meta = g_meta[2 * ms];
+        if (meta.x < 0) break;
+        const int ntok = meta.w & 0xffff;
+        const bool first = (meta.w >> 16) & 1, last = (meta.w >> 17) & 1;
+        // the V slot first (normally there already), so that nothing but the MMAs follows the softmax threads' hand-over
+        if ((ntok > 0 && !warp_wait(s_vfull + 8 * vs, (n / NV) & 1u, s_abort)) ||
+            !warp_wait(s_pready + 8 * (n & 1), (n >> 1) & 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        if (ntok > 0) {
+          tc_fence_after_sync();
+          if (lane == 0) {
+            const uint64_t dv = umma_smem_desc(s_v + (uint32_t)vs * kTc2SlotBytes, kTc2HalfBytes, 1024);
+            const uint32_t tp = tmem + 256u * (n & 1);
+#pragma unroll
+            for (int k = 0; k < kTc2StageTok / 16; ++k)  // 16 tokens: 8 columns of P, 16 rows of 128 bytes of V in either half
+              umma_ts(tmem + 128, tp + 8 * k, dv + (uint64_t)(k * (2048 >> 4)), idesc_o, (first && k == 0) ? 0u : 1u);
+            if (last) umma_commit(s_pvdone);
+            umma_commit(s_pvstage + 8 * (n & 1));
+            umma_commit(s_vempty + 8 * vs);
+          }
+          __syncwarp();
+          issued = true;
+        } else {
+          if (lane == 0) {
+            if (last) mbar_arrive(s_pvdone);  // a unit without tokens: nothing to wait for
+            mbar_arrive(s_pvstage + 8 * (n & 1));
+            mbar_arrive(s_vempty + 8 * vs);
+          }
+          __syncwarp();
+        }
+      }
+    }
+    if (!ok && lane == 0) atomicOr(&p.hdr->status, kStatusWaitTimeout);
+    if (!ok && issued) {  // the tensor memory must not be released under MMAs in flight
+      if (lane == 0) umma_commit(s_drain + 8 * t);
+      __syncwarp();
+      int dummy = 0;
+      mbar_wait_bounded(s_drain + 8 * t, 0u, &dummy, kWaitLimitNs / 8);
+    }
   } else if (warp >= kWarpM) {
     // ================================================================= MMA warps: warp kWarpM + t issues tile t's MMAs
     // One thread issues an MMA about every 110 to 130 cycles whatever its size (measured: M128 N64 or N128 K16, either
@@ -432,7 +554,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       fence_proxy_async_smem();  // the tile is read by the MMAs through the async proxy
       mbar_arrive(s_qready + 8 * t);
     };
-    for (uint32_t n = 0;; ++n) {
+    for (uint32_t n = 0; !(solo && t == 1); ++n) {  // (one-tile mode: the warps of tile 1 have nothing to do)
       const int ms = n % NM;
       if (!warp_wait(s_mfull + 8 * ms, (n / NM) & 1u, s_abort)) {
         ok = false;
@@ -469,8 +591,9 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         // tokens [0, e) of the stage are visible to the row
         const int e0 = min(min(meta2.z, lim_row[0]) - meta2.x, ntok), e1 = min(min(meta2.z, lim_row[1]) - meta2.x, ntok);
         const bool masked = __any_sync(0xffffffffu, min(e0, e1) < kTc2StageTok);
+        const uint32_t srow = trow + (solo ? 256u * (n & 1) : 0u);  // the stage's S (and P) columns
         auto load_half = [&](int h2, uint32_t (&sh)[32]) {
-          tmem_ld_16x256b_x8(trow + 64 * h2, sh);
+          tmem_ld_16x256b_x8(srow + 64 * h2, sh);
           tmem_ld_wait();
           if (masked) {
 #pragma unroll
@@ -520,6 +643,12 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
         if (__any_sync(0xffffffffu, raise_any)) {
           // P.V of the previous stage was issued before this stage's score MMAs, so it is complete: O may be rescaled
+          // (one-tile mode: another thread issues it, so its own barrier is waited on; never on a unit's first stage)
+          if (solo && !warp_wait(s_pvstage + 8 * ((n - 1) & 1), ((n - 1) >> 1) & 1u, s_abort)) {
+            ok = false;
+            break;
+          }
+          if (solo) tc_fence_after_sync();
 #pragma unroll 1
           for (int c2 = 0; c2 < 2; ++c2) {
             uint32_t o[32];
@@ -554,7 +683,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             pw[2 * i] = pack_bf16x2(w0.x, w0.y);
             pw[2 * i + 1] = pack_bf16x2(w1.x, w1.y);
           }
-          tmem_st_16x128b_x8(trow + 32 * h2, pw);
+          tmem_st_16x128b_x8(srow + 32 * h2, pw);
         }
         l_part[0] += add0.x + add0.y;
         l_part[1] += add1.x + add1.y;

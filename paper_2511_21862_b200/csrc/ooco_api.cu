@@ -24,7 +24,7 @@ namespace ooco {
 // Launch-shape knobs (benchmark sweeps); defaults are the tuned configuration.
 enum Knob { kKnobWarps = 0, kKnobStages, kKnobCtasPerSm, kKnobChunkMin, kKnobChunkMax, kKnobItemsPerCta,
             kKnobSplitHalves, kKnobTilesPerWarp, kKnobPdl, kKnobCopyCtasPerSm, kKnobHostStageKernel, kKnobRowLayout16, kKnobChunkTcgen05, kKnobOutF32, kKnobKv8Tcgen05, kKnobChunkTwoTiles, kKnobCount };
-static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}, {0}, {1}, {1}};
+static std::atomic<int> g_knobs[kKnobCount] = {{4}, {0}, {2}, {256}, {8192}, {6}, {0}, {1}, {1}, {1}, {1}, {1}, {1}, {0}, {1}, {2}};
 static std::atomic<int> g_overridden[kKnobCount];  // knob set through ooco_set_tuning
 constexpr int kGridCap = 592;  // 148 SMs x 4 CTAs: most CTAs any launch shape uses (host-only workspace bound)
 
@@ -321,8 +321,8 @@ static int launch_chunk(const CUtensorMap& tk, const CUtensorMap& tv, DecodePara
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the chunk attention kernel", (long)e);
 }
 
-// Prefill chunk on tcgen05 (head_dim 128, more than 32 score columns: from there on it beats the mma.sync
-// kernel on every workload measured, a half-empty 128-row tile included): two CTAs per SM.
+// Prefill chunk on tcgen05 with one 128-row tile per CTA and two CTAs per SM (head_dim 128): what the 8-bit cache
+// runs, and the bf16 cache when the kernel below is switched off.
 template <bool KV8>
 static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                            int ctas_per_sm, cudaStream_t st, int dev, bool dry) {
@@ -358,8 +358,10 @@ static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeP
   return e == cudaSuccess ? OOCO_OK : fail_cuda("launch of the tcgen05 chunk attention kernel", (long)e);
 }
 
-// Prefill chunk on tcgen05 with two 128-row tiles per CTA (head_dim 128, bf16 cache, more than 128 score columns):
-// one persistent CTA per SM, 512 tensor-memory columns, 128-token K / V slots.
+// Prefill chunk on tcgen05, one persistent CTA per SM, 512 tensor-memory columns, 128-token K / V slots (head_dim 128,
+// bf16 cache): two 128-row tiles per CTA beyond 128 score columns; up to 128 columns its one-tile mode, in which the
+// second tile's resources (score columns, issuing warp, Q region) pipeline the one tile -- it beats the one-tile
+// kernel and the mma.sync kernel on every workload measured, from 17 columns on.
 static int launch_chunk_tc2(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                             cudaStream_t st, int dev, bool dry) {
   auto kern = chunk_tc2_kernel;
@@ -636,7 +638,9 @@ int ooco_set_tuning(int knob, int value) {
   if (knob == kKnobItemsPerCta && (value < 1 || value > 64)) return OOCO_E_SHAPE;
   if (knob == kKnobTilesPerWarp && value != 1 && value != 2) return OOCO_E_SHAPE;
   if (knob == kKnobCopyCtasPerSm && (value < 1 || value > 3)) return OOCO_E_SHAPE;
-  if ((knob == kKnobOutF32 || knob == kKnobKv8Tcgen05 || knob == kKnobChunkTwoTiles) && value != 0 && value != 1) return OOCO_E_SHAPE;
+  if ((knob == kKnobOutF32 || knob == kKnobKv8Tcgen05) && value != 0 && value != 1) return OOCO_E_SHAPE;
+  if (knob == kKnobChunkTwoTiles && (value < 0 || value > 2)) return OOCO_E_SHAPE;
+  if (knob == kKnobChunkTcgen05 && value != 0 && value != 1 && (value < 17 || value > 65536)) return OOCO_E_SHAPE;
   g_knobs[knob].store(value);
   g_overridden[knob].store(1);
   return OOCO_OK;
@@ -745,9 +749,13 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // column layout of the decode kernel needs a second MMA tile and a transposition per tile there)
   const bool row16 = !chunk && !kv8 && G_ > 8 && g_knobs[kKnobRowLayout16].load() != 0;
   // (the 8-bit cache has no mma.sync chunk kernel: every chunk over it runs the tcgen05 kernel)
-  const bool chunk_tc = chunk && s->head_dim == 128 && (kv8 || (G_ > 32 && g_knobs[kKnobChunkTcgen05].load() != 0));
+  // (knob 12: 0 = never; 1 = every prefill chunk, i.e. from 17 score columns; n >= 17 = from n columns)
+  const int tc_knob = g_knobs[kKnobChunkTcgen05].load();
+  const int tc_from = tc_knob == 1 ? 17 : tc_knob;
+  const bool chunk_tc = chunk && s->head_dim == 128 && (kv8 || (tc_knob != 0 && G_ >= tc_from));
   // (more than one 128-row tile per item, bf16: the kernel that keeps two tiles per CTA on the tensor pipe in turns)
-  const bool chunk_tc2 = chunk_tc && !kv8 && G_ > kTcRows && g_knobs[kKnobChunkTwoTiles].load() != 0;
+  const int two_tiles = g_knobs[kKnobChunkTwoTiles].load();  // 1: beyond 128 columns only; 2: its one-tile mode below, too
+  const bool chunk_tc2 = chunk_tc && !kv8 && two_tiles != 0 && (G_ > kTcRows || two_tiles == 2);
   if (chunk) {
     ncw = chunk_warps(G_);
     cps = (ncw == 8 && !chunk_tc) ? 1 : 2;

@@ -150,7 +150,11 @@ def test_query_length_limits_and_workspace_growth_without_a_device():
     assert attn(64, q=odd) == -3 and attn(64, out=odd) == -3
     assert attn(64, ws_bytes=binding.workspace_bytes_mq(sh, 4)) == -4
     assert L.ooco_set_tuning(11, 0) == 0 and L.ooco_set_tuning(11, 1) == 0 and L.ooco_set_tuning(12, 1) == 0 and L.ooco_set_tuning(16, 1) == -2
-    assert L.ooco_set_tuning(15, 0) == 0 and L.ooco_set_tuning(15, 2) == -2 and L.ooco_set_tuning(15, 1) == 0   # two-tile chunk kernel
+    assert L.ooco_set_tuning(15, 0) == 0 and L.ooco_set_tuning(15, 3) == -2 and L.ooco_set_tuning(15, 1) == 0   # two-tile chunk kernel
+    assert L.ooco_set_tuning(15, 2) == 0
+    # knob 12: off, every prefill chunk, or a first column count of 17 or more
+    assert L.ooco_set_tuning(12, 16) == -2 and L.ooco_set_tuning(12, 33) == 0 and L.ooco_set_tuning(12, 0) == 0
+    assert L.ooco_set_tuning(12, 1) == 0
 
 
 def test_missing_library_fails_loudly(monkeypatch):

@@ -65,8 +65,10 @@ def test_multi_query_matches_oracle(cfg, Sq):
 # More than 16 score columns per (sequence, kv head): the prefill-chunk kernel (row tiles of 32 / 64 / 128
 # columns).  Contexts shorter than, equal to and just above the chunk; ragged last row tile; every block size.
 CHUNK_CASES = [
+    # 20 columns.  (sigma 0.5: with contexts of a few tokens the rows are single V entries or means of a few, and at
+    # |out| >= 2 the rounding of the bf16 output, 2^-7, plus that of the bf16 weights, 2^-9 |v|, alone passes 1e-2)
     (C("ck-g4-sq5", 32, 8, 128, 16, fixed(0, 1, 4, 5, 6, 63, 64, 65, 129, 700), seed=101, pool_fill=0.7,
-       shuffle_batch=False), 5),                                              # 20 columns: 2-warp CTAs
+       shuffle_batch=False, sigma=0.5), 5),
     (C("ck-g4-sq16", 32, 8, 128, 16, fixed(3, 16, 17, 64, 100, 1000), seed=102, shuffle_batch=False), 16),   # 64 columns
     (C("ck-g4-sq33", 32, 8, 128, 16, fixed(33, 34, 200, 1500), seed=103, shuffle_batch=False), 33),          # 132: ragged tile
     (C("ck-g4-sq128-fresh", 32, 8, 128, 16, fixed(128, 128, 500, 1290), seed=104, shuffle_batch=False), 128),  # T = S_q: a whole prompt
@@ -83,6 +85,11 @@ CHUNK_CASES = [
     # 1e-2 beyond |v| = 2.56)
     (C("ck-g4-sq80", 32, 8, 128, 16, fixed(80, 81, 127, 128, 129, 208, 2600, 9100), seed=112, pool_fill=0.8,
        shuffle_batch=False, sigma=0.5), 80),
+    # up to 128 columns on the kernel's one-tile mode: many short units (one to four 128-token slots each, contexts
+    # shorter than the chunk included), so that unit boundaries, stages without tokens and the end marker come close
+    # together; then exactly 128 columns with blocks of 32 tokens
+    (C("ck-g4-sq10-short", 32, 8, 128, 16, (G(48, 1, 400),), seed=113, pool_fill=0.8), 10),
+    (C("ck-g8-sq16-bs32", 64, 8, 128, 32, (G(24, 16, 700),), seed=114, sigma=0.5), 16),
 ]
 
 
@@ -92,11 +99,12 @@ def test_prefill_chunk_matches_oracle(cfg, Sq):
 
 
 @pytest.mark.parametrize("cfg,Sq", [c for c in CHUNK_CASES if c[0].name in
-                                    ("ck-g4-sq33", "ck-g4-sq128-fresh", "ck-g8-sq64-bs64", "ck-split")],
+                                    ("ck-g4-sq5", "ck-g4-sq33", "ck-g4-sq128-fresh", "ck-g8-sq64-bs64", "ck-split",
+                                     "ck-split-g2", "ck-token-major")],
                          ids=lambda v: getattr(v, "name", str(v)))
 def test_prefill_chunk_on_the_mma_sync_kernel(cfg, Sq):
-    """head_dim 128 with more than 32 score columns runs the tcgen05 kernel by default; the mma.sync kernel
-    of the same shape stays selectable and must agree with the oracle too."""
+    """Prefill chunks at head_dim 128 run the tcgen05 kernels by default; the mma.sync kernel of the same
+    shape stays selectable and must agree with the oracle too."""
     binding.set_tuning(chunk_tcgen05=0)
     try:
         run_case(cfg, Sq, seed=cfg.seed)
@@ -104,17 +112,20 @@ def test_prefill_chunk_on_the_mma_sync_kernel(cfg, Sq):
         binding.set_tuning(chunk_tcgen05=1)
 
 
+@pytest.mark.parametrize("two_tiles", [0, 1], ids=["never-two-tiles", "two-tiles-beyond-128-columns"])
 @pytest.mark.parametrize("cfg,Sq", [c for c in CHUNK_CASES if c[0].name in
-                                    ("ck-g4-sq33", "ck-g4-sq128-fresh", "ck-g8-sq64-bs64", "ck-split", "ck-g4-sq80")],
+                                    ("ck-g4-sq5", "ck-g4-sq16", "ck-g4-sq33", "ck-g4-sq128-fresh", "ck-g8-sq64-bs64",
+                                     "ck-split", "ck-g4-sq80", "ck-g4-sq10-short")],
                          ids=lambda v: getattr(v, "name", str(v)))
-def test_prefill_chunk_on_the_one_tile_tcgen05_kernel(cfg, Sq):
-    """More than 128 score columns over a bf16 cache run the kernel with two 128-row tiles per CTA by default;
-    the one-tile tcgen05 kernel stays selectable and must agree with the oracle too."""
-    binding.set_tuning(chunk_two_tiles=0)
+def test_prefill_chunk_on_the_one_tile_tcgen05_kernel(cfg, Sq, two_tiles):
+    """Over a bf16 cache the kernel with one CTA per SM (two 128-row tiles, or one tile in its one-tile mode) runs
+    every chunk by default; the kernel with one tile per CTA and two CTAs per SM stays selectable, for all chunks
+    or for those of up to 128 columns, and must agree with the oracle too."""
+    binding.set_tuning(chunk_two_tiles=two_tiles)
     try:
         run_case(cfg, Sq, seed=cfg.seed)
     finally:
-        binding.set_tuning(chunk_two_tiles=1)
+        binding.set_tuning(chunk_two_tiles=2)
 
 
 def test_chunk_rows_agree_with_decode_rows():
@@ -222,7 +233,8 @@ def test_fused_step_mq():
     assert_parity(out.reshape(-1, 32, 128), ref.out.reshape(-1, 32, 128), what="fused mq step")
 
 
-@pytest.mark.parametrize("Sq,tc", [(5, 1), (40, 1), (40, 0)], ids=["20-columns", "160-columns-tcgen05", "160-columns-mma-sync"])
+@pytest.mark.parametrize("Sq,tc", [(5, 1), (5, 0), (40, 1), (40, 0)],
+                         ids=["20-columns-tcgen05", "20-columns-mma-sync", "160-columns-tcgen05", "160-columns-mma-sync"])
 def test_fused_step_prefill_chunk(Sq, tc):
     """ooco_decode_step_mq with a chunk long enough for the prefill-chunk kernels: the fused append of q_len
     tokens (bit-exact over the whole pool) is seen by the attention of the same call."""
