@@ -530,6 +530,10 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int row0 = 32 * q4 + 16 * hf + g;  // this thread's rows of the tile: row0 and row0 + 8
     const uint32_t trow = tmem + ((uint32_t)(32 * q4 + 16 * hf) << 16) + 256u * t;  // the warp's lanes, the tile's columns
     const int tid_t = threadIdx.x & 255;     // index among the tile's 256 threads
+    // Score column (query token x head) of a tile's row r: column 4 (r % 32) + r / 32 of the tile, so that the columns
+    // of a tile that is not full spread over the four lane quarters -- the warps with hf = 0 take rows before those with
+    // hf = 1, one busy warp per scheduler -- and a warp none of whose rows is a column skips the stage's arithmetic.
+    auto tile_col = [](int r) { return 4 * (r & 31) + (r >> 5); };
     uint8_t* q_gen = gen + (size_t)t * kTc2QBytes;
     float m_ref[2] = {-INFINITY, -INFINITY};  // reference maximum per row (scaled, log2 domain)
     float l_part[2] = {0.f, 0.f};             // this thread's share of the row's sum of weights
@@ -541,7 +545,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // chunk ^= row & 7): thread i of the tile writes 64 dims (half i & 1) of row i >> 1; then the q-ready arrival
     auto load_q = [&](int b_, int h_, int rt_) {
       const int r_ = tid_t >> 1, half_ = tid_t & 1;
-      const int col_ = rt_ * kTc2Rows + t * kTcRows + r_;
+      const int col_ = rt_ * kTc2Rows + t * kTcRows + tile_col(r_);
       const int qi_ = col_ / p.G, head_ = col_ - qi_ * p.G;
       const bool real_ = col_ < p.GQ;
       const uint4* src = reinterpret_cast<const uint4*>(
@@ -566,13 +570,14 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const bool first = !end && ((meta.w >> 16) & 1), last = !end && ((meta.w >> 17) & 1);
       const int b = meta.y, h = meta.z, rt = end ? 0 : meta2.w, lim_base = meta2.y;
       const bool act = !end && (t == 0 || rt * kTc2Rows + kTcRows < p.GQ);
-      const int col0 = rt * kTc2Rows + t * kTcRows + row0;  // score column (query token x head) of row0; row0 + 8: col0 + 8
+      const int col0 = rt * kTc2Rows + t * kTcRows + tile_col(row0);  // score column of row0; that of row0 + 8: col0 + 32
+      const bool warp_rows = rt * kTc2Rows + t * kTcRows + tile_col(32 * q4 + 16 * hf) < p.GQ;  // the warp's first column exists
       if (first && act) {
 #pragma unroll
         for (int rr = 0; rr < 2; ++rr) {
           m_ref[rr] = -INFINITY;
           l_part[rr] = 0.f;
-          lim_row[rr] = lim_base + (col0 + 8 * rr) / p.G;
+          lim_row[rr] = lim_base + (col0 + 32 * rr) / p.G;
         }
         if (ntok > 0 && !q_ahead) load_q(b, h, rt);
         q_ahead = false;
@@ -583,7 +588,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         break;
       }
       if (end) break;
-      if (act && ntok > 0) {
+      if (act && ntok > 0 && warp_rows) {
         tc_fence_after_sync();
         // Two passes over the stage's scores, 64 tokens at a time (32 registers): the row maxima first, then, with the
         // reference maxima known, the weights.  Reading the scores twice costs little (tensor memory is close) and
@@ -688,6 +693,8 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         l_part[0] += add0.x + add0.y;
         l_part[1] += add1.x + add1.y;
         tmem_st_wait();
+      }
+      if (act && ntok > 0) {
         if (ntok < kTc2StageTok) {
           // V rows beyond the stage's tokens may hold anything (NaN included): clear them once the slot has landed
           const int vs = n % NV;
@@ -747,7 +754,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           l += __shfl_xor_sync(0xffffffffu, l, 2);
           inv[rr] = l > 0.f ? 1.f / l : 0.f;  // l = 0: the row saw no token of this chunk
           lse[rr] = l > 0.f ? m_ref[rr] + lg2(l) : -INFINITY;
-          const int col = col0 + 8 * rr;
+          const int col = col0 + 32 * rr;
           const int qi = col / p.G, head = col - qi * p.G;
           write_row[rr] = col < p.GQ && (!kChecked || dst_ok);
           orow[rr] = p.out + (((size_t)b * p.Sq + qi) * p.Hq + (size_t)h * p.G + head) * D;
@@ -755,7 +762,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           if (write_row[rr] && tq == 0 && (n_chunks > 1 || p.out_f32)) p.part_lse[(size_t)slot_id * p.GQ + col] = lse[rr];
         }
 #pragma unroll 1
-        for (int c2 = 0; c2 < 2; ++c2) {
+        for (int c2 = 0; c2 < (warp_rows ? 2 : 0); ++c2) {
           uint32_t o[32];  // o[4 i + 2 rr + c] = row (row0 + 8 rr), dim 64 c2 + 8 i + 2 tq + c
           if (unit_has_tokens) {
             tmem_ld_16x256b_x8(trow + 128 + 64 * c2, o);
