@@ -52,26 +52,26 @@ __global__ void __launch_bounds__(kTc2Threads, 1)
 chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const DecodeParams p) {
   constexpr int D = 128;
-  constexpr int NV = kTc2VSlots, NM = kTc2MetaRing;
+  constexpr int NK = kTc2KSlots, NV = kTc2VSlots, NM = kTc2MetaRing;
   // One-tile mode: no work item has rows for tile 1 (at most 128 score columns).  The kernel is then bound by HBM,
-  // not by the tensor pipe, and what would idle serves the one tile: tile 1's Q region is a third K slot, tile 1's
-  // score columns a second S buffer, and tile 1's issuing warp issues the P.V MMAs (see the MMA warps).
+  // not by the tensor pipe, and what would idle serves the one tile: tile 1's score columns are a second S buffer
+  // and tile 1's issuing warp issues the P.V MMAs (see the MMA warps).  (Tile 1's Q region as a third K slot, and
+  // tile 1's softmax warps taking half of every row's tokens, were built and measured no faster.)
   const bool solo = p.GQ <= kTcRows;
-  const int NK = solo ? kTc2KSlots + 1 : kTc2KSlots;
   constexpr int kWarpK = 16, kWarpV = 17, kWarpM = 18;  // warps 0 .. 15: softmax; 18, 19: MMA of tile 0, 1
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const uint32_t s_q = base;                                       // [2] Q tiles
-  const uint32_t s_k = s_q + (solo ? 1u : 2u) * kTc2QBytes;        // [NK] K slots
-  const uint32_t s_v = s_q + 2u * kTc2QBytes + (uint32_t)kTc2KSlots * kTc2SlotBytes;  // [NV] V slots
+  const uint32_t s_k = s_q + 2u * kTc2QBytes;                      // [NK] K slots
+  const uint32_t s_v = s_k + (uint32_t)NK * kTc2SlotBytes;         // [NV] V slots
   const uint32_t s_meta = s_v + (uint32_t)NV * kTc2SlotBytes;      // [NM] two int4 per stage
   const uint32_t s_vdesc = s_meta + (uint32_t)NM * 32;             // [NV] VStageDesc
   const uint32_t s_bar = s_vdesc + (uint32_t)NV * sizeof(VStageDesc);
   const uint32_t s_kfull = s_bar;                  // [NK] the K slot has landed                          (TMA)
-  const uint32_t s_kempty = s_kfull + (kTc2KSlots + 1) * 8;      // [NK] the score MMAs that read it are complete       (MMA commit)
-  const uint32_t s_vfull = s_kempty + (kTc2KSlots + 1) * 8;      // [NV] the V slot has landed                          (TMA)
+  const uint32_t s_kempty = s_kfull + NK * 8;      // [NK] the score MMAs that read it are complete       (MMA commit)
+  const uint32_t s_vfull = s_kempty + NK * 8;      // [NV] the V slot has landed                          (TMA)
   const uint32_t s_vempty = s_vfull + NV * 8;      // [NV] the P.V MMAs that read it are complete         (MMA commit)
   const uint32_t s_vdfull = s_vempty + NV * 8;     // [NV] the stage's V descriptor is posted             (K producer)
   const uint32_t s_mfull = s_vdfull + NV * 8;      // [NM] the stage's meta words are posted              (K producer)

@@ -1,5 +1,6 @@
-// Prefill-chunk attention over the paged cache on the 5th-generation tensor cores (tcgen05), head_dim 128,
-// for 33 or more score columns per (sequence, kv head).  Same units of work, producer warp, stage layout and
+// Prefill-chunk attention over the paged cache on the 5th-generation tensor cores (tcgen05), head_dim 128, one
+// 128-row tile per CTA and two CTAs per SM: every chunk over the 8-bit cache; over a bf16 cache the kernel of
+// chunk_tc2_kernels.cuh runs by default and this one stays selectable.  Same units of work, producer warp, stage layout and
 // meta words as chunk_main_kernel (chunk_kernels.cuh); row tiles are 128 score rows = the MMA's M.
 //
 //   warp 4      producer: TMA K / V stages of 64 tokens ([half][64 tok][64 dims], 128-byte swizzle)
