@@ -655,7 +655,7 @@ def run_multi_query(args, local_rank):
     tc_knob, tt_knob = int(knobs.get("chunk_tcgen05", 1)), int(knobs.get("chunk_two_tiles", 2))
     tc_from = 17 if tc_knob == 1 else tc_knob                              # first column count on the tcgen05 kernels
     tcgen05 = columns > 16 and cfg.head_dim == 128 and (fp8 or (tc_knob != 0 and columns >= tc_from))
-    two_tiles = tcgen05 and not fp8 and tt_knob != 0 and (columns > 128 or tt_knob == 2)
+    two_tiles = tcgen05 and tt_knob != 0 and ((columns <= 128 and tt_knob == 2) if fp8 else (columns > 128 or tt_knob == 2))
     kernel = (("chunk_tc2_kernel" if two_tiles else "chunk_tc_kernel") if tcgen05 else "chunk_main_kernel") if columns > 16 else (
         "row16_main_kernel" if columns > 8 and not fp8 else "decode_main_kernel")   # (the 8-bit cache has no row16 kernel)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

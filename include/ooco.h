@@ -199,8 +199,9 @@ int ooco_decode_step(const ooco_shape_t* shape, const void* q, const void* k_new
  * runs on tcgen05 (scores and output in tensor memory; over a bf16 cache one CTA per SM with two
  * 128-row tiles taking turns on the tensor pipe, or, up to 128 columns, one tile whose scores run a
  * stage ahead of its softmax), otherwise on mma.sync.  Over the 8-bit cache
- * (ooco_decode_step_mq_fp8) every chunk of more than 16 columns runs the tcgen05 kernel, whose extra
- * warps widen each 8-bit stage to f16 in shared memory first.  The workspace grows with q_len: one fp32
+ * (ooco_decode_step_mq_fp8) every chunk of more than 16 columns runs a tcgen05 kernel whose spare
+ * warps widen each 8-bit stage to f16 in shared memory first (up to 128 columns the one-CTA-per-SM
+ * kernel in its one-tile mode, beyond that the kernel with two CTAs per SM).  The workspace grows with q_len: one fp32
  * partial row per (split item, score column).  q_len = 1 is ooco_decode_attention /
  * ooco_kv_append exactly.  Everything else as for those two.
  */
@@ -465,10 +466,11 @@ int ooco_profile_read(float* ms_out, int max_records, int* n_out);
  * test can separate the arithmetic's error from the output format's rounding; not for the host-buffer
  * step (OOCO_E_UNSUPPORTED).  14 non-zero = the decode kernel over the 8-bit cache (8 consumer warps)
  * computes its scores on tcgen05 from the stored codes (zero = mma.sync on codes widened in registers).
- * 15 = the tcgen05 kernel with one CTA per SM and two 128-row tiles per CTA (bf16 cache, head_dim 128): 2 (default) =
- * every chunk that knob 12 sends to tcgen05 (with 128 score columns or fewer the kernel runs one tile and gives the
- * second tile's score buffer and issuing warp to it), 1 = only chunks of more than 128 score columns, 0 = never (one
- * tile per CTA, two CTAs per SM).
+ * 15 = the tcgen05 kernel with one CTA per SM and two 128-row tiles per CTA (head_dim 128): 2 (default) = every
+ * chunk that knob 12 sends to tcgen05 (with 128 score columns or fewer the kernel runs one tile and gives the
+ * second tile's score buffer and issuing warp to it; over the 8-bit cache only these chunks, its idle warps
+ * widening the codes), 1 = only chunks of more than 128 score columns over a bf16 cache, 0 = never (one tile per
+ * CTA, two CTAs per SM).
  * Changing knobs 4 or 5 changes ooco_decode_workspace_bytes.  Returns OOCO_E_SHAPE for an
  * unknown knob or a value outside its range.  ooco_get_tuning returns a knob's current value
  * (OOCO_E_SHAPE, which is negative, for an unknown knob).

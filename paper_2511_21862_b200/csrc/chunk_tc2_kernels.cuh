@@ -36,6 +36,7 @@ constexpr int kTc2Rows = 2 * kTcRows;                // score rows of a unit
 constexpr int kTc2TmemCols = 512;
 constexpr int kTc2KSlots = 2, kTc2VSlots = 3, kTc2MetaRing = 8;
 constexpr int kTc2Threads = 20 * 32;               // 16 softmax warps, K producer, V producer, one MMA warp per tile
+constexpr int kTc2RawSlotBytes = kTc2StageTok * 128;  // 8-bit cache: K (or V) codes of one stage, one 128-byte row per token
 
 struct ChunkTc2Smem {
   __host__ __device__ static size_t total() {
@@ -48,11 +49,18 @@ struct ChunkTc2Smem {
 // included) uses K slot n % 2, V slot n % 3, meta entry n % 8 and, for each tile, barrier n & 1 of the pairs
 // [2] below with phase parity (n >> 1) & 1 -- every tile takes a turn of its barriers on every stage, with or
 // without work, so nobody can be overtaken by two completions of a barrier it waits on.
+//
+// KV8 (the caches hold E4M3 codes; one-tile mode only, the host launches nothing else): the TMA copies land 8-bit
+// stages ([128 tok][128 B] of K, of V) in rings of their own -- two K slots in tile 1's Q region, two V slots in what
+// is the third V slot otherwise -- and the eight warps that would be tile 1's softmax warps widen every stage into the
+// 16-bit slot layout, exactly, to f16 holding value / 256 (e4m3x2_to_f16x2; the factor is part of the softmax scale
+// and of the output scale), so both contractions run as kind::f16 MMAs with f16 operands (Q and P rounded to f16).
+template <bool KV8>
 __global__ void __launch_bounds__(kTc2Threads, 1)
 chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const DecodeParams p) {
   constexpr int D = 128;
-  constexpr int NK = kTc2KSlots, NV = kTc2VSlots, NM = kTc2MetaRing;
+  constexpr int NK = kTc2KSlots, NV = KV8 ? 2 : kTc2VSlots, NM = kTc2MetaRing;
   // One-tile mode: no work item has rows for tile 1 (at most 128 score columns).  The kernel is then bound by HBM,
   // not by the tensor pipe, and what would idle serves the one tile: tile 1's score columns are a second S buffer
   // and tile 1's issuing warp issues the P.V MMAs (see the MMA warps).  (Tile 1's Q region as a third K slot, and
@@ -66,9 +74,11 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const uint32_t s_q = base;                                       // [2] Q tiles
   const uint32_t s_k = s_q + 2u * kTc2QBytes;                      // [NK] K slots
   const uint32_t s_v = s_k + (uint32_t)NK * kTc2SlotBytes;         // [NV] V slots
-  const uint32_t s_meta = s_v + (uint32_t)NV * kTc2SlotBytes;      // [NM] two int4 per stage
+  const uint32_t s_rk = s_q + kTc2QBytes;                          // KV8: [NK] 8-bit K slots (tile 1's Q region)
+  const uint32_t s_rv = s_v + (uint32_t)NV * kTc2SlotBytes;        // KV8: [NV] 8-bit V slots (the third V slot's place)
+  const uint32_t s_meta = s_v + (uint32_t)kTc2VSlots * kTc2SlotBytes;  // [NM] two int4 per stage
   const uint32_t s_vdesc = s_meta + (uint32_t)NM * 32;             // [NV] VStageDesc
-  const uint32_t s_bar = s_vdesc + (uint32_t)NV * sizeof(VStageDesc);
+  const uint32_t s_bar = s_vdesc + (uint32_t)kTc2VSlots * sizeof(VStageDesc);
   const uint32_t s_kfull = s_bar;                  // [NK] the K slot has landed                          (TMA)
   const uint32_t s_kempty = s_kfull + NK * 8;      // [NK] the score MMAs that read it are complete       (MMA commit)
   const uint32_t s_vfull = s_kempty + NK * 8;      // [NV] the V slot has landed                          (TMA)
@@ -80,7 +90,11 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const uint32_t s_pvdone = s_pready + 32;         // [2 tiles] the unit's last P.V_t is complete          (MMA commit)
   const uint32_t s_qready = s_pvdone + 16;         // [2 tiles] Q_t of the unit is in shared memory        (256 threads)
   const uint32_t s_pvstage = s_qready + 16;       // [2] one-tile mode: the stage's P.V is complete              (MMA commit)
-  const uint32_t s_drain = s_pvstage + 16;
+  const uint32_t s_rkfull = s_pvstage + 16;       // KV8 [NK] the 8-bit K slot has landed                         (TMA)
+  const uint32_t s_rkempty = s_rkfull + 16;       // KV8 [NK] the 8-bit K slot has been widened                   (256 threads)
+  const uint32_t s_rvfull = s_rkempty + 16;       // KV8 [NV] the 8-bit V slot has landed                         (TMA)
+  const uint32_t s_rvempty = s_rvfull + 16;       // KV8 [NV] the 8-bit V slot has been widened                   (256 threads)
+  const uint32_t s_drain = s_rvempty + 16;
   const uint32_t s_slot = s_drain + 16;
   int4* g_meta = reinterpret_cast<int4*>(gen + (s_meta - base));
   VStageDesc* g_vdesc = reinterpret_cast<VStageDesc*>(gen + (s_vdesc - base));
@@ -91,11 +105,17 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   if (threadIdx.x == 0) {
     *s_abort = 0;
     for (int i = 0; i < NK; ++i) {
-      mbar_init(s_kfull + 8 * i, 1);
+      mbar_init(s_kfull + 8 * i, KV8 ? 256 : 1);  // (KV8: filled by the widening threads, not by TMA)
       mbar_init(s_kempty + 8 * i, solo ? 1 : 2);  // one arrival per MMA warp that reads K
     }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(s_rkfull + 8 * i, 1);
+      mbar_init(s_rkempty + 8 * i, 256);
+      mbar_init(s_rvfull + 8 * i, 1);
+      mbar_init(s_rvempty + 8 * i, 256);
+    }
     for (int i = 0; i < NV; ++i) {
-      mbar_init(s_vfull + 8 * i, 1);
+      mbar_init(s_vfull + 8 * i, KV8 ? 256 : 1);
       mbar_init(s_vempty + 8 * i, solo ? 1 : 2);
       mbar_init(s_vdfull + 8 * i, 1);
     }
@@ -139,8 +159,9 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     };
     // waits until K slot, V slot (and with it the V descriptor) of stage `it` are free; false when a wait gave up
     auto acquire = [&]() {
-      return warp_wait(s_kempty + 8 * (it % NK), (((uint32_t)(it / NK)) & 1u) ^ 1u, s_abort) &&
-             warp_wait(s_vempty + 8 * (it % NV), (((uint32_t)(it / NV)) & 1u) ^ 1u, s_abort);
+      // (KV8: the slots the copies land in are the 8-bit ones, free once they have been widened)
+      return warp_wait((KV8 ? s_rkempty : s_kempty) + 8 * (it % NK), (((uint32_t)(it / NK)) & 1u) ^ 1u, s_abort) &&
+             warp_wait((KV8 ? s_rvempty : s_vempty) + 8 * (it % NV), (((uint32_t)(it / NV)) & 1u) ^ 1u, s_abort);
     };
     while (unit < n_units && ok) {
       int nxt = 0;
@@ -183,7 +204,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           break;
         }
         const int ks = it % NK, vs = it % NV, ms = it % NM;
-        const uint32_t kfull = s_kfull + 8 * ks;
+        const uint32_t kfull = (KV8 ? s_rkfull : s_kfull) + 8 * ks;
         if (lane == 0) {
           const int flags = (s == 0 ? 1 : 0) | (s == (nstage > 0 ? nstage : 1) - 1 ? 2 : 0);
           g_meta[2 * ms] = make_int4(d.y, b, h, ntok | (flags << 16));
@@ -191,7 +212,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           g_vdesc[vs].nbox = nbox;
           g_vdesc[vs].h = h;
           if (nbox > 0)
-            mbar_arrive_expect_tx(kfull, 2u * (uint32_t)nbox * box_rows_bytes);
+            mbar_arrive_expect_tx(kfull, (KV8 ? 1u : 2u) * (uint32_t)nbox * box_rows_bytes);
           else
             mbar_arrive(kfull);
         }
@@ -200,13 +221,13 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (lane < nbox) {
           const int tb = tok0 + lane * p.tile_rows;
           const int c_tok = tb % p.bs;
-          const uint32_t k0 = s_k + (uint32_t)ks * kTc2SlotBytes;
+          const uint32_t k0 = KV8 ? s_rk + (uint32_t)ks * kTc2RawSlotBytes : s_k + (uint32_t)ks * kTc2SlotBytes;
           const uint32_t dk = k0 + (uint32_t)lane * box_rows_bytes;
           span_ok = checked(chk_span(dk, box_rows_bytes, k0, (long long)k0 + kTc2HalfBytes) && chk_span(lane, 1, 0, 8),
                             &p.hdr->status, kStatusBadSmem);
           if (span_ok) {
-            tma_load_4d(dk, &tm_k, kfull, 0, c_tok, h, blk_cur);
-            tma_load_4d(dk + kTc2HalfBytes, &tm_k, kfull, 64, c_tok, h, blk_cur);
+            tma_load_4d(dk, &tm_k, kfull, 0, c_tok, h, blk_cur);  // (KV8: the row's 128 codes; else its first 64 dims)
+            if (!KV8) tma_load_4d(dk + kTc2HalfBytes, &tm_k, kfull, 64, c_tok, h, blk_cur);
             g_vdesc[vs].blk[lane & 7] = blk_cur;
             g_vdesc[vs].c_tok[lane & 7] = c_tok;
           }
@@ -231,7 +252,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (lane == 0) {
           g_meta[2 * (it % NM)] = make_int4(-1, 0, 0, 0);
           g_vdesc[it % NV].nbox = -1;
-          mbar_arrive(s_kfull + 8 * (it % NK));
+          mbar_arrive((KV8 ? s_rkfull : s_kfull) + 8 * (it % NK));
           mbar_arrive(s_vdfull + 8 * (it % NV));
           mbar_arrive(s_mfull + 8 * (it % NM));
         }
@@ -245,7 +266,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       int dummy_abort = 0;
       for (int k = 0; k < (it < NK ? it : NK); ++k) {
         const int j = it - 1 - k;
-        mbar_wait_bounded(s_kfull + 8 * (j % NK), (uint32_t)(j / NK) & 1u, &dummy_abort, kWaitLimitNs / 8);
+        mbar_wait_bounded((KV8 ? s_rkfull : s_kfull) + 8 * (j % NK), (uint32_t)(j / NK) & 1u, &dummy_abort, kWaitLimitNs / 8);
       }
     }
   } else if (warp == kWarpV) {
@@ -262,18 +283,19 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       }
       const VStageDesc& vd = g_vdesc[vs];
       const int nbox = vd.nbox;
-      const uint32_t vfull = s_vfull + 8 * vs;
+      const uint32_t vfull = (KV8 ? s_rvfull : s_vfull) + 8 * vs;
       if (nbox <= 0) {  // a stage without tokens, or the end marker
         if (lane == 0) mbar_arrive(vfull);
         if (nbox < 0) break;
         continue;
       }
-      if (lane == 0) mbar_arrive_expect_tx(vfull, 2u * (uint32_t)nbox * box_rows_bytes);
+      if (lane == 0) mbar_arrive_expect_tx(vfull, (KV8 ? 1u : 2u) * (uint32_t)nbox * box_rows_bytes);
       __syncwarp();
       if (lane < nbox && lane < 8) {
-        const uint32_t dv = s_v + (uint32_t)vs * kTc2SlotBytes + (uint32_t)lane * box_rows_bytes;
+        const uint32_t dv = (KV8 ? s_rv + (uint32_t)vs * kTc2RawSlotBytes : s_v + (uint32_t)vs * kTc2SlotBytes) +
+                            (uint32_t)lane * box_rows_bytes;
         tma_load_4d(dv, &tm_v, vfull, 0, vd.c_tok[lane], vd.h, vd.blk[lane]);
-        tma_load_4d(dv + kTc2HalfBytes, &tm_v, vfull, 64, vd.c_tok[lane], vd.h, vd.blk[lane]);
+        if (!KV8) tma_load_4d(dv + kTc2HalfBytes, &tm_v, vfull, 64, vd.c_tok[lane], vd.h, vd.blk[lane]);
       }
     }
     if (!ok) {
@@ -281,7 +303,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       int dummy_abort = 0;
       for (int k = 0; k < (it < NV ? it : NV); ++k) {
         const int j = it - 1 - k;
-        mbar_wait_bounded(s_vfull + 8 * (j % NV), (uint32_t)(j / NV) & 1u, &dummy_abort, kWaitLimitNs / 8);
+        mbar_wait_bounded((KV8 ? s_rvfull : s_vfull) + 8 * (j % NV), (uint32_t)(j / NV) & 1u, &dummy_abort, kWaitLimitNs / 8);
       }
     }
   } else if (warp >= kWarpM && solo) {
@@ -296,7 +318,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int t = warp - kWarpM;
     bool issued = false, ok = true;
     if (t == 0) {
-      const uint32_t idesc_s = umma_idesc_16bit(kTcRows, kTc2StageTok, 0, true);
+      const uint32_t idesc_s = umma_idesc_16bit(kTcRows, kTc2StageTok, 0, !KV8);  // (KV8: f16 operands)
       const uint64_t dq = umma_smem_desc(s_q, 0, 1024);
       uint32_t n_q = 0;  // units with tokens (uses of the q-ready barrier)
       for (uint32_t n = 0;; ++n) {
@@ -351,7 +373,7 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (end) break;
       }
     } else {
-      const uint32_t idesc_o = umma_idesc_16bit(kTcRows, D, 1, true);
+      const uint32_t idesc_o = umma_idesc_16bit(kTcRows, D, 1, !KV8);
       for (uint32_t n = 0;; ++n) {
         const int vs = n % NV, ms = n % NM;
         if (!warp_wait(s_mfull + 8 * ms, (n / NM) & 1u, s_abort)) {
@@ -552,13 +574,67 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           p.q + (((size_t)b_ * p.Sq + (real_ ? qi_ : 0)) * p.Hq + (size_t)h_ * p.G + (real_ ? head_ : 0)) * D + 64 * half_);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
-        const uint4 v = real_ ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+        uint4 v = real_ ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+        if (KV8) v = make_uint4(bf16x2_to_f16x2(v.x), bf16x2_to_f16x2(v.y), bf16x2_to_f16x2(v.z), bf16x2_to_f16x2(v.w));
         *reinterpret_cast<uint4*>(q_gen + (size_t)half_ * kTc2HalfBytes + (size_t)r_ * 128 + ((c ^ (r_ & 7)) << 4)) = v;
       }
       fence_proxy_async_smem();  // the tile is read by the MMAs through the async proxy
       mbar_arrive(s_qready + 8 * t);
     };
-    for (uint32_t n = 0; !(solo && t == 1); ++n) {  // (one-tile mode: the warps of tile 1 have nothing to do)
+    if (KV8 && t == 1) {
+      // ================================================================= widening warps (8-bit cache, one-tile mode)
+      // Stage n of the 8-bit rings becomes stage n of the 16-bit slots (stages without tokens and the end marker take
+      // their turns too).  A unit of work is (token row r, 16-byte chunk c of the row's 128 codes): one 16-byte load,
+      // sixteen codes widened, two 16-byte stores into the row's 64-dim half c / 4; 1024 units per slot, four per
+      // thread.  K first: the scores need it a stage earlier than P.V needs V.
+      auto widen = [&](const uint8_t* rsrc, uint8_t* sdst, int ntok_) {
+#pragma unroll
+        for (int i = 0; i < kTc2StageTok * 8 / 256; ++i) {
+          const int u = i * 256 + tid_t;
+          const int r = u >> 3, c = u & 7;
+          if (r >= ntok_) continue;  // rows beyond the stage's tokens are never used (masked scores, cleared V rows)
+          const uint4 w = *reinterpret_cast<const uint4*>(rsrc + (size_t)r * 128 + ((c ^ (r & 7)) << 4));
+          uint8_t* drow = sdst + (size_t)(c >> 2) * kTc2HalfBytes + (size_t)r * 128;
+          *reinterpret_cast<uint4*>(drow + (((2 * (c & 3)) ^ (r & 7)) << 4)) =
+              make_uint4(e4m3x2_to_f16x2<kSelB0B1>(w.x), e4m3x2_to_f16x2<kSelB2B3>(w.x), e4m3x2_to_f16x2<kSelB0B1>(w.y),
+                         e4m3x2_to_f16x2<kSelB2B3>(w.y));
+          *reinterpret_cast<uint4*>(drow + (((2 * (c & 3) + 1) ^ (r & 7)) << 4)) =
+              make_uint4(e4m3x2_to_f16x2<kSelB0B1>(w.z), e4m3x2_to_f16x2<kSelB2B3>(w.z), e4m3x2_to_f16x2<kSelB0B1>(w.w),
+                         e4m3x2_to_f16x2<kSelB2B3>(w.w));
+        }
+      };
+      for (uint32_t n = 0;; ++n) {
+        const int ks = n % NK, vs = n % NV, ms = n % NM;
+        // the 8-bit K slot has landed (its meta words were written before its barrier was armed), the 16-bit one is free
+        if (!warp_wait(s_rkfull + 8 * ks, (n / NK) & 1u, s_abort) ||
+            !warp_wait(s_kempty + 8 * ks, ((n / NK) & 1u) ^ 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        const int4 meta = g_meta[2 * ms];
+        const bool end = meta.x < 0;
+        const int ntok = end ? 0 : (meta.w & 0xffff);
+        if (ntok > 0) {
+          widen(gen + (s_rk - base) + (size_t)ks * kTc2RawSlotBytes, gen + (s_k - base) + (size_t)ks * kTc2SlotBytes, ntok);
+          fence_proxy_async_smem();  // the widened slot is read by the MMAs through the async proxy
+        }
+        mbar_arrive(s_kfull + 8 * ks);
+        mbar_arrive(s_rkempty + 8 * ks);
+        if (end) break;
+        if (!warp_wait(s_rvfull + 8 * vs, (n / NV) & 1u, s_abort) ||
+            !warp_wait(s_vempty + 8 * vs, ((n / NV) & 1u) ^ 1u, s_abort)) {
+          ok = false;
+          break;
+        }
+        if (ntok > 0) {
+          widen(gen + (s_rv - base) + (size_t)vs * kTc2RawSlotBytes, gen + (s_v - base) + (size_t)vs * kTc2SlotBytes, ntok);
+          fence_proxy_async_smem();
+        }
+        mbar_arrive(s_vfull + 8 * vs);
+        mbar_arrive(s_rvempty + 8 * vs);
+      }
+    }
+    for (uint32_t n = 0; !(solo && t == 1); ++n) {  // (one-tile mode: the warps of tile 1 have nothing else to do)
       const int ms = n % NM;
       if (!warp_wait(s_mfull + 8 * ms, (n / NM) & 1u, s_abort)) {
         ok = false;
@@ -685,8 +761,8 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             const float2 w0 = make_float2(ex2(x0.x), ex2(x0.y)), w1 = make_float2(ex2(x1.x), ex2(x1.y));
             add0 = fadd2(add0, w0);
             add1 = fadd2(add1, w1);
-            pw[2 * i] = pack_bf16x2(w0.x, w0.y);
-            pw[2 * i + 1] = pack_bf16x2(w1.x, w1.y);
+            pw[2 * i] = KV8 ? pack_f16x2(w0.x, w0.y) : pack_bf16x2(w0.x, w0.y);
+            pw[2 * i + 1] = KV8 ? pack_f16x2(w1.x, w1.y) : pack_bf16x2(w1.x, w1.y);
           }
           tmem_st_16x128b_x8(srow + 32 * h2, pw);
         }
@@ -752,7 +828,8 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           float l = l_part[rr];
           l += __shfl_xor_sync(0xffffffffu, l, 1);
           l += __shfl_xor_sync(0xffffffffu, l, 2);
-          inv[rr] = l > 0.f ? 1.f / l : 0.f;  // l = 0: the row saw no token of this chunk
+          // l = 0: the row saw no token of this chunk; the 8-bit cache's V scale (and widening factor) comes in here
+          inv[rr] = (l > 0.f ? 1.f / l : 0.f) * (KV8 ? p.v_scale : 1.f);
           lse[rr] = l > 0.f ? m_ref[rr] + lg2(l) : -INFINITY;
           const int col = col0 + 32 * rr;
           const int qi = col / p.G, head = col - qi * p.G;

@@ -361,10 +361,12 @@ static int launch_chunk_tc(const CUtensorMap& tk, const CUtensorMap& tv, DecodeP
 // Prefill chunk on tcgen05, one persistent CTA per SM, 512 tensor-memory columns, 128-token K / V slots (head_dim 128,
 // bf16 cache): two 128-row tiles per CTA beyond 128 score columns; up to 128 columns its one-tile mode, in which the
 // second tile's resources (score columns, issuing warp, Q region) pipeline the one tile -- it beats the one-tile
-// kernel and the mma.sync kernel on every workload measured, from 17 columns on.
+// kernel and the mma.sync kernel on every workload measured, from 17 columns on.  KV8: the one-tile mode over the 8-bit
+// cache (the idle softmax warps widen the codes), 1.25 to 1.5 times as fast as the two-CTA kernel on these shapes.
+template <bool KV8>
 static int launch_chunk_tc2(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, const DeviceInfo& di,
                             cudaStream_t st, int dev, bool dry) {
-  auto kern = chunk_tc2_kernel;
+  auto kern = chunk_tc2_kernel<KV8>;
   static std::atomic<int> static_smem{-1};
   if (static_smem.load() < 0) {
     cudaFuncAttributes fa;
@@ -755,7 +757,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   const bool chunk_tc = chunk && s->head_dim == 128 && (kv8 || (tc_knob != 0 && G_ >= tc_from));
   // (more than one 128-row tile per item, bf16: the kernel that keeps two tiles per CTA on the tensor pipe in turns)
   const int two_tiles = g_knobs[kKnobChunkTwoTiles].load();  // 1: beyond 128 columns only; 2: its one-tile mode below, too
-  const bool chunk_tc2 = chunk_tc && !kv8 && two_tiles != 0 && (G_ > kTcRows || two_tiles == 2);
+  // (8-bit cache: only the one-tile mode has a variant that widens the codes, so up to 128 columns)
+  const bool chunk_tc2 = chunk_tc && two_tiles != 0 && (kv8 ? (G_ <= kTcRows && two_tiles == 2) : (G_ > kTcRows || two_tiles == 2));
   if (chunk) {
     ncw = chunk_warps(G_);
     cps = (ncw == 8 && !chunk_tc) ? 1 : 2;
@@ -826,7 +829,8 @@ static int decode_core(const ooco_shape_t* s, const void* q, const void* k_cache
   // once without launching, before the first kernel of the call is enqueued.
   const int stages = g_knobs[kKnobStages].load();
   auto launch_attention = [&](bool dry) -> int {
-    if (chunk_tc2) return launch_chunk_tc2(tk, tv, p, di, st, dev, dry);
+    if (chunk_tc2)
+      return kv8 ? launch_chunk_tc2<true>(tk, tv, p, di, st, dev, dry) : launch_chunk_tc2<false>(tk, tv, p, di, st, dev, dry);
     if (chunk_tc)
       return kv8 ? launch_chunk_tc<true>(tk, tv, p, di, cps, st, dev, dry)
                  : launch_chunk_tc<false>(tk, tv, p, di, cps, st, dev, dry);

@@ -340,6 +340,21 @@ def run_case_8bit(cfg, Sq, seed, ks=1.0 / 32, vs=0.04):
     return batch, q, out
 
 
+@pytest.mark.parametrize("cfg,Sq", [c for c in CHUNK_CASES if c[0].name in
+                                    ("ck-g4-sq5", "ck-g4-sq16", "ck-g5-sq7-bs32", "ck-g1-sq100-bs128", "ck-token-major",
+                                     "ck-split-g2", "ck-g4-sq10-short", "ck-g8-sq16-bs32")],
+                         ids=lambda v: getattr(v, "name", str(v)))
+def test_prefill_chunk_over_8bit_cache_on_the_two_cta_kernel(cfg, Sq):
+    """Up to 128 score columns over the 8-bit cache run the one-CTA-per-SM kernel's one-tile mode by default (its idle
+    warps widen the codes); the kernel with two CTAs per SM, which serves more columns, stays selectable for these
+    shapes and must agree with the oracle too."""
+    binding.set_tuning(chunk_two_tiles=1)
+    try:
+        run_case_8bit(cfg, Sq, seed=cfg.seed)
+    finally:
+        binding.set_tuning(chunk_two_tiles=2)
+
+
 @pytest.mark.parametrize("cfg,Sq", [c for c in CHUNK_CASES if c[0].head_dim == 128],
                          ids=lambda v: getattr(v, "name", str(v)))
 def test_prefill_chunk_over_8bit_cache(cfg, Sq):
