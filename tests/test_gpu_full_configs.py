@@ -104,11 +104,11 @@ def test_very_long_context_next_to_very_short_ones():
         assert err.max() <= 1e-2 and err.mean() <= 1e-3, (b, h, err.max())
 
 
-@pytest.mark.parametrize("Sq", [4, 64], ids=["16-columns", "256-columns"])
+@pytest.mark.parametrize("Sq", [4, 16, 64], ids=["16-columns", "64-columns", "256-columns"])
 def test_prefill_chunk_full_size_every_output(Sq):
     """Several query tokens per sequence at benchmark size and launch shape (cfg1 with the chunk added to every
-    context): the 16-column row-layout kernel and the tcgen05 chunk kernel; every row of every sequence
-    against the oracle."""
+    context): the 16-column row-layout kernel and the tcgen05 chunk kernel in its one-tile and its two-tile mode;
+    every row of every sequence against the oracle."""
     base = inputs.CONFIGS["cfg1"]
     cfg = inputs.replace(base, groups=tuple(inputs.replace(g, lo=g.lo + Sq, hi=g.hi + Sq) for g in base.groups))
     batch = inputs.make_batch(cfg, "cuda", poison=True)
@@ -129,10 +129,43 @@ def test_prefill_chunk_full_size_every_output(Sq):
     print(f"cfg1 with {Sq} query tokens, all {ref.out.size} outputs: max abs {mx:.3e} mean abs {mean:.3e}")
 
 
-def test_prefill_chunk_over_8bit_cache_full_size_every_output():
-    """cfg1 with a 64-token chunk per sequence over E4M3 caches (256 score columns: two row tiles of the tcgen05
-    kernel, stages widened in shared memory), every output against the 8-bit oracle."""
-    Sq, ks, vs = 64, 1.0 / 32, 1.0 / 32
+def test_small_chunk_on_the_long_context_mix_every_output():
+    """cfg3 with 8 query tokens per sequence (64 score columns: the tcgen05 chunk kernel's one-tile mode) at
+    benchmark size and launch shape: 115 short sequences of one to eight 128-token slots beside 13 of 32 K to 64 K
+    tokens, so units of every length, split and unsplit, follow each other in every CTA.  Three launches give the
+    same bits (the hand-overs between the issuing warps and the softmax threads do not depend on timing), and every
+    output agrees with the oracle."""
+    Sq = 8
+    base = inputs.CONFIGS["cfg3"]
+    cfg = inputs.replace(base, groups=tuple(inputs.replace(g, lo=g.lo + Sq, hi=g.hi + Sq) for g in base.groups))
+    batch = inputs.make_batch(cfg, "cuda", poison=True)
+    B, Hq, D, bs = cfg.batch, cfg.num_q_heads, cfg.head_dim, cfg.block_size
+    gen = torch.Generator(device="cuda").manual_seed(79)
+    q = (torch.randn((B, Sq, Hq, D), generator=gen, device="cuda") * cfg.sigma).to(torch.bfloat16)
+    sh = binding.shape_of(batch)
+    ws = torch.empty(binding.workspace_bytes_mq(sh, Sq), dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(3):
+        out = torch.full_like(q, float("nan"))
+        binding.decode_attention_mq(sh, q, batch.k_cache, batch.v_cache, batch.block_table, batch.context_lens, cfg.scale,
+                                    out, ws)
+        assert binding.workspace_status(ws) == 0
+        outs.append(out)
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+    assert torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
+    ref = oracle.decode_attention_mq(inputs.as_u16(q), inputs.as_u16(batch.k_cache), inputs.as_u16(batch.v_cache),
+                                     batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
+                                     num_kv_heads=cfg.num_kv_heads, block_size=bs, strides=batch.strides)
+    mx, mean = assert_parity(outs[0].reshape(-1, Hq, D), ref.out.reshape(-1, Hq, D), what="cfg3 + chunk of 8")
+    print(f"cfg3 with 8 query tokens, all {ref.out.size} outputs: max abs {mx:.3e} mean abs {mean:.3e}")
+
+
+@pytest.mark.parametrize("Sq", [16, 64], ids=["64-columns", "256-columns"])
+def test_prefill_chunk_over_8bit_cache_full_size_every_output(Sq):
+    """cfg1 with a chunk of 16 or 64 tokens per sequence over E4M3 caches (64 score columns: the one-CTA kernel's
+    one-tile mode, whose spare warps widen the stages; 256 columns: two row tiles of the two-CTA kernel, stages
+    widened in shared memory by warps of their own), every output against the 8-bit oracle."""
+    ks, vs = 1.0 / 32, 1.0 / 32
     base = inputs.CONFIGS["cfg1"]
     cfg = inputs.replace(base, groups=tuple(inputs.replace(g, lo=g.lo + Sq, hi=g.hi + Sq) for g in base.groups))
     batch = inputs.to_e4m3_pool(inputs.make_batch(cfg, "cuda", poison=True), ks, vs)
@@ -148,5 +181,5 @@ def test_prefill_chunk_over_8bit_cache_full_size_every_output():
     ref = oracle.decode_attention_mq_fp8(inputs.as_u16(q), inputs.as_u8(batch.k_cache), inputs.as_u8(batch.v_cache),
                                          batch.block_table.cpu().numpy(), batch.context_lens.cpu().numpy(), cfg.scale,
                                          ks, vs, num_kv_heads=cfg.num_kv_heads, block_size=bs, strides=batch.strides)
-    mx, mean = assert_parity(out.reshape(-1, Hq, D), ref.out.reshape(-1, Hq, D), what="cfg1 + chunk of 64, 8-bit cache")
-    print(f"cfg1 with 64 query tokens over an 8-bit cache, all {ref.out.size} outputs: max abs {mx:.3e} mean abs {mean:.3e}")
+    mx, mean = assert_parity(out.reshape(-1, Hq, D), ref.out.reshape(-1, Hq, D), what=f"cfg1 + chunk of {Sq}, 8-bit cache")
+    print(f"cfg1 with {Sq} query tokens over an 8-bit cache, all {ref.out.size} outputs: max abs {mx:.3e} mean abs {mean:.3e}")
