@@ -46,7 +46,7 @@ struct ChunkTc2Smem {
 };
 
 // Barrier bookkeeping.  Stage number n (counted over the whole kernel, bookkeeping stages and the end marker
-// included) uses K slot n % 2, V slot n % 3, meta entry n % 8 and, for each tile, barrier n & 1 of the pairs
+// included) uses K slot n % 2, V slot n % 3 (n % 2 over the 8-bit cache), meta entry n % 8 and, for each tile, barrier n & 1 of the pairs
 // [2] below with phase parity (n >> 1) & 1 -- every tile takes a turn of its barriers on every stage, with or
 // without work, so nobody can be overtaken by two completions of a barrier it waits on.
 //
@@ -63,8 +63,9 @@ chunk_tc2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   constexpr int NK = kTc2KSlots, NV = KV8 ? 2 : kTc2VSlots, NM = kTc2MetaRing;
   // One-tile mode: no work item has rows for tile 1 (at most 128 score columns).  The kernel is then bound by HBM,
   // not by the tensor pipe, and what would idle serves the one tile: tile 1's score columns are a second S buffer
-  // and tile 1's issuing warp issues the P.V MMAs (see the MMA warps).  (Tile 1's Q region as a third K slot, and
-  // tile 1's softmax warps taking half of every row's tokens, were built and measured no faster.)
+  // and tile 1's issuing warp issues the P.V MMAs (see the MMA warps).  (Over a bf16 cache tile 1's Q region and
+  // softmax warps stay idle: the region as a third K slot, and the warps taking half of every row's tokens, were
+  // built and measured no faster.  Over the 8-bit cache they hold and widen the 8-bit slots.)
   const bool solo = p.GQ <= kTcRows;
   constexpr int kWarpK = 16, kWarpV = 17, kWarpM = 18;  // warps 0 .. 15: softmax; 18, 19: MMA of tile 0, 1
   extern __shared__ uint8_t smem_raw[];
